@@ -1,0 +1,232 @@
+/*
+ * egtp.h - C ABI of the B200 (sm_100a) hot path of the entropy-guided length predictor:
+ * Entropy-Guided Token Pooling (EGTP, paper Sec. 3.1, Eq. 2-4), the prediction head's forward
+ * pass (Sec. 3.2, Eq. 6) and Progressive Length Prediction (PLP, Sec. 3.3, Eq. 8).
+ *
+ * Conventions that hold for every entry point
+ *   - Plain C types only.  "device" pointers are CUDA device addresses on the context's GPU,
+ *     "host" pointers are ordinary (ideally pinned) host addresses.  Each argument says which.
+ *   - The caller owns every buffer it passes in.  The library owns only egtp_ctx / plp_state
+ *     and keeps no caller pointer beyond the work a call enqueues on its stream.
+ *   - Every function returns an egtp_status (0 = success, negative = error).  Problems the
+ *     host can see (NULL pointers, sizes beyond the context's capacity, unsupported layouts)
+ *     are returned at once and nothing is launched.  Problems only the device can see
+ *     (malformed offsets, an out-of-range slot, a bounded wait that ran out) are written to
+ *     the device status word: the first error wins, later kernels of the call do nothing,
+ *     nothing traps and the CUDA context stays usable.
+ *   - Device-pointer entry points are asynchronous: they enqueue on `stream` (a cudaStream_t
+ *     passed as void*, NULL = the default stream) and return.  They never allocate device
+ *     memory and never synchronise; all workspace is created by egtp_create /
+ *     plp_state_create.  The *_host entry points copy their inputs host->device, run, copy
+ *     the result back and synchronise the stream before returning.
+ *   - Calls that use the same context must not overlap on the GPU (they share workspace).
+ *   - Same inputs give bitwise identical outputs (no floating-point atomics anywhere).
+ *   - Matrices are row-major.  The LM head is W[V][d] (row v = vocabulary entry v), so the
+ *     logit of token i for entry v is sum_k hidden[i][k] * W[v][k]; no bias, norm or
+ *     temperature is applied (the caller passes the tensor that feeds its LM head).
+ *   - Supported layouts: hidden and W in the same dtype (EGTP_F32 or EGTP_BF16); rows start
+ *     on 16-byte boundaries (d * element size and both leading dimensions are multiples of
+ *     16 bytes); d is a multiple of 16.  Anything else is EGTP_ERR_UNSUPPORTED; there is no
+ *     CPU fallback.
+ */
+#ifndef EGTP_H_
+#define EGTP_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define EGTP_API __attribute__((visibility("default")))
+#else
+#define EGTP_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct egtp_ctx egtp_ctx;     /* device workspace, tensor-map encoder, SM count */
+typedef struct plp_state plp_state;   /* per-slot running state (m, s, acc[d]) in device memory */
+
+enum {
+  EGTP_OK = 0,
+  EGTP_ERR_INVALID_ARG = -1,      /* NULL where data is required, negative size, alpha <= 0 ... */
+  EGTP_ERR_UNSUPPORTED = -2,      /* dtype / alignment / layout the kernels do not handle */
+  EGTP_ERR_CAPACITY = -3,         /* larger than what egtp_create / plp_state_create was sized for */
+  EGTP_ERR_CUDA = -4,             /* a CUDA runtime or driver call failed */
+  EGTP_ERR_BAD_OFFSETS = -5,      /* (device) offsets not non-decreasing inside [0, T_total] */
+  EGTP_ERR_DEVICE_TIMEOUT = -6,   /* (device) a bounded wait inside a kernel ran out */
+  EGTP_ERR_BAD_SLOT = -7          /* (device) slot id or reset source out of range */
+};
+
+enum { EGTP_F32 = 0, EGTP_BF16 = 1 };                 /* element type of hidden, W and head weights */
+enum { EGTP_HEAD_SCALAR = 0, EGTP_HEAD_BINS = 1 };    /* head output mode */
+enum { PLP_RESET_KEEP = -2, PLP_RESET_EMPTY = -1 };   /* values of reset_src besides row ids >= 0 */
+
+/* LM head (Sec. 3.1: the next-token distribution over the vocabulary V). Device memory, read-only. */
+typedef struct {
+  const void* W;      /* device; [V][ldw] elements, first d of each row used */
+  int64_t ldw;        /* leading dimension in elements, >= d, ldw * element size % 16 == 0 */
+  int32_t d;          /* hidden size */
+  int32_t V;          /* vocabulary size */
+  int32_t dtype;      /* EGTP_F32 or EGTP_BF16; must equal the dtype of the hidden states */
+  int32_t reserved;
+} egtp_lm_head;
+
+/* Prediction head (Sec. 3.2): u = ReLU(W1 z + b1), o = W2 u + b2.
+ * EGTP_HEAD_SCALAR (d_out == 1): y = o[0].
+ * EGTP_HEAD_BINS   (d_out == K): p = softmax(o), y = sum_k p[k] * centres[k]   (Eq. 6).
+ * Device memory, read-only. */
+typedef struct {
+  const void* W1;        /* device; [m_h][d] in `wdtype` */
+  const float* b1;       /* device; [m_h] */
+  const void* W2;        /* device; [d_out][m_h] in `wdtype` */
+  const float* b2;       /* device; [d_out] */
+  const float* centres;  /* device; [d_out] bin centres c_k, NULL in scalar mode */
+  int32_t d, m_h, d_out; /* m_h <= 8192, d_out <= 256 */
+  int32_t wdtype;        /* EGTP_F32 or EGTP_BF16 */
+  int32_t mode;          /* EGTP_HEAD_SCALAR or EGTP_HEAD_BINS */
+  int32_t reserved;
+} egtp_head;
+
+/* Creates a context on CUDA device `device` and allocates all workspace once, sized for at
+ * most max_tokens packed tokens per call, max_batch prompts (or live sequences), hidden
+ * size max_d and vocabulary max_V.  *out is set only on success.  The device must be an
+ * sm_100 GPU (EGTP_ERR_UNSUPPORTED otherwise; EGTP_ERR_CUDA if allocation fails). */
+EGTP_API int egtp_create(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_batch,
+                int32_t max_d, int32_t max_V);
+
+/* Frees the context's device memory. Outstanding work on its streams must have finished. */
+EGTP_API int egtp_destroy(egtp_ctx* ctx);
+
+/* Static description of a status code (never NULL). */
+EGTP_API const char* egtp_status_string(int status);
+
+/* Bytes of device memory the context holds. */
+EGTP_API int64_t egtp_workspace_bytes(const egtp_ctx* ctx);
+
+/* EGTP over a packed ragged batch of prompts (Sec. 3.1 Eq. 2-4, then the head of Sec. 3.2).
+ *   Eq. 2: H[i] = -sum_v p_v ln p_v with p = softmax(W hidden[i]) (natural log), for every
+ *          token row i in [0, T_total); the T x V logits are never written to memory.
+ *   Eq. 3: within prompt b (tokens offsets[b] <= i < offsets[b+1]):
+ *          w_i = exp(H_i/alpha) / sum_j exp(H_j/alpha); alpha = 1 is the equation as printed.
+ *   Eq. 4: pooled[b] = sum_i w_i hidden[i].
+ *   Eq. 6: yhat[b] = head(pooled[b]).
+ * An empty prompt gives pooled = 0, state (m, s) = (-inf, 0) and yhat = head(0).  Tokens
+ * before offsets[0] or at/after offsets[B] get an entropy but join no prompt (seg_id -1,
+ * weight 0).
+ * Arguments (all pointers device unless stated):
+ *   lm, head      host structs holding device pointers; head may be NULL (then yhat_out and
+ *                 phat_out must be NULL and the head is skipped)
+ *   hidden        [T_total][ldh] rows in lm->dtype, read-only
+ *   offsets       int32 [B+1], token units, must satisfy 0 <= offsets[0] <= ... <= offsets[B]
+ *                 <= T_total (checked on the device: EGTP_ERR_BAD_OFFSETS in the status word)
+ *   alpha         temperature dividing the entropies in Eq. 3, > 0
+ *   H_out         [T_total] or NULL      token entropies (nats)
+ *   weights_out   [T_total] or NULL      w_i of Eq. 3 (0 for tokens in no prompt)
+ *   seg_id_out    int32 [T_total] or NULL  prompt index of each token, -1 if none
+ *   pooled_out    [B][d] or NULL         Eq. 4
+ *   state_m_out, state_s_out  [B] each or NULL: max_i H_i/alpha and sum_i exp(H_i/alpha - max),
+ *                 the softmax normaliser that lets plp_step continue from this prompt
+ *   yhat_out      [B] or NULL            predicted length
+ *   phat_out      [B][d_out] or NULL     bin probabilities (bins mode only)
+ *   status_dev    int32 [1] or NULL: device status word (caller zeroes it before the call; a
+ *                 non-zero word on entry turns the whole call into a no-op). NULL = a word the
+ *                 context owns, zeroed at the start of the call.
+ *   stream        cudaStream_t
+ * Returns EGTP_OK once the work is enqueued. B = 0 or T_total = 0 enqueue nothing. */
+EGTP_API int egtp_predict(egtp_ctx* ctx, const egtp_lm_head* lm, const egtp_head* head,
+                 const void* hidden, int64_t ldh, const int32_t* offsets,
+                 int32_t B, int64_t T_total, float alpha,
+                 float* H_out, float* weights_out, int32_t* seg_id_out,
+                 float* pooled_out, float* state_m_out, float* state_s_out,
+                 float* yhat_out, float* phat_out,
+                 int32_t* status_dev, void* stream);
+
+/* Same computation with the per-call data in HOST memory: hidden_host [T_total][d] (dense,
+ * lm->dtype), offsets_host int32 [B+1], yhat_host float [B] (output), pooled_host [B][d] or NULL
+ * (output), status_host int32 [1] (output: final device status word).  lm and head still
+ * point at device-resident parameters.  Copies in, runs, copies out, synchronises `stream`. */
+EGTP_API int egtp_predict_host(egtp_ctx* ctx, const egtp_lm_head* lm, const egtp_head* head,
+                      const void* hidden_host, const int32_t* offsets_host,
+                      int32_t B, int64_t T_total, float alpha,
+                      float* yhat_host, float* pooled_host, int32_t* status_host, void* stream);
+
+/* Running PLP state for num_slots decode slots of hidden size d (Sec. 3.3): per slot the
+ * online-softmax triple (m, s, acc[d]) of Eq. 3-4 over the tokens the sequence has
+ * contributed so far; all slots start empty.  Allocates num_slots * (d + 2) floats. */
+EGTP_API int plp_state_create(egtp_ctx* ctx, plp_state** out, int32_t num_slots, int32_t d);
+EGTP_API int plp_state_destroy(plp_state* st);
+
+/* Checkpoint / restore of the running state: m [num_slots], s [num_slots], acc [num_slots][d],
+ * all device pointers, copied on `stream`. */
+EGTP_API int plp_state_export(plp_state* st, float* m, float* s, float* acc, void* stream);
+EGTP_API int plp_state_import(plp_state* st, const float* m, const float* s, const float* acc, void* stream);
+
+/* One PLP decode step over B_live live sequences, one new token each (Sec. 3.3, Eq. 8).
+ * Aggregate(h, {h'_1..h'_t}) is read as token-axis concatenation followed by EGTP: z_t is the
+ * entropy-weighted pool (one joint softmax, Eq. 3-4) over the prompt's tokens and generated
+ * tokens 1..t, kept incrementally in the slot's (m, s, acc); the head then gives the
+ * remaining length.  For row i (slot = slot_ids[i]):
+ *   reset_src[i] == PLP_RESET_KEEP : continue the slot's sequence;
+ *   reset_src[i] == PLP_RESET_EMPTY: start a new sequence with no prompt;
+ *   reset_src[i] == r >= 0         : start a new sequence from EGTP row r, i.e. from
+ *                                    (src_m[r], src_s[r], src_pooled[r]) as egtp_predict wrote them;
+ *   then the new token's entropy H' (Eq. 2) enters the softmax and hidden_step[i] the pool.
+ * Arguments (device unless stated):
+ *   hidden_step   [B_live][ldh] rows in lm->dtype
+ *   slot_ids      int32 [B_live], distinct, each in [0, num_slots); NULL = identity (row i -> slot i)
+ *   reset_src     int32 [B_live] or NULL (all keep)
+ *   src_m, src_s  [n_src]; src_pooled [n_src][d]; may be NULL when n_src == 0
+ *   Hstep_out     [B_live] or NULL   entropy of each new token
+ *   z_out         [B_live][d] or NULL  Eq. 8
+ *   yrem_out      [B_live] or NULL   predicted remaining length (needs head)
+ *   status_dev, stream as in egtp_predict. */
+EGTP_API int plp_step(egtp_ctx* ctx, plp_state* st, const egtp_lm_head* lm, const egtp_head* head,
+             const void* hidden_step, int64_t ldh,
+             const int32_t* slot_ids, const int32_t* reset_src,
+             const float* src_m, const float* src_s, const float* src_pooled, int32_t n_src,
+             int32_t B_live, float alpha,
+             float* Hstep_out, float* z_out, float* yrem_out,
+             int32_t* status_dev, void* stream);
+
+/* plp_step with the step's data in HOST memory: hidden_step_host [B_live][d] dense,
+ * reset_src_host int32 [B_live] or NULL, yrem_host float [B_live] (output), status_host int32 [1]
+ * (output).  Rows map to slots 0..B_live-1.  The EGTP source table stays on the device. */
+EGTP_API int plp_step_host(egtp_ctx* ctx, plp_state* st, const egtp_lm_head* lm, const egtp_head* head,
+                  const void* hidden_step_host, const int32_t* reset_src_host,
+                  const float* src_m, const float* src_s, const float* src_pooled, int32_t n_src,
+                  int32_t B_live, float alpha, float* yrem_host, int32_t* status_host, void* stream);
+
+/* Per-kernel timing. With profiling on, every kernel launch of this context is bracketed by
+ * CUDA events on its own stream.  egtp_profile_read synchronises the device, adds up the
+ * elapsed milliseconds and launch counts per kernel since the last read and clears them.
+ * Kernel ids index the two output arrays (host pointers, EGTP_NUM_KERNELS entries each). */
+enum {
+  EGTP_K_VALIDATE = 0,      /* offsets check */
+  EGTP_K_LMHEAD_ENTROPY,    /* tcgen05 LM-head GEMM with the online entropy epilogue */
+  EGTP_K_ENTROPY_MERGE,     /* merge of per-vocabulary-chunk partials into H */
+  EGTP_K_SEGMENT_WEIGHTS,   /* Eq. 3 per prompt */
+  EGTP_K_POOL,              /* Eq. 4, first stage */
+  EGTP_K_POOL_COMBINE,      /* Eq. 4, deterministic combine of prompts that span chunks */
+  EGTP_K_HEAD_HIDDEN,       /* head layer 1 */
+  EGTP_K_HEAD_OUT,          /* head layer 2 + output mode */
+  EGTP_K_PLP_UPDATE,        /* PLP running-state update */
+  EGTP_NUM_KERNELS
+};
+EGTP_API int egtp_profile_enable(egtp_ctx* ctx, int on);
+EGTP_API int egtp_profile_read(egtp_ctx* ctx, double* ms_by_kernel, int64_t* launches_by_kernel);
+EGTP_API const char* egtp_kernel_name(int kernel_id);
+
+/* Total number of kernels this context has launched since it was created. */
+EGTP_API int64_t egtp_launch_count(const egtp_ctx* ctx);
+
+/* Launch shape the LM-head kernel uses for T rows of hidden size d against V vocabulary rows:
+ * info[0] = grid (CTAs), [1] = row tiles, [2] = vocabulary tiles, [3] = vocabulary chunks,
+ * [4] = partial slots per row, [5] = row tiles per group, [6] = k blocks, [7] = dynamic smem bytes.
+ * Host pointer; nothing is launched. */
+EGTP_API int egtp_lmhead_plan(const egtp_ctx* ctx, int64_t T, int32_t d, int32_t V, int32_t dtype, int32_t info[8]);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EGTP_H_ */

@@ -1,0 +1,550 @@
+// C ABI of the library (see include/egtp.h): argument checks, workspace, TMA tensor maps,
+// kernel sequencing, per-kernel event timing.  No arithmetic of the method lives here.
+#include "../../include/egtp.h"
+#include "kernels.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cudaTypedefs.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+using namespace egtp;
+
+namespace {
+
+struct EventPair {
+  cudaEvent_t start, stop;
+  int kernel;
+};
+
+}  // namespace
+
+struct egtp_ctx {
+  int device = 0;
+  int num_sms = 0;
+  int64_t max_tokens = 0;
+  int32_t max_batch = 0, max_d = 0, max_V = 0;
+  PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+
+  // workspace (device)
+  float* partials = nullptr;      int64_t slot_row_capacity = 0;   // rows x slots the partial buffer holds
+  float* H = nullptr;             // [max(max_tokens, max_batch)]
+  float* weights = nullptr;       // [max_tokens]
+  float* seg_m = nullptr;         // [max_batch]
+  float* seg_s = nullptr;         // [max_batch]
+  float* pooled = nullptr;        // [max_batch][max_d]  (also z of a PLP step)
+  float* piece_a = nullptr;       // [chunks][max_d]
+  float* piece_b = nullptr;       // [chunks][max_d]
+  float* head_partial = nullptr;  int64_t head_partial_floats = 0;
+  float* yhat = nullptr;          // [max_batch]
+  int32_t* status = nullptr;      // [1]
+  // staging for the *_host entry points (device)
+  void* hidden_stage = nullptr;   // [max_tokens][max_d] in the widest supported dtype
+  int32_t* offsets_stage = nullptr;  // [max_batch + 1]
+  int32_t* reset_stage = nullptr;    // [max_batch]
+  int64_t bytes = 0;
+
+  // bookkeeping
+  int64_t launches = 0;
+  bool profiling = false;
+  std::vector<EventPair> pending;
+  std::vector<EventPair> free_events;
+  double ms_acc[EGTP_NUM_KERNELS] = {};
+  int64_t n_acc[EGTP_NUM_KERNELS] = {};
+};
+
+struct plp_state {
+  egtp_ctx* ctx = nullptr;
+  int32_t num_slots = 0, d = 0;
+  float* m = nullptr;
+  float* s = nullptr;
+  float* acc = nullptr;
+};
+
+namespace {
+
+const char* const kKernelNames[EGTP_NUM_KERNELS] = {
+    "validate_offsets", "lmhead_entropy", "entropy_merge", "segment_weights", "pool",
+    "pool_combine",     "head_hidden",    "head_out",      "plp_update"};
+
+template <typename T>
+cudaError_t dev_alloc(egtp_ctx* c, T** p, int64_t count) {
+  const size_t bytes = static_cast<size_t>(std::max<int64_t>(count, 1)) * sizeof(T);
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), bytes);
+  if (e == cudaSuccess) c->bytes += static_cast<int64_t>(bytes);
+  return e;
+}
+
+void free_ctx_memory(egtp_ctx* c) {
+  cudaFree(c->partials); cudaFree(c->H); cudaFree(c->weights); cudaFree(c->seg_m); cudaFree(c->seg_s);
+  cudaFree(c->pooled); cudaFree(c->piece_a); cudaFree(c->piece_b); cudaFree(c->head_partial); cudaFree(c->yhat);
+  cudaFree(c->status); cudaFree(c->hidden_stage); cudaFree(c->offsets_stage); cudaFree(c->reset_stage);
+  for (auto& e : c->pending) { cudaEventDestroy(e.start); cudaEventDestroy(e.stop); }
+  for (auto& e : c->free_events) { cudaEventDestroy(e.start); cudaEventDestroy(e.stop); }
+}
+
+// Brackets one kernel launch with events when profiling is on; counts launches always.
+struct LaunchScope {
+  egtp_ctx* c;
+  cudaStream_t stream;
+  EventPair ev{};
+  bool timed = false;
+  LaunchScope(egtp_ctx* ctx, int kernel, cudaStream_t s) : c(ctx), stream(s) {
+    c->launches += 1;
+    if (!c->profiling) return;
+    if (!c->free_events.empty()) {
+      ev = c->free_events.back();
+      c->free_events.pop_back();
+    } else {
+      if (cudaEventCreate(&ev.start) != cudaSuccess) return;
+      if (cudaEventCreate(&ev.stop) != cudaSuccess) { cudaEventDestroy(ev.start); return; }
+    }
+    ev.kernel = kernel;
+    timed = true;
+    cudaEventRecord(ev.start, stream);
+  }
+  ~LaunchScope() {
+    if (!timed) return;
+    cudaEventRecord(ev.stop, stream);
+    c->pending.push_back(ev);
+  }
+};
+
+int elem_bytes(int dtype) { return dtype == EGTP_BF16 ? 2 : 4; }
+
+// 2-D K-major tensor map: inner dimension = d elements, outer = rows; box = 128 bytes x box_rows,
+// 128-byte swizzle, out-of-range elements read as zero.
+int make_tensor_map(egtp_ctx* c, CUtensorMap* map, const void* base, int dtype, int64_t rows, int d, int64_t ld,
+                    int box_rows) {
+  const int eb = elem_bytes(dtype);
+  cuuint64_t gdim[2] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(rows)};
+  cuuint64_t gstride[1] = {static_cast<cuuint64_t>(ld) * eb};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(kRowBytes / eb), static_cast<cuuint32_t>(box_rows)};
+  cuuint32_t estr[2] = {1, 1};
+  const CUtensorMapDataType dt = dtype == EGTP_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+  CUresult r = c->encode(map, dt, 2, const_cast<void*>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? EGTP_OK : EGTP_ERR_CUDA;
+}
+
+int check_lm(const egtp_ctx* c, const egtp_lm_head* lm, const void* hidden, int64_t ldh) {
+  if (!lm || !lm->W || !hidden) return EGTP_ERR_INVALID_ARG;
+  if (lm->d <= 0 || lm->V <= 0 || lm->ldw < lm->d || ldh < lm->d) return EGTP_ERR_INVALID_ARG;
+  if (lm->dtype != EGTP_F32 && lm->dtype != EGTP_BF16) return EGTP_ERR_UNSUPPORTED;
+  const int eb = elem_bytes(lm->dtype);
+  if (lm->d % 16 != 0) return EGTP_ERR_UNSUPPORTED;
+  if ((lm->ldw * eb) % 16 != 0 || (ldh * eb) % 16 != 0) return EGTP_ERR_UNSUPPORTED;
+  if (reinterpret_cast<uintptr_t>(lm->W) % 16 != 0 || reinterpret_cast<uintptr_t>(hidden) % 16 != 0)
+    return EGTP_ERR_UNSUPPORTED;
+  if (lm->d > c->max_d || lm->V > c->max_V) return EGTP_ERR_CAPACITY;
+  return EGTP_OK;
+}
+
+int check_head(const egtp_ctx* c, const egtp_head* h, int d) {
+  (void)c;
+  if (!h->W1 || !h->b1 || !h->W2 || !h->b2) return EGTP_ERR_INVALID_ARG;
+  if (h->d != d || h->m_h <= 0 || h->d_out <= 0) return EGTP_ERR_INVALID_ARG;
+  if (h->wdtype != EGTP_F32 && h->wdtype != EGTP_BF16) return EGTP_ERR_UNSUPPORTED;
+  if (h->m_h > 8192 || h->d_out > 256) return EGTP_ERR_UNSUPPORTED;
+  if (h->mode == EGTP_HEAD_SCALAR) {
+    if (h->d_out != 1) return EGTP_ERR_INVALID_ARG;
+  } else if (h->mode == EGTP_HEAD_BINS) {
+    if (!h->centres) return EGTP_ERR_INVALID_ARG;
+  } else {
+    return EGTP_ERR_INVALID_ARG;
+  }
+  if (reinterpret_cast<uintptr_t>(h->W1) % 16 != 0) return EGTP_ERR_UNSUPPORTED;
+  return EGTP_OK;
+}
+
+HeadArgs head_args(const egtp_head* h) {
+  HeadArgs a{};
+  a.W1 = h->W1; a.b1 = h->b1; a.W2 = h->W2; a.b2 = h->b2; a.centres = h->centres;
+  a.d = h->d; a.m_h = h->m_h; a.d_out = h->d_out; a.bf16 = h->wdtype == EGTP_BF16; a.mode = h->mode;
+  return a;
+}
+
+#define EGTP_CUDA_TRY(expr)                       \
+  do {                                            \
+    if ((expr) != cudaSuccess) return EGTP_ERR_CUDA; \
+  } while (0)
+
+// Eq. 2 for `rows` rows: LM-head kernel + merge. Writes H (and seg ids / zeroed weights when asked).
+int run_entropy(egtp_ctx* c, const egtp_lm_head* lm, const void* hidden, int64_t ldh, int64_t rows, float* H,
+                const int32_t* offsets, int B, int32_t* seg_id, float* weights_zero, int32_t* status,
+                cudaStream_t stream) {
+  const LmheadPlan plan = make_lmhead_plan(rows, lm->d, lm->V, elem_bytes(lm->dtype), c->num_sms, c->slot_row_capacity);
+  if (plan.rows_pad * plan.slots > c->slot_row_capacity) return EGTP_ERR_CAPACITY;
+  CUtensorMap map_a, map_b;
+  int rc = make_tensor_map(c, &map_a, hidden, lm->dtype, rows, lm->d, ldh, kTileM);
+  if (rc != EGTP_OK) return rc;
+  rc = make_tensor_map(c, &map_b, lm->W, lm->dtype, lm->V, lm->d, lm->ldw, kTileN);
+  if (rc != EGTP_OK) return rc;
+  {
+    LaunchScope ls(c, EGTP_K_LMHEAD_ENTROPY, stream);
+    EGTP_CUDA_TRY(launch_lmhead_entropy(plan, lm->dtype == EGTP_F32, &map_a, &map_b, rows, lm->V, c->partials, status,
+                                        stream));
+  }
+  {
+    LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
+    EGTP_CUDA_TRY(launch_entropy_merge(c->partials, plan.slots, plan.rows_pad, rows, H, offsets, B, seg_id,
+                                       weights_zero, status, stream));
+  }
+  return EGTP_OK;
+}
+
+int run_head(egtp_ctx* c, const egtp_head* head, const float* z, int64_t ldz, int rows, float* y, float* phat,
+             const int32_t* status, cudaStream_t stream) {
+  const HeadArgs ha = head_args(head);
+  const int splits = head_pick_splits(rows, ha.d, ha.m_h, c->num_sms, c->head_partial_floats);
+  if (splits <= 0) return EGTP_ERR_CAPACITY;
+  {
+    LaunchScope ls(c, EGTP_K_HEAD_HIDDEN, stream);
+    EGTP_CUDA_TRY(launch_head_hidden(ha, z, ldz, rows, splits, c->head_partial, status, stream));
+  }
+  {
+    LaunchScope ls(c, EGTP_K_HEAD_OUT, stream);
+    EGTP_CUDA_TRY(launch_head_out(ha, c->head_partial, rows, splits, y, phat, status, stream));
+  }
+  return EGTP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* egtp_status_string(int status) {
+  switch (status) {
+    case EGTP_OK: return "ok";
+    case EGTP_ERR_INVALID_ARG: return "invalid argument";
+    case EGTP_ERR_UNSUPPORTED: return "unsupported dtype, alignment or layout";
+    case EGTP_ERR_CAPACITY: return "exceeds the capacity the context or state was created with";
+    case EGTP_ERR_CUDA: return "CUDA call failed";
+    case EGTP_ERR_BAD_OFFSETS: return "offsets are not non-decreasing within [0, T_total]";
+    case EGTP_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case EGTP_ERR_BAD_SLOT: return "slot id or reset source out of range";
+    default: return "unknown status";
+  }
+}
+
+const char* egtp_kernel_name(int kernel_id) {
+  if (kernel_id < 0 || kernel_id >= EGTP_NUM_KERNELS) return "unknown";
+  return kKernelNames[kernel_id];
+}
+
+int egtp_create(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_batch, int32_t max_d, int32_t max_V) {
+  if (!out || max_tokens <= 0 || max_batch <= 0 || max_d <= 0 || max_V <= 0) return EGTP_ERR_INVALID_ARG;
+  if (max_tokens >= (1ll << 31)) return EGTP_ERR_UNSUPPORTED;   // offsets are int32 token indices
+  if (cudaSetDevice(device) != cudaSuccess) return EGTP_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return EGTP_ERR_CUDA;
+  if (prop.major != 10) return EGTP_ERR_UNSUPPORTED;
+  egtp_ctx* c = new (std::nothrow) egtp_ctx();
+  if (!c) return EGTP_ERR_CUDA;
+  c->device = device;
+  c->num_sms = prop.multiProcessorCount;
+  c->max_tokens = max_tokens; c->max_batch = max_batch; c->max_d = max_d; c->max_V = max_V;
+
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+    delete c;
+    return EGTP_ERR_CUDA;
+  }
+  c->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+  if (lmhead_prepare_device() != cudaSuccess) { delete c; return EGTP_ERR_CUDA; }
+
+  const int64_t rows_cap = std::max<int64_t>(max_tokens, max_batch);
+  const int64_t rows_pad = (rows_cap + kTileM - 1) / kTileM * kTileM;
+  const int64_t n_tiles = (static_cast<int64_t>(max_V) + kTileN - 1) / kTileN;
+  // room for 24 vocabulary chunks at the largest token count, and for one chunk per vocabulary
+  // tile on decode-sized batches (up to 1024 rows)
+  c->slot_row_capacity = std::max<int64_t>(rows_pad * 24 * kEpiSplit, std::min<int64_t>(rows_pad, 1024) * n_tiles * kEpiSplit);
+  const int64_t pool_chunks = (max_tokens + kPoolChunkTokens - 1) / kPoolChunkTokens + 1;
+  c->head_partial_floats = std::max<int64_t>(8ll << 20, static_cast<int64_t>(max_batch) * 8192);
+
+  bool ok = true;
+  ok = ok && dev_alloc(c, &c->partials, c->slot_row_capacity * 3) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->H, rows_cap) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->weights, max_tokens) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->seg_m, max_batch) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->seg_s, max_batch) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->pooled, static_cast<int64_t>(max_batch) * max_d) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->piece_a, pool_chunks * max_d) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->piece_b, pool_chunks * max_d) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->head_partial, c->head_partial_floats) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->yhat, max_batch) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->status, 1) == cudaSuccess;
+  ok = ok && dev_alloc(c, reinterpret_cast<float**>(&c->hidden_stage), rows_cap * max_d) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->offsets_stage, static_cast<int64_t>(max_batch) + 1) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->reset_stage, max_batch) == cudaSuccess;
+  ok = ok && cudaMemset(c->status, 0, sizeof(int32_t)) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    free_ctx_memory(c);
+    delete c;
+    return EGTP_ERR_CUDA;
+  }
+  *out = c;
+  return EGTP_OK;
+}
+
+int egtp_destroy(egtp_ctx* c) {
+  if (!c) return EGTP_ERR_INVALID_ARG;
+  cudaSetDevice(c->device);
+  free_ctx_memory(c);
+  delete c;
+  return EGTP_OK;
+}
+
+int64_t egtp_workspace_bytes(const egtp_ctx* c) { return c ? c->bytes : 0; }
+int64_t egtp_launch_count(const egtp_ctx* c) { return c ? c->launches : 0; }
+
+int egtp_lmhead_plan(const egtp_ctx* c, int64_t T, int32_t d, int32_t V, int32_t dtype, int32_t info[8]) {
+  if (!c || !info || T <= 0 || d <= 0 || V <= 0) return EGTP_ERR_INVALID_ARG;
+  const LmheadPlan p = make_lmhead_plan(T, d, V, elem_bytes(dtype), c->num_sms, c->slot_row_capacity);
+  info[0] = p.grid; info[1] = p.m_tiles; info[2] = p.n_tiles; info[3] = p.chunks;
+  info[4] = p.slots; info[5] = p.group_m; info[6] = p.k_blocks; info[7] = p.smem_bytes;
+  return EGTP_OK;
+}
+
+int egtp_profile_enable(egtp_ctx* c, int on) {
+  if (!c) return EGTP_ERR_INVALID_ARG;
+  c->profiling = on != 0;
+  return EGTP_OK;
+}
+
+int egtp_profile_read(egtp_ctx* c, double* ms_by_kernel, int64_t* launches_by_kernel) {
+  if (!c) return EGTP_ERR_INVALID_ARG;
+  if (cudaSetDevice(c->device) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return EGTP_ERR_CUDA;
+  for (auto& e : c->pending) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, e.start, e.stop) == cudaSuccess) {
+      c->ms_acc[e.kernel] += ms;
+      c->n_acc[e.kernel] += 1;
+    }
+    c->free_events.push_back(e);
+  }
+  c->pending.clear();
+  for (int k = 0; k < EGTP_NUM_KERNELS; ++k) {
+    if (ms_by_kernel) ms_by_kernel[k] = c->ms_acc[k];
+    if (launches_by_kernel) launches_by_kernel[k] = c->n_acc[k];
+    c->ms_acc[k] = 0.0;
+    c->n_acc[k] = 0;
+  }
+  return EGTP_OK;
+}
+
+int egtp_predict(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, const void* hidden, int64_t ldh,
+                 const int32_t* offsets, int32_t B, int64_t T_total, float alpha, float* H_out, float* weights_out,
+                 int32_t* seg_id_out, float* pooled_out, float* state_m_out, float* state_s_out, float* yhat_out,
+                 float* phat_out, int32_t* status_dev, void* stream_v) {
+  if (!c) return EGTP_ERR_INVALID_ARG;
+  if (B < 0 || T_total < 0 || !(alpha > 0.f) || !std::isfinite(alpha)) return EGTP_ERR_INVALID_ARG;
+  if (B == 0 || T_total == 0) {
+    if (B > 0 && T_total == 0 && !offsets) return EGTP_ERR_INVALID_ARG;
+    if (T_total == 0 && B == 0) return EGTP_OK;
+  }
+  if (!offsets && B > 0) return EGTP_ERR_INVALID_ARG;
+  if (!head && (yhat_out || phat_out)) return EGTP_ERR_INVALID_ARG;
+  if (T_total > c->max_tokens || B > c->max_batch) return EGTP_ERR_CAPACITY;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  int32_t* status = status_dev ? status_dev : c->status;
+  if (T_total > 0) {
+    int rc = check_lm(c, lm, hidden, ldh);
+    if (rc != EGTP_OK) return rc;
+  } else if (!lm || lm->d <= 0 || lm->d > c->max_d) {
+    return EGTP_ERR_INVALID_ARG;
+  }
+  if (head) {
+    int rc = check_head(c, head, lm->d);
+    if (rc != EGTP_OK) return rc;
+  }
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
+
+  const int d = lm->d;
+  float* H = H_out ? H_out : c->H;
+  float* weights = weights_out ? weights_out : c->weights;
+  float* pooled = pooled_out ? pooled_out : c->pooled;
+  float* seg_m = state_m_out ? state_m_out : c->seg_m;
+  float* seg_s = state_s_out ? state_s_out : c->seg_s;
+
+  if (B > 0) {
+    LaunchScope ls(c, EGTP_K_VALIDATE, stream);
+    EGTP_CUDA_TRY(launch_validate_offsets(offsets, B, T_total, status, stream));
+  }
+  if (T_total > 0) {
+    int rc = run_entropy(c, lm, hidden, ldh, T_total, H, offsets, B, seg_id_out, weights, status, stream);
+    if (rc != EGTP_OK) return rc;
+  }
+  if (B == 0) return EGTP_OK;
+  {
+    LaunchScope ls(c, EGTP_K_SEGMENT_WEIGHTS, stream);
+    EGTP_CUDA_TRY(launch_segment_weights(H, offsets, B, 1.f / alpha, weights, seg_m, seg_s, status, stream));
+  }
+  if (T_total > 0) {
+    LaunchScope ls(c, EGTP_K_POOL, stream);
+    EGTP_CUDA_TRY(launch_pool(hidden, ldh, lm->dtype == EGTP_BF16, weights, offsets, B, T_total, d, pooled,
+                              c->piece_a, c->piece_b, status, stream));
+  }
+  {
+    LaunchScope ls(c, EGTP_K_POOL_COMBINE, stream);
+    EGTP_CUDA_TRY(launch_pool_combine(offsets, B, d, c->piece_a, c->piece_b, pooled, status, stream));
+  }
+  if (head && (yhat_out || phat_out)) {
+    int rc = run_head(c, head, pooled, d, B, yhat_out, phat_out, status, stream);
+    if (rc != EGTP_OK) return rc;
+  }
+  return EGTP_OK;
+}
+
+int egtp_predict_host(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, const void* hidden_host,
+                      const int32_t* offsets_host, int32_t B, int64_t T_total, float alpha, float* yhat_host,
+                      float* pooled_host, int32_t* status_host, void* stream_v) {
+  if (!c || !lm || !head || !hidden_host || !offsets_host || !yhat_host || !status_host) return EGTP_ERR_INVALID_ARG;
+  if (B <= 0 || T_total <= 0) return EGTP_ERR_INVALID_ARG;
+  if (T_total > c->max_tokens || B > c->max_batch || lm->d > c->max_d) return EGTP_ERR_CAPACITY;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  const size_t hbytes = static_cast<size_t>(T_total) * lm->d * elem_bytes(lm->dtype);
+  EGTP_CUDA_TRY(cudaMemcpyAsync(c->hidden_stage, hidden_host, hbytes, cudaMemcpyHostToDevice, stream));
+  EGTP_CUDA_TRY(cudaMemcpyAsync(c->offsets_stage, offsets_host, sizeof(int32_t) * (static_cast<size_t>(B) + 1),
+                                cudaMemcpyHostToDevice, stream));
+  int rc = egtp_predict(c, lm, head, c->hidden_stage, lm->d, c->offsets_stage, B, T_total, alpha, nullptr, nullptr,
+                        nullptr, nullptr, nullptr, nullptr, c->yhat, nullptr, nullptr, stream);
+  if (rc != EGTP_OK) return rc;
+  EGTP_CUDA_TRY(cudaMemcpyAsync(yhat_host, c->yhat, sizeof(float) * B, cudaMemcpyDeviceToHost, stream));
+  if (pooled_host)
+    EGTP_CUDA_TRY(cudaMemcpyAsync(pooled_host, c->pooled, sizeof(float) * static_cast<size_t>(B) * lm->d,
+                                  cudaMemcpyDeviceToHost, stream));
+  EGTP_CUDA_TRY(cudaMemcpyAsync(status_host, c->status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+  EGTP_CUDA_TRY(cudaStreamSynchronize(stream));
+  return EGTP_OK;
+}
+
+int plp_state_create(egtp_ctx* c, plp_state** out, int32_t num_slots, int32_t d) {
+  if (!c || !out || num_slots <= 0 || d <= 0) return EGTP_ERR_INVALID_ARG;
+  if (d % 16 != 0) return EGTP_ERR_UNSUPPORTED;
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  plp_state* st = new (std::nothrow) plp_state();
+  if (!st) return EGTP_ERR_CUDA;
+  st->ctx = c; st->num_slots = num_slots; st->d = d;
+  bool ok = cudaMalloc(reinterpret_cast<void**>(&st->m), sizeof(float) * num_slots) == cudaSuccess;
+  ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->s), sizeof(float) * num_slots) == cudaSuccess;
+  ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->acc), sizeof(float) * static_cast<size_t>(num_slots) * d) == cudaSuccess;
+  if (ok) {
+    std::vector<float> neg(num_slots, -INFINITY);
+    ok = cudaMemcpy(st->m, neg.data(), sizeof(float) * num_slots, cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemset(st->s, 0, sizeof(float) * num_slots) == cudaSuccess;
+    ok = ok && cudaMemset(st->acc, 0, sizeof(float) * static_cast<size_t>(num_slots) * d) == cudaSuccess;
+  }
+  if (!ok) {
+    cudaGetLastError();
+    cudaFree(st->m); cudaFree(st->s); cudaFree(st->acc);
+    delete st;
+    return EGTP_ERR_CUDA;
+  }
+  *out = st;
+  return EGTP_OK;
+}
+
+int plp_state_destroy(plp_state* st) {
+  if (!st) return EGTP_ERR_INVALID_ARG;
+  cudaSetDevice(st->ctx->device);
+  cudaFree(st->m); cudaFree(st->s); cudaFree(st->acc);
+  delete st;
+  return EGTP_OK;
+}
+
+int plp_state_export(plp_state* st, float* m, float* s, float* acc, void* stream_v) {
+  if (!st || !m || !s || !acc) return EGTP_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (cudaSetDevice(st->ctx->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  EGTP_CUDA_TRY(cudaMemcpyAsync(m, st->m, sizeof(float) * st->num_slots, cudaMemcpyDeviceToDevice, stream));
+  EGTP_CUDA_TRY(cudaMemcpyAsync(s, st->s, sizeof(float) * st->num_slots, cudaMemcpyDeviceToDevice, stream));
+  EGTP_CUDA_TRY(cudaMemcpyAsync(acc, st->acc, sizeof(float) * static_cast<size_t>(st->num_slots) * st->d,
+                                cudaMemcpyDeviceToDevice, stream));
+  return EGTP_OK;
+}
+
+int plp_state_import(plp_state* st, const float* m, const float* s, const float* acc, void* stream_v) {
+  if (!st || !m || !s || !acc) return EGTP_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (cudaSetDevice(st->ctx->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  EGTP_CUDA_TRY(cudaMemcpyAsync(st->m, m, sizeof(float) * st->num_slots, cudaMemcpyDeviceToDevice, stream));
+  EGTP_CUDA_TRY(cudaMemcpyAsync(st->s, s, sizeof(float) * st->num_slots, cudaMemcpyDeviceToDevice, stream));
+  EGTP_CUDA_TRY(cudaMemcpyAsync(st->acc, acc, sizeof(float) * static_cast<size_t>(st->num_slots) * st->d,
+                                cudaMemcpyDeviceToDevice, stream));
+  return EGTP_OK;
+}
+
+int plp_step(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head* head, const void* hidden_step,
+             int64_t ldh, const int32_t* slot_ids, const int32_t* reset_src, const float* src_m, const float* src_s,
+             const float* src_pooled, int32_t n_src, int32_t B_live, float alpha, float* Hstep_out, float* z_out,
+             float* yrem_out, int32_t* status_dev, void* stream_v) {
+  if (!c || !st || st->ctx != c) return EGTP_ERR_INVALID_ARG;
+  if (B_live < 0 || n_src < 0 || !(alpha > 0.f) || !std::isfinite(alpha)) return EGTP_ERR_INVALID_ARG;
+  if (B_live == 0) return EGTP_OK;
+  if (n_src > 0 && (!src_m || !src_s || !src_pooled)) return EGTP_ERR_INVALID_ARG;
+  if (!head && yrem_out) return EGTP_ERR_INVALID_ARG;
+  if (B_live > c->max_batch || B_live > st->num_slots) return EGTP_ERR_CAPACITY;
+  int rc = check_lm(c, lm, hidden_step, ldh);
+  if (rc != EGTP_OK) return rc;
+  if (lm->d != st->d) return EGTP_ERR_INVALID_ARG;
+  if (head) {
+    rc = check_head(c, head, lm->d);
+    if (rc != EGTP_OK) return rc;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  int32_t* status = status_dev ? status_dev : c->status;
+  if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
+  float* H = Hstep_out ? Hstep_out : c->H;
+  float* z = z_out ? z_out : c->pooled;
+  rc = run_entropy(c, lm, hidden_step, ldh, B_live, H, nullptr, 0, nullptr, nullptr, status, stream);
+  if (rc != EGTP_OK) return rc;
+  {
+    LaunchScope ls(c, EGTP_K_PLP_UPDATE, stream);
+    EGTP_CUDA_TRY(launch_plp_update(hidden_step, ldh, lm->dtype == EGTP_BF16, H, slot_ids, reset_src, src_m, src_s,
+                                    src_pooled, n_src, B_live, lm->d, st->num_slots, 1.f / alpha, st->m, st->s,
+                                    st->acc, z, lm->d, status, stream));
+  }
+  if (head && yrem_out) {
+    rc = run_head(c, head, z, lm->d, B_live, yrem_out, nullptr, status, stream);
+    if (rc != EGTP_OK) return rc;
+  }
+  return EGTP_OK;
+}
+
+int plp_step_host(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head* head,
+                  const void* hidden_step_host, const int32_t* reset_src_host, const float* src_m, const float* src_s,
+                  const float* src_pooled, int32_t n_src, int32_t B_live, float alpha, float* yrem_host,
+                  int32_t* status_host, void* stream_v) {
+  if (!c || !st || !lm || !head || !hidden_step_host || !yrem_host || !status_host) return EGTP_ERR_INVALID_ARG;
+  if (B_live <= 0) return EGTP_ERR_INVALID_ARG;
+  if (B_live > c->max_batch || lm->d > c->max_d) return EGTP_ERR_CAPACITY;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  const size_t hbytes = static_cast<size_t>(B_live) * lm->d * elem_bytes(lm->dtype);
+  EGTP_CUDA_TRY(cudaMemcpyAsync(c->hidden_stage, hidden_step_host, hbytes, cudaMemcpyHostToDevice, stream));
+  if (reset_src_host)
+    EGTP_CUDA_TRY(cudaMemcpyAsync(c->reset_stage, reset_src_host, sizeof(int32_t) * B_live, cudaMemcpyHostToDevice,
+                                  stream));
+  int rc = plp_step(c, st, lm, head, c->hidden_stage, lm->d, nullptr, reset_src_host ? c->reset_stage : nullptr,
+                    src_m, src_s, src_pooled, n_src, B_live, alpha, nullptr, nullptr, c->yhat, nullptr, stream);
+  if (rc != EGTP_OK) return rc;
+  EGTP_CUDA_TRY(cudaMemcpyAsync(yrem_host, c->yhat, sizeof(float) * B_live, cudaMemcpyDeviceToHost, stream));
+  EGTP_CUDA_TRY(cudaMemcpyAsync(status_host, c->status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+  EGTP_CUDA_TRY(cudaStreamSynchronize(stream));
+  return EGTP_OK;
+}
+
+}  // extern "C"

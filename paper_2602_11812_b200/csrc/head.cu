@@ -1,0 +1,181 @@
+// Prediction head (paper Sec. 3.2, Eq. 6): u = ReLU(W1 z + b1), o = W2 u + b2, then either the
+// scalar o[0] or the expectation of softmax(o) over the bin centres.  A few MB of weights and
+// at most a few thousand rows: plain fp32 FMA on the CUDA cores, register-tiled, split along d
+// so that small batches still fill the GPU; the split partials are added in a fixed order.
+#include "kernels.h"
+#include "../../include/egtp.h"
+
+#include <cuda_bf16.h>
+
+#include <algorithm>
+
+namespace egtp {
+
+namespace {
+
+constexpr int kHT = 64;        // rows and hidden units per block tile
+constexpr int kHK = 16;        // k extent per shared-memory stage
+constexpr int kHThreads = 256; // 16 x 16 threads, 4 x 4 outputs each
+
+template <typename TW>
+__device__ __forceinline__ float4 load4(const TW* p);
+template <>
+__device__ __forceinline__ float4 load4<float>(const float* p) {
+  return __ldg(reinterpret_cast<const float4*>(p));
+}
+template <>
+__device__ __forceinline__ float4 load4<__nv_bfloat16>(const __nv_bfloat16* p) {
+  const uint2 q = __ldg(reinterpret_cast<const uint2*>(p));
+  return make_float4(__uint_as_float(q.x << 16), __uint_as_float(q.x & 0xFFFF0000u),
+                     __uint_as_float(q.y << 16), __uint_as_float(q.y & 0xFFFF0000u));
+}
+
+// partial[split][row][j] = sum_{k in split} z[row][k] * W1[j][k]
+template <typename TW>
+__global__ void __launch_bounds__(kHThreads)
+head_hidden_kernel(const float* __restrict__ z, int64_t ldz, const TW* __restrict__ W1, int rows, int d, int m_h,
+                   int k_per_split, float* __restrict__ partial, const int32_t* __restrict__ status) {
+  if (*status != 0) return;
+  __shared__ float zs[kHK][kHT + 4];
+  __shared__ float ws[kHK][kHT + 4];
+  const int j0 = blockIdx.x * kHT, r0 = blockIdx.y * kHT, split = blockIdx.z;
+  const int k_begin = split * k_per_split;
+  const int k_end = min(d, k_begin + k_per_split);
+  const int tid = threadIdx.x;
+  const int lrow = tid >> 2, lk = (tid & 3) * 4;   // loader: 64 rows x 4 quads of k
+  const int tx = tid & 15, ty = tid >> 4;          // compute: outputs rows ty*4.., units tx*4..
+  float acc[4][4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+
+  for (int k0 = k_begin; k0 < k_end; k0 += kHK) {
+    float4 zv = make_float4(0.f, 0.f, 0.f, 0.f), wv = zv;
+    if (r0 + lrow < rows) zv = __ldg(reinterpret_cast<const float4*>(z + static_cast<int64_t>(r0 + lrow) * ldz + k0 + lk));
+    if (j0 + lrow < m_h) wv = load4<TW>(W1 + static_cast<int64_t>(j0 + lrow) * d + k0 + lk);
+    __syncthreads();
+    zs[lk + 0][lrow] = zv.x; zs[lk + 1][lrow] = zv.y; zs[lk + 2][lrow] = zv.z; zs[lk + 3][lrow] = zv.w;
+    ws[lk + 0][lrow] = wv.x; ws[lk + 1][lrow] = wv.y; ws[lk + 2][lrow] = wv.z; ws[lk + 3][lrow] = wv.w;
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < kHK; ++k) {
+      const float4 a = *reinterpret_cast<const float4*>(&zs[k][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&ws[k][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w};
+      const float bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+  }
+  float* out = partial + static_cast<int64_t>(split) * rows * m_h;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = r0 + ty * 4 + i;
+    if (r >= rows) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int jj = j0 + tx * 4 + j;
+      if (jj < m_h) out[static_cast<int64_t>(r) * m_h + jj] = acc[i][j];
+    }
+  }
+}
+
+template <typename TW>
+__device__ __forceinline__ float to_f32(TW v);
+template <>
+__device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// One block per row: u = ReLU(sum of split partials + b1) into shared memory, o_c = W2[c] . u + b2[c]
+// (one warp per output, lanes stride the hidden units), then the output mode.
+template <typename TW>
+__global__ void __launch_bounds__(128)
+head_out_kernel(const float* __restrict__ partial, int rows, int splits, int m_h, int d_out,
+                const float* __restrict__ b1, const TW* __restrict__ W2, const float* __restrict__ b2,
+                const float* __restrict__ centres, int mode, float* __restrict__ y, float* __restrict__ phat,
+                const int32_t* __restrict__ status) {
+  if (*status != 0) return;
+  extern __shared__ float smem[];
+  float* u = smem;            // [m_h]
+  float* o = smem + m_h;      // [d_out]
+  const int r = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  for (int j = tid; j < m_h; j += blockDim.x) {
+    float v = 0.f;
+    for (int s = 0; s < splits; ++s) v += partial[(static_cast<int64_t>(s) * rows + r) * m_h + j];
+    u[j] = fmaxf(0.f, v + b1[j]);
+  }
+  __syncthreads();
+  for (int c = wid; c < d_out; c += (blockDim.x >> 5)) {
+    float v = 0.f;
+    for (int j = lane; j < m_h; j += 32) v = fmaf(to_f32<TW>(W2[static_cast<int64_t>(c) * m_h + j]), u[j], v);
+#pragma unroll
+    for (int of = 16; of > 0; of >>= 1) v += __shfl_xor_sync(0xffffffffu, v, of);
+    if (lane == 0) o[c] = v + b2[c];
+  }
+  __syncthreads();
+  if (tid == 0) {
+    if (mode == EGTP_HEAD_SCALAR) {
+      if (y) y[r] = o[0];
+    } else {
+      float mx = o[0];
+      for (int c = 1; c < d_out; ++c) mx = fmaxf(mx, o[c]);
+      float den = 0.f;
+      for (int c = 0; c < d_out; ++c) den += expf(o[c] - mx);
+      float ev = 0.f;
+      for (int c = 0; c < d_out; ++c) {
+        const float pc = expf(o[c] - mx) / den;
+        ev = fmaf(pc, centres[c], ev);
+        if (phat) phat[static_cast<int64_t>(r) * d_out + c] = pc;
+      }
+      if (y) y[r] = ev;
+    }
+  }
+}
+
+}  // namespace
+
+int head_pick_splits(int rows, int d, int m_h, int num_sms, int64_t partial_capacity_floats) {
+  const int64_t tiles = static_cast<int64_t>((rows + kHT - 1) / kHT) * ((m_h + kHT - 1) / kHT);
+  int splits = static_cast<int>(std::max<int64_t>(1, (2ll * num_sms + tiles - 1) / tiles));
+  splits = std::min(splits, std::max(1, d / 256));
+  const int64_t per_split = static_cast<int64_t>(rows) * m_h;
+  while (splits > 1 && per_split * splits > partial_capacity_floats) --splits;
+  if (per_split * splits > partial_capacity_floats) return 0;
+  return splits;
+}
+
+cudaError_t launch_head_hidden(const HeadArgs& h, const float* z, int64_t ldz, int rows, int splits,
+                               float* partial, const int32_t* status, cudaStream_t stream) {
+  int k_per_split = (h.d + splits - 1) / splits;
+  k_per_split = (k_per_split + kHK - 1) / kHK * kHK;
+  dim3 grid((h.m_h + kHT - 1) / kHT, (rows + kHT - 1) / kHT, splits);
+  if (h.bf16) {
+    head_hidden_kernel<__nv_bfloat16><<<grid, kHThreads, 0, stream>>>(
+        z, ldz, static_cast<const __nv_bfloat16*>(h.W1), rows, h.d, h.m_h, k_per_split, partial, status);
+  } else {
+    head_hidden_kernel<float><<<grid, kHThreads, 0, stream>>>(z, ldz, static_cast<const float*>(h.W1), rows, h.d,
+                                                              h.m_h, k_per_split, partial, status);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_head_out(const HeadArgs& h, const float* partial, int rows, int splits, float* y, float* phat,
+                            const int32_t* status, cudaStream_t stream) {
+  const size_t smem = static_cast<size_t>(h.m_h + h.d_out) * sizeof(float);
+  if (h.bf16) {
+    head_out_kernel<__nv_bfloat16><<<rows, 128, smem, stream>>>(partial, rows, splits, h.m_h, h.d_out, h.b1,
+                                                               static_cast<const __nv_bfloat16*>(h.W2), h.b2,
+                                                               h.centres, h.mode, y, phat, status);
+  } else {
+    head_out_kernel<float><<<rows, 128, smem, stream>>>(partial, rows, splits, h.m_h, h.d_out, h.b1,
+                                                       static_cast<const float*>(h.W2), h.b2, h.centres, h.mode, y,
+                                                       phat, status);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace egtp

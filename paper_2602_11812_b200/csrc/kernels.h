@@ -1,0 +1,92 @@
+// Internal launcher interface between the C ABI (api.cu) and the kernels. Not installed.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace egtp {
+
+// Finite stand-in for "no logit seen yet" / "masked column": keeps every product finite.
+constexpr float kNegBig = -1.0e30f;
+
+// ---- K1: LM-head GEMM with online entropy epilogue ---------------------------------------
+constexpr int kTileM = 128;        // token rows per tile (UMMA M, one TMEM lane per row)
+constexpr int kTileN = 256;        // vocabulary columns per tile (UMMA N, one TMEM column each)
+constexpr int kRowBytes = 128;     // K extent of one pipeline stage in bytes (one swizzle row)
+constexpr int kStages = 4;         // TMA -> MMA pipeline depth
+constexpr int kEpiSplit = 2;       // epilogue warps per TMEM lane quadrant (column halves)
+constexpr int kLmheadThreads = (2 + 4 * kEpiSplit) * 32;
+
+struct LmheadPlan {
+  int grid;          // persistent CTAs
+  int m_tiles;       // ceil(T / 128)
+  int n_tiles;       // ceil(V / 256)
+  int chunks;        // vocabulary chunks S; a work unit is (row tile, chunk)
+  int slots;         // partial slots per row = S * kEpiSplit
+  int group_m;       // row tiles that sweep the vocabulary together (L2 reuse of W tiles)
+  int k_blocks;      // ceil(d * elem / 128)
+  int smem_bytes;    // dynamic shared memory
+  int64_t rows_pad;  // m_tiles * 128: row pitch of the partial buffer
+};
+
+// Picks chunks / grouping for T rows; slot_limit bounds chunks * kEpiSplit * rows_pad by the
+// partial buffer's capacity (in rows x slots).
+LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity);
+
+// Opts the kernels into their dynamic shared-memory size on the current device (once per device).
+cudaError_t lmhead_prepare_device();
+
+// partials layout: [slot][3][rows_pad] floats: (m, s, t2) with m the running max logit,
+// s = sum 2^((x-m) log2 e), t2 = sum 2^(...) * (x-m) log2 e over the slot's vocabulary range.
+cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const CUtensorMap* map_hidden,
+                                  const CUtensorMap* map_w, int64_t T, int V, float* partials,
+                                  int32_t* status, cudaStream_t stream);
+
+// ---- K2: entropy merge, Eq. 3 weights, Eq. 4 pooling -------------------------------------
+constexpr int kPoolChunkTokens = 64;   // tokens per first-stage pooling chunk
+constexpr int kPoolThreads = 128;      // each thread owns 8 consecutive channels
+
+cudaError_t launch_validate_offsets(const int32_t* offsets, int B, int64_t T, int32_t* status, cudaStream_t stream);
+
+cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t rows_pad, int64_t T, float* H,
+                                 const int32_t* offsets, int B, int32_t* seg_id_out, float* weights_zero,
+                                 const int32_t* status, cudaStream_t stream);
+
+cudaError_t launch_segment_weights(const float* H, const int32_t* offsets, int B, float inv_alpha, float* weights,
+                                   float* seg_m, float* seg_s, const int32_t* status, cudaStream_t stream);
+
+cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, const float* weights, const int32_t* offsets,
+                        int B, int64_t T, int d, float* pooled, float* piece_a, float* piece_b,
+                        const int32_t* status, cudaStream_t stream);
+
+cudaError_t launch_pool_combine(const int32_t* offsets, int B, int d, const float* piece_a, const float* piece_b,
+                                float* pooled, const int32_t* status, cudaStream_t stream);
+
+// ---- K3: head ------------------------------------------------------------------------------
+struct HeadArgs {
+  const void* W1;
+  const float* b1;
+  const void* W2;
+  const float* b2;
+  const float* centres;
+  int d, m_h, d_out;
+  bool bf16;
+  int mode;
+};
+int head_pick_splits(int rows, int d, int m_h, int num_sms, int64_t partial_capacity_floats);
+
+cudaError_t launch_head_hidden(const HeadArgs& h, const float* z, int64_t ldz, int rows, int splits,
+                               float* partial, const int32_t* status, cudaStream_t stream);
+
+cudaError_t launch_head_out(const HeadArgs& h, const float* partial, int rows, int splits, float* y, float* phat,
+                            const int32_t* status, cudaStream_t stream);
+
+// ---- K4: PLP running-state update ---------------------------------------------------------
+cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, const float* Hstep,
+                              const int32_t* slot_ids, const int32_t* reset_src, const float* src_m,
+                              const float* src_s, const float* src_pooled, int n_src, int rows, int d, int num_slots,
+                              float inv_alpha, float* st_m, float* st_s, float* st_acc, float* z, int64_t ldz,
+                              int32_t* status, cudaStream_t stream);
+
+}  // namespace egtp

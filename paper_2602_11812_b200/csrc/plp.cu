@@ -1,0 +1,121 @@
+// Progressive Length Prediction, running-state update (paper Sec. 3.3, Eq. 8).
+// z_t is the entropy-weighted pool (Eq. 3-4) over a sequence's prompt tokens followed by its
+// generated tokens 1..t.  Per slot the library keeps the online-softmax triple
+//   m = max_i H_i/alpha,  s = sum_i exp(H_i/alpha - m),  acc = sum_i exp(H_i/alpha - m) h_i,
+// which one new token (entropy H', hidden h') updates to
+//   m' = max(m, H'/alpha), s' = s e^(m-m') + e^(H'/alpha-m'), acc' = acc e^(m-m') + e^(H'/alpha-m') h',
+// and z = acc'/s'.  HBM-bound (acc read + write, hidden read, z write): one block per live row.
+#include "kernels.h"
+#include "../../include/egtp.h"
+
+#include <cuda_bf16.h>
+
+namespace egtp {
+
+namespace {
+
+template <typename T>
+__device__ __forceinline__ void load8(const T* p, float (&v)[8]);
+template <>
+__device__ __forceinline__ void load8<__nv_bfloat16>(const __nv_bfloat16* p, float (&v)[8]) {
+  const uint4 q = __ldg(reinterpret_cast<const uint4*>(p));
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+template <>
+__device__ __forceinline__ void load8<float>(const float* p, float (&v)[8]) {
+  const float4 a = __ldg(reinterpret_cast<const float4*>(p));
+  const float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+  v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* __restrict__ Hstep,
+                  const int32_t* __restrict__ slot_ids, const int32_t* __restrict__ reset_src,
+                  const float* __restrict__ src_m, const float* __restrict__ src_s,
+                  const float* __restrict__ src_pooled, int n_src, int d, int num_slots, float inv_alpha,
+                  float* __restrict__ st_m, float* __restrict__ st_s, float* __restrict__ st_acc,
+                  float* __restrict__ z, int64_t ldz, int32_t* status) {
+  if (*status != 0) return;
+  const int i = blockIdx.x;
+  const int slot = slot_ids ? slot_ids[i] : i;
+  const int rs = reset_src ? reset_src[i] : PLP_RESET_KEEP;
+  if (slot < 0 || slot >= num_slots || rs < PLP_RESET_KEEP || rs >= n_src) {
+    if (threadIdx.x == 0) atomicCAS(status, 0, EGTP_ERR_BAD_SLOT);
+    return;
+  }
+  // state before this token
+  float m_old, s_old;
+  const float* acc_src;   // nullptr = zeros
+  float acc_scale_in;     // factor that turns *acc_src into acc (src_pooled rows are normalised pools)
+  if (rs == PLP_RESET_KEEP) {
+    m_old = st_m[slot]; s_old = st_s[slot];
+    acc_src = st_acc + static_cast<int64_t>(slot) * d; acc_scale_in = 1.f;
+  } else if (rs == PLP_RESET_EMPTY) {
+    m_old = -INFINITY; s_old = 0.f; acc_src = nullptr; acc_scale_in = 0.f;
+  } else {
+    m_old = src_m[rs]; s_old = src_s[rs];
+    acc_src = src_pooled + static_cast<int64_t>(rs) * d; acc_scale_in = s_old;
+  }
+  const float a = Hstep[i] * inv_alpha;
+  const float m_new = fmaxf(m_old, a);
+  const float carry = (s_old > 0.f) ? expf(m_old - m_new) : 0.f;
+  const float e = expf(a - m_new);
+  const float s_new = fmaf(s_old, carry, e);
+  const float inv_s = 1.f / s_new;
+  const float acc_factor = carry * acc_scale_in;
+  __syncthreads();   // every thread has read the old state before anyone overwrites it
+  float* acc_dst = st_acc + static_cast<int64_t>(slot) * d;
+  const T* hrow = hidden_step + static_cast<int64_t>(i) * ldh;
+  float* zrow = z + static_cast<int64_t>(i) * ldz;
+  for (int col = threadIdx.x * 8; col < d; col += blockDim.x * 8) {
+    float h[8], acc[8];
+    load8<T>(hrow + col, h);
+    if (acc_src != nullptr && acc_factor != 0.f) {
+      const float4 p0 = *reinterpret_cast<const float4*>(acc_src + col);
+      const float4 p1 = *reinterpret_cast<const float4*>(acc_src + col + 4);
+      acc[0] = p0.x; acc[1] = p0.y; acc[2] = p0.z; acc[3] = p0.w;
+      acc[4] = p1.x; acc[5] = p1.y; acc[6] = p1.z; acc[7] = p1.w;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) acc[k] = fmaf(acc[k], acc_factor, e * h[k]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) acc[k] = e * h[k];
+    }
+    reinterpret_cast<float4*>(acc_dst + col)[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    reinterpret_cast<float4*>(acc_dst + col)[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+    reinterpret_cast<float4*>(zrow + col)[0] = make_float4(acc[0] * inv_s, acc[1] * inv_s, acc[2] * inv_s, acc[3] * inv_s);
+    reinterpret_cast<float4*>(zrow + col)[1] = make_float4(acc[4] * inv_s, acc[5] * inv_s, acc[6] * inv_s, acc[7] * inv_s);
+  }
+  if (threadIdx.x == 0) {
+    st_m[slot] = m_new;
+    st_s[slot] = s_new;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, const float* Hstep,
+                              const int32_t* slot_ids, const int32_t* reset_src, const float* src_m,
+                              const float* src_s, const float* src_pooled, int n_src, int rows, int d, int num_slots,
+                              float inv_alpha, float* st_m, float* st_s, float* st_acc, float* z, int64_t ldz,
+                              int32_t* status, cudaStream_t stream) {
+  if (bf16) {
+    plp_update_kernel<__nv_bfloat16><<<rows, 256, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(hidden_step), ldh, Hstep, slot_ids, reset_src, src_m, src_s, src_pooled,
+        n_src, d, num_slots, inv_alpha, st_m, st_s, st_acc, z, ldz, status);
+  } else {
+    plp_update_kernel<float><<<rows, 256, 0, stream>>>(static_cast<const float*>(hidden_step), ldh, Hstep, slot_ids,
+                                                       reset_src, src_m, src_s, src_pooled, n_src, d, num_slots,
+                                                       inv_alpha, st_m, st_s, st_acc, z, ldz, status);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace egtp

@@ -1,0 +1,178 @@
+"""GPU parity: egtp_predict through the C ABI against the fp64 oracle on the same seeded inputs."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import egtp_oracle as orc
+from paper_2602_11812_b200 import binding as egtp
+from paper_2602_11812_b200 import inputs as gen
+from tests import gpu_util as gu
+from tests.golden_io import load
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = egtp.egtp_create(0, max_tokens=16384, max_batch=256, max_d=2048, max_V=40000)
+    yield c
+    egtp.egtp_destroy(c)
+
+
+def _check_all(res, ref, wl):
+    assert res["status"] == 0
+    assert np.array_equal(res["seg_id"], ref["seg_id"])                 # bit-exact segment indexing
+    gu.assert_entropy_close(res["H"], ref["H"])
+    assert np.all(np.abs(res["weights"] - ref["weights"]) <= 5e-3 * ref["weights"] + 1e-9)
+    gu.assert_pooled_close(res["pooled"], ref["pooled"])
+    gu.assert_length_close(res["yhat"], ref["yhat"])
+    ne = np.diff(wl.offsets) > 0
+    assert np.allclose(res["state_m"][ne], ref["state_m"][ne], rtol=1e-3)
+    assert np.allclose(res["state_s"][ne], ref["state_s"][ne], rtol=5e-3)
+
+
+def test_tiny_config_matches_oracle_and_golden(ctx):
+    wl = gen.config_tiny()
+    ref = orc.egtp_predict(wl.hidden, wl.offsets, wl.W, wl.head, wl.alpha)
+    res = gu.run_egtp(ctx, wl)
+    _check_all(res, ref, wl)
+    gu.assert_entropy_close(res["H"], load("egtp_tiny_H.txt"))
+    gu.assert_pooled_close(res["pooled"], load("egtp_tiny_pooled.txt", (4, 256)))
+    gu.assert_length_close(res["yhat"], load("egtp_tiny_yhat.txt"))
+
+
+def test_tiny_config_bins_head(ctx):
+    wl = gen.config_tiny(gen.HEAD_BINS)
+    ref = orc.egtp_predict(wl.hidden, wl.offsets, wl.W, wl.head, wl.alpha)
+    res = gu.run_egtp(ctx, wl, want_phat=True)
+    _check_all(res, ref, wl)
+    gu.assert_length_close(res["yhat"], load("egtp_tiny_bins_yhat.txt"))
+    assert np.allclose(res["phat"], ref["phat"], atol=2e-4)
+    assert np.allclose(res["phat"].sum(axis=1), 1.0, atol=1e-5)
+
+
+@pytest.mark.parametrize("dtype,V,d", [("bf16", 5000, 512), ("bf16", 256, 64), ("bf16", 1000, 2048),
+                                       ("f32", 777, 96), ("bf16", 33000, 256)])
+def test_uniform_logits_give_ln_V(ctx, dtype, V, d):
+    # W = 0: every entropy is ln V exactly.  V not a multiple of the 256-wide tile catches unmasked padding.
+    rng = np.random.default_rng(0)
+    lengths = [5, 130, 1, 200]
+    hidden = gen._maybe_round(rng.standard_normal((sum(lengths), d)).astype(np.float32), dtype)
+    head = gen.make_head(1, d, 32, 1, dtype)
+    wl = gen.EgtpWorkload("uniform", dtype, hidden, gen.offsets_from_lengths(lengths), np.zeros((V, d), np.float32), head)
+    res = gu.run_egtp(ctx, wl)
+    assert res["status"] == 0
+    assert np.all(np.abs(res["H"] - math.log(V)) <= 1e-4 * math.log(V))
+    # equal entropies: the pool is the plain mean of the prompt's rows
+    off = wl.offsets
+    for b in range(4):
+        mean = hidden[off[b]:off[b + 1]].astype(np.float64).mean(axis=0)
+        assert np.abs(res["pooled"][b] - mean).max() <= 2e-3 * np.abs(mean).max() + 1e-6
+
+
+def test_two_level_closed_form_and_one_hot(ctx):
+    # hidden = e_0, W[v, 0] = a for v < k else 0:  H = ln Z - k a e^a / Z, Z = k e^a + V - k
+    V, d = 4999, 64
+    cases = [(3, 5.0), (100, 7.0), (4000, -2.0), (1, 40.0)]
+    rows, Ws = [], None
+    hidden = np.zeros((len(cases), d), np.float32)
+    expect = []
+    res_all = []
+    for i, (k, a) in enumerate(cases):
+        h = np.zeros((1, d), np.float32)
+        h[0, 0] = 1.0
+        W = np.zeros((V, d), np.float32)
+        W[:k, 0] = a
+        wl = gen.EgtpWorkload("two_level", "bf16", h, np.array([0, 1], np.int32), W, gen.make_head(1, d, 16, 1, "bf16"))
+        res = gu.run_egtp(ctx, wl)
+        Z = k * math.exp(a) + V - k
+        exp_H = math.log(Z) - k * a * math.exp(a) / Z
+        assert res["status"] == 0
+        assert abs(res["H"][0] - exp_H) <= 1e-3 * abs(exp_H) + 1e-5, (k, a, res["H"][0], exp_H)
+        assert np.allclose(res["pooled"][0], h[0], atol=1e-6)          # single token: identity
+
+
+def test_mid_config_scaled(ctx):
+    # the mid configuration's recipe (lognormal lengths, 1 % outlier channels x 20, bf16) at reduced d and V;
+    # 32 ragged prompts spanning many 128-row tiles, V not a multiple of 128
+    wl = gen.config_mid(V=20000 + 72, d=512, m_h=128)
+    ref = orc.egtp_predict(wl.hidden, wl.offsets, wl.W, wl.head, wl.alpha)
+    res = gu.run_egtp(ctx, wl)
+    _check_all(res, ref, wl)
+    assert ref["H"].std() > 0.05                                        # weights are genuinely non-uniform
+
+
+def test_segment_edge_cases(ctx):
+    # leading / trailing tokens outside every prompt, empty prompts, boundaries on and next to a 128-row tile
+    # edge and a 64-token pooling chunk edge, a one-token prompt
+    rng = np.random.default_rng(3)
+    d, V = 128, 3000
+    off = np.array([3, 3, 64, 128, 129, 129, 257, 300, 300, 511, 640], np.int32)
+    T = 650
+    hidden = gen._maybe_round(rng.standard_normal((T, d)).astype(np.float32) * 2, "bf16")
+    W = gen.make_lm_head(11, V, d, "bf16") * np.float32(3.0)
+    W = gen.round_to_bf16(W)
+    head = gen.make_head(12, d, 48, 1, "bf16")
+    wl = gen.EgtpWorkload("edges", "bf16", hidden, off, W, head)
+    ref = orc.egtp_predict(hidden, off, W, head)
+    res = gu.run_egtp(ctx, wl)
+    _check_all(res, ref, wl)
+    for b in (0, 4, 7):                                                 # empty prompts
+        assert np.all(res["pooled"][b] == 0) and res["state_s"][b] == 0 and res["state_m"][b] == -np.inf
+    assert np.all(res["weights"][:3] == 0) and np.all(res["weights"][640:] == 0)
+
+
+def test_alpha_and_determinism(ctx):
+    wl = gen.config_mid(V=4096, d=256, m_h=64, B=8)
+    wl.alpha = 0.5
+    ref = orc.egtp_predict(wl.hidden, wl.offsets, wl.W, wl.head, wl.alpha)
+    r1 = gu.run_egtp(ctx, wl)
+    r2 = gu.run_egtp(ctx, wl)
+    _check_all(r1, ref, wl)
+    for k in ("H", "weights", "pooled", "yhat", "state_m", "state_s"):
+        assert np.array_equal(r1[k], r2[k]), k                          # run-to-run bitwise determinism
+
+
+def test_errors_are_reported_not_fatal(ctx):
+    wl = gen.config_tiny()
+    bad = wl.offsets.copy()
+    bad[2] = bad[1] - 1                                                 # decreasing offsets: device-side error
+    res = gu.run_egtp(ctx, wl, offsets=bad)
+    assert res["status"] == egtp.EGTP_ERR_BAD_OFFSETS
+    bad2 = wl.offsets.copy()
+    bad2[-1] = wl.T + 1
+    assert gu.run_egtp(ctx, wl, offsets=bad2)["status"] == egtp.EGTP_ERR_BAD_OFFSETS
+    # host-side errors: returned at once
+    W = gu.dev_tensor(wl.W, wl.dtype)
+    hidden = gu.dev_tensor(wl.hidden, wl.dtype)
+    off = torch.from_numpy(wl.offsets).cuda()
+    lm = egtp.make_lm_head(W)
+    y = torch.empty(4, device="cuda")
+    hd = gu.DeviceHead(wl.head, wl.dtype)
+    assert egtp.egtp_predict(ctx, lm, hd.c, hidden, off, 4, wl.T, alpha=0.0, yhat_out=y, check=False) == egtp.EGTP_ERR_INVALID_ARG
+    assert egtp.egtp_predict(ctx, lm, hd.c, hidden, off, 4, 10**6, yhat_out=y, check=False) == egtp.EGTP_ERR_CAPACITY
+    assert egtp.egtp_predict(ctx, lm, None, hidden, off, 4, wl.T, yhat_out=y, check=False) == egtp.EGTP_ERR_INVALID_ARG
+    lm_bad = egtp.make_lm_head(W)
+    lm_bad.d = 250
+    assert egtp.egtp_predict(ctx, lm_bad, None, hidden, off, 4, wl.T, check=False) == egtp.EGTP_ERR_UNSUPPORTED
+    # and the context still works afterwards
+    ref = orc.egtp_predict(wl.hidden, wl.offsets, wl.W, wl.head, wl.alpha)
+    _check_all(gu.run_egtp(ctx, wl), ref, wl)
+
+
+def test_host_buffer_entry_point(ctx):
+    wl = gen.config_mid(V=3000, d=256, m_h=64, B=6)
+    ref = orc.egtp_predict(wl.hidden, wl.offsets, wl.W, wl.head, wl.alpha)
+    W = gu.dev_tensor(wl.W, wl.dtype)
+    hd = gu.DeviceHead(wl.head, wl.dtype)
+    hidden_host = torch.from_numpy(gen.bf16_bits(wl.hidden).view(np.int16)).view(torch.bfloat16).pin_memory()
+    off_host = torch.from_numpy(wl.offsets).pin_memory()
+    y = torch.empty(wl.B, dtype=torch.float32).pin_memory()
+    pooled = torch.empty(wl.B, wl.d, dtype=torch.float32).pin_memory()
+    st = torch.full((1,), 99, dtype=torch.int32).pin_memory()
+    egtp.egtp_predict_host(ctx, egtp.make_lm_head(W), hd.c, hidden_host, off_host, wl.B, wl.T, 1.0, y, pooled, st)
+    assert int(st.item()) == 0
+    gu.assert_pooled_close(pooled.numpy().astype(np.float64), ref["pooled"])
+    gu.assert_length_close(y.numpy().astype(np.float64), ref["yhat"])
