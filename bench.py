@@ -1,0 +1,382 @@
+#!/usr/bin/env python
+"""Benchmark of the EGTP / PLP hot path on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl mine|reference]
+
+A step is one pass of the whole EGTP hot path (LM-head GEMM with online entropy, merge,
+Eq. 3 weights, Eq. 4 pooling, head) over one synthetic batch shaped like the "EGTP mid"
+configuration: 32 prompts, lognormal(5.5, 0.8) lengths clipped to [32, 2048], d = 2048 bf16
+hidden states with 1 % outlier channels, LM head 151936 x 2048 bf16, head 2048 -> 512 -> 1.
+With N > 1 every rank (one process per GPU) runs its own batch of that shape (different seed):
+prompts are independent, so there is no collective on the data path ("weak" scaling).
+Rank 0 prints ONE JSON line.  The PLP decode step (256 live sequences, d = 4096) is timed on
+rank 0 at N = 1 and reported in the same line under "plp_decode".
+
+--impl reference times the fp64 CPU oracle (oracle/) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "egtp_prompt_tokens_per_sec"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        rows = [r for (t, r) in self.rows if t0 - 0.05 <= t <= t1 + 0.1] or [r for (_, r) in self.rows]
+        for r in rows:
+            parts = [x.strip() for x in r.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(smax) if smax else None,
+                    power_w=float(np.median(power)) if power else None, samples=len(sm), reasons=sorted(reasons))
+
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def workload_for_rank(rank: int):
+    from paper_2602_11812_b200 import inputs as gen
+    return gen.config_mid(seed=1 + rank)
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle on a bounded sample (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(wl, max_tokens: int = 192):
+    """The shortest whole prompts of the batch, up to max_tokens tokens (at least one prompt)."""
+    lens = wl.lengths
+    order = np.argsort(lens, kind="stable")
+    pick, tot = [], 0
+    for b in order:
+        if pick and tot + lens[b] > max_tokens:
+            break
+        pick.append(int(b)); tot += int(lens[b])
+    rows = np.concatenate([wl.hidden[wl.offsets[b]:wl.offsets[b + 1]] for b in pick])
+    off = np.concatenate([[0], np.cumsum([lens[b] for b in pick])]).astype(np.int32)
+    return rows, off, pick
+
+
+def time_oracle(wl, steps: int, warmup: int, max_tokens: int = 192):
+    from oracle import egtp_oracle as orc
+    rows, off, pick = oracle_sample(wl, max_tokens)
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    for _ in range(warmup):
+        orc.egtp_predict(rows, off, wl.W, wl.head, wl.alpha)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        orc.egtp_predict(rows, off, wl.W, wl.head, wl.alpha)
+    dt = time.perf_counter() - t0
+    tokens = int(rows.shape[0])
+    return dict(value=tokens * steps / dt, unit=UNIT, cores=int(threads), kind="oracle",
+                sample=f"{len(pick)} shortest whole prompts of the batch ({tokens} tokens) x {steps} passes, "
+                       f"fp64 numpy, {dt:.1f} s", ms_per_step=1e3 * dt / steps, tokens=tokens)
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    wl = workload_for_rank(0)
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    # keep the whole run to a few minutes: one oracle pass over ~64 tokens costs a few seconds
+    budget_tokens = 64 if steps + warmup > 8 else 192
+    r = time_oracle(wl, steps, warmup, budget_tokens)
+    line = dict(impl="reference", metric=METRIC, value=r["value"], unit=UNIT, n_gpus=args.gpus, steps=steps,
+                warmup=warmup, ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic",
+                config=dict(workload="egtp_mid: 32 prompts lognormal(5.5,0.8) in [32,2048], d=2048, V=151936, "
+                                     "head 2048->512->1", sample_tokens=r["tokens"]),
+                cpu_baseline=dict(value=r["value"], unit=UNIT, cores=r["cores"], kind="oracle", sample=r["sample"]),
+                e2e=dict(value=r["value"], unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA path
+# ------------------------------------------------------------------------------------------------
+def run_mine(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2602_11812_b200 import binding as egtp
+    from paper_2602_11812_b200 import inputs as gen
+    from paper_2602_11812_b200 import device as gu
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    peaks = load_peaks()
+    steps, warmup = max(1, args.steps), max(3, args.warmup)
+
+    wl = workload_for_rank(rank)
+    T, B, d, V = wl.T, wl.B, wl.d, wl.V
+    hidden = gu.dev_tensor(wl.hidden, wl.dtype)
+    W = gu.dev_tensor(wl.W, wl.dtype)
+    head = gu.DeviceHead(wl.head, wl.dtype)
+    offsets = torch.from_numpy(wl.offsets).cuda()
+    lm = egtp.make_lm_head(W)
+    ctx = egtp.egtp_create(local_rank, max_tokens=max(T, 1024), max_batch=max(B, 256), max_d=4096, max_V=V)
+    yhat = torch.empty(B, device="cuda", dtype=torch.float32)
+    status = torch.zeros(1, device="cuda", dtype=torch.int32)
+
+    def step():
+        egtp.egtp_predict(ctx, lm, head.c, hidden, offsets, B, T, wl.alpha, yhat_out=yhat, status_dev=status)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        step()
+    sync_all()
+    assert int(status.item()) == 0, egtp.status_string(int(status.item()))
+
+    # ---- timed region: K steps, device-timed, per-kernel events on the launching stream
+    egtp.egtp_profile_enable(ctx, True)
+    egtp.egtp_profile_read(ctx)
+    launches0 = egtp.egtp_launch_count(ctx)
+    sampler = ClockSampler(int(os.environ.get("CUDA_VISIBLE_DEVICES", "0").split(",")[local_rank]) if os.environ.get("CUDA_VISIBLE_DEVICES") else local_rank)
+    sampler.start()
+    time.sleep(0.15)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    t_wall0 = time.time()
+    ev0.record()
+    for _ in range(steps):
+        step()
+    ev1.record()
+    sync_all()
+    t_wall1 = time.time()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop(t_wall0, t_wall1)
+    launches = egtp.egtp_launch_count(ctx) - launches0
+    prof = egtp.egtp_profile_read(ctx)
+    egtp.egtp_profile_enable(ctx, False)
+    assert int(status.item()) == 0, egtp.status_string(int(status.item()))
+
+    tmax = torch.tensor([ms], device="cuda", dtype=torch.float64)
+    ttok = torch.tensor([float(T)], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        dist.all_reduce(ttok, op=dist.ReduceOp.SUM)
+    ms_max, tokens_all = float(tmax.item()), float(ttok.item())
+    value = tokens_all * steps / (ms_max * 1e-3)
+
+    # ---- end to end through the host-buffer entry point (pinned host memory in, result out)
+    hidden_host = gu.host_tensor(wl.hidden, wl.dtype)
+    off_host = torch.from_numpy(wl.offsets).pin_memory()
+    y_host = torch.empty(B, dtype=torch.float32).pin_memory()
+    st_host = torch.zeros(1, dtype=torch.int32).pin_memory()
+    e2e_steps = max(3, min(steps, 20))
+    for _ in range(2):
+        egtp.egtp_predict_host(ctx, lm, head.c, hidden_host, off_host, B, T, wl.alpha, y_host, None, st_host)
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        egtp.egtp_predict_host(ctx, lm, head.c, hidden_host, off_host, B, T, wl.alpha, y_host, None, st_host)
+    e1.record()
+    sync_all()
+    e2e_ms = torch.tensor([e0.elapsed_time(e1)], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+    e2e_value = tokens_all * e2e_steps / (float(e2e_ms.item()) * 1e-3)
+    h2d = hidden_host.numel() * 2 + off_host.numel() * 4
+    d2h = y_host.numel() * 4 + 4
+
+    if rank != 0:
+        egtp.egtp_destroy(ctx)
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel: LM-head GEMM + online entropy, tensor-core bound
+    k1 = prof["lmhead_entropy"]
+    k1_ms = k1["ms"] / max(1, k1["launches"])
+    flops = 2.0 * d * V * T                      # algorithmic flops of one launch: 2 d V per token
+    achieved = flops / (k1_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops"] if ms < 2000 else peaks["bf16_tflops_sustained"]
+    roofline = dict(bound="tensor", kernel="lmhead_entropy", achieved=achieved, peak=peak, unit="TFLOP/s",
+                    frac=achieved / peak, traffic=None, peak_source=peaks["source"],
+                    ms_per_launch=k1_ms, frac_of_sustained=achieved / peaks["bf16_tflops_sustained"],
+                    frac_of_nominal_2250=achieved / 2250.0)
+    pool = prof["pool"]
+    pool_ms = pool["ms"] / max(1, pool["launches"])
+    pool_gbs = (2.0 * d * T + 4.0 * T) / (pool_ms * 1e-3) / 1e9 if pool_ms > 0 else None
+    kernels = {k: dict(ms_per_launch=v["ms"] / max(1, v["launches"]), launches=v["launches"]) for k, v in prof.items()
+               if v["launches"]}
+    plan = egtp.egtp_lmhead_plan(ctx, T, d, V, egtp.EGTP_BF16)
+
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=steps, warmup=warmup,
+                ms_per_step=ms_max / steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                data="synthetic",
+                config=dict(workload="egtp_mid: 32 prompts lognormal(5.5,0.8) clipped [32,2048] per GPU, d=2048 bf16 "
+                                     "(1% outlier channels x20), LM head 151936x2048 bf16, head 2048->512->1",
+                            tokens_per_gpu=T, prompts_per_gpu=B, d=d, V=V,
+                            l2="inputs (622 MB LM head) larger than the 126 MB L2; no explicit flush",
+                            lmhead_plan=plan),
+                clocks=clocks,
+                e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                         steps=e2e_steps, api="egtp_predict_host"),
+                gpu_launches=int(launches),
+                roofline=roofline,
+                kernels=kernels,
+                pool=dict(bound="hbm", achieved=pool_gbs, peak=peaks["hbm_gbs"], unit="GB/s",
+                          frac=(pool_gbs / peaks["hbm_gbs"]) if pool_gbs else None,
+                          note="40 MB of hidden states: launch-latency sized at this workload"))
+
+    if world == 1 and not args.no_plp:
+        line["plp_decode"] = bench_plp(ctx_device=local_rank, peaks=peaks, steps=args.plp_steps)
+    if world == 1 and not args.no_cpu:
+        cb = time_oracle(wl, steps=1, warmup=0, max_tokens=256)
+        line["cpu_baseline"] = dict(value=cb["value"], unit=UNIT, cores=cb["cores"], kind="oracle", sample=cb["sample"])
+    egtp.egtp_destroy(ctx)
+    if world > 1:
+        dist.destroy_process_group()
+    print(json.dumps(line), flush=True)
+
+
+def bench_plp(ctx_device: int, peaks, steps: int):
+    """PLP decode step: 256 live sequences, d = 4096 bf16, LM head 151936 x 4096, head 4096 -> 256 -> 1."""
+    import torch
+
+    from paper_2602_11812_b200 import binding as egtp
+    from paper_2602_11812_b200 import inputs as gen
+    from paper_2602_11812_b200 import device as gu
+
+    warm = 5
+    wl = gen.config_plp_decode(steps=steps + warm)
+    slots, d, V = wl.slots, wl.d, wl.V
+    W = gu.dev_tensor(wl.W, "bf16")
+    head = gu.DeviceHead(wl.head, "bf16")
+    hs = gu.dev_tensor(wl.hidden_steps.reshape(-1, d), "bf16").reshape(steps + warm, slots, d)
+    reset = torch.from_numpy(wl.reset_src).cuda()
+    ctx = egtp.egtp_create(ctx_device, max_tokens=1024, max_batch=slots, max_d=d, max_V=V)
+    st = egtp.plp_state_create(ctx, slots, d)
+    lm = egtp.make_lm_head(W)
+    yrem = torch.empty(slots, device="cuda", dtype=torch.float32)
+    status = torch.zeros(1, device="cuda", dtype=torch.int32)
+    for t in range(warm):
+        egtp.plp_step(ctx, st, lm, head.c, hs[t], reset_src=reset[t], yrem_out=yrem, status_dev=status)
+    torch.cuda.synchronize()
+    egtp.egtp_profile_enable(ctx, True)
+    egtp.egtp_profile_read(ctx)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    evs[0].record()
+    for t in range(steps):
+        egtp.plp_step(ctx, st, lm, head.c, hs[warm + t], reset_src=reset[warm + t], yrem_out=yrem, status_dev=status)
+        evs[t + 1].record()
+    torch.cuda.synchronize()
+    prof = egtp.egtp_profile_read(ctx)
+    assert int(status.item()) == 0
+    per_step = np.array([evs[i].elapsed_time(evs[i + 1]) * 1e3 for i in range(steps)])
+    k1_us = prof["lmhead_entropy"]["ms"] / prof["lmhead_entropy"]["launches"] * 1e3
+    w_bytes = 2.0 * d * V
+    out = dict(metric="plp_decode_step_us", B=slots, d=d, V=V, steps=steps,
+               us_per_step_median=float(np.median(per_step)), us_per_step_p10=float(np.percentile(per_step, 10)),
+               us_per_step_p90=float(np.percentile(per_step, 90)), lmhead_us=k1_us,
+               hbm=dict(bound="hbm", achieved=w_bytes / (k1_us * 1e-6) / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
+                        frac=w_bytes / (k1_us * 1e-6) / 1e9 / peaks["hbm_gbs"]),
+               tensor=dict(achieved=2.0 * slots * d * V / (k1_us * 1e-6) / 1e12, peak=peaks["bf16_tflops"],
+                           unit="TFLOP/s", frac=2.0 * slots * d * V / (k1_us * 1e-6) / 1e12 / peaks["bf16_tflops"]),
+               kernels={k: v["ms"] / v["launches"] * 1e3 for k, v in prof.items() if v["launches"]},
+               plan=egtp.egtp_lmhead_plan(ctx, slots, d, V, egtp.EGTP_BF16))
+    egtp.plp_state_destroy(st)
+    egtp.egtp_destroy(ctx)
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="mine", choices=["mine", "reference"])
+    ap.add_argument("--plp-steps", type=int, default=64)
+    ap.add_argument("--no-plp", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_mine(args)
+
+
+if __name__ == "__main__":
+    main()

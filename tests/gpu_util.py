@@ -4,25 +4,7 @@ import torch
 
 from paper_2602_11812_b200 import binding as egtp
 from paper_2602_11812_b200 import inputs as gen
-
-
-def dev_tensor(x: np.ndarray, dtype: str) -> torch.Tensor:
-    """float32 numpy values -> device tensor in the workload dtype (exact for bf16-representable values)."""
-    if dtype == "bf16":
-        bits = gen.bf16_bits(x).view(np.int16)
-        return torch.from_numpy(bits).cuda().view(torch.bfloat16).reshape(x.shape)
-    return torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).cuda()
-
-
-class DeviceHead:
-    def __init__(self, head: gen.HeadParams, dtype: str):
-        self.W1 = dev_tensor(head.W1, dtype)
-        self.W2 = dev_tensor(head.W2, dtype)
-        self.b1 = torch.from_numpy(head.b1).cuda()
-        self.b2 = torch.from_numpy(head.b2).cuda()
-        self.centres = None if head.centres is None else torch.from_numpy(head.centres).cuda()
-        self.c = egtp.make_head(self.W1, self.b1, self.W2, self.b2, head.mode, self.centres)
-        self.d_out = head.d_out
+from paper_2602_11812_b200.device import DeviceHead, dev_tensor, host_tensor  # noqa: F401
 
 
 def run_egtp(ctx, wl: gen.EgtpWorkload, W_dev=None, hidden_dev=None, head_dev=None, offsets=None, want_phat=False):
