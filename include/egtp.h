@@ -197,6 +197,32 @@ EGTP_API int plp_step_host(egtp_ctx* ctx, plp_state* st, const egtp_lm_head* lm,
                   const float* src_m, const float* src_s, const float* src_pooled, int32_t n_src,
                   int32_t B_live, float alpha, float* yrem_host, int32_t* status_host, void* stream);
 
+/* Prediction head alone, for callers that cannot allocate device memory.  (The paper has no
+ * counterpart of this entry point; it exists for deployment reasons only.)
+ * Who needs it: code that runs inside a host which owns all GPU memory and rules out cudaMalloc
+ * while it serves - an inference engine whose pool was carved up at start-up, a plugin inside
+ * another runtime, a process with a fixed memory budget.  Such callers cannot use egtp_create,
+ * which allocates its workspace.  This call needs no context and calls neither cudaMalloc nor
+ * cudaFree nor any allocating library routine: the scratch for the first layer's split-K partial
+ * sums is a fixed 4 MiB (+256 B) array inside the library image, present on every GPU that has
+ * loaded the library until the process exits.
+ * Computes y_out[r] = head(z[r]) for r < rows exactly as egtp_predict / plp_step do for their
+ * pooled vectors (Eq. 6 in bins mode), on the CURRENT device.
+ *   head      host struct with device pointers, as above
+ *   z         device, float [rows][ldz], ldz >= d, ldz % 4 == 0, 16-byte aligned
+ *   rows      rows * head->m_h must not exceed 1048576 (2^20) floats of scratch;
+ *             beyond that the call returns EGTP_ERR_CAPACITY and launches nothing
+ *   y_out     device, float [rows]
+ *   phat_out  device, float [rows][d_out] or NULL (bins mode)
+ *   stream    cudaStream_t
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress) and
+ * the SM count; make that first call outside any stream capture.  Every call on a device uses
+ * the same array: two calls whose kernels may overlap on the GPU (different streams without an
+ * ordering between them) race on it, so order them.  The array keeps the previous call's
+ * contents; the call clears the one word that must start at zero itself. */
+EGTP_API int egtp_head_forward_static(const egtp_head* head, const float* z, int64_t ldz, int32_t rows,
+                                      float* y_out, float* phat_out, void* stream);
+
 /* Per-kernel timing. With profiling on, every kernel launch of this context is bracketed by
  * CUDA events on its own stream.  egtp_profile_read synchronises the device, adds up the
  * elapsed milliseconds and launch counts per kernel since the last read and clears them.

@@ -33,7 +33,7 @@ EXPORTED_SYMBOLS = [
     "egtp_create", "egtp_destroy", "egtp_status_string", "egtp_workspace_bytes", "egtp_predict",
     "egtp_predict_host", "plp_state_create", "plp_state_destroy", "plp_state_export", "plp_state_import",
     "plp_step", "plp_step_host", "egtp_profile_enable", "egtp_profile_read", "egtp_kernel_name",
-    "egtp_launch_count", "egtp_lmhead_plan",
+    "egtp_launch_count", "egtp_lmhead_plan", "egtp_head_forward_static",
 ]
 
 
@@ -92,6 +92,7 @@ def load() -> C.CDLL:
                              vp, vp, vp, vp, vp]
     lib.plp_step_host.argtypes = [vp, vp, P(egtp_lm_head), P(egtp_head), vp, vp, vp, vp, vp, i32, i32, f32,
                                   vp, vp, vp]
+    lib.egtp_head_forward_static.argtypes = [P(egtp_head), vp, i64, i32, vp, vp, vp]
     for name in EXPORTED_SYMBOLS:
         fn = getattr(lib, name)
         if name not in ("egtp_status_string", "egtp_kernel_name", "egtp_workspace_bytes", "egtp_launch_count"):
@@ -259,4 +260,22 @@ def plp_step_host(ctx: int, st: int, lm: egtp_lm_head, head: egtp_head, hidden_s
                               _ptr(status_host), _stream(stream))
     if check:
         _check(rc, "plp_step_host")
+    return rc
+
+
+def egtp_head_forward_static(head: egtp_head, z, rows: Optional[int] = None, y_out=None, phat_out=None, stream=None,
+                             ldz: Optional[int] = None, check: bool = True) -> int:
+    """Head forward pass without a context and without any device allocation (fixed in-library scratch).
+
+    For callers that may not allocate GPU memory; rows * m_h is limited to 2**20.  Calls on one
+    device share the scratch, so they must not overlap on the GPU.
+    """
+    if rows is None:
+        rows = z.shape[0]
+    if ldz is None:
+        ldz = z.stride(0) if hasattr(z, "stride") else head.d
+    rc = load().egtp_head_forward_static(C.byref(head), _ptr(z), ldz, rows, _ptr(y_out), _ptr(phat_out),
+                                         _stream(stream))
+    if check:
+        _check(rc, "egtp_head_forward_static")
     return rc
