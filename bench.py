@@ -302,9 +302,10 @@ def run_mine(args):
                           note="40 MB of hidden states: launch-latency sized at this workload"))
 
     if world == 1 and not args.no_plp:
-        line["plp_decode"] = bench_plp(ctx_device=local_rank, peaks=peaks, steps=args.plp_steps)
+        line["plp_decode"], line["egtp_long"] = bench_d4096(local_rank, peaks, args.plp_steps, args.long_steps)
     if world == 1 and not args.no_cpu:
-        cb = time_oracle(wl, steps=1, warmup=0, max_tokens=256)
+        probe = time_oracle(wl, steps=1, warmup=0, max_tokens=256)          # one pass tells how many fit in ~15 s
+        cb = time_oracle(wl, steps=int(min(40, max(2, 15.0 / (probe["ms_per_step"] * 1e-3)))), warmup=0, max_tokens=256)
         line["cpu_baseline"] = dict(value=cb["value"], unit=UNIT, cores=cb["cores"], kind="oracle", sample=cb["sample"])
     egtp.egtp_destroy(ctx)
     if world > 1:
@@ -312,54 +313,98 @@ def run_mine(args):
     print(json.dumps(line), flush=True)
 
 
-def bench_plp(ctx_device: int, peaks, steps: int):
-    """PLP decode step: 256 live sequences, d = 4096 bf16, LM head 151936 x 4096, head 4096 -> 256 -> 1."""
+def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
+    """The two d = 4096 workloads, sharing one 151936 x 4096 bf16 LM head on the device.
+
+    plp_decode: 256 live sequences, one token per step, head 4096 -> 256 -> 1, slots retire at
+                lognormal(6, 1) lengths and restart empty (batch kept full).
+    egtp_long:  64 prompts with Pareto(1.2) lengths clipped to [128, 8192], head 4096 -> 1024 -> 1;
+                this is also where the pooling kernel is large enough (210 MB) to be HBM-bound.
+    """
     import torch
 
     from paper_2602_11812_b200 import binding as egtp
-    from paper_2602_11812_b200 import inputs as gen
     from paper_2602_11812_b200 import device as gu
+    from paper_2602_11812_b200 import inputs as gen
 
     warm = 5
-    wl = gen.config_plp_decode(steps=steps + warm)
+    wl = gen.config_plp_decode(steps=plp_steps + warm)
     slots, d, V = wl.slots, wl.d, wl.V
     W = gu.dev_tensor(wl.W, "bf16")
-    head = gu.DeviceHead(wl.head, "bf16")
-    hs = gu.dev_tensor(wl.hidden_steps.reshape(-1, d), "bf16").reshape(steps + warm, slots, d)
-    reset = torch.from_numpy(wl.reset_src).cuda()
-    ctx = egtp.egtp_create(ctx_device, max_tokens=1024, max_batch=slots, max_d=d, max_V=V)
-    st = egtp.plp_state_create(ctx, slots, d)
     lm = egtp.make_lm_head(W)
-    yrem = torch.empty(slots, device="cuda", dtype=torch.float32)
+    wl3 = gen.config_long(W=wl.W)
+    ctx = egtp.egtp_create(ctx_device, max_tokens=max(wl3.T, 1024), max_batch=slots, max_d=d, max_V=V)
     status = torch.zeros(1, device="cuda", dtype=torch.int32)
+
+    # ---- PLP decode steps
+    head = gu.DeviceHead(wl.head, "bf16")
+    hs = gu.dev_tensor(wl.hidden_steps.reshape(-1, d), "bf16").reshape(plp_steps + warm, slots, d)
+    reset = torch.from_numpy(wl.reset_src).cuda()
+    st = egtp.plp_state_create(ctx, slots, d)
+    yrem = torch.empty(slots, device="cuda", dtype=torch.float32)
     for t in range(warm):
         egtp.plp_step(ctx, st, lm, head.c, hs[t], reset_src=reset[t], yrem_out=yrem, status_dev=status)
     torch.cuda.synchronize()
     egtp.egtp_profile_enable(ctx, True)
     egtp.egtp_profile_read(ctx)
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(plp_steps + 1)]
     evs[0].record()
-    for t in range(steps):
+    for t in range(plp_steps):
         egtp.plp_step(ctx, st, lm, head.c, hs[warm + t], reset_src=reset[warm + t], yrem_out=yrem, status_dev=status)
         evs[t + 1].record()
     torch.cuda.synchronize()
     prof = egtp.egtp_profile_read(ctx)
     assert int(status.item()) == 0
-    per_step = np.array([evs[i].elapsed_time(evs[i + 1]) * 1e3 for i in range(steps)])
+    per_step = np.array([evs[i].elapsed_time(evs[i + 1]) * 1e3 for i in range(plp_steps)])
     k1_us = prof["lmhead_entropy"]["ms"] / prof["lmhead_entropy"]["launches"] * 1e3
     w_bytes = 2.0 * d * V
-    out = dict(metric="plp_decode_step_us", B=slots, d=d, V=V, steps=steps,
-               us_per_step_median=float(np.median(per_step)), us_per_step_p10=float(np.percentile(per_step, 10)),
+    step_us = float(np.median(per_step))
+    plp = dict(metric="plp_decode_step_us", B=slots, d=d, V=V, steps=plp_steps,
+               us_per_step_median=step_us, us_per_step_p10=float(np.percentile(per_step, 10)),
                us_per_step_p90=float(np.percentile(per_step, 90)), lmhead_us=k1_us,
-               hbm=dict(bound="hbm", achieved=w_bytes / (k1_us * 1e-6) / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
-                        frac=w_bytes / (k1_us * 1e-6) / 1e9 / peaks["hbm_gbs"]),
+               hbm=dict(bound="hbm", kernel="lmhead_entropy", achieved=w_bytes / (k1_us * 1e-6) / 1e9,
+                        peak=peaks["hbm_gbs"], unit="GB/s", frac=w_bytes / (k1_us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                        whole_step_frac=w_bytes / (step_us * 1e-6) / 1e9 / peaks["hbm_gbs"]),
                tensor=dict(achieved=2.0 * slots * d * V / (k1_us * 1e-6) / 1e12, peak=peaks["bf16_tflops"],
                            unit="TFLOP/s", frac=2.0 * slots * d * V / (k1_us * 1e-6) / 1e12 / peaks["bf16_tflops"]),
-               kernels={k: v["ms"] / v["launches"] * 1e3 for k, v in prof.items() if v["launches"]},
+               kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof.items() if v["launches"]},
                plan=egtp.egtp_lmhead_plan(ctx, slots, d, V, egtp.EGTP_BF16))
     egtp.plp_state_destroy(st)
+    del hs
+
+    # ---- EGTP over the long-tailed prompt batch
+    hidden = gu.dev_tensor(wl3.hidden, "bf16")
+    head3 = gu.DeviceHead(wl3.head, "bf16")
+    off = torch.from_numpy(wl3.offsets).cuda()
+    yhat = torch.empty(wl3.B, device="cuda", dtype=torch.float32)
+    for _ in range(3):
+        egtp.egtp_predict(ctx, lm, head3.c, hidden, off, wl3.B, wl3.T, 1.0, yhat_out=yhat, status_dev=status)
+    torch.cuda.synchronize()
+    egtp.egtp_profile_read(ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(egtp_steps):
+        egtp.egtp_predict(ctx, lm, head3.c, hidden, off, wl3.B, wl3.T, 1.0, yhat_out=yhat, status_dev=status)
+    e1.record()
+    torch.cuda.synchronize()
+    prof3 = egtp.egtp_profile_read(ctx)
+    assert int(status.item()) == 0
+    ms_step = e0.elapsed_time(e1) / egtp_steps
+    k1_ms = prof3["lmhead_entropy"]["ms"] / prof3["lmhead_entropy"]["launches"]
+    pool_us = prof3["pool"]["ms"] / prof3["pool"]["launches"] * 1e3
+    tf = 2.0 * d * V * wl3.T / (k1_ms * 1e-3) / 1e12
+    pool_gbs = (2.0 * d + 4.0) * wl3.T / (pool_us * 1e-6) / 1e9
+    long_ = dict(metric=METRIC, workload="egtp_long: 64 prompts Pareto(1.2) in [128,8192], d=4096, V=151936, head 4096->1024->1",
+                 tokens=wl3.T, steps=egtp_steps, ms_per_step=ms_step, value=wl3.T / (ms_step * 1e-3), unit=UNIT,
+                 lmhead=dict(bound="tensor", achieved=tf, peak=peaks["bf16_tflops"], unit="TFLOP/s",
+                             frac=tf / peaks["bf16_tflops"], ms_per_launch=k1_ms),
+                 pool=dict(bound="hbm", kernel="pool", achieved=pool_gbs, peak=peaks["hbm_gbs"], unit="GB/s",
+                           frac=pool_gbs / peaks["hbm_gbs"], us_per_launch=pool_us,
+                           bytes_per_token=2 * d + 4),
+                 kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof3.items() if v["launches"]},
+                 plan=egtp.egtp_lmhead_plan(ctx, wl3.T, d, V, egtp.EGTP_BF16))
     egtp.egtp_destroy(ctx)
-    return out
+    return plp, long_
 
 
 def main():
@@ -369,6 +414,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="mine", choices=["mine", "reference"])
     ap.add_argument("--plp-steps", type=int, default=64)
+    ap.add_argument("--long-steps", type=int, default=10)
     ap.add_argument("--no-plp", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -247,9 +247,9 @@ EGTP_API const char* egtp_kernel_name(int kernel_id);
 EGTP_API int64_t egtp_launch_count(const egtp_ctx* ctx);
 
 /* Launch shape the LM-head kernel uses for T rows of hidden size d against V vocabulary rows:
- * info[0] = grid (CTAs), [1] = row tiles, [2] = vocabulary tiles, [3] = vocabulary chunks,
- * [4] = partial slots per row, [5] = row tiles per group, [6] = k blocks, [7] = dynamic smem bytes.
- * Host pointer; nothing is launched. */
+ * info[0] = grid (CTAs), [1] = row blocks, [2] = rows per block (128 or 256), [3] = vocabulary
+ * chunks, [4] = partial slots per row, [5] = vocabulary columns per tile, [6] = k blocks,
+ * [7] = dynamic shared memory bytes.  Host pointer; nothing is launched. */
 EGTP_API int egtp_lmhead_plan(const egtp_ctx* ctx, int64_t T, int32_t d, int32_t V, int32_t dtype, int32_t info[8]);
 
 #ifdef __cplusplus

@@ -179,7 +179,7 @@ def egtp_kernel_name(kernel_id: int) -> str:
 def egtp_lmhead_plan(ctx: int, T: int, d: int, V: int, dtype: int) -> dict:
     info = (C.c_int32 * 8)()
     _check(load().egtp_lmhead_plan(ctx, T, d, V, dtype, info), "egtp_lmhead_plan")
-    keys = ["grid", "m_tiles", "n_tiles", "chunks", "slots", "group_m", "k_blocks", "smem_bytes"]
+    keys = ["grid", "row_blocks", "rows_per_block", "chunks", "slots", "tile_cols", "k_blocks", "smem_bytes"]
     return dict(zip(keys, list(info)))
 
 

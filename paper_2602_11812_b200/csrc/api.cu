@@ -175,27 +175,20 @@ HeadArgs head_args(const egtp_head* h) {
     if ((expr) != cudaSuccess) return EGTP_ERR_CUDA; \
   } while (0)
 
-// Eq. 2 for `rows` rows: LM-head kernel + merge. Writes H (and seg ids / zeroed weights when asked).
-int run_entropy(egtp_ctx* c, const egtp_lm_head* lm, const void* hidden, int64_t ldh, int64_t rows, float* H,
-                const int32_t* offsets, int B, int32_t* seg_id, float* weights_zero, int32_t* status,
-                cudaStream_t stream) {
+// Eq. 2 for `rows` rows, first part: the LM-head kernel leaves per-slot partials in the workspace.
+int run_lmhead(egtp_ctx* c, const egtp_lm_head* lm, const void* hidden, int64_t ldh, int64_t rows, int32_t* status,
+               cudaStream_t stream, LmheadPlan* plan_out) {
   const LmheadPlan plan = make_lmhead_plan(rows, lm->d, lm->V, elem_bytes(lm->dtype), c->num_sms, c->slot_row_capacity);
   if (plan.rows_pad * plan.slots > c->slot_row_capacity) return EGTP_ERR_CAPACITY;
   CUtensorMap map_a, map_b;
-  int rc = make_tensor_map(c, &map_a, hidden, lm->dtype, rows, lm->d, ldh, kTileM);
+  int rc = make_tensor_map(c, &map_a, hidden, lm->dtype, rows, lm->d, ldh, plan.rows_per_block);
   if (rc != EGTP_OK) return rc;
-  rc = make_tensor_map(c, &map_b, lm->W, lm->dtype, lm->V, lm->d, lm->ldw, kTileN);
+  rc = make_tensor_map(c, &map_b, lm->W, lm->dtype, lm->V, lm->d, lm->ldw, plan.b_box_rows);
   if (rc != EGTP_OK) return rc;
-  {
-    LaunchScope ls(c, EGTP_K_LMHEAD_ENTROPY, stream);
-    EGTP_CUDA_TRY(launch_lmhead_entropy(plan, lm->dtype == EGTP_F32, &map_a, &map_b, rows, lm->V, c->partials, status,
-                                        stream));
-  }
-  {
-    LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
-    EGTP_CUDA_TRY(launch_entropy_merge(c->partials, plan.slots, plan.rows_pad, rows, H, offsets, B, seg_id,
-                                       weights_zero, status, stream));
-  }
+  LaunchScope ls(c, EGTP_K_LMHEAD_ENTROPY, stream);
+  EGTP_CUDA_TRY(launch_lmhead_entropy(plan, lm->dtype == EGTP_F32, &map_a, &map_b, rows, lm->V, c->partials, status,
+                                      stream));
+  *plan_out = plan;
   return EGTP_OK;
 }
 
@@ -263,10 +256,10 @@ int egtp_create(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_batc
 
   const int64_t rows_cap = std::max<int64_t>(max_tokens, max_batch);
   const int64_t rows_pad = (rows_cap + kTileM - 1) / kTileM * kTileM;
-  const int64_t n_tiles = (static_cast<int64_t>(max_V) + kTileN - 1) / kTileN;
-  // room for 24 vocabulary chunks at the largest token count, and for one chunk per vocabulary
-  // tile on decode-sized batches (up to 1024 rows)
-  c->slot_row_capacity = std::max<int64_t>(rows_pad * 24 * kEpiSplit, std::min<int64_t>(rows_pad, 1024) * n_tiles * kEpiSplit);
+  // room for 24 vocabulary chunks (two partial slots each) at the largest token count, and for one
+  // chunk per SM on decode-sized batches
+  c->slot_row_capacity = std::max<int64_t>(rows_pad * 24 * kEpiSplit,
+                                           static_cast<int64_t>(2 * kTileM) * c->num_sms * kEpiSplit);
   const int64_t pool_chunks = (max_tokens + kPoolChunkTokens - 1) / kPoolChunkTokens + 1;
   c->head_partial_floats = std::max<int64_t>(8ll << 20, static_cast<int64_t>(max_batch) * 8192);
 
@@ -310,8 +303,8 @@ int64_t egtp_launch_count(const egtp_ctx* c) { return c ? c->launches : 0; }
 int egtp_lmhead_plan(const egtp_ctx* c, int64_t T, int32_t d, int32_t V, int32_t dtype, int32_t info[8]) {
   if (!c || !info || T <= 0 || d <= 0 || V <= 0) return EGTP_ERR_INVALID_ARG;
   const LmheadPlan p = make_lmhead_plan(T, d, V, elem_bytes(dtype), c->num_sms, c->slot_row_capacity);
-  info[0] = p.grid; info[1] = p.m_tiles; info[2] = p.n_tiles; info[3] = p.chunks;
-  info[4] = p.slots; info[5] = p.group_m; info[6] = p.k_blocks; info[7] = p.smem_bytes;
+  info[0] = p.grid; info[1] = p.row_blocks; info[2] = p.rows_per_block; info[3] = p.chunks;
+  info[4] = p.slots; info[5] = p.tile_cols; info[6] = p.k_blocks; info[7] = p.smem_bytes;
   return EGTP_OK;
 }
 
@@ -382,8 +375,12 @@ int egtp_predict(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, con
     EGTP_CUDA_TRY(launch_validate_offsets(offsets, B, T_total, status, stream));
   }
   if (T_total > 0) {
-    int rc = run_entropy(c, lm, hidden, ldh, T_total, H, offsets, B, seg_id_out, weights, status, stream);
+    LmheadPlan plan;
+    int rc = run_lmhead(c, lm, hidden, ldh, T_total, status, stream, &plan);
     if (rc != EGTP_OK) return rc;
+    LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
+    EGTP_CUDA_TRY(launch_entropy_merge(c->partials, plan.slots, T_total, H, offsets, B, seg_id_out, weights, status,
+                                       stream));
   }
   if (B == 0) return EGTP_OK;
   {
@@ -507,13 +504,13 @@ int plp_step(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head
   if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
   int32_t* status = status_dev ? status_dev : c->status;
   if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
-  float* H = Hstep_out ? Hstep_out : c->H;
   float* z = z_out ? z_out : c->pooled;
-  rc = run_entropy(c, lm, hidden_step, ldh, B_live, H, nullptr, 0, nullptr, nullptr, status, stream);
+  LmheadPlan plan;
+  rc = run_lmhead(c, lm, hidden_step, ldh, B_live, status, stream, &plan);
   if (rc != EGTP_OK) return rc;
   {
     LaunchScope ls(c, EGTP_K_PLP_UPDATE, stream);
-    EGTP_CUDA_TRY(launch_plp_update(hidden_step, ldh, lm->dtype == EGTP_BF16, H, slot_ids, reset_src, src_m, src_s,
+    EGTP_CUDA_TRY(launch_plp_update(hidden_step, ldh, lm->dtype == EGTP_BF16, c->partials, plan.slots, Hstep_out, slot_ids, reset_src, src_m, src_s,
                                     src_pooled, n_src, B_live, lm->d, st->num_slots, 1.f / alpha, st->m, st->s,
                                     st->acc, z, lm->d, status, stream));
   }

@@ -1,0 +1,47 @@
+// Merge of the LM-head kernel's per-slot entropy partials (paper Eq. 2).
+// A partial is (m, s, t2) over a range of the vocabulary: m = max logit, s = sum 2^y,
+// t2 = sum 2^y * y with y = (x - m) log2 e.  Two partials combine by rescaling both to the
+// larger m; the token's entropy is H = ln S - ln2 * T2 / S (both terms are >= 0).
+#pragma once
+
+#include "kernels.h"
+
+namespace egtp {
+
+struct EntropyPartial {
+  float m, s, t2;
+};
+
+__device__ __forceinline__ EntropyPartial combine_partials(const EntropyPartial& a, const EntropyPartial& b) {
+  constexpr float kLog2e = 1.4426950408889634f;
+  EntropyPartial r;
+  r.m = fmaxf(a.m, b.m);
+  const float da = (a.m - r.m) * kLog2e, db = (b.m - r.m) * kLog2e;
+  const float ra = exp2f(da), rb = exp2f(db);
+  r.s = fmaf(a.s, ra, b.s * rb);
+  r.t2 = ra * fmaf(da, a.s, a.t2) + rb * fmaf(db, b.s, b.t2);
+  return r;
+}
+
+// All 32 lanes of a warp call this with the same row pointer ([slots][3] floats); every lane
+// returns H.  The order of operations is fixed, so the result is bitwise reproducible.
+__device__ __forceinline__ float merge_partials_warp(const float* __restrict__ row, int slots, int lane) {
+  constexpr float kLn2 = 0.6931471805599453f;
+  EntropyPartial acc = {kNegBig, 0.f, 0.f};
+  for (int j = lane; j < slots; j += 32) {
+    const EntropyPartial pj = {row[3 * j], row[3 * j + 1], row[3 * j + 2]};
+    acc = combine_partials(acc, pj);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    EntropyPartial other;
+    other.m = __shfl_xor_sync(0xffffffffu, acc.m, o);
+    other.s = __shfl_xor_sync(0xffffffffu, acc.s, o);
+    other.t2 = __shfl_xor_sync(0xffffffffu, acc.t2, o);
+    // lower lane first on both sides so that every lane computes the identical value
+    acc = (lane & o) ? combine_partials(other, acc) : combine_partials(acc, other);
+  }
+  return logf(acc.s) - kLn2 * acc.t2 / acc.s;
+}
+
+}  // namespace egtp

@@ -16,6 +16,7 @@ namespace {
 constexpr int kHT = 64;        // rows and hidden units per block tile
 constexpr int kHK = 16;        // k extent per shared-memory stage
 constexpr int kHThreads = 256; // 16 x 16 threads, 4 x 4 outputs each
+constexpr int kHOutThreads = 256;
 
 template <typename TW>
 __device__ __forceinline__ float4 load4(const TW* p);
@@ -31,37 +32,49 @@ __device__ __forceinline__ float4 load4<__nv_bfloat16>(const __nv_bfloat16* p) {
 }
 
 // partial[split][row][j] = sum_{k in split} z[row][k] * W1[j][k]
+// 64 x 64 outputs per block, 4 x 4 per thread; the global loads of k-block i+1 are in flight while
+// k-block i is multiplied out of shared memory (two buffers, one barrier per k-block).
 template <typename TW>
 __global__ void __launch_bounds__(kHThreads)
 head_hidden_kernel(const float* __restrict__ z, int64_t ldz, const TW* __restrict__ W1, int rows, int d, int m_h,
                    int k_per_split, float* __restrict__ partial, const int32_t* __restrict__ status) {
   if (*status != 0) return;
-  __shared__ float zs[kHK][kHT + 4];
-  __shared__ float ws[kHK][kHT + 4];
+  __shared__ float zs[2][kHK][kHT + 4];
+  __shared__ float ws[2][kHK][kHT + 4];
   const int j0 = blockIdx.x * kHT, r0 = blockIdx.y * kHT, split = blockIdx.z;
   const int k_begin = split * k_per_split;
   const int k_end = min(d, k_begin + k_per_split);
   const int tid = threadIdx.x;
   const int lrow = tid >> 2, lk = (tid & 3) * 4;   // loader: 64 rows x 4 quads of k
   const int tx = tid & 15, ty = tid >> 4;          // compute: outputs rows ty*4.., units tx*4..
+  const bool z_ok = r0 + lrow < rows, w_ok = j0 + lrow < m_h;
+  const float* zp = z + static_cast<int64_t>(r0 + lrow) * ldz + lk;
+  const TW* wp = W1 + static_cast<int64_t>(j0 + lrow) * d + lk;
   float acc[4][4];
 #pragma unroll
   for (int a = 0; a < 4; ++a)
 #pragma unroll
     for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
 
+  const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 zv = zero4, wv = zero4;
+  if (k_begin < k_end) {
+    if (z_ok) zv = __ldg(reinterpret_cast<const float4*>(zp + k_begin));
+    if (w_ok) wv = load4<TW>(wp + k_begin);
+  }
+  int buf = 0;
   for (int k0 = k_begin; k0 < k_end; k0 += kHK) {
-    float4 zv = make_float4(0.f, 0.f, 0.f, 0.f), wv = zv;
-    if (r0 + lrow < rows) zv = __ldg(reinterpret_cast<const float4*>(z + static_cast<int64_t>(r0 + lrow) * ldz + k0 + lk));
-    if (j0 + lrow < m_h) wv = load4<TW>(W1 + static_cast<int64_t>(j0 + lrow) * d + k0 + lk);
+    zs[buf][lk + 0][lrow] = zv.x; zs[buf][lk + 1][lrow] = zv.y; zs[buf][lk + 2][lrow] = zv.z; zs[buf][lk + 3][lrow] = zv.w;
+    ws[buf][lk + 0][lrow] = wv.x; ws[buf][lk + 1][lrow] = wv.y; ws[buf][lk + 2][lrow] = wv.z; ws[buf][lk + 3][lrow] = wv.w;
     __syncthreads();
-    zs[lk + 0][lrow] = zv.x; zs[lk + 1][lrow] = zv.y; zs[lk + 2][lrow] = zv.z; zs[lk + 3][lrow] = zv.w;
-    ws[lk + 0][lrow] = wv.x; ws[lk + 1][lrow] = wv.y; ws[lk + 2][lrow] = wv.z; ws[lk + 3][lrow] = wv.w;
-    __syncthreads();
+    if (k0 + kHK < k_end) {
+      zv = z_ok ? __ldg(reinterpret_cast<const float4*>(zp + k0 + kHK)) : zero4;
+      wv = w_ok ? load4<TW>(wp + k0 + kHK) : zero4;
+    }
 #pragma unroll
     for (int k = 0; k < kHK; ++k) {
-      const float4 a = *reinterpret_cast<const float4*>(&zs[k][ty * 4]);
-      const float4 b = *reinterpret_cast<const float4*>(&ws[k][tx * 4]);
+      const float4 a = *reinterpret_cast<const float4*>(&zs[buf][k][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&ws[buf][k][tx * 4]);
       const float av[4] = {a.x, a.y, a.z, a.w};
       const float bv[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
@@ -69,16 +82,21 @@ head_hidden_kernel(const float* __restrict__ z, int64_t ldz, const TW* __restric
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
     }
+    buf ^= 1;   // the other buffer was last read two k-blocks ago: the barrier above already fenced it
   }
   float* out = partial + static_cast<int64_t>(split) * rows * m_h;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int r = r0 + ty * 4 + i;
     if (r >= rows) continue;
+    const int jj = j0 + tx * 4;
+    float* o = out + static_cast<int64_t>(r) * m_h + jj;
+    if (jj + 3 < m_h && (m_h & 3) == 0) {
+      *reinterpret_cast<float4*>(o) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+    } else {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int jj = j0 + tx * 4 + j;
-      if (jj < m_h) out[static_cast<int64_t>(r) * m_h + jj] = acc[i][j];
+      for (int j = 0; j < 4; ++j)
+        if (jj + j < m_h) o[j] = acc[i][j];
     }
   }
 }
@@ -93,7 +111,7 @@ __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return
 // One block per row: u = ReLU(sum of split partials + b1) into shared memory, o_c = W2[c] . u + b2[c]
 // (one warp per output, lanes stride the hidden units), then the output mode.
 template <typename TW>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kHOutThreads)
 head_out_kernel(const float* __restrict__ partial, int rows, int splits, int m_h, int d_out,
                 const float* __restrict__ b1, const TW* __restrict__ W2, const float* __restrict__ b2,
                 const float* __restrict__ centres, int mode, float* __restrict__ y, float* __restrict__ phat,
@@ -104,8 +122,16 @@ head_out_kernel(const float* __restrict__ partial, int rows, int splits, int m_h
   float* o = smem + m_h;      // [d_out]
   const int r = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   for (int j = tid; j < m_h; j += blockDim.x) {
+    const float* pj = partial + static_cast<int64_t>(r) * m_h + j;
+    const int64_t stride = static_cast<int64_t>(rows) * m_h;
     float v = 0.f;
-    for (int s = 0; s < splits; ++s) v += partial[(static_cast<int64_t>(s) * rows + r) * m_h + j];
+    int s = 0;
+    for (; s + 4 <= splits; s += 4) {     // four loads in flight; the additions keep split order
+      const float p0 = __ldg(pj + s * stride), p1 = __ldg(pj + (s + 1) * stride), p2 = __ldg(pj + (s + 2) * stride),
+                  p3 = __ldg(pj + (s + 3) * stride);
+      v = (((v + p0) + p1) + p2) + p3;
+    }
+    for (; s < splits; ++s) v += __ldg(pj + s * stride);
     u[j] = fmaxf(0.f, v + b1[j]);
   }
   __syncthreads();
@@ -167,11 +193,11 @@ cudaError_t launch_head_out(const HeadArgs& h, const float* partial, int rows, i
                             const int32_t* status, cudaStream_t stream) {
   const size_t smem = static_cast<size_t>(h.m_h + h.d_out) * sizeof(float);
   if (h.bf16) {
-    head_out_kernel<__nv_bfloat16><<<rows, 128, smem, stream>>>(partial, rows, splits, h.m_h, h.d_out, h.b1,
+    head_out_kernel<__nv_bfloat16><<<rows, kHOutThreads, smem, stream>>>(partial, rows, splits, h.m_h, h.d_out, h.b1,
                                                                static_cast<const __nv_bfloat16*>(h.W2), h.b2,
                                                                h.centres, h.mode, y, phat, status);
   } else {
-    head_out_kernel<float><<<rows, 128, smem, stream>>>(partial, rows, splits, h.m_h, h.d_out, h.b1,
+    head_out_kernel<float><<<rows, kHOutThreads, smem, stream>>>(partial, rows, splits, h.m_h, h.d_out, h.b1,
                                                        static_cast<const float*>(h.W2), h.b2, h.centres, h.mode, y,
                                                        phat, status);
   }

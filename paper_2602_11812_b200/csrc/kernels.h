@@ -12,22 +12,25 @@ constexpr float kNegBig = -1.0e30f;
 
 // ---- K1: LM-head GEMM with online entropy epilogue ---------------------------------------
 constexpr int kTileM = 128;        // token rows per tile (UMMA M, one TMEM lane per row)
-constexpr int kTileN = 256;        // vocabulary columns per tile (UMMA N, one TMEM column each)
 constexpr int kRowBytes = 128;     // K extent of one pipeline stage in bytes (one swizzle row)
-constexpr int kStages = 4;         // TMA -> MMA pipeline depth
 constexpr int kEpiSplit = 2;       // epilogue warps per TMEM lane quadrant (column halves)
 constexpr int kLmheadThreads = (2 + 4 * kEpiSplit) * 32;
 
 struct LmheadPlan {
-  int grid;          // persistent CTAs
-  int m_tiles;       // ceil(T / 128)
-  int n_tiles;       // ceil(V / 256)
-  int chunks;        // vocabulary chunks S; a work unit is (row tile, chunk)
-  int slots;         // partial slots per row = S * kEpiSplit
-  int group_m;       // row tiles that sweep the vocabulary together (L2 reuse of W tiles)
-  int k_blocks;      // ceil(d * elem / 128)
-  int smem_bytes;    // dynamic shared memory
-  int64_t rows_pad;  // m_tiles * 128: row pitch of the partial buffer
+  int variant;        // 0 prompt shape, 1 decode <= 128 rows, 2 decode <= 256 rows
+  int grid;           // persistent CTAs
+  int row_blocks;     // ceil(T / rows_per_block)
+  int rows_per_block; // 128 or 256: rows a CTA multiplies against each W tile (box rows of the hidden map)
+  int tile_cols;      // vocabulary columns per tile
+  int b_box_rows;     // rows of one TMA box of W
+  int col_gran;       // vocabulary chunks start at multiples of this many columns
+  int n_groups;       // ceil(V / col_gran)
+  int chunks;         // vocabulary chunks S; a work unit is (row block, chunk)
+  int slots;          // partial slots per row
+  int group_rb;       // row blocks that sweep the vocabulary together (L2 reuse of W tiles)
+  int k_blocks;       // ceil(d * elem / 128)
+  int smem_bytes;     // dynamic shared memory
+  int64_t rows_pad;   // row_blocks * rows_per_block: rows of the partial buffer
 };
 
 // Picks chunks / grouping for T rows; slot_limit bounds chunks * kEpiSplit * rows_pad by the
@@ -37,7 +40,7 @@ LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms
 // Opts the kernels into their dynamic shared-memory size on the current device (once per device).
 cudaError_t lmhead_prepare_device();
 
-// partials layout: [slot][3][rows_pad] floats: (m, s, t2) with m the running max logit,
+// partials layout: [rows_pad][slots][3] floats: (m, s, t2) with m the running max logit,
 // s = sum 2^((x-m) log2 e), t2 = sum 2^(...) * (x-m) log2 e over the slot's vocabulary range.
 cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const CUtensorMap* map_hidden,
                                   const CUtensorMap* map_w, int64_t T, int V, float* partials,
@@ -49,7 +52,7 @@ constexpr int kPoolThreads = 128;      // each thread owns 8 consecutive channel
 
 cudaError_t launch_validate_offsets(const int32_t* offsets, int B, int64_t T, int32_t* status, cudaStream_t stream);
 
-cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t rows_pad, int64_t T, float* H,
+cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t T, float* H,
                                  const int32_t* offsets, int B, int32_t* seg_id_out, float* weights_zero,
                                  const int32_t* status, cudaStream_t stream);
 
@@ -83,7 +86,9 @@ cudaError_t launch_head_out(const HeadArgs& h, const float* partial, int rows, i
                             const int32_t* status, cudaStream_t stream);
 
 // ---- K4: PLP running-state update ---------------------------------------------------------
-cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, const float* Hstep,
+// Merges the row's entropy partials itself (Eq. 2), optionally writes H' to Hstep_out, then updates the slot.
+cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, const float* partials, int slots,
+                              float* Hstep_out,
                               const int32_t* slot_ids, const int32_t* reset_src, const float* src_m,
                               const float* src_s, const float* src_pooled, int n_src, int rows, int d, int num_slots,
                               float inv_alpha, float* st_m, float* st_s, float* st_acc, float* z, int64_t ldz,

@@ -8,58 +8,61 @@
 // from the per-vocabulary-chunk partials written here.
 //
 // One persistent CTA per SM, warp-specialised:
-//   warp 0      TMA producer: streams 128x(128 B) hidden tiles and 256x(128 B) W tiles through a
-//               4-stage shared-memory ring (128-byte swizzle, K-major)
+//   warp 0      TMA producer: streams hidden tiles and W tiles (rows of 128 bytes, 128-byte swizzle,
+//               K-major) through a 4-stage shared-memory ring
 //   warp 1      MMA issuer (one thread) and owner of the TMEM allocation (512 columns = two
-//               128x256 fp32 accumulators, so the epilogue of tile j overlaps the MMAs of j+1)
-//   warps 2..9  epilogue: TMEM lane quadrant = warp % 4, column half = (warp - 2) / 4;
+//               256-column fp32 accumulator sets, so the epilogue of tile j overlaps the MMAs of j+1)
+//   warps 2..9  epilogue: TMEM lane quadrant = warp % 4, accumulator column half = (warp - 2) / 4;
 //               one row per thread, 128 columns per tile, tcgen05.ld in 32-column pieces
-// A work unit is (row tile, vocabulary chunk); units are ordered so that CTAs running at the
-// same time share W tiles (same chunk, neighbouring row tiles) and hidden tiles stay in L2.
+// A work unit is (row block, vocabulary chunk); units are ordered so that CTAs running at the
+// same time share W tiles (same chunk, neighbouring row blocks) and hidden tiles stay in L2.
+// Three tile shapes: prompts (128 rows x 256 columns per tile, tensor-bound), and two decode shapes
+// for <= 128 and <= 256 rows, where the step is bound by streaming W from HBM once: every SM
+// gets its own vocabulary range (equal to within 32 columns) and, for 129..256 rows, multiplies
+// both row tiles against each W tile it loads.
 #include "kernels.h"
 #include "sm100_ptx.cuh"
 #include "../../include/egtp.h"
 
 #include <algorithm>
 
+
 namespace egtp {
 
 namespace {
 
-constexpr int kABytes = kTileM * kRowBytes;            // 16 KB
-constexpr int kBBytes = kTileN * kRowBytes;            // 32 KB
-constexpr int kStageBytes = kABytes + kBBytes;         // 48 KB
-constexpr int kBarrierBytes = 128;
-constexpr int kSmemBytes = kStages * kStageBytes + kBarrierBytes + 1024;   // + slack for 1024-B alignment
+constexpr int kBarrierBytes = 256;
 constexpr uint32_t kTmemCols = 512;
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kMaxStages = 8;
 
 struct UnitCoord {
-  int m_tile;
-  int n_begin;
-  int n_end;
+  int row_block;
   int chunk;
+  int col_begin;
+  int col_end;
 };
 
 struct KParams {
-  int m_tiles, n_tiles, chunks, group_m, k_blocks;
+  int row_blocks, chunks, group_rb, k_blocks;
+  int n_groups, col_gran;      // the vocabulary is split at multiples of col_gran columns
   int total_units;
   int V;
-  int64_t rows_pad;
+  int slots;
   float* partials;
   int32_t* status;
 };
 
 __device__ __forceinline__ UnitCoord unit_coord(int u, const KParams& p) {
-  const int per_group = p.group_m * p.chunks;
+  const int per_group = p.group_rb * p.chunks;
   const int g = u / per_group;
   const int r = u - g * per_group;
-  const int gm = min(p.group_m, p.m_tiles - g * p.group_m);
+  const int gm = min(p.group_rb, p.row_blocks - g * p.group_rb);
   UnitCoord c;
   c.chunk = r / gm;
-  c.m_tile = g * p.group_m + (r - c.chunk * gm);
-  c.n_begin = static_cast<int>((static_cast<int64_t>(c.chunk) * p.n_tiles) / p.chunks);
-  c.n_end = static_cast<int>((static_cast<int64_t>(c.chunk + 1) * p.n_tiles) / p.chunks);
+  c.row_block = g * p.group_rb + (r - c.chunk * gm);
+  c.col_begin = static_cast<int>((static_cast<int64_t>(c.chunk) * p.n_groups) / p.chunks) * p.col_gran;
+  c.col_end = static_cast<int>((static_cast<int64_t>(c.chunk + 1) * p.n_groups) / p.chunks) * p.col_gran;
   return c;
 }
 
@@ -74,7 +77,7 @@ struct RowState {
     for (int i = 0; i < 4; ++i) { s[i] = 0.f; t[i] = 0.f; }
   }
   // Folds 32 logits in. With kMasked, only the first `valid` (>= 1) columns exist (the piece
-  // straddles the end of the vocabulary); the rest are ignored.
+  // straddles the end of the vocabulary or of the tile); the rest are ignored.
   template <bool kMasked>
   __device__ __forceinline__ void fold(const uint32_t (&raw)[32], int valid) {
     float x[32];
@@ -103,22 +106,41 @@ struct RowState {
       t[j & 3] = fmaf(e, y, t[j & 3]);
     }
   }
+  __device__ __forceinline__ void fold_n(const uint32_t (&raw)[32], int valid) {
+    if (valid >= 32) fold<false>(raw, 32); else fold<true>(raw, valid);
+  }
 };
 
-template <bool kTf32>
+// kMT   row tiles (of 128 rows) a CTA multiplies against every W tile it loads: 1 for prompt
+//       batches, 2 for decode batches of 129..256 rows (each W byte is then fetched once per GPU)
+// kBN   vocabulary columns per tile; kMT * kBN TMEM columns per accumulator set (256: two sets, 512: one)
+// kBBox rows of one TMA box of W (kBN for the tensor-bound shape; 32 for decode shapes, whose
+//       vocabulary ranges end on 32-column boundaries so that all SMs get equal shares)
+template <bool kTf32, int kMT, int kBN, int kBBox, int kNumStages>
 __global__ void __launch_bounds__(kLmheadThreads, 1)
 lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                       const KParams p) {
+  constexpr int kABytes = kMT * kTileM * kRowBytes;
+  constexpr int kBBytes = kBN * kRowBytes;
+  constexpr int kStageBytes = kABytes + kBBytes;
+  constexpr int kAccCols = kMT * kBN;                 // TMEM columns of one accumulator set
+  constexpr int kNumAcc = kTmemCols / kAccCols;       // 2: epilogue of tile j overlaps MMAs of tile j+1; 1 for 256 x 256 tiles
+  constexpr int kSpan = kAccCols / kEpiSplit;         // TMEM columns one epilogue warp reads per tile
+  static_assert((kAccCols == 256 || kAccCols == 512) && kBN <= 256, "accumulator sets of 256 or 512 TMEM columns");
+  static_assert(kNumStages <= kMaxStages && kBN % kBBox == 0 && kBBox % 8 == 0, "bad tile configuration");
+  static_assert(kStageBytes % 1024 == 0 && kABytes % 1024 == 0, "stages must keep 1024-byte alignment");
+
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t bar_base = smem_base + kStages * kStageBytes;
-  // barrier layout (8 bytes each): full[kStages], empty[kStages], acc_full[2], acc_empty[2]
+  const uint32_t bar_base = smem_base + kNumStages * kStageBytes;
+  // barrier layout (8 bytes each): full[kMaxStages], empty[kMaxStages], acc_full[2], acc_empty[2]
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
-  auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * kStages + a); };
-  auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * kStages + 2 + a); };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + kStages * kStageBytes + 8 * (2 * kStages + 4));
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kMaxStages + s); };
+  auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * kMaxStages + a); };
+  auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * kMaxStages + 2 + a); };
+  volatile uint32_t* tmem_slot =
+      reinterpret_cast<volatile uint32_t*>(smem_gen + kNumStages * kStageBytes + 8 * (2 * kMaxStages + 4));
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5;
@@ -132,11 +154,11 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   __syncthreads();
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < kNumStages; ++s) {
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
-    for (int a = 0; a < 2; ++a) {
+    for (int a = 0; a < kNumAcc; ++a) {
       mbar_init(acc_full_bar(a), 1);
       mbar_init(acc_empty_bar(a), 4 * kEpiSplit);
     }
@@ -156,7 +178,7 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 
   constexpr int kElemsPerStage = kTf32 ? kRowBytes / 4 : kRowBytes / 2;   // K elements per stage
   constexpr int kMmaPerStage = 4;                                         // 32 bytes of K per MMA
-  constexpr uint32_t kIdesc = umma_idesc(kTf32 ? 2u : 1u, kTileM, kTileN);
+  constexpr uint32_t kIdescNoN = umma_idesc(kTf32 ? 2u : 1u, kTileM, 0);  // N is filled in per tile
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -166,15 +188,20 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
       bool ok = true;
       for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
         const UnitCoord uc = unit_coord(u, p);
-        for (int nt = uc.n_begin; nt < uc.n_end && ok; ++nt) {
+        for (int n0 = uc.col_begin; n0 < uc.col_end && ok; n0 += kBN) {
+          const int ncols = min(kBN, uc.col_end - n0);
+          const int b_loads = (ncols + kBBox - 1) / kBBox;
+          const uint32_t tx_bytes = kABytes + b_loads * kBBox * kRowBytes;
           for (int kb = 0; kb < p.k_blocks; ++kb) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
             const uint32_t a_dst = smem_base + stage * kStageBytes;
             const uint32_t b_dst = a_dst + kABytes;
-            mbar_arrive_expect_tx(full_bar(stage), kStageBytes);
-            tma_load_2d(a_dst, &map_a, kb * kElemsPerStage, uc.m_tile * kTileM, full_bar(stage));
-            tma_load_2d(b_dst, &map_b, kb * kElemsPerStage, nt * kTileN, full_bar(stage));
-            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            mbar_arrive_expect_tx(full_bar(stage), tx_bytes);
+            tma_load_2d(a_dst, &map_a, kb * kElemsPerStage, uc.row_block * (kMT * kTileM), full_bar(stage));
+            for (int i = 0; i < b_loads; ++i)
+              tma_load_2d(b_dst + i * (kBBox * kRowBytes), &map_b, kb * kElemsPerStage, n0 + i * kBBox,
+                          full_bar(stage));
+            if (++stage == kNumStages) { stage = 0; phase ^= 1u; }
           }
         }
       }
@@ -189,34 +216,41 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
       bool ok = true;
       for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
         const UnitCoord uc = unit_coord(u, p);
-        for (int nt = uc.n_begin; nt < uc.n_end && ok; ++nt) {
+        for (int n0 = uc.col_begin; n0 < uc.col_end && ok; n0 += kBN) {
+          const int ncols = min(kBN, uc.col_end - n0);
+          const uint32_t idesc = kIdescNoN | (static_cast<uint32_t>(ncols >> 3) << 17);
           if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
           tc_fence_after_sync();
-          const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kTileN);
+          const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kAccCols);
           for (int kb = 0; kb < p.k_blocks; ++kb) {
             if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t a_src = smem_base + stage * kStageBytes;
-            const uint64_t a_desc = umma_desc_k_major_sw128(a_src);
             const uint64_t b_desc = umma_desc_k_major_sw128(a_src + kABytes);
 #pragma unroll
-            for (int k = 0; k < kMmaPerStage; ++k) {
-              // advancing K by 32 bytes inside the swizzled row = +2 in the (address >> 4) field
-              umma_ss<kTf32>(d_tmem, a_desc + 2u * k, b_desc + 2u * k, kIdesc, (kb | k) != 0 ? 1u : 0u);
+            for (int mt = 0; mt < kMT; ++mt) {
+              const uint64_t a_desc = umma_desc_k_major_sw128(a_src + mt * (kTileM * kRowBytes));
+#pragma unroll
+              for (int k = 0; k < kMmaPerStage; ++k) {
+                // advancing K by 32 bytes inside the swizzled row = +2 in the (address >> 4) field
+                umma_ss<kTf32>(d_tmem + mt * kBN, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+              }
             }
             umma_commit(empty_bar(stage));          // stage reusable once these MMAs have read it
-            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            if (++stage == kNumStages) { stage = 0; phase ^= 1u; }
           }
           if (ok) umma_commit(acc_full_bar(acc));   // accumulator complete
-          acc ^= 1;
-          if (acc == 0) acc_phase ^= 1u;
+          if (++acc == kNumAcc) { acc = 0; acc_phase ^= 1u; }
         }
       }
     }
   } else {
     // ------------------------------------------------------------------ epilogue
-    const int quad = warp & 3;                 // TMEM lanes 32*quad .. 32*quad+31
-    const int half = (warp - 2) >> 2;          // which 128 of the tile's 256 columns
+    // Warp (quad, half) reads TMEM lanes 32*quad.. and accumulator columns [half*kSpan, (half+1)*kSpan):
+    // with kMT == 1 that is one half of the tile's 256 vocabulary columns, with kMT == 2 the whole
+    // tile of row tile `half`.
+    const int quad = warp & 3;
+    const int half = (warp - 2) >> 2;
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
@@ -224,54 +258,50 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
       const UnitCoord uc = unit_coord(u, p);
       RowState st;
       st.init();
-      for (int nt = uc.n_begin; nt < uc.n_end; ++nt) {
+      for (int n0 = uc.col_begin; n0 < uc.col_end; n0 += kBN) {
         ok = __all_sync(0xffffffffu, mbar_wait(acc_full_bar(acc), acc_phase, abort_flag));
         if (!ok) break;
         tc_fence_after_sync();
-        const int col0 = nt * kTileN + half * (kTileN / kEpiSplit);
+        const int ncols = min(min(kBN, uc.col_end - n0), p.V - n0);      // tile columns that exist
+        const int cols_valid = (kMT == 1) ? min(kSpan, ncols - half * kSpan) : ncols;   // of this warp's span
+        const int npieces = cols_valid > 0 ? (cols_valid + 31) >> 5 : 0;
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
-                               static_cast<uint32_t>(acc * kTileN + half * (kTileN / kEpiSplit));
-        static_assert(kTileN / kEpiSplit == 128, "epilogue is written for 128 columns per warp and tile");
-        const int cols_left = p.V - col0;         // columns of this warp's range that exist (may be <= 0)
+                               static_cast<uint32_t>(acc * kAccCols + half * kSpan);
+        auto release = [&]() {
+          // every read of the accumulator by this warp has completed: hand it back to the MMA warp
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+        };
         uint32_t bufA[32], bufB[32];
-        if (cols_left >= 128) {
-          // software pipeline: the load of piece c+1 is in flight while piece c is folded
+        if (npieces == 0) {
+          release();
+        } else {
+          // software pipeline: the load of piece i+1 is in flight while piece i is folded
           tmem_ld_32(taddr, bufA);
           tmem_ld_wait(bufA);
-          tmem_ld_32(taddr + 32, bufB);
-          st.fold<false>(bufA, 32);
-          tmem_ld_wait(bufB);
-          tmem_ld_32(taddr + 64, bufA);
-          st.fold<false>(bufB, 32);
-          tmem_ld_wait(bufA);
-          tmem_ld_32(taddr + 96, bufB);
-          st.fold<false>(bufA, 32);
-          tmem_ld_wait(bufB);
-          // every read of the accumulator has completed: hand it back before the last fold
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(acc_empty_bar(acc));
-          st.fold<false>(bufB, 32);
-        } else {
-          for (int c = 0; c < 4 && c * 32 < cols_left; ++c) {
-            tmem_ld_32(taddr + c * 32, bufA);
-            tmem_ld_wait(bufA);
-            st.fold<true>(bufA, min(32, cols_left - c * 32));
+          for (int pc = 0; pc < npieces; pc += 2) {
+            const bool has1 = pc + 1 < npieces;
+            if (has1) tmem_ld_32(taddr + (pc + 1) * 32, bufB); else release();
+            st.fold_n(bufA, cols_valid - pc * 32);
+            if (has1) {
+              tmem_ld_wait(bufB);
+              const bool has2 = pc + 2 < npieces;
+              if (has2) tmem_ld_32(taddr + (pc + 2) * 32, bufA); else release();
+              st.fold_n(bufB, cols_valid - (pc + 1) * 32);
+              if (has2) tmem_ld_wait(bufA);
+            }
           }
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(acc_empty_bar(acc));
         }
-        acc ^= 1;
-        if (acc == 0) acc_phase ^= 1u;
+        if (++acc == kNumAcc) { acc = 0; acc_phase ^= 1u; }
       }
       if (ok) {
-        const int64_t row = static_cast<int64_t>(uc.m_tile) * kTileM + quad * 32 + lane;
-        const int slot = uc.chunk * kEpiSplit + half;
-        float* dst = p.partials + static_cast<int64_t>(slot) * 3 * p.rows_pad + row;
+        const int64_t row = (static_cast<int64_t>(uc.row_block) * kMT + (kMT == 1 ? 0 : half)) * kTileM + quad * 32 + lane;
+        const int slot = (kMT == 1) ? uc.chunk * kEpiSplit + half : uc.chunk;
+        float* dst = p.partials + (row * p.slots + slot) * 3;
         dst[0] = st.m;
-        dst[p.rows_pad] = (st.s[0] + st.s[1]) + (st.s[2] + st.s[3]);
-        dst[2 * p.rows_pad] = (st.t[0] + st.t[1]) + (st.t[2] + st.t[3]);
+        dst[1] = (st.s[0] + st.s[1]) + (st.s[2] + st.s[3]);
+        dst[2] = (st.t[0] + st.t[1]) + (st.t[2] + st.t[3]);
       }
     }
   }
@@ -292,50 +322,103 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   }
 }
 
+constexpr int smem_bytes_for(int mt, int bn, int stages) {
+  return stages * (mt * kTileM * kRowBytes + bn * kRowBytes) + kBarrierBytes + 1024;   // + slack for alignment
+}
+
+// The three shapes the host chooses from.
+struct Shape { int mt, bn, bbox, stages, col_gran; };
+constexpr Shape kShapePrompt = {1, 256, 256, 4, 256};   // tensor-bound: many row tiles
+constexpr Shape kShapeDecode1 = {1, 256, 32, 4, 32};    // <= 128 rows: W streamed once, 32-column balance
+constexpr Shape kShapeDecode2 = {2, 256, 32, 3, 32};    // 129..256 rows: both row tiles share each W tile
+
+const Shape& shape_of(int variant) {
+  return variant == 1 ? kShapeDecode1 : (variant == 2 ? kShapeDecode2 : kShapePrompt);
+}
+
+template <bool kTf32, int kMT, int kBN, int kBBox, int kNumStages>
+cudaError_t launch_shape(const LmheadPlan& plan, const CUtensorMap* a, const CUtensorMap* b, const KParams& p,
+                         cudaStream_t stream) {
+  auto kernel = lmhead_entropy_kernel<kTf32, kMT, kBN, kBBox, kNumStages>;
+  kernel<<<plan.grid, kLmheadThreads, smem_bytes_for(kMT, kBN, kNumStages), stream>>>(*a, *b, p);
+  return cudaGetLastError();
+}
+
+template <bool kTf32, int kMT, int kBN, int kBBox, int kNumStages>
+cudaError_t prepare_shape() {
+  auto kernel = lmhead_entropy_kernel<kTf32, kMT, kBN, kBBox, kNumStages>;
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              smem_bytes_for(kMT, kBN, kNumStages));
+}
+
+// One entry per Shape above (template arguments must be literals).
+#define EGTP_SHAPE_PROMPT 1, 256, 256, 4
+#define EGTP_SHAPE_DECODE1 1, 256, 32, 4
+#define EGTP_SHAPE_DECODE2 2, 256, 32, 3
+static_assert(kShapePrompt.mt == 1 && kShapePrompt.bn == 256 && kShapePrompt.bbox == 256 && kShapePrompt.stages == 4, "");
+static_assert(kShapeDecode1.mt == 1 && kShapeDecode1.bn == 256 && kShapeDecode1.bbox == 32 && kShapeDecode1.stages == 4, "");
+static_assert(kShapeDecode2.mt == 2 && kShapeDecode2.bn == 256 && kShapeDecode2.bbox == 32 && kShapeDecode2.stages == 3, "");
+
 }  // namespace
 
 LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity) {
   LmheadPlan pl{};
-  pl.m_tiles = static_cast<int>((T + kTileM - 1) / kTileM);
-  pl.n_tiles = (V + kTileN - 1) / kTileN;
-  pl.rows_pad = static_cast<int64_t>(pl.m_tiles) * kTileM;
+  pl.variant = T <= kTileM ? 1 : (T <= 2 * kTileM ? 2 : 0);
+  const Shape& sh = shape_of(pl.variant);
+  pl.rows_per_block = sh.mt * kTileM;
+  pl.tile_cols = sh.bn;
+  pl.b_box_rows = sh.bbox;
+  pl.col_gran = sh.col_gran;
+  pl.row_blocks = static_cast<int>((T + pl.rows_per_block - 1) / pl.rows_per_block);
+  pl.n_groups = (V + sh.col_gran - 1) / sh.col_gran;
+  pl.rows_pad = static_cast<int64_t>(pl.row_blocks) * pl.rows_per_block;
   pl.k_blocks = static_cast<int>((static_cast<int64_t>(d) * elem_bytes + kRowBytes - 1) / kRowBytes);
-  pl.smem_bytes = kSmemBytes;
-  const int64_t tiles = static_cast<int64_t>(pl.m_tiles) * pl.n_tiles;
-  pl.grid = static_cast<int>(std::min<int64_t>(num_sms, tiles));
-  // Units are dealt round-robin to the CTAs, so the step takes ceil(units / grid) rounds of
-  // ceil(n_tiles / S) tiles.  Take the smallest S whose makespan is within 2 % of the best
-  // reachable one (fewer chunks = fewer partials to write and merge).
-  int64_t s_cap = std::max<int64_t>(1, slot_row_capacity / (pl.rows_pad * kEpiSplit));
-  const int s_max = static_cast<int>(std::min<int64_t>(pl.n_tiles, s_cap));
-  auto makespan = [&](int S) {
-    const int64_t units = static_cast<int64_t>(pl.m_tiles) * S;
-    const int64_t rounds = (units + pl.grid - 1) / pl.grid;
-    return rounds * ((pl.n_tiles + S - 1) / S);
-  };
-  int64_t best = makespan(1);
-  for (int S = 2; S <= s_max; ++S) best = std::min(best, makespan(S));
-  int pick = 1;
-  for (int S = 1; S <= s_max; ++S) {
-    if (makespan(S) * 100 <= best * 102) { pick = S; break; }
+  pl.smem_bytes = smem_bytes_for(sh.mt, sh.bn, sh.stages);
+  const int slots_per_chunk = sh.mt == 1 ? kEpiSplit : 1;
+  const int64_t s_cap = std::max<int64_t>(1, slot_row_capacity / (pl.rows_pad * slots_per_chunk));
+  const int s_max = static_cast<int>(std::min<int64_t>(pl.n_groups, s_cap));
+  if (pl.variant == 0) {
+    pl.grid = static_cast<int>(std::min<int64_t>(num_sms, static_cast<int64_t>(pl.row_blocks) * pl.n_groups));
+    // Units are dealt round-robin to the CTAs, so the step takes ceil(units / grid) rounds of
+    // ceil(n_tiles / S) tiles.  Take the smallest S whose makespan is within 2 % of the best
+    // reachable one (fewer chunks = fewer partials to write and merge).
+    auto makespan = [&](int S) {
+      const int64_t units = static_cast<int64_t>(pl.row_blocks) * S;
+      const int64_t rounds = (units + pl.grid - 1) / pl.grid;
+      return rounds * ((pl.n_groups + S - 1) / S);
+    };
+    int64_t best = makespan(1);
+    for (int S = 2; S <= s_max; ++S) best = std::min(best, makespan(S));
+    int pick = 1;
+    for (int S = 1; S <= s_max; ++S) {
+      if (makespan(S) * 100 <= best * 102) { pick = S; break; }
+    }
+    pl.chunks = pick;
+  } else {
+    // One row block: one vocabulary range per SM, ranges differ by at most 32 columns.
+    pl.chunks = std::max(1, std::min(s_max, num_sms));
+    pl.grid = pl.chunks;
   }
-  pl.chunks = pick;
-  pl.slots = pick * kEpiSplit;
-  // Row tiles that sweep the vocabulary together: enough of them that a W tile fetched from HBM
-  // is shared by many CTAs, few enough that their hidden tiles (re-read per vocabulary tile) stay in L2.
-  const int64_t a_tile_bytes = static_cast<int64_t>(kTileM) * d * elem_bytes;
-  int gm = static_cast<int>(std::max<int64_t>(1, (48ll << 20) / std::max<int64_t>(1, a_tile_bytes)));
-  gm = std::min(gm, pl.m_tiles);
+  pl.slots = pl.chunks * slots_per_chunk;
+  // Row blocks that sweep the vocabulary together: enough of them that a W tile fetched from HBM
+  // is shared by many CTAs, few enough that their hidden tiles (re-read per vocabulary tile) stay in
+  // L2 while W streams through it (measured: about 8 MB of hidden tiles per group is the sweet spot).
+  const int64_t a_tile_bytes = static_cast<int64_t>(pl.rows_per_block) * d * elem_bytes;
+  int gm = static_cast<int>(std::max<int64_t>(1, (8ll << 20) / std::max<int64_t>(1, a_tile_bytes)));
+  gm = std::min(gm, pl.row_blocks);
   gm = std::min(gm, std::max(1, pl.grid));
-  pl.group_m = gm;
+  pl.group_rb = gm;
   return pl;
 }
 
 cudaError_t lmhead_prepare_device() {
-  cudaError_t err = cudaFuncSetAttribute(lmhead_entropy_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kSmemBytes);
-  if (err != cudaSuccess) return err;
-  return cudaFuncSetAttribute(lmhead_entropy_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  cudaError_t e;
+  if ((e = prepare_shape<false, EGTP_SHAPE_PROMPT>()) != cudaSuccess) return e;
+  if ((e = prepare_shape<false, EGTP_SHAPE_DECODE1>()) != cudaSuccess) return e;
+  if ((e = prepare_shape<false, EGTP_SHAPE_DECODE2>()) != cudaSuccess) return e;
+  if ((e = prepare_shape<true, EGTP_SHAPE_PROMPT>()) != cudaSuccess) return e;
+  if ((e = prepare_shape<true, EGTP_SHAPE_DECODE1>()) != cudaSuccess) return e;
+  return prepare_shape<true, EGTP_SHAPE_DECODE2>();
 }
 
 cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const CUtensorMap* map_hidden,
@@ -343,22 +426,29 @@ cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const CUten
                                   int32_t* status, cudaStream_t stream) {
   (void)T;
   KParams p{};
-  p.m_tiles = plan.m_tiles;
-  p.n_tiles = plan.n_tiles;
+  p.row_blocks = plan.row_blocks;
   p.chunks = plan.chunks;
-  p.group_m = plan.group_m;
+  p.group_rb = plan.group_rb;
   p.k_blocks = plan.k_blocks;
-  p.total_units = plan.m_tiles * plan.chunks;
+  p.n_groups = plan.n_groups;
+  p.col_gran = plan.col_gran;
+  p.total_units = plan.row_blocks * plan.chunks;
   p.V = V;
-  p.rows_pad = plan.rows_pad;
+  p.slots = plan.slots;
   p.partials = partials;
   p.status = status;
   if (tf32) {
-    lmhead_entropy_kernel<true><<<plan.grid, kLmheadThreads, kSmemBytes, stream>>>(*map_hidden, *map_w, p);
-  } else {
-    lmhead_entropy_kernel<false><<<plan.grid, kLmheadThreads, kSmemBytes, stream>>>(*map_hidden, *map_w, p);
+    switch (plan.variant) {
+      case 1: return launch_shape<true, EGTP_SHAPE_DECODE1>(plan, map_hidden, map_w, p, stream);
+      case 2: return launch_shape<true, EGTP_SHAPE_DECODE2>(plan, map_hidden, map_w, p, stream);
+      default: return launch_shape<true, EGTP_SHAPE_PROMPT>(plan, map_hidden, map_w, p, stream);
+    }
   }
-  return cudaGetLastError();
+  switch (plan.variant) {
+    case 1: return launch_shape<false, EGTP_SHAPE_DECODE1>(plan, map_hidden, map_w, p, stream);
+    case 2: return launch_shape<false, EGTP_SHAPE_DECODE2>(plan, map_hidden, map_w, p, stream);
+    default: return launch_shape<false, EGTP_SHAPE_PROMPT>(plan, map_hidden, map_w, p, stream);
+  }
 }
 
 }  // namespace egtp

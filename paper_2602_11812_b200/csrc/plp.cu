@@ -4,11 +4,15 @@
 //   m = max_i H_i/alpha,  s = sum_i exp(H_i/alpha - m),  acc = sum_i exp(H_i/alpha - m) h_i,
 // which one new token (entropy H', hidden h') updates to
 //   m' = max(m, H'/alpha), s' = s e^(m-m') + e^(H'/alpha-m'), acc' = acc e^(m-m') + e^(H'/alpha-m') h',
-// and z = acc'/s'.  HBM-bound (acc read + write, hidden read, z write): one block per live row.
+// and z = acc'/s'.  H' is merged here from the LM-head kernel's partials (no separate launch).
+// HBM-bound (acc read + write, hidden read, z write): one block per live row.
 #include "kernels.h"
+#include "entropy_merge.cuh"
 #include "../../include/egtp.h"
 
 #include <cuda_bf16.h>
+
+#include <algorithm>
 
 namespace egtp {
 
@@ -34,14 +38,16 @@ __device__ __forceinline__ void load8<float>(const float* p, float (&v)[8]) {
   v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
 }
 
+constexpr int kPlpMaxThreads = 1024;
+
 template <typename T>
-__global__ void __launch_bounds__(256)
-plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* __restrict__ Hstep,
-                  const int32_t* __restrict__ slot_ids, const int32_t* __restrict__ reset_src,
-                  const float* __restrict__ src_m, const float* __restrict__ src_s,
-                  const float* __restrict__ src_pooled, int n_src, int d, int num_slots, float inv_alpha,
-                  float* __restrict__ st_m, float* __restrict__ st_s, float* __restrict__ st_acc,
-                  float* __restrict__ z, int64_t ldz, int32_t* status) {
+__global__ void __launch_bounds__(kPlpMaxThreads)
+plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* __restrict__ partials, int slots,
+                  float* __restrict__ Hstep_out, const int32_t* __restrict__ slot_ids,
+                  const int32_t* __restrict__ reset_src, const float* __restrict__ src_m,
+                  const float* __restrict__ src_s, const float* __restrict__ src_pooled, int n_src, int d,
+                  int num_slots, float inv_alpha, float* __restrict__ st_m, float* __restrict__ st_s,
+                  float* __restrict__ st_acc, float* __restrict__ z, int64_t ldz, int32_t* status) {
   if (*status != 0) return;
   const int i = blockIdx.x;
   const int slot = slot_ids ? slot_ids[i] : i;
@@ -63,7 +69,23 @@ plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* _
     m_old = src_m[rs]; s_old = src_s[rs];
     acc_src = src_pooled + static_cast<int64_t>(rs) * d; acc_scale_in = s_old;
   }
-  const float a = Hstep[i] * inv_alpha;
+  if (!(s_old > 0.f)) acc_src = nullptr;    // an empty sequence carries nothing over
+  float* acc_dst = st_acc + static_cast<int64_t>(slot) * d;
+  const T* hrow = hidden_step + static_cast<int64_t>(i) * ldh;
+  float* zrow = z + static_cast<int64_t>(i) * ldz;
+
+  // first pass of loads is issued before the entropy merge so that both latencies overlap
+  int col = threadIdx.x * 8;
+  float h[8], acc[8];
+  const bool first = col < d;
+  if (first) {
+    load8<T>(hrow + col, h);
+    if (acc_src != nullptr) load8<float>(acc_src + col, acc);
+  }
+  // Eq. 2 for this row: every warp merges the row's partials (same value in all of them)
+  const float H_new = merge_partials_warp(partials + static_cast<int64_t>(i) * slots * 3, slots, threadIdx.x & 31);
+  if (threadIdx.x == 0 && Hstep_out != nullptr) Hstep_out[i] = H_new;
+  const float a = H_new * inv_alpha;
   const float m_new = fmaxf(m_old, a);
   const float carry = (s_old > 0.f) ? expf(m_old - m_new) : 0.f;
   const float e = expf(a - m_new);
@@ -71,17 +93,12 @@ plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* _
   const float inv_s = 1.f / s_new;
   const float acc_factor = carry * acc_scale_in;
   __syncthreads();   // every thread has read the old state before anyone overwrites it
-  float* acc_dst = st_acc + static_cast<int64_t>(slot) * d;
-  const T* hrow = hidden_step + static_cast<int64_t>(i) * ldh;
-  float* zrow = z + static_cast<int64_t>(i) * ldz;
-  for (int col = threadIdx.x * 8; col < d; col += blockDim.x * 8) {
-    float h[8], acc[8];
-    load8<T>(hrow + col, h);
-    if (acc_src != nullptr && acc_factor != 0.f) {
-      const float4 p0 = *reinterpret_cast<const float4*>(acc_src + col);
-      const float4 p1 = *reinterpret_cast<const float4*>(acc_src + col + 4);
-      acc[0] = p0.x; acc[1] = p0.y; acc[2] = p0.z; acc[3] = p0.w;
-      acc[4] = p1.x; acc[5] = p1.y; acc[6] = p1.z; acc[7] = p1.w;
+  for (; col < d; col += blockDim.x * 8) {
+    if (col != static_cast<int>(threadIdx.x) * 8) {
+      load8<T>(hrow + col, h);
+      if (acc_src != nullptr) load8<float>(acc_src + col, acc);
+    }
+    if (acc_src != nullptr) {
 #pragma unroll
       for (int k = 0; k < 8; ++k) acc[k] = fmaf(acc[k], acc_factor, e * h[k]);
     } else {
@@ -101,17 +118,18 @@ plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* _
 
 }  // namespace
 
-cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, const float* Hstep,
-                              const int32_t* slot_ids, const int32_t* reset_src, const float* src_m,
+cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, const float* partials, int slots,
+                              float* Hstep_out, const int32_t* slot_ids, const int32_t* reset_src, const float* src_m,
                               const float* src_s, const float* src_pooled, int n_src, int rows, int d, int num_slots,
                               float inv_alpha, float* st_m, float* st_s, float* st_acc, float* z, int64_t ldz,
                               int32_t* status, cudaStream_t stream) {
+  const int threads = std::min(kPlpMaxThreads, std::max(32, (d / 8 + 31) / 32 * 32));
   if (bf16) {
-    plp_update_kernel<__nv_bfloat16><<<rows, 256, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(hidden_step), ldh, Hstep, slot_ids, reset_src, src_m, src_s, src_pooled,
+    plp_update_kernel<__nv_bfloat16><<<rows, threads, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(hidden_step), ldh, partials, slots, Hstep_out, slot_ids, reset_src, src_m, src_s, src_pooled,
         n_src, d, num_slots, inv_alpha, st_m, st_s, st_acc, z, ldz, status);
   } else {
-    plp_update_kernel<float><<<rows, 256, 0, stream>>>(static_cast<const float*>(hidden_step), ldh, Hstep, slot_ids,
+    plp_update_kernel<float><<<rows, threads, 0, stream>>>(static_cast<const float*>(hidden_step), ldh, partials, slots, Hstep_out, slot_ids,
                                                        reset_src, src_m, src_s, src_pooled, n_src, d, num_slots,
                                                        inv_alpha, st_m, st_s, st_acc, z, ldz, status);
   }

@@ -2,6 +2,7 @@
 // entropy-weighted ragged pooling (Eq. 4).  HBM-bound work: plain coalesced 16-byte loads,
 // fp32 accumulation, warp-shuffle / block reductions, no floating-point atomics.
 #include "kernels.h"
+#include "entropy_merge.cuh"
 #include "../../include/egtp.h"
 
 #include <cuda_bf16.h>
@@ -9,9 +10,6 @@
 namespace egtp {
 
 namespace {
-
-constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
 
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
@@ -48,32 +46,26 @@ __global__ void validate_offsets_kernel(const int32_t* __restrict__ off, int B, 
 }
 
 // --------------------------------------------------------------------------- Eq. 2: merge
-// One thread per token: combines the per-slot (m, s, t2) partials of the LM-head kernel,
-// H = ln S - ln2 * T2 / S.  Also writes the token's prompt index and clears its weight.
-__global__ void entropy_merge_kernel(const float* __restrict__ partials, int slots, int64_t rows_pad, int64_t T,
+// One warp per token: lanes stride over the token's (m, s, t2) partials (contiguous in memory),
+// fold them in a fixed order, then combine across lanes: H = ln S - ln2 * T2 / S.
+// Also writes the token's prompt index and clears its weight.
+__global__ void entropy_merge_kernel(const float* __restrict__ partials, int slots, int64_t T,
                                      float* __restrict__ H, const int32_t* __restrict__ off, int B,
                                      int32_t* __restrict__ seg_id, float* __restrict__ weights,
                                      const int32_t* __restrict__ status) {
   if (*status != 0) return;
-  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int lane = threadIdx.x & 31;
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (i >= T) return;
-  float M = kNegBig;
-  for (int j = 0; j < slots; ++j) M = fmaxf(M, partials[(static_cast<int64_t>(j) * 3) * rows_pad + i]);
-  float S = 0.f, T2 = 0.f;
-  for (int j = 0; j < slots; ++j) {
-    const float* pj = partials + (static_cast<int64_t>(j) * 3) * rows_pad + i;
-    const float m = pj[0], s = pj[rows_pad], t2 = pj[2 * rows_pad];
-    const float dm = (m - M) * kLog2e;
-    const float r = exp2f(dm);
-    S = fmaf(s, r, S);
-    T2 += r * fmaf(dm, s, t2);
-  }
-  H[i] = logf(S) - kLn2 * T2 / S;
-  if (weights != nullptr) weights[i] = 0.f;
-  if (seg_id != nullptr) {
-    int sid = -1;
-    if (B > 0 && i >= off[0] && i < off[B]) sid = upper_segment(off, B, i);
-    seg_id[i] = sid;
+  const float h = merge_partials_warp(partials + i * slots * 3, slots, lane);
+  if (lane == 0) {
+    H[i] = h;
+    if (weights != nullptr) weights[i] = 0.f;
+    if (seg_id != nullptr) {
+      int sid = -1;
+      if (B > 0 && i >= off[0] && i < off[B]) sid = upper_segment(off, B, i);
+      seg_id[i] = sid;
+    }
   }
 }
 
@@ -260,13 +252,13 @@ cudaError_t launch_validate_offsets(const int32_t* offsets, int B, int64_t T, in
   return cudaGetLastError();
 }
 
-cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t rows_pad, int64_t T, float* H,
+cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t T, float* H,
                                  const int32_t* offsets, int B, int32_t* seg_id_out, float* weights_zero,
                                  const int32_t* status, cudaStream_t stream) {
-  const int threads = 256;
-  const unsigned blocks = static_cast<unsigned>((T + threads - 1) / threads);
-  entropy_merge_kernel<<<blocks, threads, 0, stream>>>(partials, slots, rows_pad, T, H, offsets, B, seg_id_out,
-                                                       weights_zero, status);
+  const int threads = 256, rows_per_block = threads / 32;
+  const unsigned blocks = static_cast<unsigned>((T + rows_per_block - 1) / rows_per_block);
+  entropy_merge_kernel<<<blocks, threads, 0, stream>>>(partials, slots, T, H, offsets, B, seg_id_out, weights_zero,
+                                                       status);
   return cudaGetLastError();
 }
 

@@ -238,12 +238,14 @@ def make_head(seed: int, d: int, m_h: int, d_out: int, dtype: str, mode: int = H
 
 def make_egtp(name: str, seed: int, lengths, d: int, V: int, dtype: str, m_h: int, d_out: int = 1,
               mode: int = HEAD_SCALAR, outlier_frac: float = 0.0, outlier_gain: float = 1.0,
-              alpha: float = 1.0) -> EgtpWorkload:
-    """Streams: seed*1000 + {1 hidden, 2 W, 3 head}."""
+              alpha: float = 1.0, W: Optional[np.ndarray] = None) -> EgtpWorkload:
+    """Streams: seed*1000 + {1 hidden, 2 W, 3 head}. A ready-made LM head `W` [V, d] may be passed in."""
     offsets = offsets_from_lengths(lengths)
     T = int(offsets[-1])
     hidden = make_hidden(seed * 1000 + 1, T, d, dtype, outlier_frac, outlier_gain)
-    W = make_lm_head(seed * 1000 + 2, V, d, dtype)
+    if W is None:
+        W = make_lm_head(seed * 1000 + 2, V, d, dtype)
+    assert W.shape == (V, d)
     head = make_head(seed * 1000 + 3, d, m_h, d_out, dtype, mode)
     return EgtpWorkload(name=name, dtype=dtype, hidden=hidden, offsets=offsets, W=W, head=head,
                         alpha=alpha, seed=seed)
@@ -299,11 +301,11 @@ def config_mid(seed: int = 1, B: int = 32, d: int = 2048, V: int = 151936, m_h: 
 
 
 def config_long(seed: int = 1, B: int = 64, d: int = 4096, V: int = 151936, m_h: int = 1024,
-                max_len: int = 8192) -> EgtpWorkload:
+                max_len: int = 8192, W: Optional[np.ndarray] = None) -> EgtpWorkload:
     """64 prompts, lengths Pareto(1.2, x_m = 128) clipped to [128, 8192]; packed ragged rows."""
     lengths = lengths_pareto(seed * 1000, B, 1.2, 128, 128, max_len)
     return make_egtp("egtp_long", seed, lengths, d=d, V=V, dtype="bf16", m_h=m_h,
-                     outlier_frac=0.01, outlier_gain=20.0)
+                     outlier_frac=0.01, outlier_gain=20.0, W=W)
 
 
 def config_plp_decode(seed: int = 4, slots: int = 256, steps: int = 512, d: int = 4096,
