@@ -172,6 +172,7 @@ def run_mine(args):
     from paper_2602_11812_b200 import binding as egtp
     from paper_2602_11812_b200 import inputs as gen
     from paper_2602_11812_b200 import device as gu
+    from paper_2602_11812_b200 import shard
 
     rank, local_rank, world = dist_env()
     if not torch.cuda.is_available():
@@ -230,12 +231,7 @@ def run_mine(args):
     egtp.egtp_profile_enable(ctx, False)
     assert int(status.item()) == 0, egtp.status_string(int(status.item()))
 
-    tmax = torch.tensor([ms], device="cuda", dtype=torch.float64)
-    ttok = torch.tensor([float(T)], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        dist.all_reduce(ttok, op=dist.ReduceOp.SUM)
-    ms_max, tokens_all = float(tmax.item()), float(ttok.item())
+    ms_max, tokens_all = shard.reduce_time_and_work(ms, float(T), torch.device("cuda", local_rank))
     value = tokens_all * steps / (ms_max * 1e-3)
 
     # ---- end to end through the host-buffer entry point (pinned host memory in, result out)
@@ -253,10 +249,8 @@ def run_mine(args):
         egtp.egtp_predict_host(ctx, lm, head.c, hidden_host, off_host, B, T, wl.alpha, y_host, None, st_host)
     e1.record()
     sync_all()
-    e2e_ms = torch.tensor([e0.elapsed_time(e1)], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
-    e2e_value = tokens_all * e2e_steps / (float(e2e_ms.item()) * 1e-3)
+    e2e_ms_max, _ = shard.reduce_time_and_work(e0.elapsed_time(e1), float(T), torch.device("cuda", local_rank))
+    e2e_value = tokens_all * e2e_steps / (e2e_ms_max * 1e-3)
     h2d = hidden_host.numel() * 2 + off_host.numel() * 4
     d2h = y_host.numel() * 4 + 4
 
