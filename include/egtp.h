@@ -223,6 +223,14 @@ EGTP_API int plp_step_host(egtp_ctx* ctx, plp_state* st, const egtp_lm_head* lm,
 EGTP_API int egtp_head_forward_static(const egtp_head* head, const float* z, int64_t ldz, int32_t rows,
                                       float* y_out, float* phat_out, void* stream);
 
+/* Tile shape of the LM-head kernel.  EGTP_LMHEAD_AUTO (default): one CTA per SM, 128 x 256 tiles for
+ * prompt batches and the two decode shapes for <= 256 rows.  EGTP_LMHEAD_CTA_PAIRS: clusters of two
+ * CTAs work on 256 x 256 tiles with tcgen05.mma.cta_group::2 wherever more than 128 rows are given
+ * (each SM then loads half as many operand bytes per flop).  Both produce the same entropies up to
+ * summation order; on a power-capped B200 AUTO measured equal or faster, so it is the default. */
+enum { EGTP_LMHEAD_AUTO = 0, EGTP_LMHEAD_CTA_PAIRS = 1 };
+EGTP_API int egtp_set_lmhead_mode(egtp_ctx* ctx, int mode);
+
 /* Per-kernel timing. With profiling on, every kernel launch of this context is bracketed by
  * CUDA events on its own stream.  egtp_profile_read synchronises the device, adds up the
  * elapsed milliseconds and launch counts per kernel since the last read and clears them.

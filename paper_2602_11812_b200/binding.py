@@ -24,6 +24,7 @@ EGTP_ERR_BAD_SLOT = -7
 EGTP_F32, EGTP_BF16 = 0, 1
 EGTP_HEAD_SCALAR, EGTP_HEAD_BINS = 0, 1
 PLP_RESET_KEEP, PLP_RESET_EMPTY = -2, -1
+EGTP_LMHEAD_AUTO, EGTP_LMHEAD_CTA_PAIRS = 0, 1
 KERNEL_IDS = ["validate_offsets", "lmhead_entropy", "entropy_merge", "segment_weights", "pool",
               "pool_combine", "head_hidden", "head_out", "plp_update"]
 EGTP_NUM_KERNELS = len(KERNEL_IDS)
@@ -33,7 +34,7 @@ EXPORTED_SYMBOLS = [
     "egtp_create", "egtp_destroy", "egtp_status_string", "egtp_workspace_bytes", "egtp_predict",
     "egtp_predict_host", "plp_state_create", "plp_state_destroy", "plp_state_export", "plp_state_import",
     "plp_step", "plp_step_host", "egtp_profile_enable", "egtp_profile_read", "egtp_kernel_name",
-    "egtp_launch_count", "egtp_lmhead_plan", "egtp_head_forward_static",
+    "egtp_launch_count", "egtp_lmhead_plan", "egtp_head_forward_static", "egtp_set_lmhead_mode",
 ]
 
 
@@ -80,6 +81,7 @@ def load() -> C.CDLL:
     lib.egtp_launch_count.restype = i64
     lib.egtp_lmhead_plan.argtypes = [vp, i64, i32, i32, i32, P(i32)]
     lib.egtp_profile_enable.argtypes = [vp, C.c_int]
+    lib.egtp_set_lmhead_mode.argtypes = [vp, C.c_int]
     lib.egtp_profile_read.argtypes = [vp, P(C.c_double), P(i64)]
     lib.egtp_predict.argtypes = [vp, P(egtp_lm_head), P(egtp_head), vp, i64, vp, i32, i64, f32,
                                  vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -181,6 +183,10 @@ def egtp_lmhead_plan(ctx: int, T: int, d: int, V: int, dtype: int) -> dict:
     _check(load().egtp_lmhead_plan(ctx, T, d, V, dtype, info), "egtp_lmhead_plan")
     keys = ["grid", "row_blocks", "rows_per_block", "chunks", "slots", "tile_cols", "k_blocks", "smem_bytes"]
     return dict(zip(keys, list(info)))
+
+
+def egtp_set_lmhead_mode(ctx: int, mode: int):
+    _check(load().egtp_set_lmhead_mode(ctx, mode), "egtp_set_lmhead_mode")
 
 
 def egtp_profile_enable(ctx: int, on: bool):

@@ -50,6 +50,7 @@ struct egtp_ctx {
   int64_t bytes = 0;
 
   // bookkeeping
+  int lmhead_mode = EGTP_LMHEAD_AUTO;
   int64_t launches = 0;
   bool profiling = false;
   std::vector<EventPair> pending;
@@ -178,10 +179,10 @@ HeadArgs head_args(const egtp_head* h) {
 // Eq. 2 for `rows` rows, first part: the LM-head kernel leaves per-slot partials in the workspace.
 int run_lmhead(egtp_ctx* c, const egtp_lm_head* lm, const void* hidden, int64_t ldh, int64_t rows, int32_t* status,
                cudaStream_t stream, LmheadPlan* plan_out) {
-  const LmheadPlan plan = make_lmhead_plan(rows, lm->d, lm->V, elem_bytes(lm->dtype), c->num_sms, c->slot_row_capacity);
+  const LmheadPlan plan = make_lmhead_plan(rows, lm->d, lm->V, elem_bytes(lm->dtype), c->num_sms, c->slot_row_capacity, c->lmhead_mode);
   if (plan.rows_pad * plan.slots > c->slot_row_capacity) return EGTP_ERR_CAPACITY;
   CUtensorMap map_a, map_b;
-  int rc = make_tensor_map(c, &map_a, hidden, lm->dtype, rows, lm->d, ldh, plan.rows_per_block);
+  int rc = make_tensor_map(c, &map_a, hidden, lm->dtype, rows, lm->d, ldh, plan.a_box_rows);
   if (rc != EGTP_OK) return rc;
   rc = make_tensor_map(c, &map_b, lm->W, lm->dtype, lm->V, lm->d, lm->ldw, plan.b_box_rows);
   if (rc != EGTP_OK) return rc;
@@ -302,9 +303,15 @@ int64_t egtp_launch_count(const egtp_ctx* c) { return c ? c->launches : 0; }
 
 int egtp_lmhead_plan(const egtp_ctx* c, int64_t T, int32_t d, int32_t V, int32_t dtype, int32_t info[8]) {
   if (!c || !info || T <= 0 || d <= 0 || V <= 0) return EGTP_ERR_INVALID_ARG;
-  const LmheadPlan p = make_lmhead_plan(T, d, V, elem_bytes(dtype), c->num_sms, c->slot_row_capacity);
+  const LmheadPlan p = make_lmhead_plan(T, d, V, elem_bytes(dtype), c->num_sms, c->slot_row_capacity, c->lmhead_mode);
   info[0] = p.grid; info[1] = p.row_blocks; info[2] = p.rows_per_block; info[3] = p.chunks;
   info[4] = p.slots; info[5] = p.tile_cols; info[6] = p.k_blocks; info[7] = p.smem_bytes;
+  return EGTP_OK;
+}
+
+int egtp_set_lmhead_mode(egtp_ctx* c, int mode) {
+  if (!c || (mode != EGTP_LMHEAD_AUTO && mode != EGTP_LMHEAD_CTA_PAIRS)) return EGTP_ERR_INVALID_ARG;
+  c->lmhead_mode = mode;
   return EGTP_OK;
 }
 

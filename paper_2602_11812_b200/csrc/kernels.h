@@ -17,10 +17,11 @@ constexpr int kEpiSplit = 2;       // epilogue warps per TMEM lane quadrant (col
 constexpr int kLmheadThreads = (2 + 4 * kEpiSplit) * 32;
 
 struct LmheadPlan {
-  int variant;        // 0 prompt shape, 1 decode <= 128 rows, 2 decode <= 256 rows
+  int variant;        // 0 prompt shape, 1 decode <= 128 rows, 2 decode <= 256 rows, 4 / 5 CTA-pair prompt / decode
+  int a_box_rows;     // rows of one TMA box of the hidden states
   int grid;           // persistent CTAs
   int row_blocks;     // ceil(T / rows_per_block)
-  int rows_per_block; // 128 or 256: rows a CTA multiplies against each W tile (box rows of the hidden map)
+  int rows_per_block; // 128 or 256: rows a CTA (or CTA pair) multiplies against each W tile
   int tile_cols;      // vocabulary columns per tile
   int b_box_rows;     // rows of one TMA box of W
   int col_gran;       // vocabulary chunks start at multiples of this many columns
@@ -35,7 +36,8 @@ struct LmheadPlan {
 
 // Picks chunks / grouping for T rows; slot_limit bounds chunks * kEpiSplit * rows_pad by the
 // partial buffer's capacity (in rows x slots).
-LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity);
+LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity,
+                            int mode);
 
 // Opts the kernels into their dynamic shared-memory size on the current device (once per device).
 cudaError_t lmhead_prepare_device();

@@ -322,17 +322,243 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// CTA-pair form: a cluster of two CTAs (two SMs) works on one 256-row x 256-column tile with
+// tcgen05.mma.cta_group::2.  Each CTA loads only its own 128 rows of the hidden states and its own
+// half of the W tile, so the bytes an SM has to pull in per flop are halved against the one-CTA
+// form (which is limited by the SM's L2 read port, not by the tensor pipe), and each CTA's TMEM
+// still holds two 128 x 256 accumulators, so the epilogue keeps overlapping the next tile's MMAs.
+//   both CTAs, warp 0   TMA producer for the CTA's own operand halves; completion bytes are counted
+//                       on the leader CTA's "full" barrier
+//   leader, warp 1      one thread issues the MMAs for both CTAs and commits to the "empty" and
+//                       "accumulator full" barriers of both CTAs
+//   both CTAs, warp 1   TMEM allocation / release (collective over the pair)
+//   both CTAs, 2..9     epilogue on the CTA's own 128 rows; arrivals go to the leader's
+//                       "accumulator empty" barrier
+// No load in this kernel is multicast; the only multicast is the arrival of tcgen05.commit.
+template <bool kTf32, int kBBox, int kNumStages>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kLmheadThreads, 1)
+lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                           const KParams p) {
+  constexpr int kBN = 256;                        // tile columns over the pair
+  constexpr int kABytes = kTileM * kRowBytes;     // this CTA's 128 rows
+  constexpr int kBBytes = (kBN / 2) * kRowBytes;  // this CTA's half of the W tile
+  constexpr int kStageBytes = kABytes + kBBytes;
+  constexpr int kAccCols = kBN;
+  constexpr int kNumAcc = kTmemCols / kAccCols;
+  constexpr int kSpan = kAccCols / kEpiSplit;
+  static_assert(kNumStages <= kMaxStages && (kBN / 2) % kBBox == 0 && kBBox % 8 == 0, "bad tile configuration");
+  static_assert(kNumAcc == 2 && kSpan == 128, "two 256-column accumulators");
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_base = smem_base + kNumStages * kStageBytes;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kMaxStages + s); };
+  auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * kMaxStages + a); };
+  auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * kMaxStages + 2 + a); };
+  volatile uint32_t* tmem_slot =
+      reinterpret_cast<volatile uint32_t*>(smem_gen + kNumStages * kStageBytes + 8 * (2 * kMaxStages + 4));
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+  volatile uint32_t* skip_flag = tmem_slot + 2;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();        // 0 = leader
+  const bool leader = rank == 0;
+  const int pair = blockIdx.x >> 1;
+  const int num_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kNumStages; ++s) {
+      mbar_init(full_bar(s), 1);            // leader: its own arrive.expect_tx (bytes of both CTAs)
+      mbar_init(empty_bar(s), 1);           // one commit arrival, delivered to both CTAs
+    }
+    for (int a = 0; a < kNumAcc; ++a) {
+      mbar_init(acc_full_bar(a), 1);                    // commit arrival, delivered to both CTAs
+      mbar_init(acc_empty_bar(a), 2 * 4 * kEpiSplit);   // leader: the epilogue warps of both CTAs
+    }
+    *abort_flag = 0u;
+    *skip_flag = (*p.status != 0) ? 1u : 0u;            // an earlier step of this call failed
+    mbar_fence_init();
+    tma_prefetch_descriptor(&map_a);
+    tma_prefetch_descriptor(&map_b);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();           // barriers of both CTAs are initialised before anyone signals across
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  // both CTAs follow the leader's reading of the status word
+  const bool skip = ld_shared_cluster_u32(map_to_cta(smem_u32(const_cast<uint32_t*>(skip_flag)), 0)) != 0u;
+
+  constexpr int kElemsPerStage = kTf32 ? kRowBytes / 4 : kRowBytes / 2;
+  constexpr int kMmaPerStage = 4;
+  constexpr uint32_t kIdescNoN = umma_idesc(kTf32 ? 2u : 1u, 2 * kTileM, 0);   // M = 256 over the pair
+
+  if (skip) {
+    // nothing to do
+  } else if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int u = pair; u < p.total_units && ok; u += num_pairs) {
+        const UnitCoord uc = unit_coord(u, p);
+        for (int n0 = uc.col_begin; n0 < uc.col_end && ok; n0 += kBN) {
+          const int ncols = min(kBN, uc.col_end - n0);
+          const int half_cols = ncols >> 1;                       // W rows this CTA supplies
+          const int b_loads = (half_cols + kBBox - 1) / kBBox;
+          const uint32_t tx_bytes = 2u * (kABytes + b_loads * kBBox * kRowBytes);   // both CTAs
+          for (int kb = 0; kb < p.k_blocks; ++kb) {
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t a_dst = smem_base + stage * kStageBytes;
+            const uint32_t b_dst = a_dst + kABytes;
+            const uint32_t full_leader = map_to_cta(full_bar(stage), 0);
+            if (leader) mbar_arrive_expect_tx(full_bar(stage), tx_bytes);
+            tma_load_2d_pair(a_dst, &map_a, kb * kElemsPerStage, uc.row_block * (2 * kTileM) + rank * kTileM,
+                             full_leader);
+            for (int i = 0; i < b_loads; ++i)
+              tma_load_2d_pair(b_dst + i * (kBBox * kRowBytes), &map_b, kb * kElemsPerStage,
+                               n0 + rank * half_cols + i * kBBox, full_leader);
+            if (++stage == kNumStages) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader only)
+    if (leader && lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int u = pair; u < p.total_units && ok; u += num_pairs) {
+        const UnitCoord uc = unit_coord(u, p);
+        for (int n0 = uc.col_begin; n0 < uc.col_end && ok; n0 += kBN) {
+          const int ncols = min(kBN, uc.col_end - n0);
+          const uint32_t idesc = kIdescNoN | (static_cast<uint32_t>(ncols >> 3) << 17);
+          if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after_sync();
+          const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kAccCols);
+          for (int kb = 0; kb < p.k_blocks; ++kb) {
+            if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t a_src = smem_base + stage * kStageBytes;
+            const uint64_t a_desc = umma_desc_k_major_sw128(a_src);
+            const uint64_t b_desc = umma_desc_k_major_sw128(a_src + kABytes);
+#pragma unroll
+            for (int k = 0; k < kMmaPerStage; ++k)
+              umma_ss_pair<kTf32>(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            umma_commit_pair(empty_bar(stage), 0x3);        // frees the stage in both CTAs
+            if (++stage == kNumStages) { stage = 0; phase ^= 1u; }
+          }
+          if (ok) umma_commit_pair(acc_full_bar(acc), 0x3); // accumulator complete in both CTAs
+          if (++acc == kNumAcc) { acc = 0; acc_phase ^= 1u; }
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (both CTAs, own rows)
+    const int quad = warp & 3;
+    const int half = (warp - 2) >> 2;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int u = pair; u < p.total_units && ok; u += num_pairs) {
+      const UnitCoord uc = unit_coord(u, p);
+      RowState st;
+      st.init();
+      for (int n0 = uc.col_begin; n0 < uc.col_end; n0 += kBN) {
+        ok = __all_sync(0xffffffffu, mbar_wait(acc_full_bar(acc), acc_phase, abort_flag));
+        if (!ok) break;
+        tc_fence_after_sync();
+        const int ncols = min(min(kBN, uc.col_end - n0), p.V - n0);
+        const int cols_valid = min(kSpan, ncols - half * kSpan);
+        const int npieces = cols_valid > 0 ? (cols_valid + 31) >> 5 : 0;
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
+                               static_cast<uint32_t>(acc * kAccCols + half * kSpan);
+        const uint32_t acc_empty_leader = map_to_cta(acc_empty_bar(acc), 0);
+        auto release = [&]() {
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+        };
+        uint32_t bufA[32], bufB[32];
+        if (npieces == 0) {
+          release();
+        } else {
+          tmem_ld_32(taddr, bufA);
+          tmem_ld_wait(bufA);
+          for (int pc = 0; pc < npieces; pc += 2) {
+            const bool has1 = pc + 1 < npieces;
+            if (has1) tmem_ld_32(taddr + (pc + 1) * 32, bufB); else release();
+            st.fold_n(bufA, cols_valid - pc * 32);
+            if (has1) {
+              tmem_ld_wait(bufB);
+              const bool has2 = pc + 2 < npieces;
+              if (has2) tmem_ld_32(taddr + (pc + 2) * 32, bufA); else release();
+              st.fold_n(bufB, cols_valid - (pc + 1) * 32);
+              if (has2) tmem_ld_wait(bufA);
+            }
+          }
+        }
+        if (++acc == kNumAcc) { acc = 0; acc_phase ^= 1u; }
+      }
+      if (ok) {
+        const int64_t row = static_cast<int64_t>(uc.row_block) * (2 * kTileM) + rank * kTileM + quad * 32 + lane;
+        const int slot = uc.chunk * kEpiSplit + half;
+        float* dst = p.partials + (row * p.slots + slot) * 3;
+        dst[0] = st.m;
+        dst[1] = (st.s[0] + st.s[1]) + (st.s[2] + st.s[3]);
+        dst[2] = (st.t[0] + st.t[1]) + (st.t[2] + st.t[3]);
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  __syncthreads();
+  if (*abort_flag != 0u) {
+    if (threadIdx.x == 0) atomicCAS(p.status, 0, EGTP_ERR_DEVICE_TIMEOUT);
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
+    __syncthreads();
+  }
+  // neither CTA may leave (and give up its shared and tensor memory) while its partner can still signal it
+  tc_fence_before_sync();
+  cluster_sync_all();
+  tc_fence_after_sync();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
+  }
+}
+
 constexpr int smem_bytes_for(int mt, int bn, int stages) {
   return stages * (mt * kTileM * kRowBytes + bn * kRowBytes) + kBarrierBytes + 1024;   // + slack for alignment
 }
 
 // The three shapes the host chooses from.
-struct Shape { int mt, bn, bbox, stages, col_gran; };
+struct Shape { int mt, bn, bbox, stages, col_gran; };   // mt = 128-row tiles per row block (2 in pair forms too)
 constexpr Shape kShapePrompt = {1, 256, 256, 4, 256};   // tensor-bound: many row tiles
 constexpr Shape kShapeDecode1 = {1, 256, 32, 4, 32};    // <= 128 rows: W streamed once, 32-column balance
 constexpr Shape kShapeDecode2 = {2, 256, 32, 3, 32};    // 129..256 rows: both row tiles share each W tile
 
+constexpr Shape kShapePairPrompt = {2, 256, 128, 6, 256};  // CTA pairs, 256 x 256 tiles
+constexpr Shape kShapePairDecode = {2, 256, 32, 6, 64};    // CTA pairs, one vocabulary range per pair
+constexpr int kPairStages = 6;
+constexpr int kPairSmemBytes = kPairStages * (kTileM * kRowBytes + 128 * kRowBytes) + kBarrierBytes + 1024;
+
 const Shape& shape_of(int variant) {
+  if (variant == 4) return kShapePairPrompt;
+  if (variant == 5) return kShapePairDecode;
   return variant == 1 ? kShapeDecode1 : (variant == 2 ? kShapeDecode2 : kShapePrompt);
 }
 
@@ -351,6 +577,38 @@ cudaError_t prepare_shape() {
                               smem_bytes_for(kMT, kBN, kNumStages));
 }
 
+template <bool kTf32, int kBBox>
+cudaError_t launch_pair(const LmheadPlan& plan, const CUtensorMap* a, const CUtensorMap* b, const KParams& p,
+                        cudaStream_t stream) {
+  auto kernel = lmhead_entropy_pair_kernel<kTf32, kBBox, kPairStages>;
+  kernel<<<plan.grid, kLmheadThreads, kPairSmemBytes, stream>>>(*a, *b, p);
+  return cudaGetLastError();
+}
+
+// CTA pairs that can be resident at once on the current device (set by lmhead_prepare_device).
+int g_pair_workers_max = 0;
+
+template <bool kTf32, int kBBox>
+cudaError_t prepare_pair(int num_sms) {
+  auto kernel = lmhead_entropy_pair_kernel<kTf32, kBBox, kPairStages>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(num_sms / 2 * 2);
+  cfg.blockDim = dim3(kLmheadThreads);
+  cfg.dynamicSmemBytes = kPairSmemBytes;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  int clusters = 0;
+  e = cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg);
+  if (e != cudaSuccess) return e;
+  g_pair_workers_max = g_pair_workers_max == 0 ? clusters : std::min(g_pair_workers_max, clusters);
+  return cudaSuccess;
+}
+
 // One entry per Shape above (template arguments must be literals).
 #define EGTP_SHAPE_PROMPT 1, 256, 256, 4
 #define EGTP_SHAPE_DECODE1 1, 256, 32, 4
@@ -361,11 +619,19 @@ static_assert(kShapeDecode2.mt == 2 && kShapeDecode2.bn == 256 && kShapeDecode2.
 
 }  // namespace
 
-LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity) {
+LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity,
+                            int mode) {
   LmheadPlan pl{};
   pl.variant = T <= kTileM ? 1 : (T <= 2 * kTileM ? 2 : 0);
+  if (mode == EGTP_LMHEAD_CTA_PAIRS) {
+    if (pl.variant == 0) pl.variant = 4;
+    if (pl.variant == 2) pl.variant = 5;
+  }
+  const bool pair = pl.variant >= 4;
+  const bool one_block = pl.variant == 1 || pl.variant == 2 || pl.variant == 5;
   const Shape& sh = shape_of(pl.variant);
   pl.rows_per_block = sh.mt * kTileM;
+  pl.a_box_rows = pair ? kTileM : pl.rows_per_block;
   pl.tile_cols = sh.bn;
   pl.b_box_rows = sh.bbox;
   pl.col_gran = sh.col_gran;
@@ -373,18 +639,24 @@ LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms
   pl.n_groups = (V + sh.col_gran - 1) / sh.col_gran;
   pl.rows_pad = static_cast<int64_t>(pl.row_blocks) * pl.rows_per_block;
   pl.k_blocks = static_cast<int>((static_cast<int64_t>(d) * elem_bytes + kRowBytes - 1) / kRowBytes);
-  pl.smem_bytes = smem_bytes_for(sh.mt, sh.bn, sh.stages);
-  const int slots_per_chunk = sh.mt == 1 ? kEpiSplit : 1;
+  pl.smem_bytes = pair ? kPairSmemBytes : smem_bytes_for(sh.mt, sh.bn, sh.stages);
+  // partial slots a row gets per vocabulary chunk: its tile columns are split over two epilogue
+  // warps unless the two warps serve two different row tiles
+  const int slots_per_chunk = pl.variant == 2 ? 1 : kEpiSplit;
+  // CTAs, or CTA pairs that fit on the device at once
+  const int workers_max = pair ? std::max(1, g_pair_workers_max > 0 ? std::min(g_pair_workers_max, num_sms / 2) : num_sms / 2)
+                               : num_sms;
   const int64_t s_cap = std::max<int64_t>(1, slot_row_capacity / (pl.rows_pad * slots_per_chunk));
   const int s_max = static_cast<int>(std::min<int64_t>(pl.n_groups, s_cap));
-  if (pl.variant == 0) {
-    pl.grid = static_cast<int>(std::min<int64_t>(num_sms, static_cast<int64_t>(pl.row_blocks) * pl.n_groups));
-    // Units are dealt round-robin to the CTAs, so the step takes ceil(units / grid) rounds of
+  int workers;
+  if (!one_block) {
+    workers = static_cast<int>(std::min<int64_t>(workers_max, static_cast<int64_t>(pl.row_blocks) * pl.n_groups));
+    // Units are dealt round-robin to the workers, so the step takes ceil(units / workers) rounds of
     // ceil(n_tiles / S) tiles.  Take the smallest S whose makespan is within 2 % of the best
     // reachable one (fewer chunks = fewer partials to write and merge).
     auto makespan = [&](int S) {
       const int64_t units = static_cast<int64_t>(pl.row_blocks) * S;
-      const int64_t rounds = (units + pl.grid - 1) / pl.grid;
+      const int64_t rounds = (units + workers - 1) / workers;
       return rounds * ((pl.n_groups + S - 1) / S);
     };
     int64_t best = makespan(1);
@@ -395,10 +667,11 @@ LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms
     }
     pl.chunks = pick;
   } else {
-    // One row block: one vocabulary range per SM, ranges differ by at most 32 columns.
-    pl.chunks = std::max(1, std::min(s_max, num_sms));
-    pl.grid = pl.chunks;
+    // One row block: one vocabulary range per worker, ranges differ by at most col_gran columns.
+    pl.chunks = std::max(1, std::min(s_max, workers_max));
+    workers = pl.chunks;
   }
+  pl.grid = pair ? 2 * workers : workers;
   pl.slots = pl.chunks * slots_per_chunk;
   // Row blocks that sweep the vocabulary together: enough of them that a W tile fetched from HBM
   // is shared by many CTAs, few enough that their hidden tiles (re-read per vocabulary tile) stay in
@@ -406,7 +679,7 @@ LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms
   const int64_t a_tile_bytes = static_cast<int64_t>(pl.rows_per_block) * d * elem_bytes;
   int gm = static_cast<int>(std::max<int64_t>(1, (8ll << 20) / std::max<int64_t>(1, a_tile_bytes)));
   gm = std::min(gm, pl.row_blocks);
-  gm = std::min(gm, std::max(1, pl.grid));
+  gm = std::min(gm, std::max(1, workers));
   pl.group_rb = gm;
   return pl;
 }
@@ -418,7 +691,15 @@ cudaError_t lmhead_prepare_device() {
   if ((e = prepare_shape<false, EGTP_SHAPE_DECODE2>()) != cudaSuccess) return e;
   if ((e = prepare_shape<true, EGTP_SHAPE_PROMPT>()) != cudaSuccess) return e;
   if ((e = prepare_shape<true, EGTP_SHAPE_DECODE1>()) != cudaSuccess) return e;
-  return prepare_shape<true, EGTP_SHAPE_DECODE2>();
+  if ((e = prepare_shape<true, EGTP_SHAPE_DECODE2>()) != cudaSuccess) return e;
+  int device = 0, num_sms = 0;
+  if ((e = cudaGetDevice(&device)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess) return e;
+  g_pair_workers_max = 0;
+  if ((e = prepare_pair<false, 128>(num_sms)) != cudaSuccess) return e;
+  if ((e = prepare_pair<false, 32>(num_sms)) != cudaSuccess) return e;
+  if ((e = prepare_pair<true, 128>(num_sms)) != cudaSuccess) return e;
+  return prepare_pair<true, 32>(num_sms);
 }
 
 cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const CUtensorMap* map_hidden,
@@ -441,12 +722,16 @@ cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const CUten
     switch (plan.variant) {
       case 1: return launch_shape<true, EGTP_SHAPE_DECODE1>(plan, map_hidden, map_w, p, stream);
       case 2: return launch_shape<true, EGTP_SHAPE_DECODE2>(plan, map_hidden, map_w, p, stream);
+      case 4: return launch_pair<true, 128>(plan, map_hidden, map_w, p, stream);
+      case 5: return launch_pair<true, 32>(plan, map_hidden, map_w, p, stream);
       default: return launch_shape<true, EGTP_SHAPE_PROMPT>(plan, map_hidden, map_w, p, stream);
     }
   }
   switch (plan.variant) {
     case 1: return launch_shape<false, EGTP_SHAPE_DECODE1>(plan, map_hidden, map_w, p, stream);
     case 2: return launch_shape<false, EGTP_SHAPE_DECODE2>(plan, map_hidden, map_w, p, stream);
+    case 4: return launch_pair<false, 128>(plan, map_hidden, map_w, p, stream);
+    case 5: return launch_pair<false, 32>(plan, map_hidden, map_w, p, stream);
     default: return launch_shape<false, EGTP_SHAPE_PROMPT>(plan, map_hidden, map_w, p, stream);
   }
 }

@@ -176,3 +176,28 @@ def test_host_buffer_entry_point(ctx):
     assert int(st.item()) == 0
     gu.assert_pooled_close(pooled.numpy().astype(np.float64), ref["pooled"])
     gu.assert_length_close(y.numpy().astype(np.float64), ref["yhat"])
+
+
+def test_cta_pair_tile_shape_matches_oracle():
+    # the same checks with the LM-head kernel switched to clusters of two CTAs (256 x 256 tiles)
+    c = egtp.egtp_create(0, max_tokens=16384, max_batch=256, max_d=2048, max_V=40000)
+    try:
+        egtp.egtp_set_lmhead_mode(c, egtp.EGTP_LMHEAD_CTA_PAIRS)
+        wl = gen.config_mid(V=20000 + 72, d=512, m_h=128)
+        ref = orc.egtp_predict(wl.hidden, wl.offsets, wl.W, wl.head, wl.alpha)
+        _check_all(gu.run_egtp(c, wl), ref, wl)
+        # odd number of 128-row tiles, V not a multiple of 256, W = 0: every entropy is ln V
+        rng = np.random.default_rng(1)
+        hidden = gen.round_to_bf16(rng.standard_normal((3 * 128 + 5, 256)).astype(np.float32))
+        wl0 = gen.EgtpWorkload("uniform", "bf16", hidden, gen.offsets_from_lengths([200, 189]), np.zeros((33000, 256), np.float32),
+                               gen.make_head(1, 256, 32, 1, "bf16"))
+        res = gu.run_egtp(c, wl0)
+        assert res["status"] == 0 and np.all(np.abs(res["H"] - math.log(33000)) <= 1e-4 * math.log(33000))
+        # fp32 inputs (tf32 MMA) in pair form
+        wt = gen.config_tiny()
+        big = gen.EgtpWorkload("tiny_x3", "f32", np.concatenate([wt.hidden] * 3), gen.offsets_from_lengths([159, 159, 159]),
+                               wt.W, wt.head)
+        _check_all(gu.run_egtp(c, big), orc.egtp_predict(big.hidden, big.offsets, big.W, big.head), big)
+        assert egtp.load().egtp_set_lmhead_mode(c, 7) == egtp.EGTP_ERR_INVALID_ARG
+    finally:
+        egtp.egtp_destroy(c)
