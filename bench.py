@@ -409,9 +409,18 @@ def main():
     ap.add_argument("--impl", default="mine", choices=["mine", "reference"])
     ap.add_argument("--plp-steps", type=int, default=64)
     ap.add_argument("--long-steps", type=int, default=10)
-    ap.add_argument("--no-plp", action="store_true")
+    ap.add_argument("--no-plp", action="store_true", help="skip the d = 4096 workloads (PLP decode, long prompts)")
+    ap.add_argument("--only-d4096", action="store_true",
+                    help="run only the d = 4096 workloads and print their two objects as one JSON line "
+                         "(used for profiler captures of the decode and pooling kernels)")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
+    if args.only_d4096:
+        import torch
+        torch.cuda.set_device(0)
+        plp, long_ = bench_d4096(0, load_peaks(), args.plp_steps, args.long_steps)
+        print(json.dumps(dict(plp_decode=plp, egtp_long=long_)), flush=True)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
