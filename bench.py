@@ -363,8 +363,31 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
                            unit="TFLOP/s", frac=2.0 * slots * d * V / (k1_us * 1e-6) / 1e12 / peaks["bf16_tflops"]),
                kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof.items() if v["launches"]},
                plan=egtp.egtp_lmhead_plan(ctx, slots, d, V, egtp.EGTP_BF16))
+    # ---- the same decode step when the serving engine already holds the step's logits
+    torch.manual_seed(0)
+    logits = (torch.randn(slots, V, device="cuda") * 1.5).to(torch.bfloat16)
+    for t in range(3):
+        egtp.plp_step_from_logits(ctx, st, logits, head.c, hs[t], reset_src=reset[t], yrem_out=yrem, status_dev=status)
+    torch.cuda.synchronize()
+    egtp.egtp_profile_read(ctx)
+    n_fl = max(8, plp_steps)
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for t in range(n_fl):
+        egtp.plp_step_from_logits(ctx, st, logits, head.c, hs[warm + t % plp_steps], reset_src=reset[warm + t % plp_steps],
+                                  yrem_out=yrem, status_dev=status)
+    f1.record()
+    torch.cuda.synchronize()
+    prof_fl = egtp.egtp_profile_read(ctx)
+    assert int(status.item()) == 0
+    le_us = prof_fl["logits_entropy"]["ms"] / prof_fl["logits_entropy"]["launches"] * 1e3
+    le_gbs = 2.0 * slots * V / (le_us * 1e-6) / 1e9
+    plp["from_logits"] = dict(us_per_step=f0.elapsed_time(f1) / n_fl * 1e3, logits_entropy_us=le_us,
+                              hbm=dict(bound="hbm", kernel="logits_entropy", achieved=le_gbs, peak=peaks["hbm_gbs"],
+                                       unit="GB/s", frac=le_gbs / peaks["hbm_gbs"], bytes_per_row=2 * V),
+                              kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof_fl.items() if v["launches"]})
     egtp.plp_state_destroy(st)
-    del hs
+    del hs, logits
 
     # ---- EGTP over the long-tailed prompt batch
     hidden = gu.dev_tensor(wl3.hidden, "bf16")

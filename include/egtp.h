@@ -223,6 +223,30 @@ EGTP_API int plp_step_host(egtp_ctx* ctx, plp_state* st, const egtp_lm_head* lm,
 EGTP_API int egtp_head_forward_static(const egtp_head* head, const float* z, int64_t ldz, int32_t rows,
                                       float* y_out, float* phat_out, void* stream);
 
+/* Eq. 2 from logits that already exist in device memory (Sec. 3.1; the paper reuses the
+ * activations the model has produced anyway): H_out[i] = entropy of softmax(logits[i][0..V)) in nats.
+ * For a serving engine that has just run its own LM head for sampling, this replaces a second
+ * LM-head GEMM by one streaming pass over the logits.
+ *   logits  device, [rows][ldl] in logits_dtype (EGTP_F32 or EGTP_BF16), ldl >= V, rows start on
+ *           16-byte boundaries; rows <= max(max_tokens, max_batch) of the context
+ *   H_out   device, float [rows]
+ * status_dev and stream as in egtp_predict. */
+EGTP_API int egtp_entropy_from_logits(egtp_ctx* ctx, const void* logits, int64_t ldl, int32_t logits_dtype,
+                                      int64_t rows, int32_t V, float* H_out, int32_t* status_dev, void* stream);
+
+/* plp_step (Sec. 3.3, Eq. 8) with the new tokens' entropies taken from logits in memory instead
+ * of an LM-head GEMM: logits [B_live][ldl] as above; hidden_step [B_live][ldh] in hidden_dtype with
+ * d = the state's hidden size.  Everything else (slots, resets, EGTP source table, outputs, status,
+ * stream) is as in plp_step. */
+EGTP_API int plp_step_from_logits(egtp_ctx* ctx, plp_state* st, const void* logits, int64_t ldl,
+                                  int32_t logits_dtype, int32_t V, const egtp_head* head,
+                                  const void* hidden_step, int64_t ldh, int32_t hidden_dtype,
+                                  const int32_t* slot_ids, const int32_t* reset_src,
+                                  const float* src_m, const float* src_s, const float* src_pooled, int32_t n_src,
+                                  int32_t B_live, float alpha,
+                                  float* Hstep_out, float* z_out, float* yrem_out,
+                                  int32_t* status_dev, void* stream);
+
 /* Tile shape of the LM-head kernel.  EGTP_LMHEAD_AUTO (default): one CTA per SM, 128 x 256 tiles for
  * prompt batches and the two decode shapes for <= 256 rows.  EGTP_LMHEAD_CTA_PAIRS: clusters of two
  * CTAs work on 256 x 256 tiles with tcgen05.mma.cta_group::2 wherever more than 128 rows are given
@@ -245,6 +269,7 @@ enum {
   EGTP_K_HEAD_HIDDEN,       /* head layer 1 */
   EGTP_K_HEAD_OUT,          /* head layer 2 + output mode */
   EGTP_K_PLP_UPDATE,        /* PLP running-state update */
+  EGTP_K_LOGITS_ENTROPY,    /* Eq. 2 from logits already in memory */
   EGTP_NUM_KERNELS
 };
 EGTP_API int egtp_profile_enable(egtp_ctx* ctx, int on);

@@ -26,7 +26,7 @@ EGTP_HEAD_SCALAR, EGTP_HEAD_BINS = 0, 1
 PLP_RESET_KEEP, PLP_RESET_EMPTY = -2, -1
 EGTP_LMHEAD_AUTO, EGTP_LMHEAD_CTA_PAIRS = 0, 1
 KERNEL_IDS = ["validate_offsets", "lmhead_entropy", "entropy_merge", "segment_weights", "pool",
-              "pool_combine", "head_hidden", "head_out", "plp_update"]
+              "pool_combine", "head_hidden", "head_out", "plp_update", "logits_entropy"]
 EGTP_NUM_KERNELS = len(KERNEL_IDS)
 EGTP_K_LMHEAD_ENTROPY = 1
 
@@ -35,6 +35,7 @@ EXPORTED_SYMBOLS = [
     "egtp_predict_host", "plp_state_create", "plp_state_destroy", "plp_state_export", "plp_state_import",
     "plp_step", "plp_step_host", "egtp_profile_enable", "egtp_profile_read", "egtp_kernel_name",
     "egtp_launch_count", "egtp_lmhead_plan", "egtp_head_forward_static", "egtp_set_lmhead_mode",
+    "egtp_entropy_from_logits", "plp_step_from_logits",
 ]
 
 
@@ -82,6 +83,9 @@ def load() -> C.CDLL:
     lib.egtp_lmhead_plan.argtypes = [vp, i64, i32, i32, i32, P(i32)]
     lib.egtp_profile_enable.argtypes = [vp, C.c_int]
     lib.egtp_set_lmhead_mode.argtypes = [vp, C.c_int]
+    lib.egtp_entropy_from_logits.argtypes = [vp, vp, i64, i32, i64, i32, vp, vp, vp]
+    lib.plp_step_from_logits.argtypes = [vp, vp, vp, i64, i32, i32, P(egtp_head), vp, i64, i32, vp, vp, vp, vp, vp, i32, i32,
+                                         f32, vp, vp, vp, vp, vp]
     lib.egtp_profile_read.argtypes = [vp, P(C.c_double), P(i64)]
     lib.egtp_predict.argtypes = [vp, P(egtp_lm_head), P(egtp_head), vp, i64, vp, i32, i64, f32,
                                  vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -284,4 +288,33 @@ def egtp_head_forward_static(head: egtp_head, z, rows: Optional[int] = None, y_o
                                          _stream(stream))
     if check:
         _check(rc, "egtp_head_forward_static")
+    return rc
+
+
+def egtp_entropy_from_logits(ctx: int, logits, H_out, rows: Optional[int] = None, V: Optional[int] = None,
+                             status_dev=None, stream=None, check: bool = True) -> int:
+    """H_out[i] = entropy of softmax(logits[i]) for a device tensor logits [rows, V] (bf16 or fp32)."""
+    rows = logits.shape[0] if rows is None else rows
+    V = logits.shape[1] if V is None else V
+    rc = load().egtp_entropy_from_logits(ctx, _ptr(logits), logits.stride(0), _dtype_code(logits), rows, V,
+                                         _ptr(H_out), _ptr(status_dev), _stream(stream))
+    if check:
+        _check(rc, "egtp_entropy_from_logits")
+    return rc
+
+
+def plp_step_from_logits(ctx: int, st: int, logits, head: Optional[egtp_head], hidden_step, slot_ids=None,
+                         reset_src=None, src_m=None, src_s=None, src_pooled=None, n_src: int = 0,
+                         B_live: Optional[int] = None, alpha: float = 1.0, Hstep_out=None, z_out=None, yrem_out=None,
+                         status_dev=None, stream=None, check: bool = True) -> int:
+    """plp_step with the step's entropies computed from logits [B_live, V] that are already in device memory."""
+    if B_live is None:
+        B_live = hidden_step.shape[0]
+    rc = load().plp_step_from_logits(ctx, st, _ptr(logits), logits.stride(0), _dtype_code(logits), logits.shape[1],
+                                     C.byref(head) if head is not None else None, _ptr(hidden_step),
+                                     hidden_step.stride(0), _dtype_code(hidden_step), _ptr(slot_ids), _ptr(reset_src),
+                                     _ptr(src_m), _ptr(src_s), _ptr(src_pooled), n_src, B_live, alpha,
+                                     _ptr(Hstep_out), _ptr(z_out), _ptr(yrem_out), _ptr(status_dev), _stream(stream))
+    if check:
+        _check(rc, "plp_step_from_logits")
     return rc

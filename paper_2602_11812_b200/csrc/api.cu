@@ -71,7 +71,7 @@ namespace {
 
 const char* const kKernelNames[EGTP_NUM_KERNELS] = {
     "validate_offsets", "lmhead_entropy", "entropy_merge", "segment_weights", "pool",
-    "pool_combine",     "head_hidden",    "head_out",      "plp_update"};
+    "pool_combine",     "head_hidden",    "head_out",      "plp_update",    "logits_entropy"};
 
 template <typename T>
 cudaError_t dev_alloc(egtp_ctx* c, T** p, int64_t count) {
@@ -206,6 +206,49 @@ int run_head(egtp_ctx* c, const egtp_head* head, const float* z, int64_t ldz, in
     LaunchScope ls(c, EGTP_K_HEAD_OUT, stream);
     EGTP_CUDA_TRY(launch_head_out(ha, c->head_partial, rows, splits, y, phat, status, stream));
   }
+  return EGTP_OK;
+}
+
+// Eq. 2 from logits in memory: per-(row, split) partials into the workspace.
+int run_logits_entropy(egtp_ctx* c, const void* logits, int64_t ldl, int dtype, int64_t rows, int V, int32_t* status,
+                       cudaStream_t stream, int* slots_out) {
+  if (!logits || V <= 0 || ldl < V) return EGTP_ERR_INVALID_ARG;
+  if (dtype != EGTP_F32 && dtype != EGTP_BF16) return EGTP_ERR_UNSUPPORTED;
+  if ((ldl * elem_bytes(dtype)) % 16 != 0 || reinterpret_cast<uintptr_t>(logits) % 16 != 0) return EGTP_ERR_UNSUPPORTED;
+  if (rows > std::max<int64_t>(c->max_tokens, c->max_batch)) return EGTP_ERR_CAPACITY;
+  int splits = logits_entropy_pick_splits(rows, V, c->num_sms);
+  while (splits > 1 && rows * splits > c->slot_row_capacity) --splits;
+  if (rows * splits > c->slot_row_capacity) return EGTP_ERR_CAPACITY;
+  LaunchScope ls(c, EGTP_K_LOGITS_ENTROPY, stream);
+  EGTP_CUDA_TRY(launch_logits_entropy(logits, ldl, dtype == EGTP_BF16, rows, V, splits, c->partials, status, stream));
+  *slots_out = splits;
+  return EGTP_OK;
+}
+
+int check_plp_common(const egtp_ctx* c, const plp_state* st, const egtp_head* head, const float* src_m,
+                     const float* src_s, const float* src_pooled, int n_src, int B_live, float alpha,
+                     const float* yrem_out) {
+  if (B_live < 0 || n_src < 0 || !(alpha > 0.f) || !std::isfinite(alpha)) return EGTP_ERR_INVALID_ARG;
+  if (n_src > 0 && (!src_m || !src_s || !src_pooled)) return EGTP_ERR_INVALID_ARG;
+  if (!head && yrem_out) return EGTP_ERR_INVALID_ARG;
+  if (B_live > c->max_batch || B_live > st->num_slots || st->d > c->max_d) return EGTP_ERR_CAPACITY;
+  return EGTP_OK;
+}
+
+// Second half of a PLP step: merge the entropy partials, update the slots (Eq. 8), run the head.
+int plp_update_and_head(egtp_ctx* c, plp_state* st, const egtp_head* head, const void* hidden_step, int64_t ldh,
+                        int hidden_dtype, int slots, const int32_t* slot_ids, const int32_t* reset_src,
+                        const float* src_m, const float* src_s, const float* src_pooled, int n_src, int B_live,
+                        float alpha, float* Hstep_out, float* z_out, float* yrem_out, int32_t* status,
+                        cudaStream_t stream) {
+  float* z = z_out ? z_out : c->pooled;
+  {
+    LaunchScope ls(c, EGTP_K_PLP_UPDATE, stream);
+    EGTP_CUDA_TRY(launch_plp_update(hidden_step, ldh, hidden_dtype == EGTP_BF16, c->partials, slots, Hstep_out, slot_ids,
+                                    reset_src, src_m, src_s, src_pooled, n_src, B_live, st->d, st->num_slots,
+                                    1.f / alpha, st->m, st->s, st->acc, z, st->d, status, stream));
+  }
+  if (head && yrem_out) return run_head(c, head, z, st->d, B_live, yrem_out, nullptr, status, stream);
   return EGTP_OK;
 }
 
@@ -495,12 +538,10 @@ int plp_step(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head
              const float* src_pooled, int32_t n_src, int32_t B_live, float alpha, float* Hstep_out, float* z_out,
              float* yrem_out, int32_t* status_dev, void* stream_v) {
   if (!c || !st || st->ctx != c) return EGTP_ERR_INVALID_ARG;
-  if (B_live < 0 || n_src < 0 || !(alpha > 0.f) || !std::isfinite(alpha)) return EGTP_ERR_INVALID_ARG;
   if (B_live == 0) return EGTP_OK;
-  if (n_src > 0 && (!src_m || !src_s || !src_pooled)) return EGTP_ERR_INVALID_ARG;
-  if (!head && yrem_out) return EGTP_ERR_INVALID_ARG;
-  if (B_live > c->max_batch || B_live > st->num_slots) return EGTP_ERR_CAPACITY;
-  int rc = check_lm(c, lm, hidden_step, ldh);
+  int rc = check_plp_common(c, st, head, src_m, src_s, src_pooled, n_src, B_live, alpha, yrem_out);
+  if (rc != EGTP_OK) return rc;
+  rc = check_lm(c, lm, hidden_step, ldh);
   if (rc != EGTP_OK) return rc;
   if (lm->d != st->d) return EGTP_ERR_INVALID_ARG;
   if (head) {
@@ -511,21 +552,55 @@ int plp_step(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head
   if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
   int32_t* status = status_dev ? status_dev : c->status;
   if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
-  float* z = z_out ? z_out : c->pooled;
   LmheadPlan plan;
   rc = run_lmhead(c, lm, hidden_step, ldh, B_live, status, stream, &plan);
   if (rc != EGTP_OK) return rc;
-  {
-    LaunchScope ls(c, EGTP_K_PLP_UPDATE, stream);
-    EGTP_CUDA_TRY(launch_plp_update(hidden_step, ldh, lm->dtype == EGTP_BF16, c->partials, plan.slots, Hstep_out, slot_ids, reset_src, src_m, src_s,
-                                    src_pooled, n_src, B_live, lm->d, st->num_slots, 1.f / alpha, st->m, st->s,
-                                    st->acc, z, lm->d, status, stream));
-  }
-  if (head && yrem_out) {
-    rc = run_head(c, head, z, lm->d, B_live, yrem_out, nullptr, status, stream);
+  return plp_update_and_head(c, st, head, hidden_step, ldh, lm->dtype, plan.slots, slot_ids, reset_src, src_m, src_s,
+                             src_pooled, n_src, B_live, alpha, Hstep_out, z_out, yrem_out, status, stream);
+}
+
+int egtp_entropy_from_logits(egtp_ctx* c, const void* logits, int64_t ldl, int32_t logits_dtype, int64_t rows,
+                             int32_t V, float* H_out, int32_t* status_dev, void* stream_v) {
+  if (!c || !H_out || rows < 0) return EGTP_ERR_INVALID_ARG;
+  if (rows == 0) return EGTP_OK;
+  int slots = 0;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  int32_t* status = status_dev ? status_dev : c->status;
+  if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
+  int rc = run_logits_entropy(c, logits, ldl, logits_dtype, rows, V, status, stream, &slots);
+  if (rc != EGTP_OK) return rc;
+  LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
+  EGTP_CUDA_TRY(launch_entropy_merge(c->partials, slots, rows, H_out, nullptr, 0, nullptr, nullptr, status, stream));
+  return EGTP_OK;
+}
+
+int plp_step_from_logits(egtp_ctx* c, plp_state* st, const void* logits, int64_t ldl, int32_t logits_dtype, int32_t V,
+                         const egtp_head* head, const void* hidden_step, int64_t ldh, int32_t hidden_dtype,
+                         const int32_t* slot_ids, const int32_t* reset_src, const float* src_m, const float* src_s,
+                         const float* src_pooled, int32_t n_src, int32_t B_live, float alpha, float* Hstep_out,
+                         float* z_out, float* yrem_out, int32_t* status_dev, void* stream_v) {
+  if (!c || !st || st->ctx != c) return EGTP_ERR_INVALID_ARG;
+  if (B_live == 0) return EGTP_OK;
+  int rc = check_plp_common(c, st, head, src_m, src_s, src_pooled, n_src, B_live, alpha, yrem_out);
+  if (rc != EGTP_OK) return rc;
+  if (!hidden_step || ldh < st->d) return EGTP_ERR_INVALID_ARG;
+  if (hidden_dtype != EGTP_F32 && hidden_dtype != EGTP_BF16) return EGTP_ERR_UNSUPPORTED;
+  if ((ldh * elem_bytes(hidden_dtype)) % 16 != 0 || reinterpret_cast<uintptr_t>(hidden_step) % 16 != 0)
+    return EGTP_ERR_UNSUPPORTED;
+  if (head) {
+    rc = check_head(c, head, st->d);
     if (rc != EGTP_OK) return rc;
   }
-  return EGTP_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  int32_t* status = status_dev ? status_dev : c->status;
+  if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
+  int slots = 0;
+  rc = run_logits_entropy(c, logits, ldl, logits_dtype, B_live, V, status, stream, &slots);
+  if (rc != EGTP_OK) return rc;
+  return plp_update_and_head(c, st, head, hidden_step, ldh, hidden_dtype, slots, slot_ids, reset_src, src_m, src_s,
+                             src_pooled, n_src, B_live, alpha, Hstep_out, z_out, yrem_out, status, stream);
 }
 
 int plp_step_host(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head* head,

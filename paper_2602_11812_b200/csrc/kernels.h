@@ -68,6 +68,12 @@ cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, const float*
 cudaError_t launch_pool_combine(const int32_t* offsets, int B, int d, const float* piece_a, const float* piece_b,
                                 float* pooled, const int32_t* status, cudaStream_t stream);
 
+// ---- Eq. 2 from logits already in memory -------------------------------------------------------
+int logits_entropy_pick_splits(int64_t rows, int V, int num_sms);
+// partials [rows][splits][3] in the layout of the LM-head kernel's partials
+cudaError_t launch_logits_entropy(const void* logits, int64_t ldl, bool bf16, int64_t rows, int V, int splits,
+                                  float* partials, const int32_t* status, cudaStream_t stream);
+
 // ---- K3: head ------------------------------------------------------------------------------
 struct HeadArgs {
   const void* W1;

@@ -1,0 +1,145 @@
+// Token entropy (paper Sec. 3.1, Eq. 2) from logits that already exist in memory.
+// A serving engine that has just run its LM head for sampling holds the [rows, V] logits of the
+// step; the entropy then costs one pass over those values instead of a second LM-head GEMM.
+// HBM-bound: 16-byte coalesced loads, one running (m, s, t2) per thread (same definition as the
+// LM-head kernel's epilogue), warp-shuffle and shared-memory combine, one partial per
+// (row, vocabulary split) in the layout the merge kernels read.
+#include "kernels.h"
+#include "entropy_merge.cuh"
+#include "../../include/egtp.h"
+
+#include <cuda_bf16.h>
+
+#include <algorithm>
+
+namespace egtp {
+
+namespace {
+
+constexpr int kLogitsThreads = 256;
+constexpr float kLog2e = 1.4426950408889634f;
+
+__device__ __forceinline__ void fold8(EntropyPartial& st, const float (&x)[8]) {
+  float cmax = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])), fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
+  if (cmax > st.m) {
+    const float dm = (st.m - cmax) * kLog2e;
+    const float r = exp2f(dm);
+    st.t2 = r * fmaf(dm, st.s, st.t2);
+    st.s *= r;
+    st.m = cmax;
+  }
+  const float neg_m_l2 = -st.m * kLog2e;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const float y = fmaf(x[j], kLog2e, neg_m_l2);
+    const float e = exp2f(y);
+    st.s += e;
+    st.t2 = fmaf(e, y, st.t2);
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ void load8_logits(const T* p, float (&v)[8]);
+template <>
+__device__ __forceinline__ void load8_logits<__nv_bfloat16>(const __nv_bfloat16* p, float (&v)[8]) {
+  const uint4 q = __ldcs(reinterpret_cast<const uint4*>(p));   // streamed once: do not keep in cache
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+template <>
+__device__ __forceinline__ void load8_logits<float>(const float* p, float (&v)[8]) {
+  const float4 a = __ldcs(reinterpret_cast<const float4*>(p));
+  const float4 b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+  v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+template <typename T>
+__device__ __forceinline__ float to_float(T v);
+template <>
+__device__ __forceinline__ float to_float<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// block (split, row): columns [split * cols_per_split, ...) of one row
+template <typename T>
+__global__ void __launch_bounds__(kLogitsThreads)
+logits_entropy_kernel(const T* __restrict__ logits, int64_t ldl, int V, int cols_per_split, int splits,
+                      float* __restrict__ partials, const int32_t* __restrict__ status) {
+  if (*status != 0) return;
+  __shared__ EntropyPartial red[kLogitsThreads / 32];
+  const int split = blockIdx.x;
+  const int64_t row = blockIdx.y;
+  const int c0 = split * cols_per_split;
+  const int c1 = min(V, c0 + cols_per_split);
+  const T* base = logits + row * ldl;
+  EntropyPartial st = {kNegBig, 0.f, 0.f};
+  const int n_vec = max(0, c1 - c0) >> 3;                       // cols_per_split is a multiple of 8
+  int v = threadIdx.x;
+  for (; v + 3 * kLogitsThreads < n_vec; v += 4 * kLogitsThreads) {   // four 16-byte loads in flight
+    float x0[8], x1[8], x2[8], x3[8];
+    load8_logits<T>(base + c0 + 8 * v, x0);
+    load8_logits<T>(base + c0 + 8 * (v + kLogitsThreads), x1);
+    load8_logits<T>(base + c0 + 8 * (v + 2 * kLogitsThreads), x2);
+    load8_logits<T>(base + c0 + 8 * (v + 3 * kLogitsThreads), x3);
+    fold8(st, x0); fold8(st, x1); fold8(st, x2); fold8(st, x3);
+  }
+  for (; v < n_vec; v += kLogitsThreads) {
+    float x0[8];
+    load8_logits<T>(base + c0 + 8 * v, x0);
+    fold8(st, x0);
+  }
+  // ragged tail of the row (fewer than 8 columns), handled by one thread
+  if (threadIdx.x == 0) {
+    for (int c = c0 + 8 * n_vec; c < c1; ++c) {
+      const EntropyPartial one = {to_float<T>(base[c]), 1.f, 0.f};
+      st = combine_partials(st, one);
+    }
+  }
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    EntropyPartial other;
+    other.m = __shfl_xor_sync(0xffffffffu, st.m, o);
+    other.s = __shfl_xor_sync(0xffffffffu, st.s, o);
+    other.t2 = __shfl_xor_sync(0xffffffffu, st.t2, o);
+    st = (lane & o) ? combine_partials(other, st) : combine_partials(st, other);
+  }
+  if (lane == 0) red[wid] = st;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    EntropyPartial acc = red[0];
+    for (int w = 1; w < kLogitsThreads / 32; ++w) acc = combine_partials(acc, red[w]);
+    float* dst = partials + (row * splits + split) * 3;
+    dst[0] = acc.m; dst[1] = acc.s; dst[2] = acc.t2;
+  }
+}
+
+}  // namespace
+
+int logits_entropy_pick_splits(int64_t rows, int V, int num_sms) {
+  // enough blocks to fill the GPU a few times over, at least 4096 columns each
+  int64_t want = (4ll * num_sms + rows - 1) / std::max<int64_t>(rows, 1);
+  want = std::min<int64_t>(want, std::max(1, V / 4096));
+  return static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(want, 64)));
+}
+
+cudaError_t launch_logits_entropy(const void* logits, int64_t ldl, bool bf16, int64_t rows, int V, int splits,
+                                  float* partials, const int32_t* status, cudaStream_t stream) {
+  int cols_per_split = (V + splits - 1) / splits;
+  cols_per_split = (cols_per_split + 7) / 8 * 8;
+  dim3 grid(splits, static_cast<unsigned>(rows));
+  if (bf16) {
+    logits_entropy_kernel<__nv_bfloat16><<<grid, kLogitsThreads, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(logits), ldl, V, cols_per_split, splits, partials, status);
+  } else {
+    logits_entropy_kernel<float><<<grid, kLogitsThreads, 0, stream>>>(static_cast<const float*>(logits), ldl, V,
+                                                                     cols_per_split, splits, partials, status);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace egtp
