@@ -23,6 +23,26 @@ __device__ __forceinline__ EntropyPartial combine_partials(const EntropyPartial&
   return r;
 }
 
+// Combines the 32 lanes' partials: every lane returns the same (m, s, t2).  The warp maximum is found
+// first, then each lane rescales once and the sums go through an xor butterfly (commutative pairs, so
+// all lanes hold bitwise the same result and the result does not depend on scheduling).
+__device__ __forceinline__ EntropyPartial warp_combine_partials(EntropyPartial p) {
+  constexpr float kLog2e = 1.4426950408889634f;
+  float M = p.m;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  const float dm = (p.m - M) * kLog2e;
+  const float r = exp2f(dm);
+  float s = p.s * r;
+  float t2 = r * fmaf(dm, p.s, p.t2);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    s += __shfl_xor_sync(0xffffffffu, s, o);
+    t2 += __shfl_xor_sync(0xffffffffu, t2, o);
+  }
+  return {M, s, t2};
+}
+
 // All 32 lanes of a warp call this with the same row pointer ([slots][3] floats); every lane
 // returns H.  The order of operations is fixed, so the result is bitwise reproducible.
 __device__ __forceinline__ float merge_partials_warp(const float* __restrict__ row, int slots, int lane) {
@@ -32,15 +52,7 @@ __device__ __forceinline__ float merge_partials_warp(const float* __restrict__ r
     const EntropyPartial pj = {row[3 * j], row[3 * j + 1], row[3 * j + 2]};
     acc = combine_partials(acc, pj);
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    EntropyPartial other;
-    other.m = __shfl_xor_sync(0xffffffffu, acc.m, o);
-    other.s = __shfl_xor_sync(0xffffffffu, acc.s, o);
-    other.t2 = __shfl_xor_sync(0xffffffffu, acc.t2, o);
-    // lower lane first on both sides so that every lane computes the identical value
-    acc = (lane & o) ? combine_partials(other, acc) : combine_partials(acc, other);
-  }
+  acc = warp_combine_partials(acc);
   return logf(acc.s) - kLn2 * acc.t2 / acc.s;
 }
 

@@ -14,21 +14,28 @@ namespace egtp {
 namespace {
 
 constexpr int kHT = 64;        // rows and hidden units per block tile
-constexpr int kHK = 16;        // k extent per shared-memory stage
+constexpr int kHK = 32;        // k extent per shared-memory stage
 constexpr int kHThreads = 256; // 16 x 16 threads, 4 x 4 outputs each
 constexpr int kHOutThreads = 256;
 
 template <typename TW>
-__device__ __forceinline__ float4 load4(const TW* p);
+__device__ __forceinline__ void load8w(const TW* p, float (&v)[8]);
 template <>
-__device__ __forceinline__ float4 load4<float>(const float* p) {
-  return __ldg(reinterpret_cast<const float4*>(p));
+__device__ __forceinline__ void load8w<float>(const float* p, float (&v)[8]) {
+  const float4 a = __ldg(reinterpret_cast<const float4*>(p));
+  const float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+  v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
 }
 template <>
-__device__ __forceinline__ float4 load4<__nv_bfloat16>(const __nv_bfloat16* p) {
-  const uint2 q = __ldg(reinterpret_cast<const uint2*>(p));
-  return make_float4(__uint_as_float(q.x << 16), __uint_as_float(q.x & 0xFFFF0000u),
-                     __uint_as_float(q.y << 16), __uint_as_float(q.y & 0xFFFF0000u));
+__device__ __forceinline__ void load8w<__nv_bfloat16>(const __nv_bfloat16* p, float (&v)[8]) {
+  const uint4 q = __ldg(reinterpret_cast<const uint4*>(p));
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
 }
 
 // partial[split][row][j] = sum_{k in split} z[row][k] * W1[j][k]
@@ -45,7 +52,7 @@ head_hidden_kernel(const float* __restrict__ z, int64_t ldz, const TW* __restric
   const int k_begin = split * k_per_split;
   const int k_end = min(d, k_begin + k_per_split);
   const int tid = threadIdx.x;
-  const int lrow = tid >> 2, lk = (tid & 3) * 4;   // loader: 64 rows x 4 quads of k
+  const int lrow = tid >> 2, lk = (tid & 3) * 8;   // loader: 64 rows x 4 groups of 8 k
   const int tx = tid & 15, ty = tid >> 4;          // compute: outputs rows ty*4.., units tx*4..
   const bool z_ok = r0 + lrow < rows, w_ok = j0 + lrow < m_h;
   const float* zp = z + static_cast<int64_t>(r0 + lrow) * ldz + lk;
@@ -56,21 +63,32 @@ head_hidden_kernel(const float* __restrict__ z, int64_t ldz, const TW* __restric
 #pragma unroll
     for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
 
-  const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
-  float4 zv = zero4, wv = zero4;
-  if (k_begin < k_end) {
-    if (z_ok) zv = __ldg(reinterpret_cast<const float4*>(zp + k_begin));
-    if (w_ok) wv = load4<TW>(wp + k_begin);
-  }
+  float zv[8], wv[8];
+  auto fetch = [&](int k0) {
+    const bool k_in = k0 + lk < k_end;     // d is a multiple of 16: a group of 8 is wholly inside or outside
+    if (z_ok && k_in) {
+      load8w<float>(zp + k0, zv);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) zv[i] = 0.f;
+    }
+    if (w_ok && k_in) {
+      load8w<TW>(wp + k0, wv);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) wv[i] = 0.f;
+    }
+  };
+  if (k_begin < k_end) fetch(k_begin);
   int buf = 0;
   for (int k0 = k_begin; k0 < k_end; k0 += kHK) {
-    zs[buf][lk + 0][lrow] = zv.x; zs[buf][lk + 1][lrow] = zv.y; zs[buf][lk + 2][lrow] = zv.z; zs[buf][lk + 3][lrow] = zv.w;
-    ws[buf][lk + 0][lrow] = wv.x; ws[buf][lk + 1][lrow] = wv.y; ws[buf][lk + 2][lrow] = wv.z; ws[buf][lk + 3][lrow] = wv.w;
-    __syncthreads();
-    if (k0 + kHK < k_end) {
-      zv = z_ok ? __ldg(reinterpret_cast<const float4*>(zp + k0 + kHK)) : zero4;
-      wv = w_ok ? load4<TW>(wp + k0 + kHK) : zero4;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      zs[buf][lk + i][lrow] = zv[i];
+      ws[buf][lk + i][lrow] = wv[i];
     }
+    __syncthreads();
+    if (k0 + kHK < k_end) fetch(k0 + kHK);
 #pragma unroll
     for (int k = 0; k < kHK; ++k) {
       const float4 a = *reinterpret_cast<const float4*>(&zs[buf][k][ty * 4]);

@@ -6,6 +6,7 @@
 // (row, vocabulary split) in the layout the merge kernels read.
 #include "kernels.h"
 #include "entropy_merge.cuh"
+#include "sm100_ptx.cuh"
 #include "../../include/egtp.h"
 
 #include <cuda_bf16.h>
@@ -19,24 +20,41 @@ namespace {
 constexpr int kLogitsThreads = 256;
 constexpr float kLog2e = 1.4426950408889634f;
 
-__device__ __forceinline__ void fold8(EntropyPartial& st, const float (&x)[8]) {
-  float cmax = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])), fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
-  if (cmax > st.m) {
-    const float dm = (st.m - cmax) * kLog2e;
-    const float r = exp2f(dm);
-    st.t2 = r * fmaf(dm, st.s, st.t2);
-    st.s *= r;
-    st.m = cmax;
-  }
-  const float neg_m_l2 = -st.m * kLog2e;
+// Running state of one thread: max m and four independent (s, t2) accumulators (short dependency chains).
+struct ThreadState {
+  float m;
+  float s[4];
+  float t[4];
+  __device__ __forceinline__ void init() {
+    m = kNegBig;
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const float y = fmaf(x[j], kLog2e, neg_m_l2);
-    const float e = exp2f(y);
-    st.s += e;
-    st.t2 = fmaf(e, y, st.t2);
+    for (int i = 0; i < 4; ++i) { s[i] = 0.f; t[i] = 0.f; }
   }
-}
+  __device__ __forceinline__ void fold8(const float (&x)[8]) {
+    const float cmax = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])), fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
+    if (cmax > m) {
+      const float dm = (m - cmax) * kLog2e;
+      const float r = ex2_approx(dm);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        t[i] = r * fmaf(dm, s[i], t[i]);
+        s[i] *= r;
+      }
+      m = cmax;
+    }
+    const float neg_m_l2 = -m * kLog2e;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float y = fmaf(x[j], kLog2e, neg_m_l2);
+      const float e = ex2_approx(y);
+      s[j & 3] += e;
+      t[j & 3] = fmaf(e, y, t[j & 3]);
+    }
+  }
+  __device__ __forceinline__ EntropyPartial total() const {
+    return {m, (s[0] + s[1]) + (s[2] + s[3]), (t[0] + t[1]) + (t[2] + t[3])};
+  }
+};
 
 template <typename T>
 __device__ __forceinline__ void load8_logits(const T* p, float (&v)[8]);
@@ -76,7 +94,8 @@ logits_entropy_kernel(const T* __restrict__ logits, int64_t ldl, int V, int cols
   const int c0 = split * cols_per_split;
   const int c1 = min(V, c0 + cols_per_split);
   const T* base = logits + row * ldl;
-  EntropyPartial st = {kNegBig, 0.f, 0.f};
+  ThreadState ts;
+  ts.init();
   const int n_vec = max(0, c1 - c0) >> 3;                       // cols_per_split is a multiple of 8
   int v = threadIdx.x;
   for (; v + 3 * kLogitsThreads < n_vec; v += 4 * kLogitsThreads) {   // four 16-byte loads in flight
@@ -85,13 +104,14 @@ logits_entropy_kernel(const T* __restrict__ logits, int64_t ldl, int V, int cols
     load8_logits<T>(base + c0 + 8 * (v + kLogitsThreads), x1);
     load8_logits<T>(base + c0 + 8 * (v + 2 * kLogitsThreads), x2);
     load8_logits<T>(base + c0 + 8 * (v + 3 * kLogitsThreads), x3);
-    fold8(st, x0); fold8(st, x1); fold8(st, x2); fold8(st, x3);
+    ts.fold8(x0); ts.fold8(x1); ts.fold8(x2); ts.fold8(x3);
   }
   for (; v < n_vec; v += kLogitsThreads) {
     float x0[8];
     load8_logits<T>(base + c0 + 8 * v, x0);
-    fold8(st, x0);
+    ts.fold8(x0);
   }
+  EntropyPartial st = ts.total();
   // ragged tail of the row (fewer than 8 columns), handled by one thread
   if (threadIdx.x == 0) {
     for (int c = c0 + 8 * n_vec; c < c1; ++c) {
@@ -100,14 +120,7 @@ logits_entropy_kernel(const T* __restrict__ logits, int64_t ldl, int V, int cols
     }
   }
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    EntropyPartial other;
-    other.m = __shfl_xor_sync(0xffffffffu, st.m, o);
-    other.s = __shfl_xor_sync(0xffffffffu, st.s, o);
-    other.t2 = __shfl_xor_sync(0xffffffffu, st.t2, o);
-    st = (lane & o) ? combine_partials(other, st) : combine_partials(st, other);
-  }
+  st = warp_combine_partials(st);
   if (lane == 0) red[wid] = st;
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -121,10 +134,13 @@ logits_entropy_kernel(const T* __restrict__ logits, int64_t ldl, int V, int cols
 }  // namespace
 
 int logits_entropy_pick_splits(int64_t rows, int V, int num_sms) {
-  // enough blocks to fill the GPU a few times over, at least 4096 columns each
-  int64_t want = (4ll * num_sms + rows - 1) / std::max<int64_t>(rows, 1);
-  want = std::min<int64_t>(want, std::max(1, V / 4096));
-  return static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(want, 64)));
+  // About 16K columns per block (8 vector loads per thread) so that many short blocks even out over the
+  // SMs; finer (down to 2K columns) when there are too few rows to fill the GPU otherwise.
+  int64_t splits = std::max(1, V / 16384);
+  const int64_t want_blocks = 4ll * num_sms;
+  if (rows * splits < want_blocks) splits = (want_blocks + rows - 1) / std::max<int64_t>(rows, 1);
+  splits = std::min<int64_t>(splits, std::max(1, V / 2048));
+  return static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(splits, 128)));
 }
 
 cudaError_t launch_logits_entropy(const void* logits, int64_t ldl, bool bf16, int64_t rows, int V, int splits,
