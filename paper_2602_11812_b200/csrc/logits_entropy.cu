@@ -51,6 +51,35 @@ struct ThreadState {
       t[j & 3] = fmaf(e, y, t[j & 3]);
     }
   }
+  // 32 values at once: one running-max update, then 32 independent exponentials (more work in flight)
+  __device__ __forceinline__ void fold32(const float (&a)[8], const float (&b)[8], const float (&c)[8],
+                                         const float (&d)[8]) {
+    float ma = a[0], mb = b[0], mc = c[0], md = d[0];
+#pragma unroll
+    for (int j = 1; j < 8; ++j) {
+      ma = fmaxf(ma, a[j]); mb = fmaxf(mb, b[j]); mc = fmaxf(mc, c[j]); md = fmaxf(md, d[j]);
+    }
+    const float cmax = fmaxf(fmaxf(ma, mb), fmaxf(mc, md));
+    if (cmax > m) {
+      const float dm = (m - cmax) * kLog2e;
+      const float r = ex2_approx(dm);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        t[i] = r * fmaf(dm, s[i], t[i]);
+        s[i] *= r;
+      }
+      m = cmax;
+    }
+    const float neg_m_l2 = -m * kLog2e;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float ya = fmaf(a[j], kLog2e, neg_m_l2), yb = fmaf(b[j], kLog2e, neg_m_l2);
+      const float yc = fmaf(c[j], kLog2e, neg_m_l2), yd = fmaf(d[j], kLog2e, neg_m_l2);
+      const float ea = ex2_approx(ya), eb = ex2_approx(yb), ec = ex2_approx(yc), ed = ex2_approx(yd);
+      s[0] += ea; s[1] += eb; s[2] += ec; s[3] += ed;
+      t[0] = fmaf(ea, ya, t[0]); t[1] = fmaf(eb, yb, t[1]); t[2] = fmaf(ec, yc, t[2]); t[3] = fmaf(ed, yd, t[3]);
+    }
+  }
   __device__ __forceinline__ EntropyPartial total() const {
     return {m, (s[0] + s[1]) + (s[2] + s[3]), (t[0] + t[1]) + (t[2] + t[3])};
   }
@@ -104,7 +133,7 @@ logits_entropy_kernel(const T* __restrict__ logits, int64_t ldl, int V, int cols
     load8_logits<T>(base + c0 + 8 * (v + kLogitsThreads), x1);
     load8_logits<T>(base + c0 + 8 * (v + 2 * kLogitsThreads), x2);
     load8_logits<T>(base + c0 + 8 * (v + 3 * kLogitsThreads), x3);
-    ts.fold8(x0); ts.fold8(x1); ts.fold8(x2); ts.fold8(x3);
+    ts.fold32(x0, x1, x2, x3);
   }
   for (; v < n_vec; v += kLogitsThreads) {
     float x0[8];
