@@ -201,3 +201,33 @@ def test_cta_pair_tile_shape_matches_oracle():
         assert egtp.load().egtp_set_lmhead_mode(c, 7) == egtp.EGTP_ERR_INVALID_ARG
     finally:
         egtp.egtp_destroy(c)
+
+
+def test_many_tokens_small_model_64bit_indexing():
+    # 300k tokens (2343.75 row tiles, > 2^31 / d / ... byte offsets in play) against a small LM head:
+    # entropies are checked on sampled tokens, pooling against fp64 pooling with the device's own entropies
+    T, d, V, B = 300_000, 64, 520, 40
+    rng = np.random.default_rng(11)
+    lengths = rng.multinomial(T - 1000, np.ones(B) / B)
+    off = np.concatenate([[500], 500 + np.cumsum(lengths)]).astype(np.int32)
+    hidden = gen.make_hidden(21, T, d, "bf16")
+    W = gen.round_to_bf16(gen.make_lm_head(22, V, d, "bf16") * np.float32(6.0))
+    head = gen.make_head(23, d, 32, 1, "bf16")
+    wl = gen.EgtpWorkload("many_tokens", "bf16", hidden, off, W, head)
+    c = egtp.egtp_create(0, max_tokens=T, max_batch=64, max_d=d, max_V=V)
+    try:
+        res = gu.run_egtp(c, wl)
+    finally:
+        egtp.egtp_destroy(c)
+    assert res["status"] == 0
+    idx = np.concatenate([[0, 1, T - 1, T - 2, 127, 128, 299_904], rng.choice(T, size=200, replace=False)])
+    gu.assert_entropy_close(res["H"][idx], orc.token_entropy(hidden[idx], W))
+    ref_seg = np.searchsorted(off, np.arange(T), side="right").astype(np.int32) - 1
+    ref_seg[(np.arange(T) < off[0]) | (np.arange(T) >= off[-1])] = -1
+    assert np.array_equal(res["seg_id"], ref_seg)
+    for b in (0, 17, B - 1):
+        s, e = off[b], off[b + 1]
+        w = orc.entropy_weights(res["H"][s:e])
+        gu.assert_pooled_close(res["pooled"][[b]], orc.pool(hidden[s:e], w)[None, :])
+    y_ref, _ = orc.head_forward(res["pooled"], head.W1, head.b1, head.W2, head.b2)
+    gu.assert_length_close(res["yhat"], y_ref)
