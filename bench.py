@@ -339,13 +339,18 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     for t in range(warm):
         egtp.plp_step(ctx, st, lm, head.c, hs[t], reset_src=reset[t], yrem_out=yrem, status_dev=status)
     torch.cuda.synchronize()
-    egtp.egtp_profile_enable(ctx, True)
-    egtp.egtp_profile_read(ctx)
+    # pass 1: step times, no per-kernel events in the stream (they cost a few microseconds per step here)
     evs = [torch.cuda.Event(enable_timing=True) for _ in range(plp_steps + 1)]
     evs[0].record()
     for t in range(plp_steps):
         egtp.plp_step(ctx, st, lm, head.c, hs[warm + t], reset_src=reset[warm + t], yrem_out=yrem, status_dev=status)
         evs[t + 1].record()
+    torch.cuda.synchronize()
+    # pass 2: the same steps again with every kernel bracketed by events (per-kernel breakdown)
+    egtp.egtp_profile_enable(ctx, True)
+    egtp.egtp_profile_read(ctx)
+    for t in range(plp_steps):
+        egtp.plp_step(ctx, st, lm, head.c, hs[warm + t], reset_src=reset[warm + t], yrem_out=yrem, status_dev=status)
     torch.cuda.synchronize()
     prof = egtp.egtp_profile_read(ctx)
     assert int(status.item()) == 0
@@ -369,14 +374,22 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     for t in range(3):
         egtp.plp_step_from_logits(ctx, st, logits, head.c, hs[t], reset_src=reset[t], yrem_out=yrem, status_dev=status)
     torch.cuda.synchronize()
-    egtp.egtp_profile_read(ctx)
     n_fl = max(8, plp_steps)
+
+    def from_logits_steps():
+        for t in range(n_fl):
+            egtp.plp_step_from_logits(ctx, st, logits, head.c, hs[warm + t % plp_steps],
+                                      reset_src=reset[warm + t % plp_steps], yrem_out=yrem, status_dev=status)
+
+    egtp.egtp_profile_enable(ctx, False)
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     f0.record()
-    for t in range(n_fl):
-        egtp.plp_step_from_logits(ctx, st, logits, head.c, hs[warm + t % plp_steps], reset_src=reset[warm + t % plp_steps],
-                                  yrem_out=yrem, status_dev=status)
+    from_logits_steps()
     f1.record()
+    torch.cuda.synchronize()
+    egtp.egtp_profile_enable(ctx, True)
+    egtp.egtp_profile_read(ctx)
+    from_logits_steps()
     torch.cuda.synchronize()
     prof_fl = egtp.egtp_profile_read(ctx)
     assert int(status.item()) == 0
