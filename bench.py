@@ -30,6 +30,11 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes (read + write) of one launch of the dominant kernel on the bench workload, from the ncu
+# capture summarised in profiles/lmhead_entropy_egtp_mid.md (seed-1 batch, 9555 tokens).  Set to None
+# whenever the kernel or its launch plan changes after the capture.
+NCU_TRAFFIC_LMHEAD_MID_BYTES = 962.4e6 + 10.1e6
+
 METRIC = "egtp_prompt_tokens_per_sec"
 UNIT = "tokens/s"
 
@@ -267,7 +272,8 @@ def run_mine(args):
     achieved = flops / (k1_ms * 1e-3) / 1e12
     peak = peaks["bf16_tflops"] if ms < 2000 else peaks["bf16_tflops_sustained"]
     roofline = dict(bound="tensor", kernel="lmhead_entropy", achieved=achieved, peak=peak, unit="TFLOP/s",
-                    frac=achieved / peak, traffic=None, peak_source=peaks["source"],
+                    frac=achieved / peak, traffic=NCU_TRAFFIC_LMHEAD_MID_BYTES if (world == 1 and T == 9555) else None,
+                    algorithmic_bytes=2.0 * V * d + 2.0 * T * d, peak_source=peaks["source"],
                     ms_per_launch=k1_ms, frac_of_sustained=achieved / peaks["bf16_tflops_sustained"],
                     frac_of_nominal_2250=achieved / 2250.0)
     pool = prof["pool"]
