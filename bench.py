@@ -439,6 +439,22 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
                            bytes_per_token=2 * d + 4),
                  kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof3.items() if v["launches"]},
                  plan=egtp.egtp_lmhead_plan(ctx, wl3.T, d, V, egtp.EGTP_BF16))
+    # ---- the paper's pooling comparators (Table 3) on the same batch: pooling alone, no LM head
+    comp = {}
+    pooled = torch.empty(wl3.B, d, device="cuda", dtype=torch.float32)
+    for name, mode in (("mean", egtp.EGTP_POOL_MEAN), ("max", egtp.EGTP_POOL_MAX), ("last", egtp.EGTP_POOL_LAST)):
+        for _ in range(3):
+            egtp.egtp_pool_baseline(ctx, None, hidden, off, wl3.B, wl3.T, mode, pooled_out=pooled, status_dev=status)
+        torch.cuda.synchronize()
+        egtp.egtp_profile_read(ctx)
+        for _ in range(10):
+            egtp.egtp_pool_baseline(ctx, None, hidden, off, wl3.B, wl3.T, mode, pooled_out=pooled, status_dev=status)
+        pr = egtp.egtp_profile_read(ctx)
+        us = pr["pool"]["ms"] / pr["pool"]["launches"] * 1e3
+        touched = 2.0 * d * (wl3.B if name == "last" else wl3.T)      # last-token pooling reads one row per prompt
+        comp[name] = dict(pool_us=us, gbs=touched / (us * 1e-6) / 1e9)
+    long_["pooling_comparators"] = comp
+    assert int(status.item()) == 0
     egtp.egtp_destroy(ctx)
     return plp, long_
 

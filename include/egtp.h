@@ -247,6 +247,20 @@ EGTP_API int plp_step_from_logits(egtp_ctx* ctx, plp_state* st, const void* logi
                                   float* Hstep_out, float* z_out, float* yrem_out,
                                   int32_t* status_dev, void* stream);
 
+/* The pooling alternatives the paper compares EGTP against (ablation, Table 3): average pooling,
+ * max pooling and last-token pooling over the same ragged batch, followed by the same head.  No LM
+ * head and no entropy are involved.  An empty prompt pools to zero.
+ *   hidden      device, [T_total][ldh] rows in `dtype` (EGTP_F32 / EGTP_BF16), d a multiple of 16
+ *   offsets     device, int32 [B+1], as in egtp_predict (checked on the device)
+ *   mode        EGTP_POOL_MEAN, EGTP_POOL_MAX or EGTP_POOL_LAST
+ *   pooled_out  device, float [B][d] or NULL;  yhat_out device, float [B] or NULL (needs head)
+ * status_dev and stream as in egtp_predict. */
+enum { EGTP_POOL_MEAN = 1, EGTP_POOL_MAX = 2, EGTP_POOL_LAST = 3 };
+EGTP_API int egtp_pool_baseline(egtp_ctx* ctx, const egtp_head* head, const void* hidden, int64_t ldh,
+                                int32_t dtype, int32_t d, const int32_t* offsets, int32_t B, int64_t T_total,
+                                int32_t mode, float* pooled_out, float* yhat_out,
+                                int32_t* status_dev, void* stream);
+
 /* Tile shape of the LM-head kernel.  EGTP_LMHEAD_AUTO (default): one CTA per SM, 128 x 256 tiles for
  * prompt batches and the two decode shapes for <= 256 rows.  EGTP_LMHEAD_CTA_PAIRS: clusters of two
  * CTAs work on 256 x 256 tiles with tcgen05.mma.cta_group::2 wherever more than 128 rows are given

@@ -35,6 +35,9 @@ HEAD_SCALAR = 0
 HEAD_BINS = 1
 RESET_KEEP = -2
 RESET_EMPTY = -1
+POOL_MEAN = 1
+POOL_MAX = 2
+POOL_LAST = 3
 
 
 # --------------------------------------------------------------------------- #
@@ -113,6 +116,33 @@ def softmax_state(H_seg: np.ndarray, alpha: float = 1.0):
     a = np.asarray(H_seg, dtype=np.float64) / float(alpha)
     M = float(a.max())
     return M, float(np.exp(a - M).sum())
+
+
+def pool_baseline(hidden_seg: np.ndarray, mode: int) -> np.ndarray:
+    """The pooling alternatives of the paper's ablation (Table 3): average, max and last-token pooling."""
+    h = np.asarray(hidden_seg, dtype=np.float64)
+    if mode == POOL_MEAN:
+        return h.sum(axis=0) / h.shape[0]
+    if mode == POOL_MAX:
+        return h.max(axis=0)
+    if mode == POOL_LAST:
+        return h[-1].copy()
+    raise ValueError("unknown pooling mode")
+
+
+def baseline_predict(hidden, offsets, head, mode: int):
+    """Table 3 comparators over a ragged batch: pooled [B, d] (zeros for an empty prompt) and the head's prediction."""
+    hidden = np.asarray(hidden)
+    off = np.asarray(offsets, dtype=np.int64)
+    if not offsets_valid(off, hidden.shape[0]):
+        raise ValueError("offsets must be non-decreasing and lie in [0, T]")
+    B = off.shape[0] - 1
+    pooled = np.zeros((B, hidden.shape[1]), dtype=np.float64)
+    for b in range(B):
+        if off[b + 1] > off[b]:
+            pooled[b] = pool_baseline(hidden[off[b]:off[b + 1]], mode)
+    yhat, phat = head_forward(pooled, head.W1, head.b1, head.W2, head.b2, head.mode, head.centres)
+    return dict(pooled=pooled, yhat=yhat, phat=phat)
 
 
 # --------------------------------------------------------------------------- #

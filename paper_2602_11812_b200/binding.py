@@ -25,6 +25,7 @@ EGTP_F32, EGTP_BF16 = 0, 1
 EGTP_HEAD_SCALAR, EGTP_HEAD_BINS = 0, 1
 PLP_RESET_KEEP, PLP_RESET_EMPTY = -2, -1
 EGTP_LMHEAD_AUTO, EGTP_LMHEAD_CTA_PAIRS = 0, 1
+EGTP_POOL_MEAN, EGTP_POOL_MAX, EGTP_POOL_LAST = 1, 2, 3
 KERNEL_IDS = ["validate_offsets", "lmhead_entropy", "entropy_merge", "segment_weights", "pool",
               "pool_combine", "head_hidden", "head_out", "plp_update", "logits_entropy"]
 EGTP_NUM_KERNELS = len(KERNEL_IDS)
@@ -35,7 +36,7 @@ EXPORTED_SYMBOLS = [
     "egtp_predict_host", "plp_state_create", "plp_state_destroy", "plp_state_export", "plp_state_import",
     "plp_step", "plp_step_host", "egtp_profile_enable", "egtp_profile_read", "egtp_kernel_name",
     "egtp_launch_count", "egtp_lmhead_plan", "egtp_head_forward_static", "egtp_set_lmhead_mode",
-    "egtp_entropy_from_logits", "plp_step_from_logits",
+    "egtp_entropy_from_logits", "plp_step_from_logits", "egtp_pool_baseline",
 ]
 
 
@@ -83,6 +84,7 @@ def load() -> C.CDLL:
     lib.egtp_lmhead_plan.argtypes = [vp, i64, i32, i32, i32, P(i32)]
     lib.egtp_profile_enable.argtypes = [vp, C.c_int]
     lib.egtp_set_lmhead_mode.argtypes = [vp, C.c_int]
+    lib.egtp_pool_baseline.argtypes = [vp, P(egtp_head), vp, i64, i32, i32, vp, i32, i64, i32, vp, vp, vp, vp]
     lib.egtp_entropy_from_logits.argtypes = [vp, vp, i64, i32, i64, i32, vp, vp, vp]
     lib.plp_step_from_logits.argtypes = [vp, vp, vp, i64, i32, i32, P(egtp_head), vp, i64, i32, vp, vp, vp, vp, vp, i32, i32,
                                          f32, vp, vp, vp, vp, vp]
@@ -317,4 +319,15 @@ def plp_step_from_logits(ctx: int, st: int, logits, head: Optional[egtp_head], h
                                      _ptr(Hstep_out), _ptr(z_out), _ptr(yrem_out), _ptr(status_dev), _stream(stream))
     if check:
         _check(rc, "plp_step_from_logits")
+    return rc
+
+
+def egtp_pool_baseline(ctx: int, head: Optional[egtp_head], hidden, offsets, B: int, T_total: int, mode: int,
+                       pooled_out=None, yhat_out=None, status_dev=None, stream=None, check: bool = True) -> int:
+    """Average / max / last-token pooling (the paper's ablation comparators) over a ragged batch, then the head."""
+    rc = load().egtp_pool_baseline(ctx, C.byref(head) if head is not None else None, _ptr(hidden), hidden.stride(0),
+                                   _dtype_code(hidden), hidden.shape[1], _ptr(offsets), B, T_total, mode,
+                                   _ptr(pooled_out), _ptr(yhat_out), _ptr(status_dev), _stream(stream))
+    if check:
+        _check(rc, "egtp_pool_baseline")
     return rc

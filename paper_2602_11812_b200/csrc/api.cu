@@ -441,17 +441,59 @@ int egtp_predict(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, con
   }
   if (T_total > 0) {
     LaunchScope ls(c, EGTP_K_POOL, stream);
-    EGTP_CUDA_TRY(launch_pool(hidden, ldh, lm->dtype == EGTP_BF16, weights, offsets, B, T_total, d, pooled,
+    EGTP_CUDA_TRY(launch_pool(hidden, ldh, lm->dtype == EGTP_BF16, false, weights, offsets, B, T_total, d, pooled,
                               c->piece_a, c->piece_b, status, stream));
   }
   {
     LaunchScope ls(c, EGTP_K_POOL_COMBINE, stream);
-    EGTP_CUDA_TRY(launch_pool_combine(offsets, B, d, c->piece_a, c->piece_b, pooled, status, stream));
+    EGTP_CUDA_TRY(launch_pool_combine(offsets, B, d, false, c->piece_a, c->piece_b, pooled, status, stream));
   }
   if (head && (yhat_out || phat_out)) {
     int rc = run_head(c, head, pooled, d, B, yhat_out, phat_out, status, stream);
     if (rc != EGTP_OK) return rc;
   }
+  return EGTP_OK;
+}
+
+int egtp_pool_baseline(egtp_ctx* c, const egtp_head* head, const void* hidden, int64_t ldh, int32_t dtype, int32_t d,
+                       const int32_t* offsets, int32_t B, int64_t T_total, int32_t mode, float* pooled_out,
+                       float* yhat_out, int32_t* status_dev, void* stream_v) {
+  if (!c || !hidden || !offsets || B < 0 || T_total < 0 || d <= 0 || ldh < d) return EGTP_ERR_INVALID_ARG;
+  if (mode != EGTP_POOL_MEAN && mode != EGTP_POOL_MAX && mode != EGTP_POOL_LAST) return EGTP_ERR_INVALID_ARG;
+  if (!head && yhat_out) return EGTP_ERR_INVALID_ARG;
+  if (dtype != EGTP_F32 && dtype != EGTP_BF16) return EGTP_ERR_UNSUPPORTED;
+  if (d % 16 != 0 || (ldh * elem_bytes(dtype)) % 16 != 0 || reinterpret_cast<uintptr_t>(hidden) % 16 != 0)
+    return EGTP_ERR_UNSUPPORTED;
+  if (T_total > c->max_tokens || B > c->max_batch || d > c->max_d) return EGTP_ERR_CAPACITY;
+  if (B == 0) return EGTP_OK;
+  if (head) {
+    int rc = check_head(c, head, d);
+    if (rc != EGTP_OK) return rc;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  int32_t* status = status_dev ? status_dev : c->status;
+  if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
+  float* pooled = pooled_out ? pooled_out : c->pooled;
+  const bool take_max = mode == EGTP_POOL_MAX;
+  {
+    LaunchScope ls(c, EGTP_K_VALIDATE, stream);
+    EGTP_CUDA_TRY(launch_validate_offsets(offsets, B, T_total, status, stream));
+  }
+  if (!take_max && T_total > 0) {
+    LaunchScope ls(c, EGTP_K_SEGMENT_WEIGHTS, stream);
+    EGTP_CUDA_TRY(launch_baseline_weights(offsets, B, mode, c->weights, status, stream));
+  }
+  if (T_total > 0) {
+    LaunchScope ls(c, EGTP_K_POOL, stream);
+    EGTP_CUDA_TRY(launch_pool(hidden, ldh, dtype == EGTP_BF16, take_max, c->weights, offsets, B, T_total, d, pooled,
+                              c->piece_a, c->piece_b, status, stream));
+  }
+  {
+    LaunchScope ls(c, EGTP_K_POOL_COMBINE, stream);
+    EGTP_CUDA_TRY(launch_pool_combine(offsets, B, d, take_max, c->piece_a, c->piece_b, pooled, status, stream));
+  }
+  if (head && yhat_out) return run_head(c, head, pooled, d, B, yhat_out, nullptr, status, stream);
   return EGTP_OK;
 }
 

@@ -61,12 +61,17 @@ cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t T, fl
 cudaError_t launch_segment_weights(const float* H, const int32_t* offsets, int B, float inv_alpha, float* weights,
                                    float* seg_m, float* seg_s, const int32_t* status, cudaStream_t stream);
 
-cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, const float* weights, const int32_t* offsets,
-                        int B, int64_t T, int d, float* pooled, float* piece_a, float* piece_b,
-                        const int32_t* status, cudaStream_t stream);
+// weights of average (w = 1/n) or last-token (one-hot) pooling for every prompt
+cudaError_t launch_baseline_weights(const int32_t* offsets, int B, int mode, float* weights, const int32_t* status,
+                                    cudaStream_t stream);
 
-cudaError_t launch_pool_combine(const int32_t* offsets, int B, int d, const float* piece_a, const float* piece_b,
-                                float* pooled, const int32_t* status, cudaStream_t stream);
+// take_max: channel-wise maximum instead of the weighted sum (weights unused)
+cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, bool take_max, const float* weights,
+                        const int32_t* offsets, int B, int64_t T, int d, float* pooled, float* piece_a,
+                        float* piece_b, const int32_t* status, cudaStream_t stream);
+
+cudaError_t launch_pool_combine(const int32_t* offsets, int B, int d, bool take_max, const float* piece_a,
+                                const float* piece_b, float* pooled, const int32_t* status, cudaStream_t stream);
 
 // ---- Eq. 2 from logits already in memory -------------------------------------------------------
 int logits_entropy_pick_splits(int64_t rows, int V, int num_sms);

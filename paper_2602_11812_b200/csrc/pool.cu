@@ -120,6 +120,19 @@ __global__ void segment_weights_kernel(const float* __restrict__ H, const int32_
   }
 }
 
+// Weights of the pooling alternatives in the paper's ablation (Table 3) that are weighted sums:
+// average pooling (w = 1/n) and last-token pooling (w = 1 on the prompt's last token).
+__global__ void baseline_weights_kernel(const int32_t* __restrict__ off, int B, int mode, float* __restrict__ weights,
+                                        const int32_t* __restrict__ status) {
+  if (*status != 0) return;
+  const int b = blockIdx.x;
+  const int s0 = off[b], s1 = off[b + 1];
+  if (s1 <= s0) return;
+  const float inv_n = 1.f / static_cast<float>(s1 - s0);
+  for (int i = s0 + threadIdx.x; i < s1; i += blockDim.x)
+    weights[i] = mode == EGTP_POOL_MEAN ? inv_n : (i == s1 - 1 ? 1.f : 0.f);
+}
+
 // --------------------------------------------------------------------------- Eq. 4: pooling
 template <typename T>
 struct Row8;
@@ -155,7 +168,9 @@ __device__ __forceinline__ void store8(float* p, const float (&v)[8]) {
 // that crosses chunk borders leaves one piece per chunk: piece_a[c] if it entered from the
 // left, piece_b[c] if it starts here and leaves to the right.  The combine kernel adds the
 // pieces of each prompt in chunk order.
-template <typename T>
+// With kMax the weights are ignored and the channel-wise maximum is taken instead of the weighted sum
+// (max pooling, Table 3); pieces of a prompt that spans chunks are then combined with max.
+template <typename T, bool kMax>
 __global__ void __launch_bounds__(kPoolThreads)
 pool_kernel(const T* __restrict__ hidden, int64_t ldh, const float* __restrict__ weights,
             const int32_t* __restrict__ off, int B, int d, float* __restrict__ pooled,
@@ -174,32 +189,46 @@ pool_kernel(const T* __restrict__ hidden, int64_t ldh, const float* __restrict__
     const int64_t run_end = min(seg_end, t1);
     float acc[8];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+    for (int k = 0; k < 8; ++k) acc[k] = kMax ? -INFINITY : 0.f;
     const T* rowp = hidden + t0 * ldh + col;
     int64_t t = t0;
     for (; t + 4 <= run_end; t += 4) {           // four rows in flight per thread
+      float w0 = 0.f, w1 = 0.f, w2 = 0.f, w3 = 0.f;
+      if constexpr (!kMax) {
+        w0 = __ldg(weights + t); w1 = __ldg(weights + t + 1); w2 = __ldg(weights + t + 2); w3 = __ldg(weights + t + 3);
+        // rows that carry no weight (last-token pooling: all but one) are not read at all
+        if (w0 == 0.f && w1 == 0.f && w2 == 0.f && w3 == 0.f) { rowp += 4 * ldh; continue; }
+      }
       float v0[8], v1[8], v2[8], v3[8];
       Row8<T>::load(rowp, v0);
       Row8<T>::load(rowp + ldh, v1);
       Row8<T>::load(rowp + 2 * ldh, v2);
       Row8<T>::load(rowp + 3 * ldh, v3);
-      const float w0 = __ldg(weights + t), w1 = __ldg(weights + t + 1), w2 = __ldg(weights + t + 2),
-                  w3 = __ldg(weights + t + 3);
+      if constexpr (kMax) {
 #pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        acc[k] = fmaf(w0, v0[k], acc[k]);
-        acc[k] = fmaf(w1, v1[k], acc[k]);
-        acc[k] = fmaf(w2, v2[k], acc[k]);
-        acc[k] = fmaf(w3, v3[k], acc[k]);
+        for (int k = 0; k < 8; ++k) acc[k] = fmaxf(fmaxf(acc[k], fmaxf(v0[k], v1[k])), fmaxf(v2[k], v3[k]));
+      } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          acc[k] = fmaf(w0, v0[k], acc[k]);
+          acc[k] = fmaf(w1, v1[k], acc[k]);
+          acc[k] = fmaf(w2, v2[k], acc[k]);
+          acc[k] = fmaf(w3, v3[k], acc[k]);
+        }
       }
       rowp += 4 * ldh;
     }
     for (; t < run_end; ++t) {
       float v0[8];
       Row8<T>::load(rowp, v0);
-      const float w0 = __ldg(weights + t);
+      if constexpr (kMax) {
 #pragma unroll
-      for (int k = 0; k < 8; ++k) acc[k] = fmaf(w0, v0[k], acc[k]);
+        for (int k = 0; k < 8; ++k) acc[k] = fmaxf(acc[k], v0[k]);
+      } else {
+        const float w0 = __ldg(weights + t);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) acc[k] = fmaf(w0, v0[k], acc[k]);
+      }
       rowp += ldh;
     }
     float* dst;
@@ -214,6 +243,7 @@ pool_kernel(const T* __restrict__ hidden, int64_t ldh, const float* __restrict__
 
 // One block per prompt (x) and 1024-channel slab (y): zero for an empty prompt, nothing for a
 // prompt finished by the first stage, else piece_b[c0] + piece_a[c0+1] + ... + piece_a[c1].
+template <bool kMax>
 __global__ void __launch_bounds__(kPoolThreads)
 pool_combine_kernel(const int32_t* __restrict__ off, int B, int d, const float* __restrict__ piece_a,
                     const float* __restrict__ piece_b, float* __restrict__ pooled,
@@ -239,8 +269,9 @@ pool_combine_kernel(const int32_t* __restrict__ off, int B, int d, const float* 
   for (int64_t c = c0 + 1; c <= c1; ++c) {
     const float4* p = reinterpret_cast<const float4*>(piece_a + c * d + col);
     const float4 a = p[0], bq = p[1];
-    acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
-    acc[4] += bq.x; acc[5] += bq.y; acc[6] += bq.z; acc[7] += bq.w;
+    const float pv[8] = {a.x, a.y, a.z, a.w, bq.x, bq.y, bq.z, bq.w};
+#pragma unroll
+    for (int k = 0; k < 8; ++k) acc[k] = kMax ? fmaxf(acc[k], pv[k]) : acc[k] + pv[k];
   }
   store8(dst, acc);
 }
@@ -268,28 +299,39 @@ cudaError_t launch_segment_weights(const float* H, const int32_t* offsets, int B
   return cudaGetLastError();
 }
 
-cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, const float* weights, const int32_t* offsets,
-                        int B, int64_t T, int d, float* pooled, float* piece_a, float* piece_b,
-                        const int32_t* status, cudaStream_t stream) {
-  const unsigned chunks = static_cast<unsigned>((T + kPoolChunkTokens - 1) / kPoolChunkTokens);
-  const unsigned slabs = static_cast<unsigned>((d + kPoolThreads * 8 - 1) / (kPoolThreads * 8));
-  dim3 grid(chunks, slabs);
-  if (bf16) {
-    pool_kernel<__nv_bfloat16><<<grid, kPoolThreads, 0, stream>>>(static_cast<const __nv_bfloat16*>(hidden), ldh,
-                                                                  weights, offsets, B, d, pooled, piece_a, piece_b,
-                                                                  status);
-  } else {
-    pool_kernel<float><<<grid, kPoolThreads, 0, stream>>>(static_cast<const float*>(hidden), ldh, weights, offsets,
-                                                          B, d, pooled, piece_a, piece_b, status);
-  }
+cudaError_t launch_baseline_weights(const int32_t* offsets, int B, int mode, float* weights, const int32_t* status,
+                                    cudaStream_t stream) {
+  baseline_weights_kernel<<<B, 256, 0, stream>>>(offsets, B, mode, weights, status);
   return cudaGetLastError();
 }
 
-cudaError_t launch_pool_combine(const int32_t* offsets, int B, int d, const float* piece_a, const float* piece_b,
-                                float* pooled, const int32_t* status, cudaStream_t stream) {
+cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, bool take_max, const float* weights,
+                        const int32_t* offsets, int B, int64_t T, int d, float* pooled, float* piece_a,
+                        float* piece_b, const int32_t* status, cudaStream_t stream) {
+  const unsigned chunks = static_cast<unsigned>((T + kPoolChunkTokens - 1) / kPoolChunkTokens);
+  const unsigned slabs = static_cast<unsigned>((d + kPoolThreads * 8 - 1) / (kPoolThreads * 8));
+  dim3 grid(chunks, slabs);
+  const __nv_bfloat16* hb = static_cast<const __nv_bfloat16*>(hidden);
+  const float* hf = static_cast<const float*>(hidden);
+  if (bf16 && take_max)
+    pool_kernel<__nv_bfloat16, true><<<grid, kPoolThreads, 0, stream>>>(hb, ldh, weights, offsets, B, d, pooled, piece_a, piece_b, status);
+  else if (bf16)
+    pool_kernel<__nv_bfloat16, false><<<grid, kPoolThreads, 0, stream>>>(hb, ldh, weights, offsets, B, d, pooled, piece_a, piece_b, status);
+  else if (take_max)
+    pool_kernel<float, true><<<grid, kPoolThreads, 0, stream>>>(hf, ldh, weights, offsets, B, d, pooled, piece_a, piece_b, status);
+  else
+    pool_kernel<float, false><<<grid, kPoolThreads, 0, stream>>>(hf, ldh, weights, offsets, B, d, pooled, piece_a, piece_b, status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pool_combine(const int32_t* offsets, int B, int d, bool take_max, const float* piece_a,
+                                const float* piece_b, float* pooled, const int32_t* status, cudaStream_t stream) {
   const unsigned slabs = static_cast<unsigned>((d + kPoolThreads * 8 - 1) / (kPoolThreads * 8));
   dim3 grid(B, slabs);
-  pool_combine_kernel<<<grid, kPoolThreads, 0, stream>>>(offsets, B, d, piece_a, piece_b, pooled, status);
+  if (take_max)
+    pool_combine_kernel<true><<<grid, kPoolThreads, 0, stream>>>(offsets, B, d, piece_a, piece_b, pooled, status);
+  else
+    pool_combine_kernel<false><<<grid, kPoolThreads, 0, stream>>>(offsets, B, d, piece_a, piece_b, pooled, status);
   return cudaGetLastError();
 }
 

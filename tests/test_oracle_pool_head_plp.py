@@ -244,3 +244,30 @@ def test_plp_fan_out_identical_streams_stay_identical():
     out = orc.plp_run(hs, reset, W, head, prompts=dict(hidden=p_hidden, offsets=p_off, H=eg["H"]))
     for s in range(1, 4):
         assert np.array_equal(out["z"][:, s], out["z"][:, 0]) and np.array_equal(out["yrem"][:, s], out["yrem"][:, 0])
+
+
+# ----------------------------- Table 3: pooling alternatives ----------------- #
+def test_baseline_pooling_definitions():
+    rng = np.random.default_rng(10)
+    rows = rng.standard_normal((7, 5))
+    mean, mx, last = (orc.pool_baseline(rows, m) for m in (orc.POOL_MEAN, orc.POOL_MAX, orc.POOL_LAST))
+    for k in range(5):
+        assert abs(mean[k] - math.fsum(rows[i, k] for i in range(7)) / 7) < 1e-15
+        assert mx[k] == max(rows[i, k] for i in range(7))
+        assert last[k] == rows[6, k]
+    # average pooling is EGTP with equal entropies; a one-token prompt makes all variants that token
+    assert np.allclose(mean, orc.pool(rows, orc.entropy_weights(np.zeros(7))), atol=1e-15)
+    for m in (orc.POOL_MEAN, orc.POOL_MAX, orc.POOL_LAST):
+        assert np.array_equal(orc.pool_baseline(rows[2:3], m), rows[2])
+    # max and mean ignore token order, last-token pooling does not
+    perm = rng.permutation(7)
+    assert np.array_equal(orc.pool_baseline(rows[perm], orc.POOL_MAX), mx)
+    assert np.allclose(orc.pool_baseline(rows[perm], orc.POOL_MEAN), mean, atol=1e-15)
+    assert np.all(mx >= mean) and np.all(mx >= last)
+    head = _head(rng, 5, 3, 1)
+    out = orc.baseline_predict(rows, np.array([0, 3, 3, 7]), head, orc.POOL_LAST)
+    assert np.array_equal(out["pooled"][0], rows[2]) and np.all(out["pooled"][1] == 0) and np.array_equal(out["pooled"][2], rows[6])
+    y, _ = orc.head_forward(rows[6], head.W1, head.b1, head.W2, head.b2)
+    assert out["yhat"][2] == y[0]
+    with pytest.raises(ValueError):
+        orc.pool_baseline(rows, 9)
