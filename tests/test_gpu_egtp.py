@@ -231,3 +231,17 @@ def test_many_tokens_small_model_64bit_indexing():
         gu.assert_pooled_close(res["pooled"][[b]], orc.pool(hidden[s:e], w)[None, :])
     y_ref, _ = orc.head_forward(res["pooled"], head.W1, head.b1, head.W2, head.b2)
     gu.assert_length_close(res["yhat"], y_ref)
+
+
+@pytest.mark.parametrize("T,d,V", [(3, 16, 40), (129, 32, 300), (256, 48, 1000), (257, 80, 1000), (128, 272, 31), (1, 2048, 9)])
+def test_small_and_boundary_shapes(ctx, T, d, V):
+    # row counts on both sides of the 128 / 256-row launch shapes, hidden sizes that are not multiples of
+    # the 64-element k block, vocabularies smaller than one tile
+    rng = np.random.default_rng(T * 1000 + d + V)
+    lengths = [T] if T < 4 else [T // 3, T - T // 3 - 1, 1]
+    hidden = gen.round_to_bf16((rng.standard_normal((T, d)) * 1.5).astype(np.float32))
+    W = gen.round_to_bf16((rng.standard_normal((V, d)) * (2.0 / np.sqrt(d))).astype(np.float32))
+    head = gen.make_head(5, d, 24, 1, "bf16")
+    wl = gen.EgtpWorkload("small", "bf16", hidden, gen.offsets_from_lengths(lengths), W, head)
+    ref = orc.egtp_predict(hidden, wl.offsets, W, head)
+    _check_all(gu.run_egtp(ctx, wl), ref, wl)
