@@ -374,6 +374,39 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
                            unit="TFLOP/s", frac=2.0 * slots * d * V / (k1_us * 1e-6) / 1e12 / peaks["bf16_tflops"]),
                kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof.items() if v["launches"]},
                plan=egtp.egtp_lmhead_plan(ctx, slots, d, V, egtp.EGTP_BF16))
+    # ---- the same step captured once in a CUDA graph and replayed (fixed buffers; removes launch gaps)
+    try:
+        static_h = hs[warm].clone()
+        static_r = reset[warm].clone()
+        static_r.fill_(-2)                       # keep: replays continue the running state
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            egtp.plp_step(ctx, st, lm, head.c, static_h, reset_src=static_r, yrem_out=yrem, status_dev=status)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        egtp.egtp_profile_enable(ctx, False)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            egtp.plp_step(ctx, st, lm, head.c, static_h, reset_src=static_r, yrem_out=yrem, status_dev=status)
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for t in range(plp_steps):
+            static_h.copy_(hs[warm + t], non_blocking=True)      # the step's new tokens (0.2 MB device copy)
+            graph.replay()
+        g1.record()
+        torch.cuda.synchronize()
+        plp["cuda_graph_us_per_step"] = g0.elapsed_time(g1) / plp_steps * 1e3
+        del graph
+    except Exception as exc:  # capture is a convenience measurement, never a requirement
+        plp["cuda_graph_us_per_step"] = None
+        plp["cuda_graph_error"] = str(exc)[:200]
+    egtp.egtp_profile_enable(ctx, True)
+    assert int(status.item()) == 0
+
     # ---- the same decode step when the serving engine already holds the step's logits
     torch.manual_seed(0)
     logits = (torch.randn(slots, V, device="cuda") * 1.5).to(torch.bfloat16)
