@@ -247,6 +247,32 @@ EGTP_API int plp_step_from_logits(egtp_ctx* ctx, plp_state* st, const void* logi
                                   float* Hstep_out, float* z_out, float* yrem_out,
                                   int32_t* status_dev, void* stream);
 
+/* Vocabulary-parallel form of Eq. 2 for LM heads that are sharded over several GPUs (tensor-parallel
+ * serving): each GPU holds the rows [v0, v1) of W and can only see its part of every token's
+ * distribution.  A shard reduces its part to one triple per token,
+ *   m = max_v x_v,  s = sum_v 2^((x_v - m) log2 e),  t2 = sum_v 2^(..) * (x_v - m) log2 e,
+ * the ranks exchange the triples (one all-gather of rows * 3 floats per rank: the path's only
+ * collective, done by the caller, e.g. with NCCL), and every rank merges them: triples of disjoint
+ * vocabulary ranges combine exactly like the per-chunk partials inside one GPU.
+ *
+ * egtp_entropy_partials: partial_out (device, float [rows][3]) for this GPU's shard `lm_shard`
+ *   (W pointing at the shard's first row, V = rows of the shard), hidden [rows][ldh] as in egtp_predict.
+ * egtp_entropy_from_partials: gathered (device, float [num_shards][rows][3], rank-major as an
+ *   all-gather leaves it) -> H_out (device, float [rows]).
+ * plp_step_from_partials: plp_step with the step's entropies taken from such gathered triples
+ *   (gathered [num_shards][B_live][3]); all other arguments as in plp_step_from_logits. */
+EGTP_API int egtp_entropy_partials(egtp_ctx* ctx, const egtp_lm_head* lm_shard, const void* hidden, int64_t ldh,
+                                   int64_t rows, float* partial_out, int32_t* status_dev, void* stream);
+EGTP_API int egtp_entropy_from_partials(egtp_ctx* ctx, const float* gathered, int32_t num_shards, int64_t rows,
+                                        float* H_out, int32_t* status_dev, void* stream);
+EGTP_API int plp_step_from_partials(egtp_ctx* ctx, plp_state* st, const float* gathered, int32_t num_shards,
+                                    const egtp_head* head, const void* hidden_step, int64_t ldh, int32_t hidden_dtype,
+                                    const int32_t* slot_ids, const int32_t* reset_src,
+                                    const float* src_m, const float* src_s, const float* src_pooled, int32_t n_src,
+                                    int32_t B_live, float alpha,
+                                    float* Hstep_out, float* z_out, float* yrem_out,
+                                    int32_t* status_dev, void* stream);
+
 /* The pooling alternatives the paper compares EGTP against (ablation, Table 3): average pooling,
  * max pooling and last-token pooling over the same ragged batch, followed by the same head.  No LM
  * head and no entropy are involved.  An empty prompt pools to zero.

@@ -37,6 +37,7 @@ EXPORTED_SYMBOLS = [
     "plp_step", "plp_step_host", "egtp_profile_enable", "egtp_profile_read", "egtp_kernel_name",
     "egtp_launch_count", "egtp_lmhead_plan", "egtp_head_forward_static", "egtp_set_lmhead_mode",
     "egtp_entropy_from_logits", "plp_step_from_logits", "egtp_pool_baseline",
+    "egtp_entropy_partials", "egtp_entropy_from_partials", "plp_step_from_partials",
 ]
 
 
@@ -84,6 +85,10 @@ def load() -> C.CDLL:
     lib.egtp_lmhead_plan.argtypes = [vp, i64, i32, i32, i32, P(i32)]
     lib.egtp_profile_enable.argtypes = [vp, C.c_int]
     lib.egtp_set_lmhead_mode.argtypes = [vp, C.c_int]
+    lib.egtp_entropy_partials.argtypes = [vp, P(egtp_lm_head), vp, i64, i64, vp, vp, vp]
+    lib.egtp_entropy_from_partials.argtypes = [vp, vp, i32, i64, vp, vp, vp]
+    lib.plp_step_from_partials.argtypes = [vp, vp, vp, i32, P(egtp_head), vp, i64, i32, vp, vp, vp, vp, vp, i32, i32, f32,
+                                           vp, vp, vp, vp, vp]
     lib.egtp_pool_baseline.argtypes = [vp, P(egtp_head), vp, i64, i32, i32, vp, i32, i64, i32, vp, vp, vp, vp]
     lib.egtp_entropy_from_logits.argtypes = [vp, vp, i64, i32, i64, i32, vp, vp, vp]
     lib.plp_step_from_logits.argtypes = [vp, vp, vp, i64, i32, i32, P(egtp_head), vp, i64, i32, vp, vp, vp, vp, vp, i32, i32,
@@ -330,4 +335,39 @@ def egtp_pool_baseline(ctx: int, head: Optional[egtp_head], hidden, offsets, B: 
                                    _ptr(pooled_out), _ptr(yhat_out), _ptr(status_dev), _stream(stream))
     if check:
         _check(rc, "egtp_pool_baseline")
+    return rc
+
+
+def egtp_entropy_partials(ctx: int, lm_shard: egtp_lm_head, hidden, partial_out, rows: Optional[int] = None,
+                          status_dev=None, stream=None, check: bool = True) -> int:
+    """(m, s, t2) per row over this GPU's shard of the vocabulary; partial_out float32 [rows, 3]."""
+    rows = hidden.shape[0] if rows is None else rows
+    rc = load().egtp_entropy_partials(ctx, C.byref(lm_shard), _ptr(hidden), hidden.stride(0), rows, _ptr(partial_out),
+                                      _ptr(status_dev), _stream(stream))
+    if check:
+        _check(rc, "egtp_entropy_partials")
+    return rc
+
+
+def egtp_entropy_from_partials(ctx: int, gathered, H_out, status_dev=None, stream=None, check: bool = True) -> int:
+    """gathered float32 [num_shards, rows, 3] (rank-major, as an all-gather leaves it) -> H_out [rows]."""
+    rc = load().egtp_entropy_from_partials(ctx, _ptr(gathered), gathered.shape[0], gathered.shape[1], _ptr(H_out),
+                                           _ptr(status_dev), _stream(stream))
+    if check:
+        _check(rc, "egtp_entropy_from_partials")
+    return rc
+
+
+def plp_step_from_partials(ctx: int, st: int, gathered, head: Optional[egtp_head], hidden_step, slot_ids=None,
+                           reset_src=None, src_m=None, src_s=None, src_pooled=None, n_src: int = 0,
+                           alpha: float = 1.0, Hstep_out=None, z_out=None, yrem_out=None, status_dev=None, stream=None,
+                           check: bool = True) -> int:
+    """plp_step with the step's entropies merged from vocabulary-shard triples gathered [num_shards, B_live, 3]."""
+    rc = load().plp_step_from_partials(ctx, st, _ptr(gathered), gathered.shape[0], C.byref(head) if head is not None else None,
+                                       _ptr(hidden_step), hidden_step.stride(0), _dtype_code(hidden_step), _ptr(slot_ids),
+                                       _ptr(reset_src), _ptr(src_m), _ptr(src_s), _ptr(src_pooled), n_src,
+                                       gathered.shape[1], alpha, _ptr(Hstep_out), _ptr(z_out), _ptr(yrem_out),
+                                       _ptr(status_dev), _stream(stream))
+    if check:
+        _check(rc, "plp_step_from_partials")
     return rc

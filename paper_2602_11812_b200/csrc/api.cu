@@ -239,14 +239,16 @@ int check_plp_common(const egtp_ctx* c, const plp_state* st, const egtp_head* he
 
 // Second half of a PLP step: merge the entropy partials, update the slots (Eq. 8), run the head.
 int plp_update_and_head(egtp_ctx* c, plp_state* st, const egtp_head* head, const void* hidden_step, int64_t ldh,
-                        int hidden_dtype, int slots, const int32_t* slot_ids, const int32_t* reset_src,
+                        int hidden_dtype, const float* partials, int slots, int64_t row_stride, int64_t slot_stride,
+                        const int32_t* slot_ids, const int32_t* reset_src,
                         const float* src_m, const float* src_s, const float* src_pooled, int n_src, int B_live,
                         float alpha, float* Hstep_out, float* z_out, float* yrem_out, int32_t* status,
                         cudaStream_t stream) {
   float* z = z_out ? z_out : c->pooled;
   {
     LaunchScope ls(c, EGTP_K_PLP_UPDATE, stream);
-    EGTP_CUDA_TRY(launch_plp_update(hidden_step, ldh, hidden_dtype == EGTP_BF16, c->partials, slots, Hstep_out, slot_ids,
+    EGTP_CUDA_TRY(launch_plp_update(hidden_step, ldh, hidden_dtype == EGTP_BF16, partials, slots, row_stride, slot_stride, Hstep_out,
+                                    slot_ids,
                                     reset_src, src_m, src_s, src_pooled, n_src, B_live, st->d, st->num_slots,
                                     1.f / alpha, st->m, st->s, st->acc, z, st->d, status, stream));
   }
@@ -431,7 +433,7 @@ int egtp_predict(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, con
     int rc = run_lmhead(c, lm, hidden, ldh, T_total, status, stream, &plan);
     if (rc != EGTP_OK) return rc;
     LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
-    EGTP_CUDA_TRY(launch_entropy_merge(c->partials, plan.slots, T_total, H, offsets, B, seg_id_out, weights, status,
+    EGTP_CUDA_TRY(launch_entropy_merge(c->partials, plan.slots, plan.slots * 3, 3, T_total, H, offsets, B, seg_id_out, weights, status,
                                        stream));
   }
   if (B == 0) return EGTP_OK;
@@ -599,7 +601,7 @@ int plp_step(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head
   LmheadPlan plan;
   rc = run_lmhead(c, lm, hidden_step, ldh, B_live, status, stream, &plan);
   if (rc != EGTP_OK) return rc;
-  return plp_update_and_head(c, st, head, hidden_step, ldh, lm->dtype, plan.slots, slot_ids, reset_src, src_m, src_s,
+  return plp_update_and_head(c, st, head, hidden_step, ldh, lm->dtype, c->partials, plan.slots, plan.slots * 3, 3, slot_ids, reset_src, src_m, src_s,
                              src_pooled, n_src, B_live, alpha, Hstep_out, z_out, yrem_out, status, stream);
 }
 
@@ -615,7 +617,7 @@ int egtp_entropy_from_logits(egtp_ctx* c, const void* logits, int64_t ldl, int32
   int rc = run_logits_entropy(c, logits, ldl, logits_dtype, rows, V, status, stream, &slots);
   if (rc != EGTP_OK) return rc;
   LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
-  EGTP_CUDA_TRY(launch_entropy_merge(c->partials, slots, rows, H_out, nullptr, 0, nullptr, nullptr, status, stream));
+  EGTP_CUDA_TRY(launch_entropy_merge(c->partials, slots, slots * 3, 3, rows, H_out, nullptr, 0, nullptr, nullptr, status, stream));
   return EGTP_OK;
 }
 
@@ -643,8 +645,67 @@ int plp_step_from_logits(egtp_ctx* c, plp_state* st, const void* logits, int64_t
   int slots = 0;
   rc = run_logits_entropy(c, logits, ldl, logits_dtype, B_live, V, status, stream, &slots);
   if (rc != EGTP_OK) return rc;
-  return plp_update_and_head(c, st, head, hidden_step, ldh, hidden_dtype, slots, slot_ids, reset_src, src_m, src_s,
+  return plp_update_and_head(c, st, head, hidden_step, ldh, hidden_dtype, c->partials, slots, slots * 3, 3, slot_ids, reset_src, src_m, src_s,
                              src_pooled, n_src, B_live, alpha, Hstep_out, z_out, yrem_out, status, stream);
+}
+
+int egtp_entropy_partials(egtp_ctx* c, const egtp_lm_head* lm_shard, const void* hidden, int64_t ldh, int64_t rows,
+                          float* partial_out, int32_t* status_dev, void* stream_v) {
+  if (!c || !partial_out || rows < 0) return EGTP_ERR_INVALID_ARG;
+  if (rows == 0) return EGTP_OK;
+  if (rows > std::max<int64_t>(c->max_tokens, c->max_batch)) return EGTP_ERR_CAPACITY;
+  int rc = check_lm(c, lm_shard, hidden, ldh);
+  if (rc != EGTP_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  int32_t* status = status_dev ? status_dev : c->status;
+  if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
+  LmheadPlan plan;
+  rc = run_lmhead(c, lm_shard, hidden, ldh, rows, status, stream, &plan);
+  if (rc != EGTP_OK) return rc;
+  LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
+  EGTP_CUDA_TRY(launch_partials_reduce(c->partials, plan.slots, rows, partial_out, status, stream));
+  return EGTP_OK;
+}
+
+int egtp_entropy_from_partials(egtp_ctx* c, const float* gathered, int32_t num_shards, int64_t rows, float* H_out,
+                               int32_t* status_dev, void* stream_v) {
+  if (!c || !gathered || !H_out || num_shards <= 0 || rows < 0) return EGTP_ERR_INVALID_ARG;
+  if (rows == 0) return EGTP_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  int32_t* status = status_dev ? status_dev : c->status;
+  if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
+  LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
+  EGTP_CUDA_TRY(launch_entropy_merge(gathered, num_shards, 3, rows * 3, rows, H_out, nullptr, 0, nullptr, nullptr, status,
+                                     stream));
+  return EGTP_OK;
+}
+
+int plp_step_from_partials(egtp_ctx* c, plp_state* st, const float* gathered, int32_t num_shards,
+                           const egtp_head* head, const void* hidden_step, int64_t ldh, int32_t hidden_dtype,
+                           const int32_t* slot_ids, const int32_t* reset_src, const float* src_m, const float* src_s,
+                           const float* src_pooled, int32_t n_src, int32_t B_live, float alpha, float* Hstep_out,
+                           float* z_out, float* yrem_out, int32_t* status_dev, void* stream_v) {
+  if (!c || !st || st->ctx != c || !gathered || num_shards <= 0) return EGTP_ERR_INVALID_ARG;
+  if (B_live == 0) return EGTP_OK;
+  int rc = check_plp_common(c, st, head, src_m, src_s, src_pooled, n_src, B_live, alpha, yrem_out);
+  if (rc != EGTP_OK) return rc;
+  if (!hidden_step || ldh < st->d) return EGTP_ERR_INVALID_ARG;
+  if (hidden_dtype != EGTP_F32 && hidden_dtype != EGTP_BF16) return EGTP_ERR_UNSUPPORTED;
+  if ((ldh * elem_bytes(hidden_dtype)) % 16 != 0 || reinterpret_cast<uintptr_t>(hidden_step) % 16 != 0)
+    return EGTP_ERR_UNSUPPORTED;
+  if (head) {
+    rc = check_head(c, head, st->d);
+    if (rc != EGTP_OK) return rc;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  int32_t* status = status_dev ? status_dev : c->status;
+  if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
+  return plp_update_and_head(c, st, head, hidden_step, ldh, hidden_dtype, gathered, num_shards, 3,
+                             static_cast<int64_t>(B_live) * 3, slot_ids, reset_src, src_m, src_s, src_pooled, n_src,
+                             B_live, alpha, Hstep_out, z_out, yrem_out, status, stream);
 }
 
 int plp_step_host(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head* head,

@@ -45,15 +45,27 @@ __device__ __forceinline__ EntropyPartial warp_combine_partials(EntropyPartial p
 
 // All 32 lanes of a warp call this with the same row pointer ([slots][3] floats); every lane
 // returns H.  The order of operations is fixed, so the result is bitwise reproducible.
-__device__ __forceinline__ float merge_partials_warp(const float* __restrict__ row, int slots, int lane) {
-  constexpr float kLn2 = 0.6931471805599453f;
+// slot j of the row lives at row + j * slot_stride (floats): 3 for the LM-head kernel's [row][slot][3]
+// layout, rows * 3 for partials gathered rank-major from several GPUs ([rank][row][3]).
+__device__ __forceinline__ EntropyPartial merge_partials_warp_raw(const float* __restrict__ row, int slots,
+                                                                  int64_t slot_stride, int lane) {
   EntropyPartial acc = {kNegBig, 0.f, 0.f};
   for (int j = lane; j < slots; j += 32) {
-    const EntropyPartial pj = {row[3 * j], row[3 * j + 1], row[3 * j + 2]};
-    acc = combine_partials(acc, pj);
+    const float* pj = row + j * slot_stride;
+    const EntropyPartial q = {pj[0], pj[1], pj[2]};
+    acc = combine_partials(acc, q);
   }
-  acc = warp_combine_partials(acc);
-  return logf(acc.s) - kLn2 * acc.t2 / acc.s;
+  return warp_combine_partials(acc);
+}
+
+__device__ __forceinline__ float entropy_of(const EntropyPartial& p) {
+  constexpr float kLn2 = 0.6931471805599453f;
+  return logf(p.s) - kLn2 * p.t2 / p.s;
+}
+
+__device__ __forceinline__ float merge_partials_warp(const float* __restrict__ row, int slots, int64_t slot_stride,
+                                                     int lane) {
+  return entropy_of(merge_partials_warp_raw(row, slots, slot_stride, lane));
 }
 
 }  // namespace egtp

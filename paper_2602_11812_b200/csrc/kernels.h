@@ -54,7 +54,11 @@ constexpr int kPoolThreads = 128;      // each thread owns 8 consecutive channel
 
 cudaError_t launch_validate_offsets(const int32_t* offsets, int B, int64_t T, int32_t* status, cudaStream_t stream);
 
-cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t T, float* H,
+// slot j of row i is read at partials + i * row_stride + j * slot_stride (floats)
+cudaError_t launch_partials_reduce(const float* partials, int slots, int64_t rows, float* out, const int32_t* status,
+                                   cudaStream_t stream);
+cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t row_stride, int64_t slot_stride, int64_t T,
+                                 float* H,
                                  const int32_t* offsets, int B, int32_t* seg_id_out, float* weights_zero,
                                  const int32_t* status, cudaStream_t stream);
 
@@ -101,7 +105,7 @@ cudaError_t launch_head_out(const HeadArgs& h, const float* partial, int rows, i
 // ---- K4: PLP running-state update ---------------------------------------------------------
 // Merges the row's entropy partials itself (Eq. 2), optionally writes H' to Hstep_out, then updates the slot.
 cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, const float* partials, int slots,
-                              float* Hstep_out,
+                              int64_t row_stride, int64_t slot_stride, float* Hstep_out,
                               const int32_t* slot_ids, const int32_t* reset_src, const float* src_m,
                               const float* src_s, const float* src_pooled, int n_src, int rows, int d, int num_slots,
                               float inv_alpha, float* st_m, float* st_s, float* st_acc, float* z, int64_t ldz,

@@ -43,7 +43,7 @@ constexpr int kPlpMaxThreads = 1024;
 template <typename T>
 __global__ void __launch_bounds__(kPlpMaxThreads)
 plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* __restrict__ partials, int slots,
-                  float* __restrict__ Hstep_out, const int32_t* __restrict__ slot_ids,
+                  int64_t row_stride, int64_t slot_stride, float* __restrict__ Hstep_out, const int32_t* __restrict__ slot_ids,
                   const int32_t* __restrict__ reset_src, const float* __restrict__ src_m,
                   const float* __restrict__ src_s, const float* __restrict__ src_pooled, int n_src, int d,
                   int num_slots, float inv_alpha, float* __restrict__ st_m, float* __restrict__ st_s,
@@ -83,7 +83,7 @@ plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* _
     if (acc_src != nullptr) load8<float>(acc_src + col, acc);
   }
   // Eq. 2 for this row: every warp merges the row's partials (same value in all of them)
-  const float H_new = merge_partials_warp(partials + static_cast<int64_t>(i) * slots * 3, slots, threadIdx.x & 31);
+  const float H_new = merge_partials_warp(partials + static_cast<int64_t>(i) * row_stride, slots, slot_stride, threadIdx.x & 31);
   if (threadIdx.x == 0 && Hstep_out != nullptr) Hstep_out[i] = H_new;
   const float a = H_new * inv_alpha;
   const float m_new = fmaxf(m_old, a);
@@ -119,17 +119,17 @@ plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* _
 }  // namespace
 
 cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, const float* partials, int slots,
-                              float* Hstep_out, const int32_t* slot_ids, const int32_t* reset_src, const float* src_m,
+                              int64_t row_stride, int64_t slot_stride, float* Hstep_out, const int32_t* slot_ids, const int32_t* reset_src, const float* src_m,
                               const float* src_s, const float* src_pooled, int n_src, int rows, int d, int num_slots,
                               float inv_alpha, float* st_m, float* st_s, float* st_acc, float* z, int64_t ldz,
                               int32_t* status, cudaStream_t stream) {
   const int threads = std::min(kPlpMaxThreads, std::max(32, (d / 8 + 31) / 32 * 32));
   if (bf16) {
     plp_update_kernel<__nv_bfloat16><<<rows, threads, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(hidden_step), ldh, partials, slots, Hstep_out, slot_ids, reset_src, src_m, src_s, src_pooled,
+        static_cast<const __nv_bfloat16*>(hidden_step), ldh, partials, slots, row_stride, slot_stride, Hstep_out, slot_ids, reset_src, src_m, src_s, src_pooled,
         n_src, d, num_slots, inv_alpha, st_m, st_s, st_acc, z, ldz, status);
   } else {
-    plp_update_kernel<float><<<rows, threads, 0, stream>>>(static_cast<const float*>(hidden_step), ldh, partials, slots, Hstep_out, slot_ids,
+    plp_update_kernel<float><<<rows, threads, 0, stream>>>(static_cast<const float*>(hidden_step), ldh, partials, slots, row_stride, slot_stride, Hstep_out, slot_ids,
                                                        reset_src, src_m, src_s, src_pooled, n_src, d, num_slots,
                                                        inv_alpha, st_m, st_s, st_acc, z, ldz, status);
   }

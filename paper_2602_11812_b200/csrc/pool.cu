@@ -49,15 +49,15 @@ __global__ void validate_offsets_kernel(const int32_t* __restrict__ off, int B, 
 // One warp per token: lanes stride over the token's (m, s, t2) partials (contiguous in memory),
 // fold them in a fixed order, then combine across lanes: H = ln S - ln2 * T2 / S.
 // Also writes the token's prompt index and clears its weight.
-__global__ void entropy_merge_kernel(const float* __restrict__ partials, int slots, int64_t T,
-                                     float* __restrict__ H, const int32_t* __restrict__ off, int B,
+__global__ void entropy_merge_kernel(const float* __restrict__ partials, int slots, int64_t row_stride,
+                                     int64_t slot_stride, int64_t T, float* __restrict__ H, const int32_t* __restrict__ off, int B,
                                      int32_t* __restrict__ seg_id, float* __restrict__ weights,
                                      const int32_t* __restrict__ status) {
   if (*status != 0) return;
   const int lane = threadIdx.x & 31;
   const int64_t i = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (i >= T) return;
-  const float h = merge_partials_warp(partials + i * slots * 3, slots, lane);
+  const float h = merge_partials_warp(partials + i * row_stride, slots, slot_stride, lane);
   if (lane == 0) {
     H[i] = h;
     if (weights != nullptr) weights[i] = 0.f;
@@ -66,6 +66,22 @@ __global__ void entropy_merge_kernel(const float* __restrict__ partials, int slo
       if (B > 0 && i >= off[0] && i < off[B]) sid = upper_segment(off, B, i);
       seg_id[i] = sid;
     }
+  }
+}
+
+// One warp per row: folds the row's per-chunk partials into a single (m, s, t2) triple, the unit that
+// GPUs holding different vocabulary shards exchange.
+__global__ void partials_reduce_kernel(const float* __restrict__ partials, int slots, int64_t rows,
+                                       float* __restrict__ out, const int32_t* __restrict__ status) {
+  if (*status != 0) return;
+  const int lane = threadIdx.x & 31;
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (i >= rows) return;
+  const EntropyPartial p = merge_partials_warp_raw(partials + i * slots * 3, slots, 3, lane);
+  if (lane == 0) {
+    out[3 * i] = p.m;
+    out[3 * i + 1] = p.s;
+    out[3 * i + 2] = p.t2;
   }
 }
 
@@ -283,13 +299,21 @@ cudaError_t launch_validate_offsets(const int32_t* offsets, int B, int64_t T, in
   return cudaGetLastError();
 }
 
-cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t T, float* H,
-                                 const int32_t* offsets, int B, int32_t* seg_id_out, float* weights_zero,
+cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t row_stride, int64_t slot_stride, int64_t T,
+                                 float* H, const int32_t* offsets, int B, int32_t* seg_id_out, float* weights_zero,
                                  const int32_t* status, cudaStream_t stream) {
   const int threads = 256, rows_per_block = threads / 32;
   const unsigned blocks = static_cast<unsigned>((T + rows_per_block - 1) / rows_per_block);
-  entropy_merge_kernel<<<blocks, threads, 0, stream>>>(partials, slots, T, H, offsets, B, seg_id_out, weights_zero,
-                                                       status);
+  entropy_merge_kernel<<<blocks, threads, 0, stream>>>(partials, slots, row_stride, slot_stride, T, H, offsets, B,
+                                                       seg_id_out, weights_zero, status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_partials_reduce(const float* partials, int slots, int64_t rows, float* out, const int32_t* status,
+                                   cudaStream_t stream) {
+  const int threads = 256, rows_per_block = threads / 32;
+  const unsigned blocks = static_cast<unsigned>((rows + rows_per_block - 1) / rows_per_block);
+  partials_reduce_kernel<<<blocks, threads, 0, stream>>>(partials, slots, rows, out, status);
   return cudaGetLastError();
 }
 

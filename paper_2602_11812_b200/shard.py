@@ -73,3 +73,18 @@ def reduce_time_and_work(ms_local: float, units_local: float, device, group=None
         dist.all_reduce(t, op=dist.ReduceOp.MAX, group=group)
         dist.all_reduce(u, op=dist.ReduceOp.SUM, group=group)
     return float(t.item()), float(u.item())
+
+
+def vocab_shards(V: int, world: int, multiple: int = 256):
+    """Row ranges [v0, v1) of a vocabulary-sharded LM head, boundaries on multiples of `multiple` (the tile width)."""
+    units = (V + multiple - 1) // multiple
+    cuts = [min(V, (r * units // world) * multiple) for r in range(world)] + [V]
+    return [(cuts[r], cuts[r + 1]) for r in range(world)]
+
+
+def all_gather_partials(partial_local: torch.Tensor, group=None) -> torch.Tensor:
+    """The vocabulary-parallel path's one collective: [rows, 3] per rank -> [world, rows, 3] on every rank."""
+    world = dist.get_world_size(group)
+    out = torch.empty((world,) + tuple(partial_local.shape), device=partial_local.device, dtype=partial_local.dtype)
+    dist.all_gather(list(out.unbind(0)), partial_local.contiguous(), group=group)   # writes into the views of `out`
+    return out

@@ -36,9 +36,14 @@ def _worker(rank, world, port, q):
         y = orc.egtp_predict(rows, off, wl.W, wl.head)["yhat"] if len(mine) else np.zeros(0)
         y_all = shard.gather_predictions(torch.from_numpy(y.astype(np.float32)), mine, wl.B)
         t_max, units = shard.reduce_time_and_work(10.0 + rank, float(rows.shape[0]), torch.device("cpu"))
+        # the vocabulary-parallel exchange: every rank contributes a [rows, 3] block, all ranks receive all blocks
+        part = torch.full((5, 3), float(rank), dtype=torch.float32) + torch.arange(15, dtype=torch.float32).reshape(5, 3)
+        gathered = shard.all_gather_partials(part)
+        g_ok = gathered.shape == (world, 5, 3) and all(bool(torch.equal(gathered[r], part - rank + r)) for r in range(world))
         if rank == 0:
             ref = orc.egtp_predict(wl.hidden, wl.offsets, wl.W, wl.head)["yhat"]
-            q.put(dict(ok=bool(np.allclose(y_all.numpy(), ref, rtol=1e-6, atol=1e-6)), t_max=t_max, units=units, T=wl.T))
+            q.put(dict(ok=bool(np.allclose(y_all.numpy(), ref, rtol=1e-6, atol=1e-6)) and g_ok, t_max=t_max, units=units,
+                       T=wl.T))
     finally:
         dist.destroy_process_group()
 
@@ -51,6 +56,8 @@ def test_partition_is_balanced_and_complete():
         loads = [int(lengths[p].sum()) for p in parts]
         assert max(loads) - min(loads) <= int(lengths.max())         # LPT bound
     assert [p.tolist() for p in shard.partition_prompts([5, 5, 5], 2)] == [[0, 2], [1]]
+    assert shard.vocab_shards(151936, 4) == [(0, 37888), (37888, 76032), (76032, 113920), (113920, 151936)]
+    assert shard.vocab_shards(100, 3, multiple=256) == [(0, 0), (0, 0), (0, 100)]
     rows, off = shard.local_batch(np.arange(20).reshape(10, 2), np.array([0, 3, 4, 10]), np.array([2, 0]))
     assert off.tolist() == [0, 6, 9] and rows[:, 0].tolist() == [8, 10, 12, 14, 16, 18, 0, 2, 4]
 
