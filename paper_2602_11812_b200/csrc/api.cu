@@ -51,6 +51,11 @@ struct egtp_ctx {
 
   // bookkeeping
   int lmhead_mode = EGTP_LMHEAD_AUTO;
+  // host-buffer entry points: copies run on their own stream, one event per piece of the batch
+  static constexpr int kMaxPieces = 4;
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t piece_ready[kMaxPieces] = {};
+  cudaEvent_t stage_free = nullptr;
   int64_t launches = 0;
   bool profiling = false;
   std::vector<EventPair> pending;
@@ -85,6 +90,9 @@ void free_ctx_memory(egtp_ctx* c) {
   cudaFree(c->partials); cudaFree(c->H); cudaFree(c->weights); cudaFree(c->seg_m); cudaFree(c->seg_s);
   cudaFree(c->pooled); cudaFree(c->piece_a); cudaFree(c->piece_b); cudaFree(c->head_partial); cudaFree(c->yhat);
   cudaFree(c->status); cudaFree(c->hidden_stage); cudaFree(c->offsets_stage); cudaFree(c->reset_stage);
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+  for (auto& e : c->piece_ready) if (e) cudaEventDestroy(e);
+  if (c->stage_free) cudaEventDestroy(c->stage_free);
   for (auto& e : c->pending) { cudaEventDestroy(e.start); cudaEventDestroy(e.stop); }
   for (auto& e : c->free_events) { cudaEventDestroy(e.start); cudaEventDestroy(e.stop); }
 }
@@ -256,6 +264,84 @@ int plp_update_and_head(egtp_ctx* c, plp_state* st, const egtp_head* head, const
   return EGTP_OK;
 }
 
+// The whole EGTP chain.  With pieces > 1 the LM-head phase runs over row ranges of the batch one after the
+// other, each waiting for its own event (the host entry point records one when that range's copy has
+// landed), so that the copy of range i+1 overlaps the GEMM of range i.
+int predict_impl(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, const void* hidden, int64_t ldh,
+                 const int32_t* offsets, int32_t B, int64_t T_total, float alpha, float* H_out, float* weights_out,
+                 int32_t* seg_id_out, float* pooled_out, float* state_m_out, float* state_s_out, float* yhat_out,
+                 float* phat_out, int32_t* status_dev, void* stream_v, int pieces, int64_t piece_rows,
+                 const cudaEvent_t* piece_ready) {
+  if (!c) return EGTP_ERR_INVALID_ARG;
+  if (B < 0 || T_total < 0 || !(alpha > 0.f) || !std::isfinite(alpha)) return EGTP_ERR_INVALID_ARG;
+  if (B == 0 || T_total == 0) {
+    if (B > 0 && T_total == 0 && !offsets) return EGTP_ERR_INVALID_ARG;
+    if (T_total == 0 && B == 0) return EGTP_OK;
+  }
+  if (!offsets && B > 0) return EGTP_ERR_INVALID_ARG;
+  if (!head && (yhat_out || phat_out)) return EGTP_ERR_INVALID_ARG;
+  if (T_total > c->max_tokens || B > c->max_batch) return EGTP_ERR_CAPACITY;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  int32_t* status = status_dev ? status_dev : c->status;
+  if (T_total > 0) {
+    int rc = check_lm(c, lm, hidden, ldh);
+    if (rc != EGTP_OK) return rc;
+  } else if (!lm || lm->d <= 0 || lm->d > c->max_d) {
+    return EGTP_ERR_INVALID_ARG;
+  }
+  if (head) {
+    int rc = check_head(c, head, lm->d);
+    if (rc != EGTP_OK) return rc;
+  }
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
+
+  const int d = lm->d;
+  float* H = H_out ? H_out : c->H;
+  float* weights = weights_out ? weights_out : c->weights;
+  float* pooled = pooled_out ? pooled_out : c->pooled;
+  float* seg_m = state_m_out ? state_m_out : c->seg_m;
+  float* seg_s = state_s_out ? state_s_out : c->seg_s;
+
+  if (B > 0) {
+    LaunchScope ls(c, EGTP_K_VALIDATE, stream);
+    EGTP_CUDA_TRY(launch_validate_offsets(offsets, B, T_total, status, stream));
+  }
+  for (int p = 0; p < pieces && T_total > 0; ++p) {
+    const int64_t r0 = p * piece_rows;
+    const int64_t rows = std::min<int64_t>(piece_rows, T_total - r0);
+    if (rows <= 0) break;
+    if (piece_ready) EGTP_CUDA_TRY(cudaStreamWaitEvent(stream, piece_ready[p], 0));
+    const char* piece_ptr = static_cast<const char*>(hidden) + r0 * ldh * elem_bytes(lm->dtype);
+    LmheadPlan plan;
+    int rc = run_lmhead(c, lm, piece_ptr, ldh, rows, status, stream, &plan);
+    if (rc != EGTP_OK) return rc;
+    LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
+    EGTP_CUDA_TRY(launch_entropy_merge(c->partials, plan.slots, plan.slots * 3, 3, rows, r0, H, offsets, B, seg_id_out,
+                                       weights, status, stream));
+  }
+  if (B == 0) return EGTP_OK;
+  {
+    LaunchScope ls(c, EGTP_K_SEGMENT_WEIGHTS, stream);
+    EGTP_CUDA_TRY(launch_segment_weights(H, offsets, B, 1.f / alpha, weights, seg_m, seg_s, status, stream));
+  }
+  if (T_total > 0) {
+    LaunchScope ls(c, EGTP_K_POOL, stream);
+    EGTP_CUDA_TRY(launch_pool(hidden, ldh, lm->dtype == EGTP_BF16, false, weights, offsets, B, T_total, d, pooled,
+                              c->piece_a, c->piece_b, status, stream));
+  }
+  {
+    LaunchScope ls(c, EGTP_K_POOL_COMBINE, stream);
+    EGTP_CUDA_TRY(launch_pool_combine(offsets, B, d, false, c->piece_a, c->piece_b, pooled, status, stream));
+  }
+  if (head && (yhat_out || phat_out)) {
+    int rc = run_head(c, head, pooled, d, B, yhat_out, phat_out, status, stream);
+    if (rc != EGTP_OK) return rc;
+  }
+  return EGTP_OK;
+}
+
+
 }  // namespace
 
 extern "C" {
@@ -327,6 +413,9 @@ int egtp_create(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_batc
   ok = ok && dev_alloc(c, &c->offsets_stage, static_cast<int64_t>(max_batch) + 1) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->reset_stage, max_batch) == cudaSuccess;
   ok = ok && cudaMemset(c->status, 0, sizeof(int32_t)) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+  for (auto& e : c->piece_ready) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&c->stage_free, cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     free_ctx_memory(c);
@@ -393,68 +482,8 @@ int egtp_predict(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, con
                  const int32_t* offsets, int32_t B, int64_t T_total, float alpha, float* H_out, float* weights_out,
                  int32_t* seg_id_out, float* pooled_out, float* state_m_out, float* state_s_out, float* yhat_out,
                  float* phat_out, int32_t* status_dev, void* stream_v) {
-  if (!c) return EGTP_ERR_INVALID_ARG;
-  if (B < 0 || T_total < 0 || !(alpha > 0.f) || !std::isfinite(alpha)) return EGTP_ERR_INVALID_ARG;
-  if (B == 0 || T_total == 0) {
-    if (B > 0 && T_total == 0 && !offsets) return EGTP_ERR_INVALID_ARG;
-    if (T_total == 0 && B == 0) return EGTP_OK;
-  }
-  if (!offsets && B > 0) return EGTP_ERR_INVALID_ARG;
-  if (!head && (yhat_out || phat_out)) return EGTP_ERR_INVALID_ARG;
-  if (T_total > c->max_tokens || B > c->max_batch) return EGTP_ERR_CAPACITY;
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
-  int32_t* status = status_dev ? status_dev : c->status;
-  if (T_total > 0) {
-    int rc = check_lm(c, lm, hidden, ldh);
-    if (rc != EGTP_OK) return rc;
-  } else if (!lm || lm->d <= 0 || lm->d > c->max_d) {
-    return EGTP_ERR_INVALID_ARG;
-  }
-  if (head) {
-    int rc = check_head(c, head, lm->d);
-    if (rc != EGTP_OK) return rc;
-  }
-  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
-  if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
-
-  const int d = lm->d;
-  float* H = H_out ? H_out : c->H;
-  float* weights = weights_out ? weights_out : c->weights;
-  float* pooled = pooled_out ? pooled_out : c->pooled;
-  float* seg_m = state_m_out ? state_m_out : c->seg_m;
-  float* seg_s = state_s_out ? state_s_out : c->seg_s;
-
-  if (B > 0) {
-    LaunchScope ls(c, EGTP_K_VALIDATE, stream);
-    EGTP_CUDA_TRY(launch_validate_offsets(offsets, B, T_total, status, stream));
-  }
-  if (T_total > 0) {
-    LmheadPlan plan;
-    int rc = run_lmhead(c, lm, hidden, ldh, T_total, status, stream, &plan);
-    if (rc != EGTP_OK) return rc;
-    LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
-    EGTP_CUDA_TRY(launch_entropy_merge(c->partials, plan.slots, plan.slots * 3, 3, T_total, H, offsets, B, seg_id_out, weights, status,
-                                       stream));
-  }
-  if (B == 0) return EGTP_OK;
-  {
-    LaunchScope ls(c, EGTP_K_SEGMENT_WEIGHTS, stream);
-    EGTP_CUDA_TRY(launch_segment_weights(H, offsets, B, 1.f / alpha, weights, seg_m, seg_s, status, stream));
-  }
-  if (T_total > 0) {
-    LaunchScope ls(c, EGTP_K_POOL, stream);
-    EGTP_CUDA_TRY(launch_pool(hidden, ldh, lm->dtype == EGTP_BF16, false, weights, offsets, B, T_total, d, pooled,
-                              c->piece_a, c->piece_b, status, stream));
-  }
-  {
-    LaunchScope ls(c, EGTP_K_POOL_COMBINE, stream);
-    EGTP_CUDA_TRY(launch_pool_combine(offsets, B, d, false, c->piece_a, c->piece_b, pooled, status, stream));
-  }
-  if (head && (yhat_out || phat_out)) {
-    int rc = run_head(c, head, pooled, d, B, yhat_out, phat_out, status, stream);
-    if (rc != EGTP_OK) return rc;
-  }
-  return EGTP_OK;
+  return predict_impl(c, lm, head, hidden, ldh, offsets, B, T_total, alpha, H_out, weights_out, seg_id_out, pooled_out,
+                      state_m_out, state_s_out, yhat_out, phat_out, status_dev, stream_v, 1, T_total, nullptr);
 }
 
 int egtp_pool_baseline(egtp_ctx* c, const egtp_head* head, const void* hidden, int64_t ldh, int32_t dtype, int32_t d,
@@ -507,13 +536,34 @@ int egtp_predict_host(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head
   if (T_total > c->max_tokens || B > c->max_batch || lm->d > c->max_d) return EGTP_ERR_CAPACITY;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
   if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
-  const size_t hbytes = static_cast<size_t>(T_total) * lm->d * elem_bytes(lm->dtype);
-  EGTP_CUDA_TRY(cudaMemcpyAsync(c->hidden_stage, hidden_host, hbytes, cudaMemcpyHostToDevice, stream));
+  // The hidden states travel in up to four row ranges on the context's copy stream; the LM-head kernel of
+  // range i starts when its copy has landed, while range i+1 is still on the bus.
+  const int eb = elem_bytes(lm->dtype);
+  const int64_t min_piece = 2048;
+  int pieces = static_cast<int>(std::min<int64_t>(egtp_ctx::kMaxPieces, std::max<int64_t>(1, T_total / min_piece)));
+  const int64_t piece_rows = ((T_total + pieces - 1) / pieces + 255) / 256 * 256;
+  pieces = static_cast<int>((T_total + piece_rows - 1) / piece_rows);
+  // the staging buffer may still be read by earlier work on `stream`
+  EGTP_CUDA_TRY(cudaEventRecord(c->stage_free, stream));
+  EGTP_CUDA_TRY(cudaStreamWaitEvent(c->copy_stream, c->stage_free, 0));
+  for (int p = 0; p < pieces; ++p) {
+    const int64_t r0 = p * piece_rows;
+    const int64_t rows = std::min<int64_t>(piece_rows, T_total - r0);
+    const size_t off_bytes = static_cast<size_t>(r0) * lm->d * eb;
+    EGTP_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(c->hidden_stage) + off_bytes,
+                                  static_cast<const char*>(hidden_host) + off_bytes,
+                                  static_cast<size_t>(rows) * lm->d * eb, cudaMemcpyHostToDevice, c->copy_stream));
+    EGTP_CUDA_TRY(cudaEventRecord(c->piece_ready[p], c->copy_stream));
+  }
   EGTP_CUDA_TRY(cudaMemcpyAsync(c->offsets_stage, offsets_host, sizeof(int32_t) * (static_cast<size_t>(B) + 1),
                                 cudaMemcpyHostToDevice, stream));
-  int rc = egtp_predict(c, lm, head, c->hidden_stage, lm->d, c->offsets_stage, B, T_total, alpha, nullptr, nullptr,
-                        nullptr, nullptr, nullptr, nullptr, c->yhat, nullptr, nullptr, stream);
-  if (rc != EGTP_OK) return rc;
+  int rc = predict_impl(c, lm, head, c->hidden_stage, lm->d, c->offsets_stage, B, T_total, alpha, nullptr, nullptr,
+                        nullptr, nullptr, nullptr, nullptr, c->yhat, nullptr, nullptr, stream, pieces, piece_rows,
+                        c->piece_ready);
+  if (rc != EGTP_OK) {
+    cudaStreamSynchronize(c->copy_stream);
+    return rc;
+  }
   EGTP_CUDA_TRY(cudaMemcpyAsync(yhat_host, c->yhat, sizeof(float) * B, cudaMemcpyDeviceToHost, stream));
   if (pooled_host)
     EGTP_CUDA_TRY(cudaMemcpyAsync(pooled_host, c->pooled, sizeof(float) * static_cast<size_t>(B) * lm->d,
@@ -617,7 +667,7 @@ int egtp_entropy_from_logits(egtp_ctx* c, const void* logits, int64_t ldl, int32
   int rc = run_logits_entropy(c, logits, ldl, logits_dtype, rows, V, status, stream, &slots);
   if (rc != EGTP_OK) return rc;
   LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
-  EGTP_CUDA_TRY(launch_entropy_merge(c->partials, slots, slots * 3, 3, rows, H_out, nullptr, 0, nullptr, nullptr, status, stream));
+  EGTP_CUDA_TRY(launch_entropy_merge(c->partials, slots, slots * 3, 3, rows, 0, H_out, nullptr, 0, nullptr, nullptr, status, stream));
   return EGTP_OK;
 }
 
@@ -677,7 +727,7 @@ int egtp_entropy_from_partials(egtp_ctx* c, const float* gathered, int32_t num_s
   int32_t* status = status_dev ? status_dev : c->status;
   if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
   LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
-  EGTP_CUDA_TRY(launch_entropy_merge(gathered, num_shards, 3, rows * 3, rows, H_out, nullptr, 0, nullptr, nullptr, status,
+  EGTP_CUDA_TRY(launch_entropy_merge(gathered, num_shards, 3, rows * 3, rows, 0, H_out, nullptr, 0, nullptr, nullptr, status,
                                      stream));
   return EGTP_OK;
 }

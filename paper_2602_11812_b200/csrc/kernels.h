@@ -54,11 +54,12 @@ constexpr int kPoolThreads = 128;      // each thread owns 8 consecutive channel
 
 cudaError_t launch_validate_offsets(const int32_t* offsets, int B, int64_t T, int32_t* status, cudaStream_t stream);
 
-// slot j of row i is read at partials + i * row_stride + j * slot_stride (floats)
+// slot j of row i is read at partials + i * row_stride + j * slot_stride (floats); row i is token row0 + i of
+// the batch (H, weights and segment ids are indexed by the batch-wide token index)
 cudaError_t launch_partials_reduce(const float* partials, int slots, int64_t rows, float* out, const int32_t* status,
                                    cudaStream_t stream);
 cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t row_stride, int64_t slot_stride, int64_t T,
-                                 float* H,
+                                 int64_t row0, float* H,
                                  const int32_t* offsets, int B, int32_t* seg_id_out, float* weights_zero,
                                  const int32_t* status, cudaStream_t stream);
 

@@ -50,7 +50,7 @@ __global__ void validate_offsets_kernel(const int32_t* __restrict__ off, int B, 
 // fold them in a fixed order, then combine across lanes: H = ln S - ln2 * T2 / S.
 // Also writes the token's prompt index and clears its weight.
 __global__ void entropy_merge_kernel(const float* __restrict__ partials, int slots, int64_t row_stride,
-                                     int64_t slot_stride, int64_t T, float* __restrict__ H, const int32_t* __restrict__ off, int B,
+                                     int64_t slot_stride, int64_t T, int64_t row0, float* __restrict__ H, const int32_t* __restrict__ off, int B,
                                      int32_t* __restrict__ seg_id, float* __restrict__ weights,
                                      const int32_t* __restrict__ status) {
   if (*status != 0) return;
@@ -59,12 +59,13 @@ __global__ void entropy_merge_kernel(const float* __restrict__ partials, int slo
   if (i >= T) return;
   const float h = merge_partials_warp(partials + i * row_stride, slots, slot_stride, lane);
   if (lane == 0) {
-    H[i] = h;
-    if (weights != nullptr) weights[i] = 0.f;
+    const int64_t g = row0 + i;      // token index in the whole batch (the partials may cover one piece of it)
+    H[g] = h;
+    if (weights != nullptr) weights[g] = 0.f;
     if (seg_id != nullptr) {
       int sid = -1;
-      if (B > 0 && i >= off[0] && i < off[B]) sid = upper_segment(off, B, i);
-      seg_id[i] = sid;
+      if (B > 0 && g >= off[0] && g < off[B]) sid = upper_segment(off, B, g);
+      seg_id[g] = sid;
     }
   }
 }
@@ -300,11 +301,11 @@ cudaError_t launch_validate_offsets(const int32_t* offsets, int B, int64_t T, in
 }
 
 cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t row_stride, int64_t slot_stride, int64_t T,
-                                 float* H, const int32_t* offsets, int B, int32_t* seg_id_out, float* weights_zero,
+                                 int64_t row0, float* H, const int32_t* offsets, int B, int32_t* seg_id_out, float* weights_zero,
                                  const int32_t* status, cudaStream_t stream) {
   const int threads = 256, rows_per_block = threads / 32;
   const unsigned blocks = static_cast<unsigned>((T + rows_per_block - 1) / rows_per_block);
-  entropy_merge_kernel<<<blocks, threads, 0, stream>>>(partials, slots, row_stride, slot_stride, T, H, offsets, B,
+  entropy_merge_kernel<<<blocks, threads, 0, stream>>>(partials, slots, row_stride, slot_stride, T, row0, H, offsets, B,
                                                        seg_id_out, weights_zero, status);
   return cudaGetLastError();
 }

@@ -162,8 +162,10 @@ def test_errors_are_reported_not_fatal(ctx):
     _check_all(gu.run_egtp(ctx, wl), ref, wl)
 
 
-def test_host_buffer_entry_point(ctx):
-    wl = gen.config_mid(V=3000, d=256, m_h=64, B=6)
+@pytest.mark.parametrize("B", [6, 32])
+def test_host_buffer_entry_point(ctx, B):
+    # B = 32 gives 9555 tokens: the copy is split into four row ranges that overlap the LM-head kernel
+    wl = gen.config_mid(V=3000, d=256, m_h=64, B=B)
     ref = orc.egtp_predict(wl.hidden, wl.offsets, wl.W, wl.head, wl.alpha)
     W = gu.dev_tensor(wl.W, wl.dtype)
     hd = gu.DeviceHead(wl.head, wl.dtype)
