@@ -259,6 +259,28 @@ def run_mine(args):
     h2d = hidden_host.numel() * 2 + off_host.numel() * 4
     d2h = y_host.numel() * 4 + 4
 
+    # ---- context only: a library GEMM of the same shape (it also has to write the T x V logits), same run
+    lib_gemm = None
+    if world == 1:
+        try:
+            logits = torch.empty(T, V, device="cuda", dtype=torch.bfloat16)
+            for _ in range(2):
+                torch.matmul(hidden, W.t(), out=logits)
+            torch.cuda.synchronize()
+            m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n_mm = 20
+            m0.record()
+            for _ in range(n_mm):
+                torch.matmul(hidden, W.t(), out=logits)
+            m1.record()
+            torch.cuda.synchronize()
+            mm_ms = m0.elapsed_time(m1) / n_mm
+            lib_gemm = dict(what="torch.matmul (cuBLAS) bf16 [T,d] x [d,V] -> bf16 logits, no entropy", ms=mm_ms,
+                            tflops=2.0 * d * V * T / (mm_ms * 1e-3) / 1e12)
+            del logits
+        except Exception as exc:
+            lib_gemm = dict(error=str(exc)[:200])
+
     if rank != 0:
         egtp.egtp_destroy(ctx)
         if world > 1:
@@ -297,6 +319,7 @@ def run_mine(args):
                 gpu_launches=int(launches),
                 roofline=roofline,
                 kernels=kernels,
+                library_gemm_same_shape=lib_gemm,
                 pool=dict(bound="hbm", achieved=pool_gbs, peak=peaks["hbm_gbs"], unit="GB/s",
                           frac=(pool_gbs / peaks["hbm_gbs"]) if pool_gbs else None,
                           note="40 MB of hidden states: launch-latency sized at this workload"))
