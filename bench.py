@@ -397,6 +397,25 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
                            unit="TFLOP/s", frac=2.0 * slots * d * V / (k1_us * 1e-6) / 1e12 / peaks["bf16_tflops"]),
                kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof.items() if v["launches"]},
                plan=egtp.egtp_lmhead_plan(ctx, slots, d, V, egtp.EGTP_BF16))
+    # ---- context only: a library GEMM of the decode shape (writes the [256, V] logits, no entropy)
+    try:
+        lg = torch.empty(slots, V, device="cuda", dtype=torch.bfloat16)
+        for t in range(3):
+            torch.matmul(hs[t], W.t(), out=lg)
+        torch.cuda.synchronize()
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record()
+        for t in range(plp_steps):
+            torch.matmul(hs[warm + t], W.t(), out=lg)
+        c1.record()
+        torch.cuda.synchronize()
+        mm_us = c0.elapsed_time(c1) / plp_steps * 1e3
+        plp["library_gemm_same_shape"] = dict(what="torch.matmul (cuBLAS) bf16 [256,d] x [d,V] -> bf16 logits", us=mm_us,
+                                              w_stream_gbs=w_bytes / (mm_us * 1e-6) / 1e9)
+        del lg
+    except Exception as exc:
+        plp["library_gemm_same_shape"] = dict(error=str(exc)[:200])
+
     # ---- the same step captured once in a CUDA graph and replayed (fixed buffers; removes launch gaps)
     try:
         static_h = hs[warm].clone()
