@@ -17,7 +17,7 @@ namespace egtp {
 
 namespace {
 
-constexpr int kLogitsThreads = 256;
+constexpr int kLogitsThreads = 128;
 constexpr float kLog2e = 1.4426950408889634f;
 
 // Running state of one thread: max m and four independent (s, t2) accumulators (short dependency chains).
@@ -163,11 +163,9 @@ logits_entropy_kernel(const T* __restrict__ logits, int64_t ldl, int V, int cols
 }  // namespace
 
 int logits_entropy_pick_splits(int64_t rows, int V, int num_sms) {
-  // About 16K columns per block (8 vector loads per thread) so that many short blocks even out over the
-  // SMs; finer (down to 2K columns) when there are too few rows to fill the GPU otherwise.
-  int64_t splits = std::max(1, V / 16384);
-  const int64_t want_blocks = 4ll * num_sms;
-  if (rows * splits < want_blocks) splits = (want_blocks + rows - 1) / std::max<int64_t>(rows, 1);
+  // One wave of blocks: about seven 128-thread blocks per SM fit at once, and every thread should see a few
+  // hundred logits so that the per-block combine is amortised; never less than 2K columns per block.
+  int64_t splits = std::max<int64_t>(1, (7ll * num_sms) / std::max<int64_t>(rows, 1));
   splits = std::min<int64_t>(splits, std::max(1, V / 2048));
   return static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(splits, 128)));
 }
