@@ -297,6 +297,15 @@ EGTP_API int egtp_pool_baseline(egtp_ctx* ctx, const egtp_head* head, const void
 enum { EGTP_LMHEAD_AUTO = 0, EGTP_LMHEAD_CTA_PAIRS = 1 };
 EGTP_API int egtp_set_lmhead_mode(egtp_ctx* ctx, int mode);
 
+/* Failure-detection self-test.  Every wait inside the pipeline kernels (on an mbarrier fed by TMA, by the
+ * tensor core or by another warp) is bounded: when its limit runs out the kernel writes
+ * EGTP_ERR_DEVICE_TIMEOUT to the status word, releases its tensor memory and returns, so a protocol
+ * fault becomes an error code instead of a hung GPU.  This call runs the same wait primitive on a
+ * barrier that nothing ever signals, with a limit of limit_ms (1..1000) milliseconds: afterwards
+ * *status_dev (device, int32, zeroed by the caller) holds EGTP_ERR_DEVICE_TIMEOUT and the context
+ * is usable as before. */
+EGTP_API int egtp_selftest_wait_timeout(egtp_ctx* ctx, int32_t limit_ms, int32_t* status_dev, void* stream);
+
 /* Per-kernel timing. With profiling on, every kernel launch of this context is bracketed by
  * CUDA events on its own stream.  egtp_profile_read synchronises the device, adds up the
  * elapsed milliseconds and launch counts per kernel since the last read and clears them.

@@ -37,7 +37,7 @@ EXPORTED_SYMBOLS = [
     "plp_step", "plp_step_host", "egtp_profile_enable", "egtp_profile_read", "egtp_kernel_name",
     "egtp_launch_count", "egtp_lmhead_plan", "egtp_head_forward_static", "egtp_set_lmhead_mode",
     "egtp_entropy_from_logits", "plp_step_from_logits", "egtp_pool_baseline",
-    "egtp_entropy_partials", "egtp_entropy_from_partials", "plp_step_from_partials",
+    "egtp_entropy_partials", "egtp_entropy_from_partials", "plp_step_from_partials", "egtp_selftest_wait_timeout",
 ]
 
 
@@ -85,6 +85,7 @@ def load() -> C.CDLL:
     lib.egtp_lmhead_plan.argtypes = [vp, i64, i32, i32, i32, P(i32)]
     lib.egtp_profile_enable.argtypes = [vp, C.c_int]
     lib.egtp_set_lmhead_mode.argtypes = [vp, C.c_int]
+    lib.egtp_selftest_wait_timeout.argtypes = [vp, i32, vp, vp]
     lib.egtp_entropy_partials.argtypes = [vp, P(egtp_lm_head), vp, i64, i64, vp, vp, vp]
     lib.egtp_entropy_from_partials.argtypes = [vp, vp, i32, i64, vp, vp, vp]
     lib.plp_step_from_partials.argtypes = [vp, vp, vp, i32, P(egtp_head), vp, i64, i32, vp, vp, vp, vp, vp, i32, i32, f32,
@@ -370,4 +371,12 @@ def plp_step_from_partials(ctx: int, st: int, gathered, head: Optional[egtp_head
                                        _ptr(status_dev), _stream(stream))
     if check:
         _check(rc, "plp_step_from_partials")
+    return rc
+
+
+def egtp_selftest_wait_timeout(ctx: int, limit_ms: int, status_dev, stream=None, check: bool = True) -> int:
+    """Runs a bounded wait that nothing will satisfy; status_dev ends up holding EGTP_ERR_DEVICE_TIMEOUT."""
+    rc = load().egtp_selftest_wait_timeout(ctx, limit_ms, _ptr(status_dev), _stream(stream))
+    if check:
+        _check(rc, "egtp_selftest_wait_timeout")
     return rc

@@ -16,7 +16,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 OBJ_DIR = os.path.join(PKG_DIR, "_build")
 LIB_PATH = os.path.join(PKG_DIR, "libegtp_b200.so")
-SOURCES = ["api.cu", "lmhead_entropy.cu", "pool.cu", "head.cu", "plp.cu", "logits_entropy.cu", "head_static.cu"]
+SOURCES = ["api.cu", "lmhead_entropy.cu", "pool.cu", "head.cu", "plp.cu", "logits_entropy.cu", "selftest.cu", "head_static.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

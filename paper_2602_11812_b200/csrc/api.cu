@@ -451,6 +451,15 @@ int egtp_set_lmhead_mode(egtp_ctx* c, int mode) {
   return EGTP_OK;
 }
 
+int egtp_selftest_wait_timeout(egtp_ctx* c, int32_t limit_ms, int32_t* status_dev, void* stream_v) {
+  if (!c || !status_dev || limit_ms <= 0 || limit_ms > 1000) return EGTP_ERR_INVALID_ARG;
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  c->launches += 1;
+  EGTP_CUDA_TRY(launch_wait_timeout_selftest(static_cast<uint64_t>(limit_ms) * 1000000ull, status_dev,
+                                             static_cast<cudaStream_t>(stream_v)));
+  return EGTP_OK;
+}
+
 int egtp_profile_enable(egtp_ctx* c, int on) {
   if (!c) return EGTP_ERR_INVALID_ARG;
   c->profiling = on != 0;

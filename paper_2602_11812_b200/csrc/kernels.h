@@ -103,6 +103,9 @@ cudaError_t launch_head_hidden(const HeadArgs& h, const float* z, int64_t ldz, i
 cudaError_t launch_head_out(const HeadArgs& h, const float* partial, int rows, int splits, float* y, float* phat,
                             const int32_t* status, cudaStream_t stream);
 
+// ---- self-test of the bounded wait (a wait on a barrier nobody signals must end with an error status)
+cudaError_t launch_wait_timeout_selftest(uint64_t limit_ns, int32_t* status, cudaStream_t stream);
+
 // ---- K4: PLP running-state update ---------------------------------------------------------
 // Merges the row's entropy partials itself (Eq. 2), optionally writes H' to Hstep_out, then updates the slot.
 cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, const float* partials, int slots,

@@ -247,3 +247,28 @@ def test_small_and_boundary_shapes(ctx, T, d, V):
     wl = gen.EgtpWorkload("small", "bf16", hidden, gen.offsets_from_lengths(lengths), W, head)
     ref = orc.egtp_predict(hidden, wl.offsets, W, head)
     _check_all(gu.run_egtp(ctx, wl), ref, wl)
+
+
+def test_bounded_wait_reports_timeout_and_context_survives(ctx):
+    # a wait on a barrier that nothing signals must end by itself with an error status (no trap, no hang)
+    status = torch.zeros(1, device="cuda", dtype=torch.int32)
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    egtp.egtp_selftest_wait_timeout(ctx, 50, status)
+    t1.record()
+    torch.cuda.synchronize()
+    assert int(status.item()) == egtp.EGTP_ERR_DEVICE_TIMEOUT
+    assert 40.0 <= t0.elapsed_time(t1) <= 500.0                         # the 50 ms limit, not the 4 s production limit
+    assert egtp.status_string(egtp.EGTP_ERR_DEVICE_TIMEOUT).startswith("a bounded wait")
+    # a non-zero status word turns a following call into a no-op instead of computing on top of a failure ...
+    wl = gen.config_tiny()
+    H = torch.full((wl.T,), -1.0, device="cuda")
+    W = gu.dev_tensor(wl.W, wl.dtype); hidden = gu.dev_tensor(wl.hidden, wl.dtype)
+    off = torch.from_numpy(wl.offsets).cuda()
+    egtp.egtp_predict(ctx, egtp.make_lm_head(W), None, hidden, off, wl.B, wl.T, H_out=H, status_dev=status)
+    torch.cuda.synchronize()
+    assert torch.all(H == -1.0) and int(status.item()) == egtp.EGTP_ERR_DEVICE_TIMEOUT
+    # ... and with a cleared word the same context works as before
+    ref = orc.egtp_predict(wl.hidden, wl.offsets, wl.W, wl.head, wl.alpha)
+    _check_all(gu.run_egtp(ctx, wl), ref, wl)
+    assert egtp.egtp_selftest_wait_timeout(ctx, 0, status, check=False) == egtp.EGTP_ERR_INVALID_ARG
