@@ -274,10 +274,7 @@ int predict_impl(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, con
                  const cudaEvent_t* piece_ready) {
   if (!c) return EGTP_ERR_INVALID_ARG;
   if (B < 0 || T_total < 0 || !(alpha > 0.f) || !std::isfinite(alpha)) return EGTP_ERR_INVALID_ARG;
-  if (B == 0 || T_total == 0) {
-    if (B > 0 && T_total == 0 && !offsets) return EGTP_ERR_INVALID_ARG;
-    if (T_total == 0 && B == 0) return EGTP_OK;
-  }
+  if (B == 0 && T_total == 0) return EGTP_OK;
   if (!offsets && B > 0) return EGTP_ERR_INVALID_ARG;
   if (!head && (yhat_out || phat_out)) return EGTP_ERR_INVALID_ARG;
   if (T_total > c->max_tokens || B > c->max_batch) return EGTP_ERR_CAPACITY;
