@@ -15,7 +15,7 @@ namespace {
 
 constexpr int kHT = 64;        // rows and hidden units per block tile
 constexpr int kHK = 32;        // k extent per shared-memory stage
-constexpr int kHThreads = 256; // 16 x 16 threads, 4 x 4 outputs each
+constexpr int kHThreads = 128; // 16 x 8 threads, 8 x 4 outputs each
 constexpr int kHOutThreads = 256;
 
 template <typename TW>
@@ -39,7 +39,7 @@ __device__ __forceinline__ void load8w<__nv_bfloat16>(const __nv_bfloat16* p, fl
 }
 
 // partial[split][row][j] = sum_{k in split} z[row][k] * W1[j][k]
-// 64 x 64 outputs per block, 4 x 4 per thread; the global loads of k-block i+1 are in flight while
+// 64 x 64 outputs per block, 8 x 4 per thread; the global loads of k-block i+1 are in flight while
 // k-block i is multiplied out of shared memory (two buffers, one barrier per k-block).
 template <typename TW>
 __global__ void __launch_bounds__(kHThreads)
@@ -52,38 +52,36 @@ head_hidden_kernel(const float* __restrict__ z, int64_t ldz, const TW* __restric
   const int k_begin = split * k_per_split;
   const int k_end = min(d, k_begin + k_per_split);
   const int tid = threadIdx.x;
-  const int lrow = tid >> 2, lk = (tid & 3) * 8;   // loader: 64 rows x 4 groups of 8 k
-  const int tx = tid & 15, ty = tid >> 4;          // compute: outputs rows ty*4.., units tx*4..
+  const int lrow = tid >> 1, lk = (tid & 1) * 16;  // loader: 64 rows x 2 groups of 16 k
+  const int tx = tid & 15, ty = tid >> 4;          // compute: outputs rows ty*8.., units tx*4..
   const bool z_ok = r0 + lrow < rows, w_ok = j0 + lrow < m_h;
   const float* zp = z + static_cast<int64_t>(r0 + lrow) * ldz + lk;
   const TW* wp = W1 + static_cast<int64_t>(j0 + lrow) * d + lk;
-  float acc[4][4];
+  float acc[8][4];
 #pragma unroll
-  for (int a = 0; a < 4; ++a)
+  for (int a = 0; a < 8; ++a)
 #pragma unroll
     for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
 
-  float zv[8], wv[8];
+  float zv[16], wv[16];
   auto fetch = [&](int k0) {
-    const bool k_in = k0 + lk < k_end;     // d is a multiple of 16: a group of 8 is wholly inside or outside
-    if (z_ok && k_in) {
-      load8w<float>(zp + k0, zv);
-    } else {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) zv[i] = 0.f;
-    }
-    if (w_ok && k_in) {
-      load8w<TW>(wp + k0, wv);
-    } else {
+    for (int h = 0; h < 2; ++h) {
+      const bool k_in = k0 + lk + 8 * h < k_end;   // d is a multiple of 16: a group of 8 is wholly inside or outside
+      float tz[8], tw[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) wv[i] = 0.f;
+      for (int i = 0; i < 8; ++i) { tz[i] = 0.f; tw[i] = 0.f; }
+      if (z_ok && k_in) load8w<float>(zp + k0 + 8 * h, tz);
+      if (w_ok && k_in) load8w<TW>(wp + k0 + 8 * h, tw);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { zv[8 * h + i] = tz[i]; wv[8 * h + i] = tw[i]; }
     }
   };
   if (k_begin < k_end) fetch(k_begin);
   int buf = 0;
   for (int k0 = k_begin; k0 < k_end; k0 += kHK) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < 16; ++i) {
       zs[buf][lk + i][lrow] = zv[i];
       ws[buf][lk + i][lrow] = wv[i];
     }
@@ -91,12 +89,13 @@ head_hidden_kernel(const float* __restrict__ z, int64_t ldz, const TW* __restric
     if (k0 + kHK < k_end) fetch(k0 + kHK);
 #pragma unroll
     for (int k = 0; k < kHK; ++k) {
-      const float4 a = *reinterpret_cast<const float4*>(&zs[buf][k][ty * 4]);
+      const float4 a0 = *reinterpret_cast<const float4*>(&zs[buf][k][ty * 8]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&zs[buf][k][ty * 8 + 4]);
       const float4 b = *reinterpret_cast<const float4*>(&ws[buf][k][tx * 4]);
-      const float av[4] = {a.x, a.y, a.z, a.w};
+      const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
       const float bv[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int i = 0; i < 8; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
     }
@@ -104,8 +103,8 @@ head_hidden_kernel(const float* __restrict__ z, int64_t ldz, const TW* __restric
   }
   float* out = partial + static_cast<int64_t>(split) * rows * m_h;
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int r = r0 + ty * 4 + i;
+  for (int i = 0; i < 8; ++i) {
+    const int r = r0 + ty * 8 + i;
     if (r >= rows) continue;
     const int jj = j0 + tx * 4;
     float* o = out + static_cast<int64_t>(r) * m_h + jj;
