@@ -363,40 +363,54 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     head = gu.DeviceHead(wl.head, "bf16")
     hs = gu.dev_tensor(wl.hidden_steps.reshape(-1, d), "bf16").reshape(plp_steps + warm, slots, d)
     reset = torch.from_numpy(wl.reset_src).cuda()
-    st = egtp.plp_state_create(ctx, slots, d)
     yrem = torch.empty(slots, device="cuda", dtype=torch.float32)
-    for t in range(warm):
-        egtp.plp_step(ctx, st, lm, head.c, hs[t], reset_src=reset[t], yrem_out=yrem, status_dev=status)
-    torch.cuda.synchronize()
-    # pass 1: step times, no per-kernel events in the stream (they cost a few microseconds per step here)
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(plp_steps + 1)]
-    evs[0].record()
-    for t in range(plp_steps):
-        egtp.plp_step(ctx, st, lm, head.c, hs[warm + t], reset_src=reset[warm + t], yrem_out=yrem, status_dev=status)
-        evs[t + 1].record()
-    torch.cuda.synchronize()
-    # pass 2: the same steps again with every kernel bracketed by events (per-kernel breakdown)
-    egtp.egtp_profile_enable(ctx, True)
-    egtp.egtp_profile_read(ctx)
-    for t in range(plp_steps):
-        egtp.plp_step(ctx, st, lm, head.c, hs[warm + t], reset_src=reset[warm + t], yrem_out=yrem, status_dev=status)
-    torch.cuda.synchronize()
-    prof = egtp.egtp_profile_read(ctx)
-    assert int(status.item()) == 0
-    per_step = np.array([evs[i].elapsed_time(evs[i + 1]) * 1e3 for i in range(plp_steps)])
-    k1_us = prof["lmhead_entropy"]["ms"] / prof["lmhead_entropy"]["launches"] * 1e3
     w_bytes = 2.0 * d * V
-    step_us = float(np.median(per_step))
+
+    def measure_steps(st):
+        for t in range(warm):
+            egtp.plp_step(ctx, st, lm, head.c, hs[t], reset_src=reset[t], yrem_out=yrem, status_dev=status)
+        torch.cuda.synchronize()
+        # pass 1: step times, no per-kernel events in the stream (they cost a few microseconds per step here)
+        egtp.egtp_profile_enable(ctx, False)
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(plp_steps + 1)]
+        evs[0].record()
+        for t in range(plp_steps):
+            egtp.plp_step(ctx, st, lm, head.c, hs[warm + t], reset_src=reset[warm + t], yrem_out=yrem, status_dev=status)
+            evs[t + 1].record()
+        torch.cuda.synchronize()
+        # pass 2: the same steps again with every kernel bracketed by events (per-kernel breakdown)
+        egtp.egtp_profile_enable(ctx, True)
+        egtp.egtp_profile_read(ctx)
+        for t in range(plp_steps):
+            egtp.plp_step(ctx, st, lm, head.c, hs[warm + t], reset_src=reset[warm + t], yrem_out=yrem, status_dev=status)
+        torch.cuda.synchronize()
+        prof = egtp.egtp_profile_read(ctx)
+        assert int(status.item()) == 0
+        per_step = np.array([evs[i].elapsed_time(evs[i + 1]) * 1e3 for i in range(plp_steps)])
+        k1_us = prof["lmhead_entropy"]["ms"] / prof["lmhead_entropy"]["launches"] * 1e3
+        step_us = float(np.median(per_step))
+        return dict(us_per_step_median=step_us, us_per_step_p10=float(np.percentile(per_step, 10)),
+                    us_per_step_p90=float(np.percentile(per_step, 90)), lmhead_us=k1_us,
+                    hbm=dict(bound="hbm", kernel="lmhead_entropy", achieved=w_bytes / (k1_us * 1e-6) / 1e9,
+                             peak=peaks["hbm_gbs"], unit="GB/s", frac=w_bytes / (k1_us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                             whole_step_frac=w_bytes / (step_us * 1e-6) / 1e9 / peaks["hbm_gbs"]),
+                    tensor=dict(achieved=2.0 * slots * d * V / (k1_us * 1e-6) / 1e12, peak=peaks["bf16_tflops"],
+                                unit="TFLOP/s", frac=2.0 * slots * d * V / (k1_us * 1e-6) / 1e12 / peaks["bf16_tflops"]),
+                    kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof.items() if v["launches"]},
+                    launches_per_step=sum(v["launches"] for v in prof.values()) / plp_steps)
+
+    # the ordinary route first (head layer 1 as its own GEMM over z), then the state bound to its head
+    # (W1 h' from the LM-head kernel's extra columns; one kernel finishes the step): the headline numbers
+    st_plain = egtp.plp_state_create(ctx, slots, d)
+    plain = measure_steps(st_plain)
+    egtp.plp_state_destroy(st_plain)
+    st = egtp.plp_state_create(ctx, slots, d)
+    egtp.plp_state_bind_head(st, head.c)
     plp = dict(metric="plp_decode_step_us", B=slots, d=d, V=V, steps=plp_steps,
-               us_per_step_median=step_us, us_per_step_p10=float(np.percentile(per_step, 10)),
-               us_per_step_p90=float(np.percentile(per_step, 90)), lmhead_us=k1_us,
-               hbm=dict(bound="hbm", kernel="lmhead_entropy", achieved=w_bytes / (k1_us * 1e-6) / 1e9,
-                        peak=peaks["hbm_gbs"], unit="GB/s", frac=w_bytes / (k1_us * 1e-6) / 1e9 / peaks["hbm_gbs"],
-                        whole_step_frac=w_bytes / (step_us * 1e-6) / 1e9 / peaks["hbm_gbs"]),
-               tensor=dict(achieved=2.0 * slots * d * V / (k1_us * 1e-6) / 1e12, peak=peaks["bf16_tflops"],
-                           unit="TFLOP/s", frac=2.0 * slots * d * V / (k1_us * 1e-6) / 1e12 / peaks["bf16_tflops"]),
-               kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof.items() if v["launches"]},
-               plan=egtp.egtp_lmhead_plan(ctx, slots, d, V, egtp.EGTP_BF16))
+               route="state bound to its head (plp_state_bind_head)")
+    plp.update(measure_steps(st))
+    plp["plan"] = egtp.egtp_lmhead_plan(ctx, slots, d, V, egtp.EGTP_BF16)
+    plp["unbound_state"] = plain
     # ---- context only: a library GEMM of the decode shape (writes the [256, V] logits, no entropy)
     try:
         lg = torch.empty(slots, V, device="cuda", dtype=torch.bfloat16)

@@ -191,6 +191,27 @@ EGTP_API int plp_step(egtp_ctx* ctx, plp_state* st, const egtp_lm_head* lm, cons
              float* Hstep_out, float* z_out, float* yrem_out,
              int32_t* status_dev, void* stream);
 
+/* Binds a PLP state to one prediction head so that a decode step needs no separate layer-1 GEMM
+ * (Sec. 3.2 head on the Sec. 3.3 aggregate).  Layer 1 of the head is linear before its ReLU and z = acc / s,
+ * so W1 z = (W1 acc) / s.  A bound state keeps P = W1 acc [num_slots][m_h] next to acc and advances it with
+ * the recurrence of the pool itself, P' = P e^(m-m') + e^(H'/alpha-m') (W1 h').  W1 h' for all live rows is
+ * produced by the LM-head kernel: the m_h rows of W1 are appended to the vocabulary as extra output columns
+ * whose products are written out instead of entering the entropy (0.2 % more GEMM work at m_h = 256).  One
+ * kernel then merges the entropy partials, updates (m, s, acc, P) and finishes the head for its row.  The
+ * result equals the unbound plp_step up to floating-point summation order.
+ *   head   host struct with device pointers; wdtype must be EGTP_BF16 (EGTP_ERR_UNSUPPORTED otherwise).  The
+ *          struct is copied; the weights it points at must stay in place and unchanged while bound.
+ * Allocates num_slots * m_h + max_batch * m_h + (padded rows) * (padded m_h) floats and synchronises the device
+ * (a create-time call, not for the decode loop).  Binding again replaces the previous binding.
+ * plp_step takes the bound route when it is given the same head (same W1 pointer, m_h, d, dtype) with
+ * yrem_out != NULL, bf16 hidden states and LM head, and n_src <= the context's max_batch; every other call
+ * (another head, no head, plp_step_from_logits / _from_partials, plp_state_import) takes the ordinary route or
+ * changes acc directly, and the next bound step first recomputes P = W1 acc for all slots (one layer-1 pass
+ * over num_slots rows).  A bound step that restarts rows from EGTP rows (reset_src != NULL and n_src > 0)
+ * first projects the n_src source rows (W1 src_pooled), so pass reset_src = NULL on steps without restarts
+ * or keep n_src small.  All calls on one state must be ordered on the GPU (one stream, or events). */
+EGTP_API int plp_state_bind_head(plp_state* st, const egtp_head* head);
+
 /* plp_step with the step's data in HOST memory: hidden_step_host [B_live][d] dense,
  * reset_src_host int32 [B_live] or NULL, yrem_host float [B_live] (output), status_host int32 [1]
  * (output).  Rows map to slots 0..B_live-1.  The EGTP source table stays on the device. */

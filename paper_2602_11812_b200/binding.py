@@ -38,6 +38,7 @@ EXPORTED_SYMBOLS = [
     "egtp_launch_count", "egtp_lmhead_plan", "egtp_head_forward_static", "egtp_set_lmhead_mode",
     "egtp_entropy_from_logits", "plp_step_from_logits", "egtp_pool_baseline",
     "egtp_entropy_partials", "egtp_entropy_from_partials", "plp_step_from_partials", "egtp_selftest_wait_timeout",
+    "plp_state_bind_head",
 ]
 
 
@@ -102,6 +103,7 @@ def load() -> C.CDLL:
     lib.plp_state_destroy.argtypes = [vp]
     lib.plp_state_export.argtypes = [vp, vp, vp, vp, vp]
     lib.plp_state_import.argtypes = [vp, vp, vp, vp, vp]
+    lib.plp_state_bind_head.argtypes = [vp, P(egtp_head)]
     lib.plp_step.argtypes = [vp, vp, P(egtp_lm_head), P(egtp_head), vp, i64, vp, vp, vp, vp, vp, i32, i32, f32,
                              vp, vp, vp, vp, vp]
     lib.plp_step_host.argtypes = [vp, vp, P(egtp_lm_head), P(egtp_head), vp, vp, vp, vp, vp, i32, i32, f32,
@@ -252,6 +254,14 @@ def plp_state_export(st: int, m, s, acc, stream=None):
 
 def plp_state_import(st: int, m, s, acc, stream=None):
     _check(load().plp_state_import(st, _ptr(m), _ptr(s), _ptr(acc), _stream(stream)), "plp_state_import")
+
+
+def plp_state_bind_head(st: int, head: egtp_head, check: bool = True) -> int:
+    """Fixes the head a PLP state is used with: plp_step then gets W1 h' from the LM-head kernel itself."""
+    rc = load().plp_state_bind_head(st, C.byref(head))
+    if check:
+        _check(rc, "plp_state_bind_head")
+    return rc
 
 
 def plp_step(ctx: int, st: int, lm: egtp_lm_head, head: Optional[egtp_head], hidden_step, slot_ids=None,

@@ -70,6 +70,14 @@ struct plp_state {
   float* m = nullptr;
   float* s = nullptr;
   float* acc = nullptr;
+  // binding to one prediction head (plp_state_bind_head)
+  bool bound = false;
+  egtp_head bound_head{};
+  float* proj = nullptr;        // [num_slots][m_h]: W1 acc
+  bool proj_valid = false;      // false: acc was changed without proj (import, a step through another route)
+  float* src_proj = nullptr;    // [ctx->max_batch][m_h]: W1 src_pooled of the current step
+  float* head_g = nullptr;      // [g_rows][ldg_max]: W1 h' of the current step, written by the LM-head kernel
+  int64_t g_rows = 0, ldg_max = 0;
 };
 
 namespace {
@@ -187,18 +195,42 @@ HeadArgs head_args(const egtp_head* h) {
   } while (0)
 
 // Eq. 2 for `rows` rows, first part: the LM-head kernel leaves per-slot partials in the workspace.
+// With fuse_W1 != NULL (bf16 only) the m_h rows of that matrix ride along as extra output columns and
+// head_g [plan.rows_pad][plan.head_cols_pad] receives W1 hidden[i] for every row.
 int run_lmhead(egtp_ctx* c, const egtp_lm_head* lm, const void* hidden, int64_t ldh, int64_t rows, int32_t* status,
-               cudaStream_t stream, LmheadPlan* plan_out) {
-  const LmheadPlan plan = make_lmhead_plan(rows, lm->d, lm->V, elem_bytes(lm->dtype), c->num_sms, c->slot_row_capacity, c->lmhead_mode);
+               cudaStream_t stream, LmheadPlan* plan_out, const void* fuse_W1 = nullptr, int fuse_m_h = 0,
+               float* head_g = nullptr) {
+  const bool fuse = fuse_W1 != nullptr;
+  const LmheadPlan plan = make_lmhead_plan(rows, lm->d, lm->V, elem_bytes(lm->dtype), c->num_sms, c->slot_row_capacity,
+                                           fuse ? static_cast<int>(EGTP_LMHEAD_AUTO) : c->lmhead_mode, fuse ? fuse_m_h : 0);
   if (plan.rows_pad * plan.slots > c->slot_row_capacity) return EGTP_ERR_CAPACITY;
-  CUtensorMap map_a, map_b;
+  CUtensorMap map_a, map_b, map_b_tile, map_c, map_c_tile;
+  LmheadMaps maps;
   int rc = make_tensor_map(c, &map_a, hidden, lm->dtype, rows, lm->d, ldh, plan.a_box_rows);
   if (rc != EGTP_OK) return rc;
   rc = make_tensor_map(c, &map_b, lm->W, lm->dtype, lm->V, lm->d, lm->ldw, plan.b_box_rows);
   if (rc != EGTP_OK) return rc;
+  maps.hidden = &map_a;
+  maps.w = maps.w_tile = &map_b;
+  const bool pair = plan.variant >= 4;
+  if (!pair && plan.b_box_rows != plan.tile_cols) {
+    rc = make_tensor_map(c, &map_b_tile, lm->W, lm->dtype, lm->V, lm->d, lm->ldw, plan.tile_cols);
+    if (rc != EGTP_OK) return rc;
+    maps.w_tile = &map_b_tile;
+  }
+  if (fuse) {
+    rc = make_tensor_map(c, &map_c, fuse_W1, lm->dtype, fuse_m_h, lm->d, lm->d, plan.b_box_rows);
+    if (rc != EGTP_OK) return rc;
+    maps.w1 = maps.w1_tile = &map_c;
+    if (plan.b_box_rows != plan.tile_cols) {
+      rc = make_tensor_map(c, &map_c_tile, fuse_W1, lm->dtype, fuse_m_h, lm->d, lm->d, plan.tile_cols);
+      if (rc != EGTP_OK) return rc;
+      maps.w1_tile = &map_c_tile;
+    }
+  }
   LaunchScope ls(c, EGTP_K_LMHEAD_ENTROPY, stream);
-  EGTP_CUDA_TRY(launch_lmhead_entropy(plan, lm->dtype == EGTP_F32, &map_a, &map_b, rows, lm->V, c->partials, status,
-                                      stream));
+  EGTP_CUDA_TRY(launch_lmhead_entropy(plan, lm->dtype == EGTP_F32, maps, rows, lm->V, c->partials, status, stream,
+                                      head_g));
   *plan_out = plan;
   return EGTP_OK;
 }
@@ -253,6 +285,7 @@ int plp_update_and_head(egtp_ctx* c, plp_state* st, const egtp_head* head, const
                         float alpha, float* Hstep_out, float* z_out, float* yrem_out, int32_t* status,
                         cudaStream_t stream) {
   float* z = z_out ? z_out : c->pooled;
+  st->proj_valid = false;   // acc moves on without the projection a bound state keeps
   {
     LaunchScope ls(c, EGTP_K_PLP_UPDATE, stream);
     EGTP_CUDA_TRY(launch_plp_update(hidden_step, ldh, hidden_dtype == EGTP_BF16, partials, slots, row_stride, slot_stride, Hstep_out,
@@ -262,6 +295,41 @@ int plp_update_and_head(egtp_ctx* c, plp_state* st, const egtp_head* head, const
   }
   if (head && yrem_out) return run_head(c, head, z, st->d, B_live, yrem_out, nullptr, status, stream);
   return EGTP_OK;
+}
+
+// out[r] = W1 x[r] for rows of fp32 vectors x (layer 1 of the head without bias and ReLU), in row chunks that fit
+// the split-K workspace.
+int project_rows(egtp_ctx* c, const egtp_head* head, const float* x, int64_t ldx, int rows, float* out, int64_t ld_out,
+                 const int32_t* status, cudaStream_t stream) {
+  const HeadArgs ha = head_args(head);
+  const int chunk = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(rows, c->head_partial_floats / ha.m_h)));
+  for (int r0 = 0; r0 < rows; r0 += chunk) {
+    const int n = std::min(chunk, rows - r0);
+    const int splits = head_pick_splits(n, ha.d, ha.m_h, c->num_sms, c->head_partial_floats);
+    if (splits <= 0) return EGTP_ERR_CAPACITY;
+    {
+      LaunchScope ls(c, EGTP_K_HEAD_HIDDEN, stream);
+      EGTP_CUDA_TRY(launch_head_hidden(ha, x + r0 * ldx, ldx, n, splits, c->head_partial, status, stream));
+    }
+    {
+      LaunchScope ls(c, EGTP_K_HEAD_OUT, stream);
+      EGTP_CUDA_TRY(launch_head_partial_sum(c->head_partial, n, splits, ha.m_h, out + r0 * ld_out, ld_out, status, stream));
+    }
+  }
+  return EGTP_OK;
+}
+
+// True when this step can take the route of a state bound to `head`: the LM-head kernel also produces W1 h'.
+bool plp_fused_route(const egtp_ctx* c, const plp_state* st, const egtp_lm_head* lm, const egtp_head* head,
+                     int B_live, int n_src, const float* yrem_out) {
+  if (!st->bound || !head || !yrem_out) return false;
+  const egtp_head& b = st->bound_head;
+  if (head->W1 != b.W1 || head->m_h != b.m_h || head->d != b.d || head->wdtype != b.wdtype) return false;
+  if (lm->dtype != EGTP_BF16 || head->wdtype != EGTP_BF16) return false;
+  if (n_src > c->max_batch) return false;
+  const int64_t rows_pad = B_live <= 2 * kTileM ? (B_live <= kTileM ? kTileM : 2 * kTileM)
+                                                : (static_cast<int64_t>(B_live) + kTileM - 1) / kTileM * kTileM;
+  return rows_pad <= st->g_rows;
 }
 
 // The whole EGTP chain.  With pieces > 1 the LM-head phase runs over row ranges of the batch one after the
@@ -609,6 +677,7 @@ int plp_state_destroy(plp_state* st) {
   if (!st) return EGTP_ERR_INVALID_ARG;
   cudaSetDevice(st->ctx->device);
   cudaFree(st->m); cudaFree(st->s); cudaFree(st->acc);
+  cudaFree(st->proj); cudaFree(st->src_proj); cudaFree(st->head_g);
   delete st;
   return EGTP_OK;
 }
@@ -632,6 +701,7 @@ int plp_state_import(plp_state* st, const float* m, const float* s, const float*
   EGTP_CUDA_TRY(cudaMemcpyAsync(st->s, s, sizeof(float) * st->num_slots, cudaMemcpyDeviceToDevice, stream));
   EGTP_CUDA_TRY(cudaMemcpyAsync(st->acc, acc, sizeof(float) * static_cast<size_t>(st->num_slots) * st->d,
                                 cudaMemcpyDeviceToDevice, stream));
+  st->proj_valid = false;
   return EGTP_OK;
 }
 
@@ -655,10 +725,62 @@ int plp_step(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head
   int32_t* status = status_dev ? status_dev : c->status;
   if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
   LmheadPlan plan;
+  if (plp_fused_route(c, st, lm, head, B_live, n_src, yrem_out)) {
+    // bound state: W1 h' comes out of the LM-head kernel, one kernel finishes the step
+    if (!st->proj_valid) {
+      rc = project_rows(c, head, st->acc, st->d, st->num_slots, st->proj, head->m_h, status, stream);
+      if (rc != EGTP_OK) return rc;
+      st->proj_valid = true;
+    }
+    if (reset_src && n_src > 0) {
+      rc = project_rows(c, head, src_pooled, st->d, n_src, st->src_proj, head->m_h, status, stream);
+      if (rc != EGTP_OK) return rc;
+    }
+    rc = run_lmhead(c, lm, hidden_step, ldh, B_live, status, stream, &plan, head->W1, head->m_h, st->head_g);
+    if (rc != EGTP_OK) return rc;
+    if (plan.rows_pad > st->g_rows || plan.head_cols_pad > st->ldg_max) return EGTP_ERR_CAPACITY;
+    LaunchScope ls(c, EGTP_K_PLP_UPDATE, stream);
+    EGTP_CUDA_TRY(launch_plp_update_bound(hidden_step, ldh, c->partials, plan.slots, plan.slots * 3, 3, Hstep_out, slot_ids,
+                                          reset_src, src_m, src_s, src_pooled, st->src_proj, n_src, B_live, st->d,
+                                          st->num_slots, 1.f / alpha, st->m, st->s, st->acc, st->proj, z_out, st->d,
+                                          st->head_g, plan.head_cols_pad, head_args(head), yrem_out, status, stream));
+    return EGTP_OK;
+  }
   rc = run_lmhead(c, lm, hidden_step, ldh, B_live, status, stream, &plan);
   if (rc != EGTP_OK) return rc;
   return plp_update_and_head(c, st, head, hidden_step, ldh, lm->dtype, c->partials, plan.slots, plan.slots * 3, 3, slot_ids, reset_src, src_m, src_s,
                              src_pooled, n_src, B_live, alpha, Hstep_out, z_out, yrem_out, status, stream);
+}
+
+int plp_state_bind_head(plp_state* st, const egtp_head* head) {
+  if (!st || !head) return EGTP_ERR_INVALID_ARG;
+  egtp_ctx* c = st->ctx;
+  int rc = check_head(c, head, st->d);
+  if (rc != EGTP_OK) return rc;
+  if (head->wdtype != EGTP_BF16) return EGTP_ERR_UNSUPPORTED;
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  if (cudaDeviceSynchronize() != cudaSuccess) return EGTP_ERR_CUDA;   // buffers of an earlier binding may be in use
+  cudaFree(st->proj); cudaFree(st->src_proj); cudaFree(st->head_g);
+  st->proj = st->src_proj = st->head_g = nullptr;
+  st->bound = false;
+  // head_g: one row per padded LM-head row (decode shapes pad to 128 / 256 rows, larger batches to 128),
+  // columns padded to the coarsest column granularity of the LM-head shapes (256)
+  const int64_t cap = std::min<int64_t>(c->max_batch, st->num_slots);
+  st->g_rows = std::max<int64_t>(2 * kTileM, (cap + kTileM - 1) / kTileM * kTileM);
+  st->ldg_max = (static_cast<int64_t>(head->m_h) + 255) / 256 * 256;
+  bool ok = cudaMalloc(reinterpret_cast<void**>(&st->proj), sizeof(float) * static_cast<size_t>(st->num_slots) * head->m_h) == cudaSuccess;
+  ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->src_proj), sizeof(float) * static_cast<size_t>(c->max_batch) * head->m_h) == cudaSuccess;
+  ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->head_g), sizeof(float) * static_cast<size_t>(st->g_rows) * st->ldg_max) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    cudaFree(st->proj); cudaFree(st->src_proj); cudaFree(st->head_g);
+    st->proj = st->src_proj = st->head_g = nullptr;
+    return EGTP_ERR_CUDA;
+  }
+  st->bound_head = *head;
+  st->bound = true;
+  st->proj_valid = false;   // the first step through the bound route projects the current acc
+  return EGTP_OK;
 }
 
 int egtp_entropy_from_logits(egtp_ctx* c, const void* logits, int64_t ldl, int32_t logits_dtype, int64_t rows,

@@ -3,6 +3,7 @@
 // at most a few thousand rows: plain fp32 FMA on the CUDA cores, register-tiled, split along d
 // so that small batches still fill the GPU; the split partials are added in a fixed order.
 #include "kernels.h"
+#include "head_out.cuh"
 #include "../../include/egtp.h"
 
 #include <cuda_bf16.h>
@@ -118,13 +119,6 @@ head_hidden_kernel(const float* __restrict__ z, int64_t ldz, const TW* __restric
   }
 }
 
-template <typename TW>
-__device__ __forceinline__ float to_f32(TW v);
-template <>
-__device__ __forceinline__ float to_f32<float>(float v) { return v; }
-template <>
-__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
-
 // One block per row: u = ReLU(sum of split partials + b1) into shared memory, o_c = W2[c] . u + b2[c]
 // (one warp per output, lanes stride the hidden units), then the output mode.
 template <typename TW>
@@ -137,7 +131,7 @@ head_out_kernel(const float* __restrict__ partial, int rows, int splits, int m_h
   extern __shared__ float smem[];
   float* u = smem;            // [m_h]
   float* o = smem + m_h;      // [d_out]
-  const int r = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int r = blockIdx.x, tid = threadIdx.x;
   for (int j = tid; j < m_h; j += blockDim.x) {
     const float* pj = partial + static_cast<int64_t>(r) * m_h + j;
     const int64_t stride = static_cast<int64_t>(rows) * m_h;
@@ -151,31 +145,22 @@ head_out_kernel(const float* __restrict__ partial, int rows, int splits, int m_h
     for (; s < splits; ++s) v += __ldg(pj + s * stride);
     u[j] = fmaxf(0.f, v + b1[j]);
   }
-  __syncthreads();
-  for (int c = wid; c < d_out; c += (blockDim.x >> 5)) {
+  head_output_stage<TW>(u, o, m_h, d_out, W2, b2, centres, mode, y, phat, r);
+}
+
+// out[r][j] = sum over splits of partial[split][r][j], added in split order: the projection W1 x of rows x
+// that are not pooled vectors (the running sums of a PLP state bound to a head).
+__global__ void __launch_bounds__(256)
+head_partial_sum_kernel(const float* __restrict__ partial, int rows, int splits, int m_h, float* __restrict__ out,
+                        int64_t ld_out, const int32_t* __restrict__ status) {
+  if (*status != 0) return;
+  const int64_t n = static_cast<int64_t>(rows) * m_h;
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
     float v = 0.f;
-    for (int j = lane; j < m_h; j += 32) v = fmaf(to_f32<TW>(W2[static_cast<int64_t>(c) * m_h + j]), u[j], v);
-#pragma unroll
-    for (int of = 16; of > 0; of >>= 1) v += __shfl_xor_sync(0xffffffffu, v, of);
-    if (lane == 0) o[c] = v + b2[c];
-  }
-  __syncthreads();
-  if (tid == 0) {
-    if (mode == EGTP_HEAD_SCALAR) {
-      if (y) y[r] = o[0];
-    } else {
-      float mx = o[0];
-      for (int c = 1; c < d_out; ++c) mx = fmaxf(mx, o[c]);
-      float den = 0.f;
-      for (int c = 0; c < d_out; ++c) den += expf(o[c] - mx);
-      float ev = 0.f;
-      for (int c = 0; c < d_out; ++c) {
-        const float pc = expf(o[c] - mx) / den;
-        ev = fmaf(pc, centres[c], ev);
-        if (phat) phat[static_cast<int64_t>(r) * d_out + c] = pc;
-      }
-      if (y) y[r] = ev;
-    }
+    for (int s = 0; s < splits; ++s) v += __ldg(partial + s * n + i);
+    const int64_t r = i / m_h;
+    out[r * ld_out + (i - r * m_h)] = v;
   }
 }
 
@@ -218,6 +203,14 @@ cudaError_t launch_head_out(const HeadArgs& h, const float* partial, int rows, i
                                                        static_cast<const float*>(h.W2), h.b2, h.centres, h.mode, y,
                                                        phat, status);
   }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_head_partial_sum(const float* partial, int rows, int splits, int m_h, float* out, int64_t ld_out,
+                                    const int32_t* status, cudaStream_t stream) {
+  const int64_t n = static_cast<int64_t>(rows) * m_h;
+  const int blocks = static_cast<int>(std::min<int64_t>(1184, (n + 255) / 256));
+  head_partial_sum_kernel<<<std::max(1, blocks), 256, 0, stream>>>(partial, rows, splits, m_h, out, ld_out, status);
   return cudaGetLastError();
 }
 

@@ -25,7 +25,9 @@ struct LmheadPlan {
   int tile_cols;      // vocabulary columns per tile
   int b_box_rows;     // rows of one TMA box of W
   int col_gran;       // vocabulary chunks start at multiples of this many columns
-  int n_groups;       // ceil(V / col_gran)
+  int n_groups;       // ceil(V / col_gran) + head_cols_pad / col_gran
+  int v_pad;          // V rounded up to col_gran: column index of the first fused head column
+  int head_cols_pad;  // fused head columns (rows of the head's W1) rounded up to col_gran; 0 = none
   int chunks;         // vocabulary chunks S; a work unit is (row block, chunk)
   int slots;          // partial slots per row
   int group_rb;       // row blocks that sweep the vocabulary together (L2 reuse of W tiles)
@@ -36,17 +38,30 @@ struct LmheadPlan {
 
 // Picks chunks / grouping for T rows; slot_limit bounds chunks * kEpiSplit * rows_pad by the
 // partial buffer's capacity (in rows x slots).
+// head_cols > 0: that many rows of a second matrix (the head's W1) are appended to the vocabulary as
+// extra columns whose raw products the kernel writes out (bf16, one-CTA shapes only).
 LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity,
-                            int mode);
+                            int mode, int head_cols = 0);
 
 // Opts the kernels into their dynamic shared-memory size on the current device (once per device).
 cudaError_t lmhead_prepare_device();
 
 // partials layout: [rows_pad][slots][3] floats: (m, s, t2) with m the running max logit,
 // s = sum 2^((x-m) log2 e), t2 = sum 2^(...) * (x-m) log2 e over the slot's vocabulary range.
-cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const CUtensorMap* map_hidden,
-                                  const CUtensorMap* map_w, int64_t T, int V, float* partials,
-                                  int32_t* status, cudaStream_t stream);
+// Tensor maps of one launch (K-major, 128-byte rows, 128-byte swizzle).  w / w1: boxes of plan.b_box_rows rows;
+// w_tile / w1_tile: boxes of plan.tile_cols rows (one copy per full tile; may equal w / w1 when the two box
+// heights are the same, must be NULL for the CTA-pair variants that do not use them).  w1 and w1_tile describe
+// the head's W1 [m_h][d] and are needed only with plan.head_cols_pad > 0; head_g [plan.rows_pad][plan.head_cols_pad]
+// then receives head_g[i][j] = W1[j] . hidden[i].
+struct LmheadMaps {
+  const CUtensorMap* hidden = nullptr;
+  const CUtensorMap* w = nullptr;
+  const CUtensorMap* w_tile = nullptr;
+  const CUtensorMap* w1 = nullptr;
+  const CUtensorMap* w1_tile = nullptr;
+};
+cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const LmheadMaps& maps, int64_t T, int V,
+                                  float* partials, int32_t* status, cudaStream_t stream, float* head_g = nullptr);
 
 // ---- K2: entropy merge, Eq. 3 weights, Eq. 4 pooling -------------------------------------
 constexpr int kPoolChunkTokens = 64;   // tokens per first-stage pooling chunk
@@ -103,6 +118,10 @@ cudaError_t launch_head_hidden(const HeadArgs& h, const float* z, int64_t ldz, i
 cudaError_t launch_head_out(const HeadArgs& h, const float* partial, int rows, int splits, float* y, float* phat,
                             const int32_t* status, cudaStream_t stream);
 
+// out[r][j] = sum_s partial[s][r][j] (split order): W1 x for rows x that are not pooled vectors
+cudaError_t launch_head_partial_sum(const float* partial, int rows, int splits, int m_h, float* out, int64_t ld_out,
+                                    const int32_t* status, cudaStream_t stream);
+
 // ---- self-test of the bounded wait (a wait on a barrier nobody signals must end with an error status)
 cudaError_t launch_wait_timeout_selftest(uint64_t limit_ns, int32_t* status, cudaStream_t stream);
 
@@ -114,5 +133,16 @@ cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, c
                               const float* src_s, const float* src_pooled, int n_src, int rows, int d, int num_slots,
                               float inv_alpha, float* st_m, float* st_s, float* st_acc, float* z, int64_t ldz,
                               int32_t* status, cudaStream_t stream);
+
+// The update for a state bound to a head (bf16 hidden states and head weights): also advances the slot's
+// projection st_proj = W1 acc with g = W1 h' from the LM-head kernel and finishes the head for the row.
+// src_proj [n_src][m_h] = W1 src_pooled; z may be NULL.
+cudaError_t launch_plp_update_bound(const void* hidden_step, int64_t ldh, const float* partials, int slots,
+                                    int64_t row_stride, int64_t slot_stride, float* Hstep_out, const int32_t* slot_ids,
+                                    const int32_t* reset_src, const float* src_m, const float* src_s,
+                                    const float* src_pooled, const float* src_proj, int n_src, int rows, int d,
+                                    int num_slots, float inv_alpha, float* st_m, float* st_s, float* st_acc,
+                                    float* st_proj, float* z, int64_t ldz, const float* g, int64_t ldg,
+                                    const HeadArgs& h, float* y, int32_t* status, cudaStream_t stream);
 
 }  // namespace egtp

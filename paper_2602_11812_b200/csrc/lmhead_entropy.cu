@@ -25,6 +25,7 @@
 #include "../../include/egtp.h"
 
 #include <algorithm>
+#include <type_traits>
 
 
 namespace egtp {
@@ -51,6 +52,10 @@ struct KParams {
   int slots;
   float* partials;
   int32_t* status;
+  // head columns appended to the vocabulary (fused form only): column v_pad + j is row j of the head's W1
+  int v_pad;          // first head column: V rounded up to col_gran
+  int ldg;            // floats per row of head_g (head columns rounded up to col_gran)
+  float* head_g;      // [rows_pad][ldg]: head_g[i][j] = W1[j] . hidden[i]
 };
 
 __device__ __forceinline__ UnitCoord unit_coord(int u, const KParams& p) {
@@ -116,10 +121,17 @@ struct RowState {
 // kBN   vocabulary columns per tile; kMT * kBN TMEM columns per accumulator set (256: two sets, 512: one)
 // kBBox rows of one TMA box of W (kBN for the tensor-bound shape; 32 for decode shapes, whose
 //       vocabulary ranges end on 32-column boundaries so that all SMs get equal shares)
-template <bool kTf32, int kMT, int kBN, int kBBox, int kNumStages>
+// kFuse the column space continues past the vocabulary with the rows of a second matrix (map_c: the
+//       prediction head's W1, Sec. 3.2); the accumulators of those columns are written to p.head_g as they
+//       are instead of entering the entropy.  Layer 1 of the head is linear before its ReLU, so W1 h' for
+//       the step's new tokens is all a PLP step needs to advance W1 acc (Sec. 3.3) without a second GEMM.
+template <bool kTf32, int kMT, int kBN, int kBBox, int kNumStages, bool kFuse>
 __global__ void __launch_bounds__(kLmheadThreads, 1)
 lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                      const KParams p) {
+                      const __grid_constant__ CUtensorMap map_b_tile, const __grid_constant__ CUtensorMap map_c,
+                      const __grid_constant__ CUtensorMap map_c_tile, const KParams p) {
+  // map_b / map_c: boxes of kBBox rows of W / W1; map_b_tile / map_c_tile: boxes of kBN rows (a whole tile in
+  // one copy; the same maps when kBBox == kBN)
   constexpr int kABytes = kMT * kTileM * kRowBytes;
   constexpr int kBBytes = kBN * kRowBytes;
   constexpr int kStageBytes = kABytes + kBBytes;
@@ -166,6 +178,8 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     mbar_fence_init();
     tma_prefetch_descriptor(&map_a);
     tma_prefetch_descriptor(&map_b);
+    if (kBBox < kBN) tma_prefetch_descriptor(&map_b_tile);
+    if (kFuse) tma_prefetch_descriptor(&map_c);
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
@@ -190,19 +204,43 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         const UnitCoord uc = unit_coord(u, p);
         for (int n0 = uc.col_begin; n0 < uc.col_end && ok; n0 += kBN) {
           const int ncols = min(kBN, uc.col_end - n0);
-          const int b_loads = (ncols + kBBox - 1) / kBBox;
+          // A full tile that lies wholly in W or wholly in W1 is fetched with one copy, a ragged tile (the end of
+          // an SM's column range, or a tile that straddles v_pad) box by box, each box from the matrix its rows
+          // belong to.  Every source gets a copy loop of its own: a tensor-map address picked per copy at run
+          // time made the copy instruction issue twice and cost a quarter of the decode step.
+          const bool in_w1 = kFuse && n0 >= p.v_pad;
+          const bool whole = kBBox < kBN && ncols == kBN && (!kFuse || in_w1 || n0 + kBN <= p.v_pad);
+          const int b_loads = whole ? kBN / kBBox : (ncols + kBBox - 1) / kBBox;
+          const int b_loads_w = kFuse ? max(0, min(b_loads, (p.v_pad - n0) / kBBox)) : b_loads;   // boxes from W
           const uint32_t tx_bytes = kABytes + b_loads * kBBox * kRowBytes;
-          for (int kb = 0; kb < p.k_blocks; ++kb) {
-            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
-            const uint32_t a_dst = smem_base + stage * kStageBytes;
-            const uint32_t b_dst = a_dst + kABytes;
-            mbar_arrive_expect_tx(full_bar(stage), tx_bytes);
-            tma_load_2d(a_dst, &map_a, kb * kElemsPerStage, uc.row_block * (kMT * kTileM), full_bar(stage));
-            for (int i = 0; i < b_loads; ++i)
-              tma_load_2d(b_dst + i * (kBBox * kRowBytes), &map_b, kb * kElemsPerStage, n0 + i * kBBox,
-                          full_bar(stage));
-            if (++stage == kNumStages) { stage = 0; phase ^= 1u; }
-          }
+          // kSource 0: whole tile of W, 1: whole tile of W1, 2: boxes
+          auto stream_tile = [&](auto source) {
+            constexpr int kSource = decltype(source)::value;
+            for (int kb = 0; kb < p.k_blocks; ++kb) {
+              if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+              const uint32_t a_dst = smem_base + stage * kStageBytes;
+              const uint32_t b_dst = a_dst + kABytes;
+              const int kx = kb * kElemsPerStage;
+              mbar_arrive_expect_tx(full_bar(stage), tx_bytes);
+              tma_load_2d(a_dst, &map_a, kx, uc.row_block * (kMT * kTileM), full_bar(stage));
+              if constexpr (kSource == 0) {
+                tma_load_2d(b_dst, &map_b_tile, kx, n0, full_bar(stage));
+              } else if constexpr (kSource == 1) {
+                tma_load_2d(b_dst, &map_c_tile, kx, n0 - p.v_pad, full_bar(stage));
+              } else {
+                for (int i = 0; i < b_loads_w; ++i)
+                  tma_load_2d(b_dst + i * (kBBox * kRowBytes), &map_b, kx, n0 + i * kBBox, full_bar(stage));
+                if constexpr (kFuse) {
+                  for (int i = b_loads_w; i < b_loads; ++i)
+                    tma_load_2d(b_dst + i * (kBBox * kRowBytes), &map_c, kx, n0 + i * kBBox - p.v_pad, full_bar(stage));
+                }
+              }
+              if (++stage == kNumStages) { stage = 0; phase ^= 1u; }
+            }
+          };
+          if (whole && !in_w1) stream_tile(std::integral_constant<int, 0>{});
+          else if (kFuse && whole) stream_tile(std::integral_constant<int, 1>{});
+          else stream_tile(std::integral_constant<int, 2>{});
         }
       }
     }
@@ -256,15 +294,20 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     bool ok = true;
     for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
       const UnitCoord uc = unit_coord(u, p);
+      const int64_t row = (static_cast<int64_t>(uc.row_block) * kMT + (kMT == 1 ? 0 : half)) * kTileM + quad * 32 + lane;
       RowState st;
       st.init();
       for (int n0 = uc.col_begin; n0 < uc.col_end; n0 += kBN) {
         ok = __all_sync(0xffffffffu, mbar_wait(acc_full_bar(acc), acc_phase, abort_flag));
         if (!ok) break;
         tc_fence_after_sync();
-        const int ncols = min(min(kBN, uc.col_end - n0), p.V - n0);      // tile columns that exist
+        // tile columns this warp has to look at: all that were computed in the fused form (head columns
+        // lie beyond V), otherwise only those that exist in the vocabulary
+        const int tile_cols = min(kBN, uc.col_end - n0);
+        const int ncols = kFuse ? tile_cols : min(tile_cols, p.V - n0);
         const int cols_valid = (kMT == 1) ? min(kSpan, ncols - half * kSpan) : ncols;   // of this warp's span
         const int npieces = cols_valid > 0 ? (cols_valid + 31) >> 5 : 0;
+        const int c_base = n0 + (kMT == 1 ? half * kSpan : 0);                          // first column of the span
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
                                static_cast<uint32_t>(acc * kAccCols + half * kSpan);
         auto release = [&]() {
@@ -272,6 +315,24 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+        };
+        // piece pc = 32 accumulator columns starting at vocabulary / head column c_base + 32 pc
+        auto consume = [&](const uint32_t (&buf)[32], int pc) {
+          if constexpr (kFuse) {
+            const int c0 = c_base + pc * 32;
+            if (c0 >= p.v_pad) {
+              float4* dst = reinterpret_cast<float4*>(p.head_g + row * p.ldg + (c0 - p.v_pad));
+#pragma unroll
+              for (int q = 0; q < 8; ++q)
+                dst[q] = make_float4(__uint_as_float(buf[4 * q]), __uint_as_float(buf[4 * q + 1]),
+                                     __uint_as_float(buf[4 * q + 2]), __uint_as_float(buf[4 * q + 3]));
+            } else {
+              const int valid = min(cols_valid - pc * 32, p.V - c0);   // <= 0: padding between V and v_pad
+              if (valid > 0) st.fold_n(buf, valid);
+            }
+          } else {
+            st.fold_n(buf, cols_valid - pc * 32);
+          }
         };
         uint32_t bufA[32], bufB[32];
         if (npieces == 0) {
@@ -283,12 +344,12 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
           for (int pc = 0; pc < npieces; pc += 2) {
             const bool has1 = pc + 1 < npieces;
             if (has1) tmem_ld_32(taddr + (pc + 1) * 32, bufB); else release();
-            st.fold_n(bufA, cols_valid - pc * 32);
+            consume(bufA, pc);
             if (has1) {
               tmem_ld_wait(bufB);
               const bool has2 = pc + 2 < npieces;
               if (has2) tmem_ld_32(taddr + (pc + 2) * 32, bufA); else release();
-              st.fold_n(bufB, cols_valid - (pc + 1) * 32);
+              consume(bufB, pc + 1);
               if (has2) tmem_ld_wait(bufA);
             }
           }
@@ -296,7 +357,6 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         if (++acc == kNumAcc) { acc = 0; acc_phase ^= 1u; }
       }
       if (ok) {
-        const int64_t row = (static_cast<int64_t>(uc.row_block) * kMT + (kMT == 1 ? 0 : half)) * kTileM + quad * 32 + lane;
         const int slot = (kMT == 1) ? uc.chunk * kEpiSplit + half : uc.chunk;
         float* dst = p.partials + (row * p.slots + slot) * 3;
         dst[0] = st.m;
@@ -562,17 +622,19 @@ const Shape& shape_of(int variant) {
   return variant == 1 ? kShapeDecode1 : (variant == 2 ? kShapeDecode2 : kShapePrompt);
 }
 
-template <bool kTf32, int kMT, int kBN, int kBBox, int kNumStages>
-cudaError_t launch_shape(const LmheadPlan& plan, const CUtensorMap* a, const CUtensorMap* b, const KParams& p,
-                         cudaStream_t stream) {
-  auto kernel = lmhead_entropy_kernel<kTf32, kMT, kBN, kBBox, kNumStages>;
-  kernel<<<plan.grid, kLmheadThreads, smem_bytes_for(kMT, kBN, kNumStages), stream>>>(*a, *b, p);
+template <bool kTf32, int kMT, int kBN, int kBBox, int kNumStages, bool kFuse = false>
+cudaError_t launch_shape(const LmheadPlan& plan, const LmheadMaps& m, const KParams& p, cudaStream_t stream) {
+  auto kernel = lmhead_entropy_kernel<kTf32, kMT, kBN, kBBox, kNumStages, kFuse>;
+  const CUtensorMap* c = kFuse ? m.w1 : m.w;
+  const CUtensorMap* c_tile = kFuse ? m.w1_tile : m.w_tile;
+  kernel<<<plan.grid, kLmheadThreads, smem_bytes_for(kMT, kBN, kNumStages), stream>>>(*m.hidden, *m.w, *m.w_tile, *c,
+                                                                                     *c_tile, p);
   return cudaGetLastError();
 }
 
-template <bool kTf32, int kMT, int kBN, int kBBox, int kNumStages>
+template <bool kTf32, int kMT, int kBN, int kBBox, int kNumStages, bool kFuse = false>
 cudaError_t prepare_shape() {
-  auto kernel = lmhead_entropy_kernel<kTf32, kMT, kBN, kBBox, kNumStages>;
+  auto kernel = lmhead_entropy_kernel<kTf32, kMT, kBN, kBBox, kNumStages, kFuse>;
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               smem_bytes_for(kMT, kBN, kNumStages));
 }
@@ -620,7 +682,7 @@ static_assert(kShapeDecode2.mt == 2 && kShapeDecode2.bn == 256 && kShapeDecode2.
 }  // namespace
 
 LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity,
-                            int mode) {
+                            int mode, int head_cols) {
   LmheadPlan pl{};
   pl.variant = T <= kTileM ? 1 : (T <= 2 * kTileM ? 2 : 0);
   if (mode == EGTP_LMHEAD_CTA_PAIRS) {
@@ -637,6 +699,9 @@ LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms
   pl.col_gran = sh.col_gran;
   pl.row_blocks = static_cast<int>((T + pl.rows_per_block - 1) / pl.rows_per_block);
   pl.n_groups = (V + sh.col_gran - 1) / sh.col_gran;
+  pl.v_pad = pl.n_groups * sh.col_gran;
+  pl.head_cols_pad = (head_cols + sh.col_gran - 1) / sh.col_gran * sh.col_gran;
+  pl.n_groups += pl.head_cols_pad / sh.col_gran;     // head columns follow the (padded) vocabulary
   pl.rows_pad = static_cast<int64_t>(pl.row_blocks) * pl.rows_per_block;
   pl.k_blocks = static_cast<int>((static_cast<int64_t>(d) * elem_bytes + kRowBytes - 1) / kRowBytes);
   pl.smem_bytes = pair ? kPairSmemBytes : smem_bytes_for(sh.mt, sh.bn, sh.stages);
@@ -695,6 +760,9 @@ cudaError_t lmhead_prepare_device() {
   if ((e = prepare_shape<true, EGTP_SHAPE_PROMPT>()) != cudaSuccess) return e;
   if ((e = prepare_shape<true, EGTP_SHAPE_DECODE1>()) != cudaSuccess) return e;
   if ((e = prepare_shape<true, EGTP_SHAPE_DECODE2>()) != cudaSuccess) return e;
+  if ((e = prepare_shape<false, EGTP_SHAPE_PROMPT, true>()) != cudaSuccess) return e;
+  if ((e = prepare_shape<false, EGTP_SHAPE_DECODE1, true>()) != cudaSuccess) return e;
+  if ((e = prepare_shape<false, EGTP_SHAPE_DECODE2, true>()) != cudaSuccess) return e;
   int device = 0, num_sms = 0;
   if ((e = cudaGetDevice(&device)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess) return e;
@@ -705,9 +773,8 @@ cudaError_t lmhead_prepare_device() {
   return prepare_pair<true, 32>(num_sms);
 }
 
-cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const CUtensorMap* map_hidden,
-                                  const CUtensorMap* map_w, int64_t T, int V, float* partials,
-                                  int32_t* status, cudaStream_t stream) {
+cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const LmheadMaps& maps, int64_t T, int V,
+                                  float* partials, int32_t* status, cudaStream_t stream, float* head_g) {
   (void)T;
   KParams p{};
   p.row_blocks = plan.row_blocks;
@@ -721,21 +788,35 @@ cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const CUten
   p.slots = plan.slots;
   p.partials = partials;
   p.status = status;
+  p.v_pad = plan.v_pad;
+  p.ldg = plan.head_cols_pad;
+  p.head_g = head_g;
+  if (maps.hidden == nullptr || maps.w == nullptr || maps.w_tile == nullptr) return cudaErrorInvalidValue;
+  if (plan.head_cols_pad > 0) {
+    // fused head columns: bf16, one CTA per SM only
+    if (tf32 || maps.w1 == nullptr || maps.w1_tile == nullptr || head_g == nullptr) return cudaErrorInvalidValue;
+    switch (plan.variant) {
+      case 0: return launch_shape<false, EGTP_SHAPE_PROMPT, true>(plan, maps, p, stream);
+      case 1: return launch_shape<false, EGTP_SHAPE_DECODE1, true>(plan, maps, p, stream);
+      case 2: return launch_shape<false, EGTP_SHAPE_DECODE2, true>(plan, maps, p, stream);
+      default: return cudaErrorInvalidValue;
+    }
+  }
   if (tf32) {
     switch (plan.variant) {
-      case 1: return launch_shape<true, EGTP_SHAPE_DECODE1>(plan, map_hidden, map_w, p, stream);
-      case 2: return launch_shape<true, EGTP_SHAPE_DECODE2>(plan, map_hidden, map_w, p, stream);
-      case 4: return launch_pair<true, 128>(plan, map_hidden, map_w, p, stream);
-      case 5: return launch_pair<true, 32>(plan, map_hidden, map_w, p, stream);
-      default: return launch_shape<true, EGTP_SHAPE_PROMPT>(plan, map_hidden, map_w, p, stream);
+      case 1: return launch_shape<true, EGTP_SHAPE_DECODE1>(plan, maps, p, stream);
+      case 2: return launch_shape<true, EGTP_SHAPE_DECODE2>(plan, maps, p, stream);
+      case 4: return launch_pair<true, 128>(plan, maps.hidden, maps.w, p, stream);
+      case 5: return launch_pair<true, 32>(plan, maps.hidden, maps.w, p, stream);
+      default: return launch_shape<true, EGTP_SHAPE_PROMPT>(plan, maps, p, stream);
     }
   }
   switch (plan.variant) {
-    case 1: return launch_shape<false, EGTP_SHAPE_DECODE1>(plan, map_hidden, map_w, p, stream);
-    case 2: return launch_shape<false, EGTP_SHAPE_DECODE2>(plan, map_hidden, map_w, p, stream);
-    case 4: return launch_pair<false, 128>(plan, map_hidden, map_w, p, stream);
-    case 5: return launch_pair<false, 32>(plan, map_hidden, map_w, p, stream);
-    default: return launch_shape<false, EGTP_SHAPE_PROMPT>(plan, map_hidden, map_w, p, stream);
+    case 1: return launch_shape<false, EGTP_SHAPE_DECODE1>(plan, maps, p, stream);
+    case 2: return launch_shape<false, EGTP_SHAPE_DECODE2>(plan, maps, p, stream);
+    case 4: return launch_pair<false, 128>(plan, maps.hidden, maps.w, p, stream);
+    case 5: return launch_pair<false, 32>(plan, maps.hidden, maps.w, p, stream);
+    default: return launch_shape<false, EGTP_SHAPE_PROMPT>(plan, maps, p, stream);
   }
 }
 

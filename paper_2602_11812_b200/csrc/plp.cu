@@ -8,6 +8,7 @@
 // HBM-bound (acc read + write, hidden read, z write): one block per live row.
 #include "kernels.h"
 #include "entropy_merge.cuh"
+#include "head_out.cuh"
 #include "../../include/egtp.h"
 
 #include <cuda_bf16.h>
@@ -116,7 +117,123 @@ plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* _
   }
 }
 
+// The same update for a state that is bound to a prediction head (Sec. 3.2-3.3).  Layer 1 of the head is linear
+// before its ReLU, W1 z = (W1 acc) / s, so next to acc the slot keeps P = W1 acc [m_h] and advances it with the
+// same recurrence, P' = P e^(m-m') + e^(H'/alpha-m') (W1 h'), where g = W1 h' was produced by the LM-head kernel
+// as extra output columns.  The block then finishes the head for its row: u = ReLU(P'/s' + b1), o = W2 u + b2,
+// output mode (Eq. 6).  A row that restarts from EGTP row r takes P from src_proj[r] = W1 src_pooled[r].
+// z is written only when the caller asked for it.
+template <typename T, typename TW>
+__global__ void __launch_bounds__(kPlpMaxThreads)
+plp_update_bound_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* __restrict__ partials, int slots,
+                        int64_t row_stride, int64_t slot_stride, float* __restrict__ Hstep_out,
+                        const int32_t* __restrict__ slot_ids, const int32_t* __restrict__ reset_src,
+                        const float* __restrict__ src_m, const float* __restrict__ src_s,
+                        const float* __restrict__ src_pooled, const float* __restrict__ src_proj, int n_src, int d,
+                        int num_slots, float inv_alpha, float* __restrict__ st_m, float* __restrict__ st_s,
+                        float* __restrict__ st_acc, float* __restrict__ st_proj, float* __restrict__ z, int64_t ldz,
+                        const float* __restrict__ g, int64_t ldg, int m_h, int d_out, const float* __restrict__ b1,
+                        const TW* __restrict__ W2, const float* __restrict__ b2, const float* __restrict__ centres,
+                        int mode, float* __restrict__ y, int32_t* status) {
+  if (*status != 0) return;
+  extern __shared__ float smem[];
+  float* u = smem;            // [m_h]
+  float* o = smem + m_h;      // [d_out]
+  const int i = blockIdx.x;
+  const int slot = slot_ids ? slot_ids[i] : i;
+  const int rs = reset_src ? reset_src[i] : PLP_RESET_KEEP;
+  if (slot < 0 || slot >= num_slots || rs < PLP_RESET_KEEP || rs >= n_src) {
+    if (threadIdx.x == 0) atomicCAS(status, 0, EGTP_ERR_BAD_SLOT);
+    return;
+  }
+  float m_old, s_old;
+  const float* acc_src;    // nullptr = zeros
+  const float* proj_src;   // W1 times the vector acc_src points at
+  float acc_scale_in;
+  if (rs == PLP_RESET_KEEP) {
+    m_old = st_m[slot]; s_old = st_s[slot];
+    acc_src = st_acc + static_cast<int64_t>(slot) * d; proj_src = st_proj + static_cast<int64_t>(slot) * m_h;
+    acc_scale_in = 1.f;
+  } else if (rs == PLP_RESET_EMPTY) {
+    m_old = -INFINITY; s_old = 0.f; acc_src = nullptr; proj_src = nullptr; acc_scale_in = 0.f;
+  } else {
+    m_old = src_m[rs]; s_old = src_s[rs];
+    acc_src = src_pooled + static_cast<int64_t>(rs) * d; proj_src = src_proj + static_cast<int64_t>(rs) * m_h;
+    acc_scale_in = s_old;
+  }
+  if (!(s_old > 0.f)) { acc_src = nullptr; proj_src = nullptr; }
+  float* acc_dst = st_acc + static_cast<int64_t>(slot) * d;
+  const T* hrow = hidden_step + static_cast<int64_t>(i) * ldh;
+  float* zrow = z ? z + static_cast<int64_t>(i) * ldz : nullptr;
+
+  int col = threadIdx.x * 8;
+  float h[8], acc[8];
+  const bool first = col < d;
+  if (first) {
+    load8<T>(hrow + col, h);
+    if (acc_src != nullptr) load8<float>(acc_src + col, acc);
+  }
+  const float H_new = merge_partials_warp(partials + static_cast<int64_t>(i) * row_stride, slots, slot_stride, threadIdx.x & 31);
+  if (threadIdx.x == 0 && Hstep_out != nullptr) Hstep_out[i] = H_new;
+  const float a = H_new * inv_alpha;
+  const float m_new = fmaxf(m_old, a);
+  const float carry = (s_old > 0.f) ? expf(m_old - m_new) : 0.f;
+  const float e = expf(a - m_new);
+  const float s_new = fmaf(s_old, carry, e);
+  const float inv_s = 1.f / s_new;
+  const float acc_factor = carry * acc_scale_in;
+  // the projected state and the head's hidden layer
+  const float* grow = g + static_cast<int64_t>(i) * ldg;
+  float* proj_dst = st_proj + static_cast<int64_t>(slot) * m_h;
+  for (int j = threadIdx.x; j < m_h; j += blockDim.x) {
+    const float pj = (proj_src != nullptr) ? fmaf(proj_src[j], acc_factor, e * grow[j]) : e * grow[j];
+    u[j] = fmaxf(0.f, fmaf(pj, inv_s, b1[j]));
+    proj_dst[j] = pj;      // element j is read and written by this thread only
+  }
+  __syncthreads();   // every thread has read the old state before anyone overwrites it
+  for (; col < d; col += blockDim.x * 8) {
+    if (col != static_cast<int>(threadIdx.x) * 8) {
+      load8<T>(hrow + col, h);
+      if (acc_src != nullptr) load8<float>(acc_src + col, acc);
+    }
+    if (acc_src != nullptr) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) acc[k] = fmaf(acc[k], acc_factor, e * h[k]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) acc[k] = e * h[k];
+    }
+    reinterpret_cast<float4*>(acc_dst + col)[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    reinterpret_cast<float4*>(acc_dst + col)[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+    if (zrow != nullptr) {
+      reinterpret_cast<float4*>(zrow + col)[0] = make_float4(acc[0] * inv_s, acc[1] * inv_s, acc[2] * inv_s, acc[3] * inv_s);
+      reinterpret_cast<float4*>(zrow + col)[1] = make_float4(acc[4] * inv_s, acc[5] * inv_s, acc[6] * inv_s, acc[7] * inv_s);
+    }
+  }
+  if (threadIdx.x == 0) {
+    st_m[slot] = m_new;
+    st_s[slot] = s_new;
+  }
+  head_output_stage<TW>(u, o, m_h, d_out, W2, b2, centres, mode, y, nullptr, i);
+}
+
 }  // namespace
+
+cudaError_t launch_plp_update_bound(const void* hidden_step, int64_t ldh, const float* partials, int slots,
+                                    int64_t row_stride, int64_t slot_stride, float* Hstep_out, const int32_t* slot_ids,
+                                    const int32_t* reset_src, const float* src_m, const float* src_s,
+                                    const float* src_pooled, const float* src_proj, int n_src, int rows, int d,
+                                    int num_slots, float inv_alpha, float* st_m, float* st_s, float* st_acc,
+                                    float* st_proj, float* z, int64_t ldz, const float* g, int64_t ldg,
+                                    const HeadArgs& h, float* y, int32_t* status, cudaStream_t stream) {
+  const int threads = std::min(kPlpMaxThreads, std::max(64, (d / 8 + 31) / 32 * 32));
+  const size_t smem = static_cast<size_t>(h.m_h + h.d_out) * sizeof(float);
+  plp_update_bound_kernel<__nv_bfloat16, __nv_bfloat16><<<rows, threads, smem, stream>>>(
+      static_cast<const __nv_bfloat16*>(hidden_step), ldh, partials, slots, row_stride, slot_stride, Hstep_out, slot_ids,
+      reset_src, src_m, src_s, src_pooled, src_proj, n_src, d, num_slots, inv_alpha, st_m, st_s, st_acc, st_proj, z, ldz,
+      g, ldg, h.m_h, h.d_out, h.b1, static_cast<const __nv_bfloat16*>(h.W2), h.b2, h.centres, h.mode, y, status);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, const float* partials, int slots,
                               int64_t row_stride, int64_t slot_stride, float* Hstep_out, const int32_t* slot_ids, const int32_t* reset_src, const float* src_m,

@@ -1,0 +1,142 @@
+"""GPU parity of plp_step on a state bound to its head (plp_state_bind_head): W1 h' comes out of the LM-head
+kernel as extra output columns and one kernel finishes the step.  Checked against the oracle, which knows nothing
+of that shortcut (it recomputes Eq. 8 and the head from explicit token lists), and against the unbound route."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import egtp_oracle as orc
+from paper_2602_11812_b200 import binding as egtp
+from paper_2602_11812_b200 import inputs as gen
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = egtp.egtp_create(0, max_tokens=8192, max_batch=512, max_d=1024, max_V=40000)
+    yield c
+    egtp.egtp_destroy(c)
+
+
+def _run(ctx, wl: gen.PlpWorkload, bind=True, src=None, want_z=True, head=None, W=None):
+    steps, slots, d = wl.steps, wl.slots, wl.d
+    W = gu.dev_tensor(wl.W, wl.dtype) if W is None else W
+    head = gu.DeviceHead(wl.head, wl.dtype) if head is None else head
+    hs = gu.dev_tensor(wl.hidden_steps.reshape(-1, d), wl.dtype).reshape(steps, slots, d)
+    reset = torch.from_numpy(wl.reset_src).cuda()
+    st = egtp.plp_state_create(ctx, slots, d)
+    if bind:
+        egtp.plp_state_bind_head(st, head.c)
+    lm = egtp.make_lm_head(W)
+    f = dict(device="cuda", dtype=torch.float32)
+    H = torch.zeros(steps, slots, **f)
+    z = torch.zeros(steps, slots, d, **f)
+    y = torch.full((steps, slots), float("nan"), **f)
+    status = torch.zeros(1, device="cuda", dtype=torch.int32)
+    sm, ss, sp, n_src = (None, None, None, 0) if src is None else src
+    n0 = egtp.egtp_launch_count(ctx)
+    for t in range(steps):
+        egtp.plp_step(ctx, st, lm, head.c, hs[t], reset_src=reset[t], src_m=sm, src_s=ss, src_pooled=sp, n_src=n_src,
+                      Hstep_out=H[t], z_out=z[t] if want_z else None, yrem_out=y[t], status_dev=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, egtp.status_string(int(status.item()))
+    launches = egtp.egtp_launch_count(ctx) - n0
+    to64 = lambda a: a.cpu().numpy().astype(np.float64)
+    return st, to64(H), to64(z), to64(y), launches
+
+
+def _compare(H, z, y, ref, slots):
+    gu.assert_entropy_close(H[:, slots].ravel(), ref["H"].ravel())
+    for t in range(z.shape[0]):
+        gu.assert_pooled_close(z[t, slots], ref["z"][t])
+    gu.assert_length_close(y[:, slots].ravel(), ref["yrem"].ravel())
+
+
+@pytest.mark.parametrize("slots,V,m_h", [(130, 9000, 64),      # two row tiles; V not a multiple of 32: padded gap before W1
+                                         (77, 4096 + 32, 40),   # one row tile; m_h not a multiple of 32
+                                         (300, 7000, 96)])      # three row blocks of the prompt shape, 256-column boxes
+def test_bound_decode_loop_matches_oracle(ctx, slots, V, m_h):
+    wl = gen.config_plp_decode(slots=slots, steps=12, d=256, V=V, m_h=m_h, mu=1.5, sigma=0.8)
+    assert (wl.reset_src[1:] == gen.RESET_EMPTY).sum() > 10
+    st, H, z, y, launches = _run(ctx, wl)
+    # first step projects the (empty) state: 2 launches; then 2 launches per step (LM head, fused update + head)
+    assert launches == 2 + 2 * wl.steps
+    follow = sorted({0, 1, slots // 2, slots - 2, slots - 1})
+    ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=follow)
+    _compare(H, z, y, ref, follow)
+    egtp.plp_state_destroy(st)
+    # the unbound route on the same inputs: same entropies bit for bit (same vocabulary columns per tile only when
+    # the column split is the same, so compare within tolerance), same lengths within tolerance
+    st2, H2, z2, y2, launches2 = _run(ctx, wl, bind=False)
+    assert launches2 == 4 * wl.steps
+    gu.assert_entropy_close(H.ravel(), H2.ravel())
+    assert np.abs(y - y2).max() <= 1e-3 * max(1.0, np.abs(y2).max())
+    assert np.array_equal(z, z2) or np.abs(z - z2).max() <= 1e-5 * np.abs(z2).max()
+    egtp.plp_state_destroy(st2)
+
+
+def test_bound_bins_head_without_z(ctx):
+    wl = gen.config_plp_decode(slots=140, steps=6, d=256, V=5000, m_h=64, mu=1.5, sigma=0.5)
+    head_bins = gen.make_head(11, 256, 64, 20, "bf16", mode=gen.HEAD_BINS)
+    wl = gen.PlpWorkload("bins", "bf16", wl.hidden_steps, wl.reset_src, wl.W, head_bins)
+    st, H, z, y, _ = _run(ctx, wl, want_z=False)
+    assert np.all(z == 0)            # z_out was not requested: nothing is written
+    follow = [0, 128, 139]
+    ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=follow)
+    gu.assert_length_close(y[:, follow].ravel(), ref["yrem"].ravel())
+    c = np.asarray(head_bins.centres, dtype=np.float64)
+    assert np.all(y >= c.min() - 1e-3) and np.all(y <= c.max() + 1e-3)
+    egtp.plp_state_destroy(st)
+
+
+def test_bound_rl_group_continues_from_egtp_rows(ctx):
+    wl = gen.config_rl_group(prompts=5, group=4, steps=8, d=256, V=7000, m_h=64, min_len=3, max_len=200)
+    eg = wl.prompts
+    res = gu.run_egtp(ctx, eg)
+    ref_eg = orc.egtp_predict(eg.hidden, eg.offsets, eg.W, eg.head)
+    src = (torch.from_numpy(res["state_m"].astype(np.float32)).cuda(), torch.from_numpy(res["state_s"].astype(np.float32)).cuda(),
+           torch.from_numpy(res["pooled"].astype(np.float32)).cuda(), eg.B)
+    st, H, z, y, _ = _run(ctx, wl, src=src)
+    follow = [0, 3, 4, 19]
+    ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=follow,
+                      prompts=dict(hidden=eg.hidden, offsets=eg.offsets, H=ref_eg["H"]))
+    _compare(H, z, y, ref, follow)
+    egtp.plp_state_destroy(st)
+
+
+def test_projection_is_rebuilt_after_other_routes(ctx):
+    # bound steps, then an unbound step with another head, an import, and bound steps again: the oracle's
+    # answer for the original head must come out every time the bound head is used
+    wl = gen.config_plp_decode(slots=40, steps=9, d=128, V=3000, m_h=32, mu=3.0, sigma=0.3)
+    W = gu.dev_tensor(wl.W, "bf16"); lm = egtp.make_lm_head(W)
+    head = gu.DeviceHead(wl.head, "bf16")
+    other = gu.DeviceHead(gen.make_head(99, 128, 48, 1, "bf16"), "bf16")
+    hs = gu.dev_tensor(wl.hidden_steps.reshape(-1, 128), "bf16").reshape(wl.steps, 40, 128)
+    reset = torch.from_numpy(wl.reset_src).cuda()
+    st = egtp.plp_state_create(ctx, 40, 128)
+    egtp.plp_state_bind_head(st, head.c)
+    y = torch.full((wl.steps, 40), float("nan"), device="cuda")
+    y_other = torch.zeros(40, device="cuda")
+    m = torch.empty(40, device="cuda"); s = torch.empty(40, device="cuda"); acc = torch.empty(40, 128, device="cuda")
+    for t in range(wl.steps):
+        if t == 3:       # another head: ordinary route, the projection goes stale
+            egtp.plp_step(ctx, st, lm, other.c, hs[t], reset_src=reset[t], yrem_out=y_other)
+            continue
+        if t == 6:       # checkpoint and restore into the same state
+            egtp.plp_state_export(st, m, s, acc)
+            egtp.plp_state_import(st, m, s, acc)
+        egtp.plp_step(ctx, st, lm, head.c, hs[t], reset_src=reset[t], yrem_out=y[t])
+    torch.cuda.synchronize()
+    ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head)
+    keep = [t for t in range(wl.steps) if t != 3]
+    gu.assert_length_close(y.cpu().numpy().astype(np.float64)[keep].ravel(), ref["yrem"][keep].ravel())
+    egtp.plp_state_destroy(st)
+
+
+def test_bind_rejects_fp32_heads(ctx):
+    st = egtp.plp_state_create(ctx, 8, 128)
+    head32 = gu.DeviceHead(gen.make_head(5, 128, 32, 1, "f32"), "f32")
+    assert egtp.plp_state_bind_head(st, head32.c, check=False) == egtp.EGTP_ERR_UNSUPPORTED
+    egtp.plp_state_destroy(st)
