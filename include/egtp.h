@@ -310,12 +310,17 @@ EGTP_API int egtp_pool_baseline(egtp_ctx* ctx, const egtp_head* head, const void
                                 int32_t mode, float* pooled_out, float* yhat_out,
                                 int32_t* status_dev, void* stream);
 
-/* Tile shape of the LM-head kernel.  EGTP_LMHEAD_AUTO (default): one CTA per SM, 128 x 256 tiles for
- * prompt batches and the two decode shapes for <= 256 rows.  EGTP_LMHEAD_CTA_PAIRS: clusters of two
- * CTAs work on 256 x 256 tiles with tcgen05.mma.cta_group::2 wherever more than 128 rows are given
- * (each SM then loads half as many operand bytes per flop).  Both produce the same entropies up to
- * summation order; on a power-capped B200 AUTO measured equal or faster, so it is the default. */
-enum { EGTP_LMHEAD_AUTO = 0, EGTP_LMHEAD_CTA_PAIRS = 1 };
+/* Tile shape of the LM-head kernel (Sec. 3.1, Eq. 2).
+ *   EGTP_LMHEAD_AUTO (default): one CTA per SM on 128 x 256 tiles for prompt batches and for up to 128 rows;
+ *     batches of 129..256 rows (decode steps) run as clusters of two CTAs on 256 x 512 tiles with
+ *     tcgen05.mma.cta_group::2: every SM then loads half of the hidden rows per 512 instead of 256 vocabulary
+ *     columns, a quarter less operand traffic per flop where the step is bound by streaming W (measured
+ *     4 % faster per decode step than the one-CTA form, in short bursts and sustained).
+ *   EGTP_LMHEAD_CTA_PAIRS: CTA pairs for prompt batches too (256 x 256 tiles).  On a power-capped B200 this
+ *     measured equal or slower than AUTO for prompts, so it is an option.
+ *   EGTP_LMHEAD_SINGLE_CTA: never use CTA pairs (129..256 rows then run both row tiles in one CTA).
+ * All modes give the same entropies up to summation order. */
+enum { EGTP_LMHEAD_AUTO = 0, EGTP_LMHEAD_CTA_PAIRS = 1, EGTP_LMHEAD_SINGLE_CTA = 2 };
 EGTP_API int egtp_set_lmhead_mode(egtp_ctx* ctx, int mode);
 
 /* Failure-detection self-test.  Every wait inside the pipeline kernels (on an mbarrier fed by TMA, by the

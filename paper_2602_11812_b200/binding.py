@@ -24,7 +24,7 @@ EGTP_ERR_BAD_SLOT = -7
 EGTP_F32, EGTP_BF16 = 0, 1
 EGTP_HEAD_SCALAR, EGTP_HEAD_BINS = 0, 1
 PLP_RESET_KEEP, PLP_RESET_EMPTY = -2, -1
-EGTP_LMHEAD_AUTO, EGTP_LMHEAD_CTA_PAIRS = 0, 1
+EGTP_LMHEAD_AUTO, EGTP_LMHEAD_CTA_PAIRS, EGTP_LMHEAD_SINGLE_CTA = 0, 1, 2
 EGTP_POOL_MEAN, EGTP_POOL_MAX, EGTP_POOL_LAST = 1, 2, 3
 KERNEL_IDS = ["validate_offsets", "lmhead_entropy", "entropy_merge", "segment_weights", "pool",
               "pool_combine", "head_hidden", "head_out", "plp_update", "logits_entropy"]

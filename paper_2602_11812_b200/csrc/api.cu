@@ -202,7 +202,7 @@ int run_lmhead(egtp_ctx* c, const egtp_lm_head* lm, const void* hidden, int64_t 
                float* head_g = nullptr) {
   const bool fuse = fuse_W1 != nullptr;
   const LmheadPlan plan = make_lmhead_plan(rows, lm->d, lm->V, elem_bytes(lm->dtype), c->num_sms, c->slot_row_capacity,
-                                           fuse ? static_cast<int>(EGTP_LMHEAD_AUTO) : c->lmhead_mode, fuse ? fuse_m_h : 0);
+                                           c->lmhead_mode, fuse ? fuse_m_h : 0);
   if (plan.rows_pad * plan.slots > c->slot_row_capacity) return EGTP_ERR_CAPACITY;
   CUtensorMap map_a, map_b, map_b_tile, map_c, map_c_tile;
   LmheadMaps maps;
@@ -222,7 +222,7 @@ int run_lmhead(egtp_ctx* c, const egtp_lm_head* lm, const void* hidden, int64_t 
     rc = make_tensor_map(c, &map_c, fuse_W1, lm->dtype, fuse_m_h, lm->d, lm->d, plan.b_box_rows);
     if (rc != EGTP_OK) return rc;
     maps.w1 = maps.w1_tile = &map_c;
-    if (plan.b_box_rows != plan.tile_cols) {
+    if (!pair && plan.b_box_rows != plan.tile_cols) {
       rc = make_tensor_map(c, &map_c_tile, fuse_W1, lm->dtype, fuse_m_h, lm->d, lm->d, plan.tile_cols);
       if (rc != EGTP_OK) return rc;
       maps.w1_tile = &map_c_tile;
@@ -511,7 +511,8 @@ int egtp_lmhead_plan(const egtp_ctx* c, int64_t T, int32_t d, int32_t V, int32_t
 }
 
 int egtp_set_lmhead_mode(egtp_ctx* c, int mode) {
-  if (!c || (mode != EGTP_LMHEAD_AUTO && mode != EGTP_LMHEAD_CTA_PAIRS)) return EGTP_ERR_INVALID_ARG;
+  if (!c || (mode != EGTP_LMHEAD_AUTO && mode != EGTP_LMHEAD_CTA_PAIRS && mode != EGTP_LMHEAD_SINGLE_CTA))
+    return EGTP_ERR_INVALID_ARG;
   c->lmhead_mode = mode;
   return EGTP_OK;
 }
@@ -767,7 +768,7 @@ int plp_state_bind_head(plp_state* st, const egtp_head* head) {
   // columns padded to the coarsest column granularity of the LM-head shapes (256)
   const int64_t cap = std::min<int64_t>(c->max_batch, st->num_slots);
   st->g_rows = std::max<int64_t>(2 * kTileM, (cap + kTileM - 1) / kTileM * kTileM);
-  st->ldg_max = (static_cast<int64_t>(head->m_h) + 255) / 256 * 256;
+  st->ldg_max = (static_cast<int64_t>(head->m_h) + 255) / 256 * 256;   // covers every shape's column granularity
   bool ok = cudaMalloc(reinterpret_cast<void**>(&st->proj), sizeof(float) * static_cast<size_t>(st->num_slots) * head->m_h) == cudaSuccess;
   ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->src_proj), sizeof(float) * static_cast<size_t>(c->max_batch) * head->m_h) == cudaSuccess;
   ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->head_g), sizeof(float) * static_cast<size_t>(st->g_rows) * st->ldg_max) == cudaSuccess;

@@ -116,6 +116,29 @@ struct RowState {
   }
 };
 
+// One piece of an accumulator row: 32 columns starting at column c0 of the (extended) column space, of which the
+// first `produced` were computed and belong to this warp's span.  Without kFuse they are vocabulary columns (the
+// caller has already cut `produced` at V).  With kFuse, columns from p.v_pad on are rows of the prediction head's
+// W1 (Sec. 3.2) and are written to p.head_g as they are; columns between V and v_pad are padding.
+template <bool kFuse>
+__device__ __forceinline__ void consume_piece(RowState& st, const uint32_t (&buf)[32], int c0, int produced,
+                                              const KParams& p, int64_t row) {
+  if constexpr (kFuse) {
+    if (c0 >= p.v_pad) {
+      float4* dst = reinterpret_cast<float4*>(p.head_g + row * p.ldg + (c0 - p.v_pad));
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        dst[q] = make_float4(__uint_as_float(buf[4 * q]), __uint_as_float(buf[4 * q + 1]),
+                             __uint_as_float(buf[4 * q + 2]), __uint_as_float(buf[4 * q + 3]));
+    } else {
+      const int valid = min(produced, p.V - c0);
+      if (valid > 0) st.fold_n(buf, valid);
+    }
+  } else {
+    st.fold_n(buf, produced);
+  }
+}
+
 // kMT   row tiles (of 128 rows) a CTA multiplies against every W tile it loads: 1 for prompt
 //       batches, 2 for decode batches of 129..256 rows (each W byte is then fetched once per GPU)
 // kBN   vocabulary columns per tile; kMT * kBN TMEM columns per accumulator set (256: two sets, 512: one)
@@ -318,21 +341,7 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         };
         // piece pc = 32 accumulator columns starting at vocabulary / head column c_base + 32 pc
         auto consume = [&](const uint32_t (&buf)[32], int pc) {
-          if constexpr (kFuse) {
-            const int c0 = c_base + pc * 32;
-            if (c0 >= p.v_pad) {
-              float4* dst = reinterpret_cast<float4*>(p.head_g + row * p.ldg + (c0 - p.v_pad));
-#pragma unroll
-              for (int q = 0; q < 8; ++q)
-                dst[q] = make_float4(__uint_as_float(buf[4 * q]), __uint_as_float(buf[4 * q + 1]),
-                                     __uint_as_float(buf[4 * q + 2]), __uint_as_float(buf[4 * q + 3]));
-            } else {
-              const int valid = min(cols_valid - pc * 32, p.V - c0);   // <= 0: padding between V and v_pad
-              if (valid > 0) st.fold_n(buf, valid);
-            }
-          } else {
-            st.fold_n(buf, cols_valid - pc * 32);
-          }
+          consume_piece<kFuse>(st, buf, c_base + pc * 32, cols_valid - pc * 32, p, row);
         };
         uint32_t bufA[32], bufB[32];
         if (npieces == 0) {
@@ -396,19 +405,27 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 //   both CTAs, 2..9     epilogue on the CTA's own 128 rows; arrivals go to the leader's
 //                       "accumulator empty" barrier
 // No load in this kernel is multicast; the only multicast is the arrival of tcgen05.commit.
-template <bool kTf32, int kBBox, int kNumStages>
+// kNT  256-column subtiles per tile: 1 = 256 x 256 tiles, two accumulator sets; 2 = 256 x 512 tiles (two MMAs of
+//      N = 256 per k step into the two halves of one 512-column accumulator set): every 128 rows of hidden states
+//      an SM loads then meet 512 instead of 256 vocabulary columns, a quarter less operand traffic per flop, at
+//      the price of an epilogue that no longer overlaps the next tile's MMAs
+// kFuse as in the one-CTA kernel: the column space continues past the vocabulary with the rows of W1 (map_c)
+template <bool kTf32, int kBBox, int kNumStages, int kNT, bool kFuse>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kLmheadThreads, 1)
 lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                           const KParams p) {
-  constexpr int kBN = 256;                        // tile columns over the pair
+                           const __grid_constant__ CUtensorMap map_c, const KParams p) {
+  constexpr int kSubN = 256;                      // columns of one MMA over the pair
+  constexpr int kBN = kSubN * kNT;                // tile columns over the pair
   constexpr int kABytes = kTileM * kRowBytes;     // this CTA's 128 rows
-  constexpr int kBBytes = (kBN / 2) * kRowBytes;  // this CTA's half of the W tile
+  constexpr int kSubBBytes = (kSubN / 2) * kRowBytes;   // this CTA's half of one subtile of W
+  constexpr int kBBytes = kNT * kSubBBytes;
   constexpr int kStageBytes = kABytes + kBBytes;
   constexpr int kAccCols = kBN;
   constexpr int kNumAcc = kTmemCols / kAccCols;
   constexpr int kSpan = kAccCols / kEpiSplit;
-  static_assert(kNumStages <= kMaxStages && (kBN / 2) % kBBox == 0 && kBBox % 8 == 0, "bad tile configuration");
-  static_assert(kNumAcc == 2 && kSpan == 128, "two 256-column accumulators");
+  static_assert(kNumStages <= kMaxStages && (kSubN / 2) % kBBox == 0 && kBBox % 8 == 0, "bad tile configuration");
+  static_assert((kNT == 1 && kNumAcc == 2 && kSpan == 128) || (kNT == 2 && kNumAcc == 1 && kSpan == 256),
+                "two 256-column accumulators or one of 512 columns");
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -444,6 +461,7 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
     mbar_fence_init();
     tma_prefetch_descriptor(&map_a);
     tma_prefetch_descriptor(&map_b);
+    if (kFuse) tma_prefetch_descriptor(&map_c);
   }
   if (warp == 1) {
     tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
@@ -473,9 +491,17 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         const UnitCoord uc = unit_coord(u, p);
         for (int n0 = uc.col_begin; n0 < uc.col_end && ok; n0 += kBN) {
           const int ncols = min(kBN, uc.col_end - n0);
-          const int half_cols = ncols >> 1;                       // W rows this CTA supplies
-          const int b_loads = (half_cols + kBBox - 1) / kBBox;
-          const uint32_t tx_bytes = 2u * (kABytes + b_loads * kBBox * kRowBytes);   // both CTAs
+          // per subtile t: its columns, the W rows this CTA supplies (one half), and the boxes that takes
+          int half_cols[kNT], b_loads[kNT];
+          uint32_t b_bytes = 0;
+#pragma unroll
+          for (int t = 0; t < kNT; ++t) {
+            const int nc = max(0, min(kSubN, ncols - t * kSubN));
+            half_cols[t] = nc >> 1;
+            b_loads[t] = (half_cols[t] + kBBox - 1) / kBBox;
+            b_bytes += b_loads[t] * kBBox * kRowBytes;
+          }
+          const uint32_t tx_bytes = 2u * (kABytes + b_bytes);   // both CTAs
           for (int kb = 0; kb < p.k_blocks; ++kb) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
             const uint32_t a_dst = smem_base + stage * kStageBytes;
@@ -484,9 +510,21 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
             if (leader) mbar_arrive_expect_tx(full_bar(stage), tx_bytes);
             tma_load_2d_pair(a_dst, &map_a, kb * kElemsPerStage, uc.row_block * (2 * kTileM) + rank * kTileM,
                              full_leader);
-            for (int i = 0; i < b_loads; ++i)
-              tma_load_2d_pair(b_dst + i * (kBBox * kRowBytes), &map_b, kb * kElemsPerStage,
-                               n0 + rank * half_cols + i * kBBox, full_leader);
+#pragma unroll
+            for (int t = 0; t < kNT; ++t) {
+              // this CTA's rows of subtile t start at r0; boxes below v_pad come from W, the others from W1
+              // (a loop per matrix: a tensor-map address picked per copy at run time makes the copy issue twice)
+              const int r0 = n0 + t * kSubN + rank * half_cols[t];
+              const int from_w = kFuse ? max(0, min(b_loads[t], (p.v_pad - r0) / kBBox)) : b_loads[t];
+              for (int i = 0; i < from_w; ++i)
+                tma_load_2d_pair(b_dst + t * kSubBBytes + i * (kBBox * kRowBytes), &map_b, kb * kElemsPerStage,
+                                 r0 + i * kBBox, full_leader);
+              if constexpr (kFuse) {
+                for (int i = from_w; i < b_loads[t]; ++i)
+                  tma_load_2d_pair(b_dst + t * kSubBBytes + i * (kBBox * kRowBytes), &map_c, kb * kElemsPerStage,
+                                   r0 + i * kBBox - p.v_pad, full_leader);
+              }
+            }
             if (++stage == kNumStages) { stage = 0; phase ^= 1u; }
           }
         }
@@ -504,7 +542,10 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         const UnitCoord uc = unit_coord(u, p);
         for (int n0 = uc.col_begin; n0 < uc.col_end && ok; n0 += kBN) {
           const int ncols = min(kBN, uc.col_end - n0);
-          const uint32_t idesc = kIdescNoN | (static_cast<uint32_t>(ncols >> 3) << 17);
+          uint32_t idesc[kNT];
+#pragma unroll
+          for (int t = 0; t < kNT; ++t)
+            idesc[t] = kIdescNoN | (static_cast<uint32_t>(max(0, min(kSubN, ncols - t * kSubN)) >> 3) << 17);
           if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
           tc_fence_after_sync();
           const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kAccCols);
@@ -513,10 +554,14 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
             tc_fence_after_sync();
             const uint32_t a_src = smem_base + stage * kStageBytes;
             const uint64_t a_desc = umma_desc_k_major_sw128(a_src);
-            const uint64_t b_desc = umma_desc_k_major_sw128(a_src + kABytes);
 #pragma unroll
-            for (int k = 0; k < kMmaPerStage; ++k)
-              umma_ss_pair<kTf32>(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            for (int t = 0; t < kNT; ++t) {
+              if (ncols <= t * kSubN) break;                // ragged tile without this subtile
+              const uint64_t b_desc = umma_desc_k_major_sw128(a_src + kABytes + t * kSubBBytes);
+#pragma unroll
+              for (int k = 0; k < kMmaPerStage; ++k)
+                umma_ss_pair<kTf32>(d_tmem + t * kSubN, a_desc + 2u * k, b_desc + 2u * k, idesc[t], (kb | k) != 0 ? 1u : 0u);
+            }
             umma_commit_pair(empty_bar(stage), 0x3);        // frees the stage in both CTAs
             if (++stage == kNumStages) { stage = 0; phase ^= 1u; }
           }
@@ -534,15 +579,18 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
     bool ok = true;
     for (int u = pair; u < p.total_units && ok; u += num_pairs) {
       const UnitCoord uc = unit_coord(u, p);
+      const int64_t row = static_cast<int64_t>(uc.row_block) * (2 * kTileM) + rank * kTileM + quad * 32 + lane;
       RowState st;
       st.init();
       for (int n0 = uc.col_begin; n0 < uc.col_end; n0 += kBN) {
         ok = __all_sync(0xffffffffu, mbar_wait(acc_full_bar(acc), acc_phase, abort_flag));
         if (!ok) break;
         tc_fence_after_sync();
-        const int ncols = min(min(kBN, uc.col_end - n0), p.V - n0);
+        const int tile_cols = min(kBN, uc.col_end - n0);
+        const int ncols = kFuse ? tile_cols : min(tile_cols, p.V - n0);
         const int cols_valid = min(kSpan, ncols - half * kSpan);
         const int npieces = cols_valid > 0 ? (cols_valid + 31) >> 5 : 0;
+        const int c_base = n0 + half * kSpan;
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
                                static_cast<uint32_t>(acc * kAccCols + half * kSpan);
         const uint32_t acc_empty_leader = map_to_cta(acc_empty_bar(acc), 0);
@@ -550,6 +598,9 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+        };
+        auto consume = [&](const uint32_t (&buf)[32], int pc) {
+          consume_piece<kFuse>(st, buf, c_base + pc * 32, cols_valid - pc * 32, p, row);
         };
         uint32_t bufA[32], bufB[32];
         if (npieces == 0) {
@@ -560,12 +611,12 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
           for (int pc = 0; pc < npieces; pc += 2) {
             const bool has1 = pc + 1 < npieces;
             if (has1) tmem_ld_32(taddr + (pc + 1) * 32, bufB); else release();
-            st.fold_n(bufA, cols_valid - pc * 32);
+            consume(bufA, pc);
             if (has1) {
               tmem_ld_wait(bufB);
               const bool has2 = pc + 2 < npieces;
               if (has2) tmem_ld_32(taddr + (pc + 2) * 32, bufA); else release();
-              st.fold_n(bufB, cols_valid - (pc + 1) * 32);
+              consume(bufB, pc + 1);
               if (has2) tmem_ld_wait(bufA);
             }
           }
@@ -573,7 +624,6 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         if (++acc == kNumAcc) { acc = 0; acc_phase ^= 1u; }
       }
       if (ok) {
-        const int64_t row = static_cast<int64_t>(uc.row_block) * (2 * kTileM) + rank * kTileM + quad * 32 + lane;
         const int slot = uc.chunk * kEpiSplit + half;
         float* dst = p.partials + (row * p.slots + slot) * 3;
         dst[0] = st.m;
@@ -612,9 +662,11 @@ constexpr Shape kShapeDecode1 = {1, 256, 32, 4, 32};    // <= 128 rows: W stream
 constexpr Shape kShapeDecode2 = {2, 256, 32, 3, 32};    // 129..256 rows: both row tiles share each W tile
 
 constexpr Shape kShapePairPrompt = {2, 256, 128, 6, 256};  // CTA pairs, 256 x 256 tiles
-constexpr Shape kShapePairDecode = {2, 256, 32, 6, 64};    // CTA pairs, one vocabulary range per pair
-constexpr int kPairStages = 6;
+constexpr Shape kShapePairDecode = {2, 512, 32, 4, 64};    // CTA pairs, 256 x 512 tiles, one vocabulary range per pair
+constexpr int kPairStages = 6;         // 256 x 256 tiles: 6 x 32 KB
+constexpr int kPairWideStages = 4;     // 256 x 512 tiles: 4 x 48 KB
 constexpr int kPairSmemBytes = kPairStages * (kTileM * kRowBytes + 128 * kRowBytes) + kBarrierBytes + 1024;
+static_assert(kPairWideStages * (kTileM * kRowBytes + 2 * 128 * kRowBytes) + kBarrierBytes + 1024 == kPairSmemBytes, "both pair forms use the same shared memory");
 
 const Shape& shape_of(int variant) {
   if (variant == 4) return kShapePairPrompt;
@@ -639,20 +691,22 @@ cudaError_t prepare_shape() {
                               smem_bytes_for(kMT, kBN, kNumStages));
 }
 
-template <bool kTf32, int kBBox>
-cudaError_t launch_pair(const LmheadPlan& plan, const CUtensorMap* a, const CUtensorMap* b, const KParams& p,
-                        cudaStream_t stream) {
-  auto kernel = lmhead_entropy_pair_kernel<kTf32, kBBox, kPairStages>;
-  kernel<<<plan.grid, kLmheadThreads, kPairSmemBytes, stream>>>(*a, *b, p);
+// kBBox 128: 256 x 256 tiles (prompt batches); 32: 256 x 512 tiles (decode batches), optionally with head columns
+template <bool kTf32, int kBBox, bool kFuse = false>
+cudaError_t launch_pair(const LmheadPlan& plan, const LmheadMaps& m, const KParams& p, cudaStream_t stream) {
+  auto kernel = kBBox == 32 ? lmhead_entropy_pair_kernel<kTf32, kBBox, kPairWideStages, 2, kFuse>
+                            : lmhead_entropy_pair_kernel<kTf32, kBBox, kPairStages, 1, kFuse>;
+  kernel<<<plan.grid, kLmheadThreads, kPairSmemBytes, stream>>>(*m.hidden, *m.w, kFuse ? *m.w1 : *m.w, p);
   return cudaGetLastError();
 }
 
 // CTA pairs that can be resident at once on the current device (set by lmhead_prepare_device).
 int g_pair_workers_max = 0;
 
-template <bool kTf32, int kBBox>
+template <bool kTf32, int kBBox, bool kFuse = false>
 cudaError_t prepare_pair(int num_sms) {
-  auto kernel = lmhead_entropy_pair_kernel<kTf32, kBBox, kPairStages>;
+  auto kernel = kBBox == 32 ? lmhead_entropy_pair_kernel<kTf32, kBBox, kPairWideStages, 2, kFuse>
+                            : lmhead_entropy_pair_kernel<kTf32, kBBox, kPairStages, 1, kFuse>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
@@ -684,11 +738,12 @@ static_assert(kShapeDecode2.mt == 2 && kShapeDecode2.bn == 256 && kShapeDecode2.
 LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity,
                             int mode, int head_cols) {
   LmheadPlan pl{};
+  // decode batches of 129..256 rows run as CTA pairs on 256 x 512 tiles unless single CTAs are asked for or the
+  // device cannot co-schedule the pairs; prompt batches run as pairs only on request (and never with head columns)
   pl.variant = T <= kTileM ? 1 : (T <= 2 * kTileM ? 2 : 0);
-  if (mode == EGTP_LMHEAD_CTA_PAIRS) {
-    if (pl.variant == 0) pl.variant = 4;
-    if (pl.variant == 2) pl.variant = 5;
-  }
+  const bool pairs_ok = g_pair_workers_max > 0 && mode != EGTP_LMHEAD_SINGLE_CTA;
+  if (pl.variant == 2 && pairs_ok) pl.variant = 5;
+  if (pl.variant == 0 && pairs_ok && mode == EGTP_LMHEAD_CTA_PAIRS && head_cols == 0) pl.variant = 4;
   const bool pair = pl.variant >= 4;
   const bool one_block = pl.variant == 1 || pl.variant == 2 || pl.variant == 5;
   const Shape& sh = shape_of(pl.variant);
@@ -770,6 +825,7 @@ cudaError_t lmhead_prepare_device() {
   if ((e = prepare_pair<false, 128>(num_sms)) != cudaSuccess) return e;
   if ((e = prepare_pair<false, 32>(num_sms)) != cudaSuccess) return e;
   if ((e = prepare_pair<true, 128>(num_sms)) != cudaSuccess) return e;
+  if ((e = prepare_pair<false, 32, true>(num_sms)) != cudaSuccess) return e;
   return prepare_pair<true, 32>(num_sms);
 }
 
@@ -791,14 +847,15 @@ cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const Lmhea
   p.v_pad = plan.v_pad;
   p.ldg = plan.head_cols_pad;
   p.head_g = head_g;
-  if (maps.hidden == nullptr || maps.w == nullptr || maps.w_tile == nullptr) return cudaErrorInvalidValue;
+  if (maps.hidden == nullptr || maps.w == nullptr || (plan.variant < 4 && maps.w_tile == nullptr)) return cudaErrorInvalidValue;
   if (plan.head_cols_pad > 0) {
     // fused head columns: bf16, one CTA per SM only
-    if (tf32 || maps.w1 == nullptr || maps.w1_tile == nullptr || head_g == nullptr) return cudaErrorInvalidValue;
+    if (tf32 || maps.w1 == nullptr || (plan.variant < 4 && maps.w1_tile == nullptr) || head_g == nullptr) return cudaErrorInvalidValue;
     switch (plan.variant) {
       case 0: return launch_shape<false, EGTP_SHAPE_PROMPT, true>(plan, maps, p, stream);
       case 1: return launch_shape<false, EGTP_SHAPE_DECODE1, true>(plan, maps, p, stream);
       case 2: return launch_shape<false, EGTP_SHAPE_DECODE2, true>(plan, maps, p, stream);
+      case 5: return launch_pair<false, 32, true>(plan, maps, p, stream);
       default: return cudaErrorInvalidValue;
     }
   }
@@ -806,16 +863,16 @@ cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const Lmhea
     switch (plan.variant) {
       case 1: return launch_shape<true, EGTP_SHAPE_DECODE1>(plan, maps, p, stream);
       case 2: return launch_shape<true, EGTP_SHAPE_DECODE2>(plan, maps, p, stream);
-      case 4: return launch_pair<true, 128>(plan, maps.hidden, maps.w, p, stream);
-      case 5: return launch_pair<true, 32>(plan, maps.hidden, maps.w, p, stream);
+      case 4: return launch_pair<true, 128>(plan, maps, p, stream);
+      case 5: return launch_pair<true, 32>(plan, maps, p, stream);
       default: return launch_shape<true, EGTP_SHAPE_PROMPT>(plan, maps, p, stream);
     }
   }
   switch (plan.variant) {
     case 1: return launch_shape<false, EGTP_SHAPE_DECODE1>(plan, maps, p, stream);
     case 2: return launch_shape<false, EGTP_SHAPE_DECODE2>(plan, maps, p, stream);
-    case 4: return launch_pair<false, 128>(plan, maps.hidden, maps.w, p, stream);
-    case 5: return launch_pair<false, 32>(plan, maps.hidden, maps.w, p, stream);
+    case 4: return launch_pair<false, 128>(plan, maps, p, stream);
+    case 5: return launch_pair<false, 32>(plan, maps, p, stream);
     default: return launch_shape<false, EGTP_SHAPE_PROMPT>(plan, maps, p, stream);
   }
 }

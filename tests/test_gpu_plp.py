@@ -75,6 +75,21 @@ def test_decode_loop_in_cta_pair_mode(ctx):
     egtp.plp_state_destroy(st)
 
 
+def test_decode_loop_in_single_cta_mode(ctx):
+    # 129..256 rows default to CTA pairs on 256 x 512 tiles; the one-CTA form (both row tiles per W tile) stays selectable
+    wl = gen.config_plp_decode(slots=200, steps=6, d=256, V=9000 + 40, m_h=64, mu=1.0, sigma=0.5)
+    egtp.egtp_set_lmhead_mode(ctx, egtp.EGTP_LMHEAD_SINGLE_CTA)
+    try:
+        assert egtp.egtp_lmhead_plan(ctx, 200, 256, 9040, egtp.EGTP_BF16)["rows_per_block"] == 256
+        st, H, z, y = _run_plp(ctx, wl)
+    finally:
+        egtp.egtp_set_lmhead_mode(ctx, egtp.EGTP_LMHEAD_AUTO)
+    follow = [0, 127, 128, 199]
+    ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=follow)
+    _compare(H, z, y, ref, follow)
+    egtp.plp_state_destroy(st)
+
+
 def test_rl_group_sampling_continues_from_egtp_state(ctx):
     # EGTP over shared prompts, then decode streams that start from their prompt's state (fan-out 4)
     wl = gen.config_rl_group(prompts=5, group=4, steps=12, d=256, V=7000, m_h=64, min_len=3, max_len=200)

@@ -77,6 +77,21 @@ def test_bound_decode_loop_matches_oracle(ctx, slots, V, m_h):
     egtp.plp_state_destroy(st2)
 
 
+def test_bound_decode_loop_in_single_cta_mode(ctx):
+    # 129..256 rows: the default is the CTA-pair kernel with head columns; this is the one-CTA kernel with head columns
+    wl = gen.config_plp_decode(slots=190, steps=8, d=256, V=6000 + 8, m_h=72, mu=1.5, sigma=0.8)
+    egtp.egtp_set_lmhead_mode(ctx, egtp.EGTP_LMHEAD_SINGLE_CTA)
+    try:
+        st, H, z, y, launches = _run(ctx, wl)
+    finally:
+        egtp.egtp_set_lmhead_mode(ctx, egtp.EGTP_LMHEAD_AUTO)
+    assert launches == 2 + 2 * wl.steps
+    follow = [0, 127, 128, 189]
+    ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=follow)
+    _compare(H, z, y, ref, follow)
+    egtp.plp_state_destroy(st)
+
+
 def test_bound_bins_head_without_z(ctx):
     wl = gen.config_plp_decode(slots=140, steps=6, d=256, V=5000, m_h=64, mu=1.5, sigma=0.5)
     head_bins = gen.make_head(11, 256, 64, 20, "bf16", mode=gen.HEAD_BINS)
