@@ -744,7 +744,8 @@ int plp_step(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head
     EGTP_CUDA_TRY(launch_plp_update_bound(hidden_step, ldh, c->partials, plan.slots, plan.slots * 3, 3, Hstep_out, slot_ids,
                                           reset_src, src_m, src_s, src_pooled, st->src_proj, n_src, B_live, st->d,
                                           st->num_slots, 1.f / alpha, st->m, st->s, st->acc, st->proj, z_out, st->d,
-                                          st->head_g, plan.head_cols_pad, head_args(head), yrem_out, status, stream));
+                                          st->head_g, plan.head_cols_pad, head_args(head), yrem_out, status, stream,
+                                          /*overlap_previous=*/!c->profiling));
     return EGTP_OK;
   }
   rc = run_lmhead(c, lm, hidden_step, ldh, B_live, status, stream, &plan);

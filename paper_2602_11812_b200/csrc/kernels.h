@@ -136,13 +136,16 @@ cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, c
 
 // The update for a state bound to a head (bf16 hidden states and head weights): also advances the slot's
 // projection st_proj = W1 acc with g = W1 h' from the LM-head kernel and finishes the head for the row.
-// src_proj [n_src][m_h] = W1 src_pooled; z may be NULL.
+// src_proj [n_src][m_h] = W1 src_pooled; z may be NULL.  overlap_previous: launch with programmatic stream
+// serialization, so that blocks are staged (and read their state rows) while the LM-head kernel before it in the
+// stream is still running; the kernel waits for that kernel's end before it reads its results.
 cudaError_t launch_plp_update_bound(const void* hidden_step, int64_t ldh, const float* partials, int slots,
                                     int64_t row_stride, int64_t slot_stride, float* Hstep_out, const int32_t* slot_ids,
                                     const int32_t* reset_src, const float* src_m, const float* src_s,
                                     const float* src_pooled, const float* src_proj, int n_src, int rows, int d,
                                     int num_slots, float inv_alpha, float* st_m, float* st_s, float* st_acc,
                                     float* st_proj, float* z, int64_t ldz, const float* g, int64_t ldg,
-                                    const HeadArgs& h, float* y, int32_t* status, cudaStream_t stream);
+                                    const HeadArgs& h, float* y, int32_t* status, cudaStream_t stream,
+                                    bool overlap_previous);
 
 }  // namespace egtp

@@ -187,6 +187,9 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   __syncthreads();
   if (*abort_flag != 0u) return;
   __syncthreads();
+  // the kernel that consumes the partials may be staged on SMs this grid has left (it waits for the grid's end
+  // before it reads anything written here)
+  pdl_launch_dependents();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kNumStages; ++s) {
@@ -472,6 +475,7 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
   cluster_sync_all();           // barriers of both CTAs are initialised before anyone signals across
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_launch_dependents();      // see the one-CTA kernel
   // both CTAs follow the leader's reading of the status word
   const bool skip = ld_shared_cluster_u32(map_to_cta(smem_u32(const_cast<uint32_t*>(skip_flag)), 0)) != 0u;
 

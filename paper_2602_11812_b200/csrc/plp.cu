@@ -9,6 +9,7 @@
 #include "kernels.h"
 #include "entropy_merge.cuh"
 #include "head_out.cuh"
+#include "sm100_ptx.cuh"
 #include "../../include/egtp.h"
 
 #include <cuda_bf16.h>
@@ -135,7 +136,9 @@ plp_update_bound_kernel(const T* __restrict__ hidden_step, int64_t ldh, const fl
                         const float* __restrict__ g, int64_t ldg, int m_h, int d_out, const float* __restrict__ b1,
                         const TW* __restrict__ W2, const float* __restrict__ b2, const float* __restrict__ centres,
                         int mode, float* __restrict__ y, int32_t* status) {
-  if (*status != 0) return;
+  // Launched with programmatic stream serialization: this block may start while the LM-head kernel is still
+  // running.  Its inputs and the state rows (last written by an earlier, completed kernel) are read ahead;
+  // the status word, the entropy partials and g come after pdl_wait().
   extern __shared__ float smem[];
   float* u = smem;            // [m_h]
   float* o = smem + m_h;      // [d_out]
@@ -173,6 +176,8 @@ plp_update_bound_kernel(const T* __restrict__ hidden_step, int64_t ldh, const fl
     load8<T>(hrow + col, h);
     if (acc_src != nullptr) load8<float>(acc_src + col, acc);
   }
+  pdl_wait();
+  if (*status != 0) return;     // uniform over the block
   const float H_new = merge_partials_warp(partials + static_cast<int64_t>(i) * row_stride, slots, slot_stride, threadIdx.x & 31);
   if (threadIdx.x == 0 && Hstep_out != nullptr) Hstep_out[i] = H_new;
   const float a = H_new * inv_alpha;
@@ -225,14 +230,25 @@ cudaError_t launch_plp_update_bound(const void* hidden_step, int64_t ldh, const 
                                     const float* src_pooled, const float* src_proj, int n_src, int rows, int d,
                                     int num_slots, float inv_alpha, float* st_m, float* st_s, float* st_acc,
                                     float* st_proj, float* z, int64_t ldz, const float* g, int64_t ldg,
-                                    const HeadArgs& h, float* y, int32_t* status, cudaStream_t stream) {
+                                    const HeadArgs& h, float* y, int32_t* status, cudaStream_t stream, bool overlap_previous) {
   const int threads = std::min(kPlpMaxThreads, std::max(64, (d / 8 + 31) / 32 * 32));
   const size_t smem = static_cast<size_t>(h.m_h + h.d_out) * sizeof(float);
-  plp_update_bound_kernel<__nv_bfloat16, __nv_bfloat16><<<rows, threads, smem, stream>>>(
-      static_cast<const __nv_bfloat16*>(hidden_step), ldh, partials, slots, row_stride, slot_stride, Hstep_out, slot_ids,
-      reset_src, src_m, src_s, src_pooled, src_proj, n_src, d, num_slots, inv_alpha, st_m, st_s, st_acc, st_proj, z, ldz,
-      g, ldg, h.m_h, h.d_out, h.b1, static_cast<const __nv_bfloat16*>(h.W2), h.b2, h.centres, h.mode, y, status);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(rows);
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = overlap_previous ? 1 : 0;
+  const __nv_bfloat16* hs = static_cast<const __nv_bfloat16*>(hidden_step);
+  const __nv_bfloat16* W2 = static_cast<const __nv_bfloat16*>(h.W2);
+  return cudaLaunchKernelEx(&cfg, plp_update_bound_kernel<__nv_bfloat16, __nv_bfloat16>, hs, ldh, partials, slots,
+                            row_stride, slot_stride, Hstep_out, slot_ids, reset_src, src_m, src_s, src_pooled, src_proj,
+                            n_src, d, num_slots, inv_alpha, st_m, st_s, st_acc, st_proj, z, ldz, g, ldg, h.m_h, h.d_out,
+                            h.b1, W2, h.b2, h.centres, h.mode, y, status);
 }
 
 cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, const float* partials, int slots,

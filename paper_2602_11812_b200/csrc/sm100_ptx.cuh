@@ -267,6 +267,14 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t cta_mask
                : "memory");
 }
 
+// ----------------------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-stream-serialization attribute may start while the kernel before it
+// in the stream is still running, once that kernel has executed pdl_launch_dependents() in every CTA (or
+// exited).  pdl_wait() blocks until the earlier kernel has completed and its writes are visible; everything a
+// kernel reads from its predecessor must come after it.  Both are no-ops in launches without the attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ----------------------------------------------------------------------------- scalar helpers
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
