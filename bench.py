@@ -370,8 +370,12 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
         for t in range(warm):
             egtp.plp_step(ctx, st, lm, head.c, hs[t], reset_src=reset[t], yrem_out=yrem, status_dev=status)
         torch.cuda.synchronize()
-        # pass 1: step times, no per-kernel events in the stream (they cost a few microseconds per step here)
+        # pass 1: step times, no per-kernel events in the stream (they cost a few microseconds per step here);
+        # every route starts its burst from an idle GPU (the power state of the previous burst carries over otherwise)
         egtp.egtp_profile_enable(ctx, False)
+        time.sleep(0.5)
+        for t in range(warm):
+            egtp.plp_step(ctx, st, lm, head.c, hs[t], reset_src=None, yrem_out=yrem, status_dev=status)
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(plp_steps + 1)]
         evs[0].record()
         for t in range(plp_steps):
@@ -548,6 +552,100 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     return plp, long_
 
 
+def bench_rl_group(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
+    """RL group sampling at its full sizes: EGTP over 64 shared prompts (d = 5120, V = 152064), then PLP steps over
+    1024 decode streams that start from their prompt's state (tensor-bound: 8 row blocks of 128 rows per step)."""
+    import torch
+
+    from paper_2602_11812_b200 import binding as egtp
+    from paper_2602_11812_b200 import device as gu
+    from paper_2602_11812_b200 import inputs as gen
+
+    warm = 3
+    wl = gen.config_rl_group(steps=warm + plp_steps)
+    eg = wl.prompts
+    slots, d, V = wl.slots, wl.d, wl.V
+    W = gu.dev_tensor(wl.W, "bf16")
+    lm = egtp.make_lm_head(W)
+    head = gu.DeviceHead(wl.head, "bf16")
+    ctx = egtp.egtp_create(ctx_device, max_tokens=eg.T, max_batch=slots, max_d=d, max_V=V)
+    status = torch.zeros(1, device="cuda", dtype=torch.int32)
+    f = dict(device="cuda", dtype=torch.float32)
+    # ---- EGTP over the shared prompts
+    hidden = gu.dev_tensor(eg.hidden, "bf16")
+    off = torch.from_numpy(eg.offsets).cuda()
+    yhat, pooled = torch.empty(eg.B, **f), torch.empty(eg.B, d, **f)
+    sm, ss = torch.empty(eg.B, **f), torch.empty(eg.B, **f)
+
+    def predict():
+        egtp.egtp_predict(ctx, lm, head.c, hidden, off, eg.B, eg.T, 1.0, pooled_out=pooled, state_m_out=sm,
+                          state_s_out=ss, yhat_out=yhat, status_dev=status)
+
+    predict()
+    torch.cuda.synchronize()
+    egtp.egtp_profile_enable(ctx, True)
+    egtp.egtp_profile_read(ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(egtp_steps):
+        predict()
+    e1.record()
+    torch.cuda.synchronize()
+    prof = egtp.egtp_profile_read(ctx)
+    ms_step = e0.elapsed_time(e1) / egtp_steps
+    k1_ms = prof["lmhead_entropy"]["ms"] / prof["lmhead_entropy"]["launches"]
+    tf = 2.0 * d * V * eg.T / (k1_ms * 1e-3) / 1e12
+    out = dict(workload="rl_group: 64 prompts U[256,4096] x 16 streams, d=5120, V=152064, head 5120->512->1",
+               egtp=dict(tokens=eg.T, steps=egtp_steps, ms_per_step=ms_step, value=eg.T / (ms_step * 1e-3), unit=UNIT,
+                         lmhead=dict(bound="tensor", achieved=tf, peak=peaks["bf16_tflops"], unit="TFLOP/s",
+                                     frac=tf / peaks["bf16_tflops"], ms_per_launch=k1_ms),
+                         kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof.items() if v["launches"]}))
+    del hidden
+    # ---- PLP over the 1024 streams: ordinary route, then the state bound to the head
+    hs = gu.dev_tensor(wl.hidden_steps.reshape(-1, d), "bf16").reshape(warm + plp_steps, slots, d)
+    reset0 = torch.from_numpy(wl.reset_src[0].copy()).cuda()
+    yrem = torch.empty(slots, **f)
+
+    def measure(bind):
+        st = egtp.plp_state_create(ctx, slots, d)
+        if bind:
+            egtp.plp_state_bind_head(st, head.c)
+        # step 0 starts every stream from its prompt's EGTP state; later steps pass no reset table
+        egtp.plp_step(ctx, st, lm, head.c, hs[0], reset_src=reset0, src_m=sm, src_s=ss, src_pooled=pooled, n_src=eg.B,
+                      yrem_out=yrem, status_dev=status)
+        for t in range(1, warm):
+            egtp.plp_step(ctx, st, lm, head.c, hs[t], yrem_out=yrem, status_dev=status)
+        torch.cuda.synchronize()
+        egtp.egtp_profile_enable(ctx, False)
+        time.sleep(0.5)       # both routes start their burst from an idle GPU (the power state carries over otherwise)
+        for t in range(1, warm):
+            egtp.plp_step(ctx, st, lm, head.c, hs[t], yrem_out=yrem, status_dev=status)
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for t in range(plp_steps):
+            egtp.plp_step(ctx, st, lm, head.c, hs[warm + t], yrem_out=yrem, status_dev=status)
+        a1.record()
+        torch.cuda.synchronize()
+        egtp.egtp_profile_enable(ctx, True)
+        egtp.egtp_profile_read(ctx)
+        for t in range(plp_steps):
+            egtp.plp_step(ctx, st, lm, head.c, hs[warm + t], yrem_out=yrem, status_dev=status)
+        torch.cuda.synchronize()
+        pr = egtp.egtp_profile_read(ctx)
+        egtp.plp_state_destroy(st)
+        us = a0.elapsed_time(a1) / plp_steps * 1e3
+        k_us = pr["lmhead_entropy"]["ms"] / pr["lmhead_entropy"]["launches"] * 1e3
+        tfl = 2.0 * slots * d * V / (k_us * 1e-6) / 1e12
+        return dict(us_per_step=us, lmhead=dict(bound="tensor", achieved=tfl, peak=peaks["bf16_tflops"], unit="TFLOP/s",
+                                                frac=tfl / peaks["bf16_tflops"], us_per_launch=k_us),
+                    kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in pr.items() if v["launches"]})
+
+    out["plp_B1024"] = dict(steps=plp_steps, ordinary=measure(False), bound_to_head=measure(True))
+    assert int(status.item()) == 0
+    egtp.egtp_destroy(ctx)
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -561,7 +659,15 @@ def main():
                     help="run only the d = 4096 workloads and print their two objects as one JSON line "
                          "(used for profiler captures of the decode and pooling kernels)")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--only-rl-group", action="store_true",
+                    help="run only the RL group-sampling sizes (d = 5120, V = 152064, 1024 streams) and print one JSON line")
     args = ap.parse_args()
+    if args.only_rl_group:
+        import torch
+        torch.cuda.set_device(0)
+        print(json.dumps(dict(rl_group=bench_rl_group(0, load_peaks(), min(args.plp_steps, 16), min(args.long_steps, 3)))),
+              flush=True)
+        return
     if args.only_d4096:
         import torch
         torch.cuda.set_device(0)

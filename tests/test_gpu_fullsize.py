@@ -78,11 +78,13 @@ def test_long_configuration_full_size():
         egtp.egtp_destroy(ctx)
 
 
-def _run_plp_steps(ctx, wl, W_dev, head, src=None):
+def _run_plp_steps(ctx, wl, W_dev, head, src=None, bind=False):
     steps, slots, d = wl.steps, wl.slots, wl.d
     hs = gu.dev_tensor(wl.hidden_steps.reshape(-1, d), wl.dtype).reshape(steps, slots, d)
     reset = torch.from_numpy(wl.reset_src).cuda()
     st = egtp.plp_state_create(ctx, slots, d)
+    if bind:     # the head's first layer rides along in the LM-head kernel, one kernel finishes the step
+        egtp.plp_state_bind_head(st, head.c)
     lm = egtp.make_lm_head(W_dev)
     f = dict(device="cuda", dtype=torch.float32)
     H, z, y = torch.zeros(steps, slots, **f), torch.zeros(steps, slots, d, **f), torch.zeros(steps, slots, **f)
@@ -106,18 +108,23 @@ def test_plp_decode_configuration_full_width():
     ctx = egtp.egtp_create(0, max_tokens=1024, max_batch=256, max_d=wl.d, max_V=wl.V)
     try:
         W_dev = gu.dev_tensor(wl.W, "bf16")
-        H, z, y = _run_plp_steps(ctx, wl, W_dev, gu.DeviceHead(wl.head, "bf16"))
+        head = gu.DeviceHead(wl.head, "bf16")
+        runs = [_run_plp_steps(ctx, wl, W_dev, head, bind=bind) for bind in (False, True)]
     finally:
         egtp.egtp_destroy(ctx)
     follow = [3, 130, 255]
     ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=follow)
-    gu.assert_entropy_close(H[:, follow].ravel(), ref["H"].ravel())
-    for t in range(wl.steps):
-        gu.assert_pooled_close(z[t, follow], ref["z"][t])
-    gu.assert_length_close(y[:, follow].ravel(), ref["yrem"].ravel())
-    # every slot, every step: z is a convex combination of the tokens seen since the last reset
-    assert np.all(np.isfinite(z)) and np.all(H > 0) and np.all(H <= np.log(wl.V) + 1e-3)
-    assert np.array_equal(z[7, 3], wl.hidden_steps[7, 3].astype(np.float64))
+    for H, z, y in runs:       # the ordinary route, then the state bound to its head (the route bench.py times)
+        gu.assert_entropy_close(H[:, follow].ravel(), ref["H"].ravel())
+        for t in range(wl.steps):
+            gu.assert_pooled_close(z[t, follow], ref["z"][t])
+        gu.assert_length_close(y[:, follow].ravel(), ref["yrem"].ravel())
+        # every slot, every step: z is a convex combination of the tokens seen since the last reset
+        assert np.all(np.isfinite(z)) and np.all(H > 0) and np.all(H <= np.log(wl.V) + 1e-3)
+        assert np.array_equal(z[7, 3], wl.hidden_steps[7, 3].astype(np.float64))
+    # both routes on all 256 slots: same entropies and lengths up to summation order
+    gu.assert_entropy_close(runs[1][0].ravel(), runs[0][0].ravel())
+    gu.assert_length_close(runs[1][2].ravel(), runs[0][2].ravel())
 
 
 def test_rl_group_configuration_full_size():
@@ -131,7 +138,8 @@ def test_rl_group_configuration_full_size():
         src = (torch.from_numpy(res["state_m"].astype(np.float32)).cuda(),
                torch.from_numpy(res["state_s"].astype(np.float32)).cuda(),
                torch.from_numpy(res["pooled"].astype(np.float32)).cuda(), eg.B)
-        H, z, y = _run_plp_steps(ctx, wl, W_dev, gu.DeviceHead(wl.head, "bf16"), src=src)
+        head = gu.DeviceHead(wl.head, "bf16")
+        runs = [_run_plp_steps(ctx, wl, W_dev, head, src=src, bind=bind) for bind in (False, True)]
     finally:
         egtp.egtp_destroy(ctx)
     b = _shortest_prompts(eg, 1)[0]
@@ -143,9 +151,11 @@ def test_rl_group_configuration_full_size():
     reset[0, follow] = 0
     ref = orc.plp_run(wl.hidden_steps, reset, wl.W, wl.head, slots=follow,
                       prompts=dict(hidden=rows, offsets=np.array([0, rows.shape[0]]), H=H_prompt))
-    gu.assert_entropy_close(H[:, follow].ravel(), ref["H"].ravel())
-    for t in range(wl.steps):
-        gu.assert_pooled_close(z[t, follow], ref["z"][t])
-    gu.assert_length_close(y[:, follow].ravel(), ref["yrem"].ravel())
-    # streams of one group that were fed different tokens differ; all are finite
-    assert np.all(np.isfinite(y)) and not np.array_equal(z[-1, follow[0]], z[-1, follow[1]])
+    for H, z, y in runs:       # the ordinary route, then the state bound to its head (1024 rows: 8 row blocks)
+        gu.assert_entropy_close(H[:, follow].ravel(), ref["H"].ravel())
+        for t in range(wl.steps):
+            gu.assert_pooled_close(z[t, follow], ref["z"][t])
+        gu.assert_length_close(y[:, follow].ravel(), ref["yrem"].ravel())
+        # streams of one group that were fed different tokens differ; all are finite
+        assert np.all(np.isfinite(y)) and not np.array_equal(z[-1, follow[0]], z[-1, follow[1]])
+    gu.assert_length_close(runs[1][2].ravel(), runs[0][2].ravel())
