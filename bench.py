@@ -470,34 +470,40 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     # ---- the same decode step when the serving engine already holds the step's logits
     torch.manual_seed(0)
     logits = (torch.randn(slots, V, device="cuda") * 1.5).to(torch.bfloat16)
-    for t in range(3):
-        egtp.plp_step_from_logits(ctx, st, logits, head.c, hs[t], reset_src=reset[t], yrem_out=yrem, status_dev=status)
-    torch.cuda.synchronize()
     n_fl = max(8, plp_steps)
 
-    def from_logits_steps():
-        for t in range(n_fl):
-            egtp.plp_step_from_logits(ctx, st, logits, head.c, hs[warm + t % plp_steps],
-                                      reset_src=reset[warm + t % plp_steps], yrem_out=yrem, status_dev=status)
+    def measure_from_logits(state):
+        def steps_():
+            for t in range(n_fl):
+                egtp.plp_step_from_logits(ctx, state, logits, head.c, hs[warm + t % plp_steps],
+                                          reset_src=reset[warm + t % plp_steps], yrem_out=yrem, status_dev=status)
+        for t in range(3):
+            egtp.plp_step_from_logits(ctx, state, logits, head.c, hs[t], reset_src=reset[t], yrem_out=yrem, status_dev=status)
+        torch.cuda.synchronize()
+        egtp.egtp_profile_enable(ctx, False)
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        steps_()
+        f1.record()
+        torch.cuda.synchronize()
+        egtp.egtp_profile_enable(ctx, True)
+        egtp.egtp_profile_read(ctx)
+        steps_()
+        torch.cuda.synchronize()
+        prof_fl = egtp.egtp_profile_read(ctx)
+        assert int(status.item()) == 0
+        le_us = prof_fl["logits_entropy"]["ms"] / prof_fl["logits_entropy"]["launches"] * 1e3
+        le_gbs = 2.0 * slots * V / (le_us * 1e-6) / 1e9
+        return dict(us_per_step=f0.elapsed_time(f1) / n_fl * 1e3, logits_entropy_us=le_us,
+                    hbm=dict(bound="hbm", kernel="logits_entropy", achieved=le_gbs, peak=peaks["hbm_gbs"],
+                             unit="GB/s", frac=le_gbs / peaks["hbm_gbs"], bytes_per_row=2 * V),
+                    kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof_fl.items() if v["launches"]})
 
-    egtp.egtp_profile_enable(ctx, False)
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record()
-    from_logits_steps()
-    f1.record()
-    torch.cuda.synchronize()
-    egtp.egtp_profile_enable(ctx, True)
-    egtp.egtp_profile_read(ctx)
-    from_logits_steps()
-    torch.cuda.synchronize()
-    prof_fl = egtp.egtp_profile_read(ctx)
-    assert int(status.item()) == 0
-    le_us = prof_fl["logits_entropy"]["ms"] / prof_fl["logits_entropy"]["launches"] * 1e3
-    le_gbs = 2.0 * slots * V / (le_us * 1e-6) / 1e9
-    plp["from_logits"] = dict(us_per_step=f0.elapsed_time(f1) / n_fl * 1e3, logits_entropy_us=le_us,
-                              hbm=dict(bound="hbm", kernel="logits_entropy", achieved=le_gbs, peak=peaks["hbm_gbs"],
-                                       unit="GB/s", frac=le_gbs / peaks["hbm_gbs"], bytes_per_row=2 * V),
-                              kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof_fl.items() if v["launches"]})
+    # bound state: W1 h' from a launch of the LM-head kernel over the head columns alone (reported as head_hidden)
+    plp["from_logits"] = measure_from_logits(st)
+    st_plain = egtp.plp_state_create(ctx, slots, d)
+    plp["from_logits"]["unbound_state"] = measure_from_logits(st_plain)
+    egtp.plp_state_destroy(st_plain)
     egtp.plp_state_destroy(st)
     del hs, logits
 

@@ -203,9 +203,10 @@ EGTP_API int plp_step(egtp_ctx* ctx, plp_state* st, const egtp_lm_head* lm, cons
  *          struct is copied; the weights it points at must stay in place and unchanged while bound.
  * Allocates num_slots * m_h + max_batch * m_h + (padded rows) * (padded m_h) floats and synchronises the device
  * (a create-time call, not for the decode loop).  Binding again replaces the previous binding.
- * plp_step takes the bound route when it is given the same head (same W1 pointer, m_h, d, dtype) with
- * yrem_out != NULL, bf16 hidden states and LM head, and n_src <= the context's max_batch; every other call
- * (another head, no head, plp_step_from_logits / _from_partials, plp_state_import) takes the ordinary route or
+ * plp_step, plp_step_from_logits and plp_step_from_partials take the bound route when they are given the same
+ * head (same W1 pointer, m_h, d, dtype) with yrem_out != NULL, bf16 hidden states (and LM head), and n_src <= the
+ * context's max_batch; the two that run no LM-head GEMM get W1 h' from a launch of the LM-head kernel over the
+ * head columns alone.  Every other call (another head, no head, plp_state_import) takes the ordinary route or
  * changes acc directly, and the next bound step first recomputes P = W1 acc for all slots (one layer-1 pass
  * over num_slots rows).  A bound step that restarts rows from EGTP rows (reset_src != NULL and n_src > 0)
  * first projects the n_src source rows (W1 src_pooled), so pass reset_src = NULL on steps without restarts

@@ -78,6 +78,7 @@ struct plp_state {
   float* src_proj = nullptr;    // [ctx->max_batch][m_h]: W1 src_pooled of the current step
   float* head_g = nullptr;      // [g_rows][ldg_max]: W1 h' of the current step, written by the LM-head kernel
   int64_t g_rows = 0, ldg_max = 0;
+  int g_max_splits = 1;         // K splits head_g has room for (projection launches without an LM head)
 };
 
 namespace {
@@ -277,26 +278,6 @@ int check_plp_common(const egtp_ctx* c, const plp_state* st, const egtp_head* he
   return EGTP_OK;
 }
 
-// Second half of a PLP step: merge the entropy partials, update the slots (Eq. 8), run the head.
-int plp_update_and_head(egtp_ctx* c, plp_state* st, const egtp_head* head, const void* hidden_step, int64_t ldh,
-                        int hidden_dtype, const float* partials, int slots, int64_t row_stride, int64_t slot_stride,
-                        const int32_t* slot_ids, const int32_t* reset_src,
-                        const float* src_m, const float* src_s, const float* src_pooled, int n_src, int B_live,
-                        float alpha, float* Hstep_out, float* z_out, float* yrem_out, int32_t* status,
-                        cudaStream_t stream) {
-  float* z = z_out ? z_out : c->pooled;
-  st->proj_valid = false;   // acc moves on without the projection a bound state keeps
-  {
-    LaunchScope ls(c, EGTP_K_PLP_UPDATE, stream);
-    EGTP_CUDA_TRY(launch_plp_update(hidden_step, ldh, hidden_dtype == EGTP_BF16, partials, slots, row_stride, slot_stride, Hstep_out,
-                                    slot_ids,
-                                    reset_src, src_m, src_s, src_pooled, n_src, B_live, st->d, st->num_slots,
-                                    1.f / alpha, st->m, st->s, st->acc, z, st->d, status, stream));
-  }
-  if (head && yrem_out) return run_head(c, head, z, st->d, B_live, yrem_out, nullptr, status, stream);
-  return EGTP_OK;
-}
-
 // out[r] = W1 x[r] for rows of fp32 vectors x (layer 1 of the head without bias and ReLU), in row chunks that fit
 // the split-K workspace.
 int project_rows(egtp_ctx* c, const egtp_head* head, const float* x, int64_t ldx, int rows, float* out, int64_t ld_out,
@@ -320,16 +301,72 @@ int project_rows(egtp_ctx* c, const egtp_head* head, const float* x, int64_t ldx
 }
 
 // True when this step can take the route of a state bound to `head`: the LM-head kernel also produces W1 h'.
-bool plp_fused_route(const egtp_ctx* c, const plp_state* st, const egtp_lm_head* lm, const egtp_head* head,
+bool plp_fused_route(const egtp_ctx* c, const plp_state* st, int hidden_dtype, const egtp_head* head,
                      int B_live, int n_src, const float* yrem_out) {
   if (!st->bound || !head || !yrem_out) return false;
   const egtp_head& b = st->bound_head;
   if (head->W1 != b.W1 || head->m_h != b.m_h || head->d != b.d || head->wdtype != b.wdtype) return false;
-  if (lm->dtype != EGTP_BF16 || head->wdtype != EGTP_BF16) return false;
+  if (hidden_dtype != EGTP_BF16 || head->wdtype != EGTP_BF16) return false;
   if (n_src > c->max_batch) return false;
   const int64_t rows_pad = B_live <= 2 * kTileM ? (B_live <= kTileM ? kTileM : 2 * kTileM)
                                                 : (static_cast<int64_t>(B_live) + kTileM - 1) / kTileM * kTileM;
   return rows_pad <= st->g_rows;
+}
+
+// Second half of a PLP step: merge the entropy partials, update the slots (Eq. 8), run the head.
+int plp_update_and_head(egtp_ctx* c, plp_state* st, const egtp_head* head, const void* hidden_step, int64_t ldh,
+                        int hidden_dtype, const float* partials, int slots, int64_t row_stride, int64_t slot_stride,
+                        const int32_t* slot_ids, const int32_t* reset_src,
+                        const float* src_m, const float* src_s, const float* src_pooled, int n_src, int B_live,
+                        float alpha, float* Hstep_out, float* z_out, float* yrem_out, int32_t* status,
+                        cudaStream_t stream) {
+  if (plp_fused_route(c, st, hidden_dtype, head, B_live, n_src, yrem_out) &&
+      reinterpret_cast<uintptr_t>(hidden_step) % 16 == 0 && (ldh * 2) % 16 == 0) {
+    // State bound to this head, entropies from elsewhere (logits in memory, gathered shard partials): W1 h' comes
+    // from a launch of the LM-head kernel over the head columns alone (K split over the SMs), then the bound update.
+    if (!st->proj_valid) {
+      int rc = project_rows(c, head, st->acc, st->d, st->num_slots, st->proj, head->m_h, status, stream);
+      if (rc != EGTP_OK) return rc;
+      st->proj_valid = true;
+    }
+    if (reset_src && n_src > 0) {
+      int rc = project_rows(c, head, src_pooled, st->d, n_src, st->src_proj, head->m_h, status, stream);
+      if (rc != EGTP_OK) return rc;
+    }
+    const LmheadPlan plan = make_headproj_plan(B_live, st->d, head->m_h, 2, c->num_sms, st->g_max_splits);
+    if (plan.rows_pad > st->g_rows || plan.head_cols_pad > st->ldg_max) return EGTP_ERR_CAPACITY;
+    CUtensorMap map_a, map_c;
+    int rc = make_tensor_map(c, &map_a, hidden_step, EGTP_BF16, B_live, st->d, ldh, plan.a_box_rows);
+    if (rc != EGTP_OK) return rc;
+    rc = make_tensor_map(c, &map_c, head->W1, EGTP_BF16, head->m_h, st->d, st->d, plan.b_box_rows);
+    if (rc != EGTP_OK) return rc;
+    LmheadMaps maps;
+    maps.hidden = &map_a;
+    maps.w = maps.w_tile = maps.w1 = maps.w1_tile = &map_c;
+    {
+      LaunchScope ls(c, EGTP_K_HEAD_HIDDEN, stream);
+      EGTP_CUDA_TRY(launch_lmhead_entropy(plan, false, maps, B_live, 0, nullptr, status, stream, st->head_g));
+    }
+    LaunchScope ls(c, EGTP_K_PLP_UPDATE, stream);
+    EGTP_CUDA_TRY(launch_plp_update_bound(hidden_step, ldh, partials, slots, row_stride, slot_stride, Hstep_out, slot_ids,
+                                          reset_src, src_m, src_s, src_pooled, st->src_proj, n_src, B_live, st->d,
+                                          st->num_slots, 1.f / alpha, st->m, st->s, st->acc, st->proj, z_out, st->d,
+                                          st->head_g, plan.head_cols_pad, plan.k_splits,
+                                          plan.rows_pad * static_cast<int64_t>(plan.head_cols_pad), head_args(head),
+                                          yrem_out, status, stream, /*overlap_previous=*/false));
+    return EGTP_OK;
+  }
+  float* z = z_out ? z_out : c->pooled;
+  st->proj_valid = false;   // acc moves on without the projection a bound state keeps
+  {
+    LaunchScope ls(c, EGTP_K_PLP_UPDATE, stream);
+    EGTP_CUDA_TRY(launch_plp_update(hidden_step, ldh, hidden_dtype == EGTP_BF16, partials, slots, row_stride, slot_stride, Hstep_out,
+                                    slot_ids,
+                                    reset_src, src_m, src_s, src_pooled, n_src, B_live, st->d, st->num_slots,
+                                    1.f / alpha, st->m, st->s, st->acc, z, st->d, status, stream));
+  }
+  if (head && yrem_out) return run_head(c, head, z, st->d, B_live, yrem_out, nullptr, status, stream);
+  return EGTP_OK;
 }
 
 // The whole EGTP chain.  With pieces > 1 the LM-head phase runs over row ranges of the batch one after the
@@ -726,7 +763,7 @@ int plp_step(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head
   int32_t* status = status_dev ? status_dev : c->status;
   if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
   LmheadPlan plan;
-  if (plp_fused_route(c, st, lm, head, B_live, n_src, yrem_out)) {
+  if (plp_fused_route(c, st, lm->dtype, head, B_live, n_src, yrem_out)) {
     // bound state: W1 h' comes out of the LM-head kernel, one kernel finishes the step
     if (!st->proj_valid) {
       rc = project_rows(c, head, st->acc, st->d, st->num_slots, st->proj, head->m_h, status, stream);
@@ -744,7 +781,7 @@ int plp_step(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head
     EGTP_CUDA_TRY(launch_plp_update_bound(hidden_step, ldh, c->partials, plan.slots, plan.slots * 3, 3, Hstep_out, slot_ids,
                                           reset_src, src_m, src_s, src_pooled, st->src_proj, n_src, B_live, st->d,
                                           st->num_slots, 1.f / alpha, st->m, st->s, st->acc, st->proj, z_out, st->d,
-                                          st->head_g, plan.head_cols_pad, head_args(head), yrem_out, status, stream,
+                                          st->head_g, plan.head_cols_pad, 1, 0, head_args(head), yrem_out, status, stream,
                                           /*overlap_previous=*/!c->profiling));
     return EGTP_OK;
   }
@@ -772,7 +809,10 @@ int plp_state_bind_head(plp_state* st, const egtp_head* head) {
   st->ldg_max = (static_cast<int64_t>(head->m_h) + 255) / 256 * 256;   // covers every shape's column granularity
   bool ok = cudaMalloc(reinterpret_cast<void**>(&st->proj), sizeof(float) * static_cast<size_t>(st->num_slots) * head->m_h) == cudaSuccess;
   ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->src_proj), sizeof(float) * static_cast<size_t>(c->max_batch) * head->m_h) == cudaSuccess;
-  ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->head_g), sizeof(float) * static_cast<size_t>(st->g_rows) * st->ldg_max) == cudaSuccess;
+  // room for up to 16 K-split slices (steps whose entropies do not come from an LM-head launch), at most 64 MB
+  const int64_t slice_bytes = static_cast<int64_t>(sizeof(float)) * st->g_rows * st->ldg_max;
+  st->g_max_splits = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(16, (64ll << 20) / slice_bytes)));
+  ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->head_g), static_cast<size_t>(slice_bytes) * st->g_max_splits) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     cudaFree(st->proj); cudaFree(st->src_proj); cudaFree(st->head_g);

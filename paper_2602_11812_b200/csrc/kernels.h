@@ -32,6 +32,7 @@ struct LmheadPlan {
   int slots;          // partial slots per row
   int group_rb;       // row blocks that sweep the vocabulary together (L2 reuse of W tiles)
   int k_blocks;       // ceil(d * elem / 128)
+  int k_splits;       // > 1: K is split over that many units per (row block, chunk); head projection launches only
   int smem_bytes;     // dynamic shared memory
   int64_t rows_pad;   // row_blocks * rows_per_block: rows of the partial buffer
 };
@@ -42,6 +43,10 @@ struct LmheadPlan {
 // extra columns whose raw products the kernel writes out (bf16, one-CTA shapes only).
 LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity,
                             int mode, int head_cols = 0);
+
+// Launch shape for W1 hidden[i] alone (no vocabulary): the head columns of the prompt shape with K split over
+// up to max_splits units, each writing its own slice head_g[split][rows_pad][head_cols_pad].
+LmheadPlan make_headproj_plan(int64_t T, int d, int m_h, int elem_bytes, int num_sms, int max_splits);
 
 // Opts the kernels into their dynamic shared-memory size on the current device (once per device).
 cudaError_t lmhead_prepare_device();
@@ -136,7 +141,7 @@ cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, c
 
 // The update for a state bound to a head (bf16 hidden states and head weights): also advances the slot's
 // projection st_proj = W1 acc with g = W1 h' from the LM-head kernel and finishes the head for the row.
-// src_proj [n_src][m_h] = W1 src_pooled; z may be NULL.  overlap_previous: launch with programmatic stream
+// src_proj [n_src][m_h] = W1 src_pooled; z may be NULL; g is the sum of g_splits slices g_split_stride floats apart.  overlap_previous: launch with programmatic stream
 // serialization, so that blocks are staged (and read their state rows) while the LM-head kernel before it in the
 // stream is still running; the kernel waits for that kernel's end before it reads its results.
 cudaError_t launch_plp_update_bound(const void* hidden_step, int64_t ldh, const float* partials, int slots,
@@ -144,8 +149,8 @@ cudaError_t launch_plp_update_bound(const void* hidden_step, int64_t ldh, const 
                                     const int32_t* reset_src, const float* src_m, const float* src_s,
                                     const float* src_pooled, const float* src_proj, int n_src, int rows, int d,
                                     int num_slots, float inv_alpha, float* st_m, float* st_s, float* st_acc,
-                                    float* st_proj, float* z, int64_t ldz, const float* g, int64_t ldg,
-                                    const HeadArgs& h, float* y, int32_t* status, cudaStream_t stream,
-                                    bool overlap_previous);
+                                    float* st_proj, float* z, int64_t ldz, const float* g, int64_t ldg, int g_splits,
+                                    int64_t g_split_stride, const HeadArgs& h, float* y, int32_t* status,
+                                    cudaStream_t stream, bool overlap_previous);
 
 }  // namespace egtp

@@ -42,6 +42,8 @@ struct UnitCoord {
   int chunk;
   int col_begin;
   int col_end;
+  int kb_begin, kb_end;   // k blocks of this unit (all of them unless the launch splits K)
+  int k_split;
 };
 
 struct KParams {
@@ -55,15 +57,30 @@ struct KParams {
   // head columns appended to the vocabulary (fused form only): column v_pad + j is row j of the head's W1
   int v_pad;          // first head column: V rounded up to col_gran
   int ldg;            // floats per row of head_g (head columns rounded up to col_gran)
-  float* head_g;      // [rows_pad][ldg]: head_g[i][j] = W1[j] . hidden[i]
+  float* head_g;      // [k_splits][rows_pad][ldg]: sum over splits of head_g[s][i][j] = W1[j] . hidden[i]
+  // K split (one-CTA kernel with head columns only; 1 = none): unit u covers k blocks
+  // [(u % k_splits) * kb_per_split, ...) of the unit u / k_splits and writes its own slice of head_g
+  int k_splits, kb_per_split;
+  int64_t g_split_stride;
 };
 
-__device__ __forceinline__ UnitCoord unit_coord(int u, const KParams& p) {
+__device__ __forceinline__ UnitCoord unit_coord(int u_in, const KParams& p) {
+  UnitCoord c;
+  int u = u_in;
+  if (p.k_splits > 1) {
+    u = u_in / p.k_splits;
+    c.k_split = u_in - u * p.k_splits;
+    c.kb_begin = c.k_split * p.kb_per_split;
+    c.kb_end = min(p.k_blocks, c.kb_begin + p.kb_per_split);
+  } else {
+    c.k_split = 0;
+    c.kb_begin = 0;
+    c.kb_end = p.k_blocks;
+  }
   const int per_group = p.group_rb * p.chunks;
   const int g = u / per_group;
   const int r = u - g * per_group;
   const int gm = min(p.group_rb, p.row_blocks - g * p.group_rb);
-  UnitCoord c;
   c.chunk = r / gm;
   c.row_block = g * p.group_rb + (r - c.chunk * gm);
   c.col_begin = static_cast<int>((static_cast<int64_t>(c.chunk) * p.n_groups) / p.chunks) * p.col_gran;
@@ -122,10 +139,10 @@ struct RowState {
 // W1 (Sec. 3.2) and are written to p.head_g as they are; columns between V and v_pad are padding.
 template <bool kFuse>
 __device__ __forceinline__ void consume_piece(RowState& st, const uint32_t (&buf)[32], int c0, int produced,
-                                              const KParams& p, int64_t row) {
+                                              const KParams& p, int64_t row, int k_split = 0) {
   if constexpr (kFuse) {
     if (c0 >= p.v_pad) {
-      float4* dst = reinterpret_cast<float4*>(p.head_g + row * p.ldg + (c0 - p.v_pad));
+      float4* dst = reinterpret_cast<float4*>(p.head_g + k_split * p.g_split_stride + row * p.ldg + (c0 - p.v_pad));
 #pragma unroll
       for (int q = 0; q < 8; ++q)
         dst[q] = make_float4(__uint_as_float(buf[4 * q]), __uint_as_float(buf[4 * q + 1]),
@@ -242,7 +259,7 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
           // kSource 0: whole tile of W, 1: whole tile of W1, 2: boxes
           auto stream_tile = [&](auto source) {
             constexpr int kSource = decltype(source)::value;
-            for (int kb = 0; kb < p.k_blocks; ++kb) {
+            for (int kb = uc.kb_begin; kb < uc.kb_end; ++kb) {
               if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
               const uint32_t a_dst = smem_base + stage * kStageBytes;
               const uint32_t b_dst = a_dst + kABytes;
@@ -286,7 +303,7 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
           if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
           tc_fence_after_sync();
           const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kAccCols);
-          for (int kb = 0; kb < p.k_blocks; ++kb) {
+          for (int kb = uc.kb_begin; kb < uc.kb_end; ++kb) {
             if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t a_src = smem_base + stage * kStageBytes;
@@ -297,7 +314,8 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 #pragma unroll
               for (int k = 0; k < kMmaPerStage; ++k) {
                 // advancing K by 32 bytes inside the swizzled row = +2 in the (address >> 4) field
-                umma_ss<kTf32>(d_tmem + mt * kBN, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                umma_ss<kTf32>(d_tmem + mt * kBN, a_desc + 2u * k, b_desc + 2u * k, idesc,
+                               (kb != uc.kb_begin || k != 0) ? 1u : 0u);
               }
             }
             umma_commit(empty_bar(stage));          // stage reusable once these MMAs have read it
@@ -344,7 +362,7 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         };
         // piece pc = 32 accumulator columns starting at vocabulary / head column c_base + 32 pc
         auto consume = [&](const uint32_t (&buf)[32], int pc) {
-          consume_piece<kFuse>(st, buf, c_base + pc * 32, cols_valid - pc * 32, p, row);
+          consume_piece<kFuse>(st, buf, c_base + pc * 32, cols_valid - pc * 32, p, row, uc.k_split);
         };
         uint32_t bufA[32], bufB[32];
         if (npieces == 0) {
@@ -368,7 +386,7 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         }
         if (++acc == kNumAcc) { acc = 0; acc_phase ^= 1u; }
       }
-      if (ok) {
+      if (ok && p.partials != nullptr) {     // no partials: a launch that only projects onto head columns
         const int slot = (kMT == 1) ? uc.chunk * kEpiSplit + half : uc.chunk;
         float* dst = p.partials + (row * p.slots + slot) * 3;
         dst[0] = st.m;
@@ -811,6 +829,37 @@ LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms
   return pl;
 }
 
+LmheadPlan make_headproj_plan(int64_t T, int d, int m_h, int elem_bytes, int num_sms, int max_splits) {
+  // The prompt shape (128-row blocks, 256-column tiles) over the head columns alone, K split so that the grid
+  // fills the GPU while every split still streams several k blocks.
+  LmheadPlan pl{};
+  const Shape& sh = kShapePrompt;
+  pl.variant = 0;
+  pl.rows_per_block = kTileM;
+  pl.a_box_rows = kTileM;
+  pl.tile_cols = sh.bn;
+  pl.b_box_rows = sh.bbox;
+  pl.col_gran = sh.col_gran;
+  pl.row_blocks = static_cast<int>((T + kTileM - 1) / kTileM);
+  pl.v_pad = 0;
+  pl.head_cols_pad = (m_h + sh.col_gran - 1) / sh.col_gran * sh.col_gran;
+  pl.n_groups = pl.head_cols_pad / sh.col_gran;
+  pl.rows_pad = static_cast<int64_t>(pl.row_blocks) * kTileM;
+  pl.k_blocks = static_cast<int>((static_cast<int64_t>(d) * elem_bytes + kRowBytes - 1) / kRowBytes);
+  pl.smem_bytes = smem_bytes_for(sh.mt, sh.bn, sh.stages);
+  pl.chunks = pl.n_groups;           // one 256-column tile per unit
+  pl.slots = pl.chunks * kEpiSplit;  // unused: no entropy partials are written
+  pl.group_rb = pl.row_blocks;
+  const int base_units = pl.row_blocks * pl.chunks;
+  int splits = std::max(1, num_sms / std::max(1, base_units));
+  splits = std::min(splits, std::max(1, pl.k_blocks / 4));
+  splits = std::max(1, std::min(splits, max_splits));
+  const int kb_per = (pl.k_blocks + splits - 1) / splits;
+  pl.k_splits = (pl.k_blocks + kb_per - 1) / kb_per;      // every split owns at least one k block
+  pl.grid = std::min(num_sms, base_units * pl.k_splits);
+  return pl;
+}
+
 cudaError_t lmhead_prepare_device() {
   cudaError_t e;
   if ((e = prepare_shape<false, EGTP_SHAPE_PROMPT>()) != cudaSuccess) return e;
@@ -843,7 +892,10 @@ cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const Lmhea
   p.k_blocks = plan.k_blocks;
   p.n_groups = plan.n_groups;
   p.col_gran = plan.col_gran;
-  p.total_units = plan.row_blocks * plan.chunks;
+  p.k_splits = std::max(1, plan.k_splits);
+  p.kb_per_split = (plan.k_blocks + p.k_splits - 1) / p.k_splits;
+  p.g_split_stride = plan.rows_pad * static_cast<int64_t>(plan.head_cols_pad);
+  p.total_units = plan.row_blocks * plan.chunks * p.k_splits;
   p.V = V;
   p.slots = plan.slots;
   p.partials = partials;
@@ -852,6 +904,7 @@ cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const Lmhea
   p.ldg = plan.head_cols_pad;
   p.head_g = head_g;
   if (maps.hidden == nullptr || maps.w == nullptr || (plan.variant < 4 && maps.w_tile == nullptr)) return cudaErrorInvalidValue;
+  if (p.k_splits > 1 && (plan.head_cols_pad == 0 || plan.variant != 0)) return cudaErrorInvalidValue;
   if (plan.head_cols_pad > 0) {
     // fused head columns: bf16, one CTA per SM only
     if (tf32 || maps.w1 == nullptr || (plan.variant < 4 && maps.w1_tile == nullptr) || head_g == nullptr) return cudaErrorInvalidValue;

@@ -121,7 +121,8 @@ plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* _
 // The same update for a state that is bound to a prediction head (Sec. 3.2-3.3).  Layer 1 of the head is linear
 // before its ReLU, W1 z = (W1 acc) / s, so next to acc the slot keeps P = W1 acc [m_h] and advances it with the
 // same recurrence, P' = P e^(m-m') + e^(H'/alpha-m') (W1 h'), where g = W1 h' was produced by the LM-head kernel
-// as extra output columns.  The block then finishes the head for its row: u = ReLU(P'/s' + b1), o = W2 u + b2,
+// as extra output columns (or by a launch of that kernel over the head columns alone, K split over g_splits
+// slices that are added here in order).  The block then finishes the head for its row: u = ReLU(P'/s' + b1), o = W2 u + b2,
 // output mode (Eq. 6).  A row that restarts from EGTP row r takes P from src_proj[r] = W1 src_pooled[r].
 // z is written only when the caller asked for it.
 template <typename T, typename TW>
@@ -133,7 +134,8 @@ plp_update_bound_kernel(const T* __restrict__ hidden_step, int64_t ldh, const fl
                         const float* __restrict__ src_pooled, const float* __restrict__ src_proj, int n_src, int d,
                         int num_slots, float inv_alpha, float* __restrict__ st_m, float* __restrict__ st_s,
                         float* __restrict__ st_acc, float* __restrict__ st_proj, float* __restrict__ z, int64_t ldz,
-                        const float* __restrict__ g, int64_t ldg, int m_h, int d_out, const float* __restrict__ b1,
+                        const float* __restrict__ g, int64_t ldg, int g_splits, int64_t g_split_stride, int m_h,
+                        int d_out, const float* __restrict__ b1,
                         const TW* __restrict__ W2, const float* __restrict__ b2, const float* __restrict__ centres,
                         int mode, float* __restrict__ y, int32_t* status) {
   // Launched with programmatic stream serialization: this block may start while the LM-head kernel is still
@@ -191,7 +193,9 @@ plp_update_bound_kernel(const T* __restrict__ hidden_step, int64_t ldh, const fl
   const float* grow = g + static_cast<int64_t>(i) * ldg;
   float* proj_dst = st_proj + static_cast<int64_t>(slot) * m_h;
   for (int j = threadIdx.x; j < m_h; j += blockDim.x) {
-    const float pj = (proj_src != nullptr) ? fmaf(proj_src[j], acc_factor, e * grow[j]) : e * grow[j];
+    float gj = grow[j];
+    for (int sp = 1; sp < g_splits; ++sp) gj += grow[sp * g_split_stride + j];   // K splits, added in order
+    const float pj = (proj_src != nullptr) ? fmaf(proj_src[j], acc_factor, e * gj) : e * gj;
     u[j] = fmaxf(0.f, fmaf(pj, inv_s, b1[j]));
     proj_dst[j] = pj;      // element j is read and written by this thread only
   }
@@ -229,8 +233,9 @@ cudaError_t launch_plp_update_bound(const void* hidden_step, int64_t ldh, const 
                                     const int32_t* reset_src, const float* src_m, const float* src_s,
                                     const float* src_pooled, const float* src_proj, int n_src, int rows, int d,
                                     int num_slots, float inv_alpha, float* st_m, float* st_s, float* st_acc,
-                                    float* st_proj, float* z, int64_t ldz, const float* g, int64_t ldg,
-                                    const HeadArgs& h, float* y, int32_t* status, cudaStream_t stream, bool overlap_previous) {
+                                    float* st_proj, float* z, int64_t ldz, const float* g, int64_t ldg, int g_splits,
+                                    int64_t g_split_stride, const HeadArgs& h, float* y, int32_t* status,
+                                    cudaStream_t stream, bool overlap_previous) {
   const int threads = std::min(kPlpMaxThreads, std::max(64, (d / 8 + 31) / 32 * 32));
   const size_t smem = static_cast<size_t>(h.m_h + h.d_out) * sizeof(float);
   cudaLaunchConfig_t cfg{};
@@ -247,7 +252,8 @@ cudaError_t launch_plp_update_bound(const void* hidden_step, int64_t ldh, const 
   const __nv_bfloat16* W2 = static_cast<const __nv_bfloat16*>(h.W2);
   return cudaLaunchKernelEx(&cfg, plp_update_bound_kernel<__nv_bfloat16, __nv_bfloat16>, hs, ldh, partials, slots,
                             row_stride, slot_stride, Hstep_out, slot_ids, reset_src, src_m, src_s, src_pooled, src_proj,
-                            n_src, d, num_slots, inv_alpha, st_m, st_s, st_acc, st_proj, z, ldz, g, ldg, h.m_h, h.d_out,
+                            n_src, d, num_slots, inv_alpha, st_m, st_s, st_acc, st_proj, z, ldz, g, ldg, g_splits, g_split_stride,
+                            h.m_h, h.d_out,
                             h.b1, W2, h.b2, h.centres, h.mode, y, status);
 }
 

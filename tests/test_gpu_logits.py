@@ -55,8 +55,11 @@ def test_entropy_from_logits_closed_forms(ctx):
                                          check=False) == egtp.EGTP_ERR_CAPACITY
 
 
-def test_plp_step_from_logits_matches_oracle_and_plp_step(ctx):
-    wl = gen.config_plp_decode(slots=130, steps=5, d=256, V=9000, m_h=64, mu=1.0, sigma=0.6)
+@pytest.mark.parametrize("bind,slots,m_h", [(False, 130, 64), (True, 130, 64), (True, 300, 264)])
+def test_plp_step_from_logits_matches_oracle_and_plp_step(ctx, bind, slots, m_h):
+    # bind: the state is bound to its head, so W1 h' comes from a launch of the LM-head kernel over the head columns
+    # alone (K split over the SMs; 264 hidden units = two column tiles) and one kernel finishes the step
+    wl = gen.config_plp_decode(slots=slots, steps=5, d=256, V=9000, m_h=m_h, mu=1.0, sigma=0.6)
     steps, slots, d = wl.steps, wl.slots, wl.d
     W = gu.dev_tensor(wl.W, "bf16")
     head = gu.DeviceHead(wl.head, "bf16")
@@ -65,11 +68,14 @@ def test_plp_step_from_logits_matches_oracle_and_plp_step(ctx):
     lm = egtp.make_lm_head(W)
     st_a = egtp.plp_state_create(ctx, slots, d)
     st_b = egtp.plp_state_create(ctx, slots, d)
+    if bind:
+        egtp.plp_state_bind_head(st_a, head.c)
     f = dict(device="cuda", dtype=torch.float32)
     Ha, za, ya = torch.zeros(steps, slots, **f), torch.zeros(steps, slots, d, **f), torch.zeros(steps, slots, **f)
     Hb, zb, yb = torch.zeros(steps, slots, **f), torch.zeros(steps, slots, d, **f), torch.zeros(steps, slots, **f)
     status = torch.zeros(1, device="cuda", dtype=torch.int32)
     logits_all = []
+    n0 = egtp.egtp_launch_count(ctx)
     for t in range(steps):
         logits = (hs[t].float() @ W.float().T).to(torch.bfloat16)       # what a serving engine would hold
         logits_all.append(logits.float().cpu().numpy())
@@ -79,9 +85,12 @@ def test_plp_step_from_logits_matches_oracle_and_plp_step(ctx):
                       status_dev=status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
+    # per step: entropy from logits + update + head layer 1 + head output, and the 4 kernels of plp_step; bound:
+    # entropy from logits + projection + fused update (and 2 launches once for the projection of the empty state)
+    assert egtp.egtp_launch_count(ctx) - n0 == ((3 + 4) * steps + 2 if bind else (4 + 4) * steps)
     # oracle on exactly the logits the kernel read (bf16-rounded), followed through the token lists
     H_ref = np.stack([orc.entropy_from_logits(x.astype(np.float64)) for x in logits_all])
-    follow = [0, 64, 129]
+    follow = [0, 64, slots - 1]
     ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=follow, H_steps=H_ref[:, follow])
     Ha_n, za_n, ya_n = (a.cpu().numpy().astype(np.float64) for a in (Ha, za, ya))
     gu.assert_entropy_close(Ha_n.ravel(), H_ref.ravel())

@@ -56,7 +56,10 @@ def test_sharded_entropy_matches_oracle_and_single_gpu(ctx, world, rows):
     assert np.abs(H - gu.run_egtp(ctx, wl)["H"]).max() < 2e-5
 
 
-def test_plp_step_from_partials_matches_plp_step(ctx):
+@pytest.mark.parametrize("bind", [False, True])
+def test_plp_step_from_partials_matches_plp_step(ctx, bind):
+    # bind: both states are bound to the head (the sharded one gets W1 h' from a projection launch, the other from
+    # the LM-head kernel's extra columns)
     wl = gen.config_plp_decode(slots=140, steps=4, d=256, V=9000, m_h=64, mu=1.0, sigma=0.6)
     steps, slots, d = wl.steps, wl.slots, wl.d
     Wd = gu.dev_tensor(wl.W, "bf16")
@@ -64,6 +67,9 @@ def test_plp_step_from_partials_matches_plp_step(ctx):
     hs = gu.dev_tensor(wl.hidden_steps.reshape(-1, d), "bf16").reshape(steps, slots, d)
     reset = torch.from_numpy(wl.reset_src).cuda()
     st_a, st_b = egtp.plp_state_create(ctx, slots, d), egtp.plp_state_create(ctx, slots, d)
+    if bind:
+        egtp.plp_state_bind_head(st_a, head.c)
+        egtp.plp_state_bind_head(st_b, head.c)
     f = dict(device="cuda", dtype=torch.float32)
     ya, yb = torch.zeros(steps, slots, **f), torch.zeros(steps, slots, **f)
     za, zb = torch.zeros(steps, slots, d, **f), torch.zeros(steps, slots, d, **f)
