@@ -324,6 +324,14 @@ EGTP_API int egtp_pool_baseline(egtp_ctx* ctx, const egtp_head* head, const void
 enum { EGTP_LMHEAD_AUTO = 0, EGTP_LMHEAD_CTA_PAIRS = 1, EGTP_LMHEAD_SINGLE_CTA = 2 };
 EGTP_API int egtp_set_lmhead_mode(egtp_ctx* ctx, int mode);
 
+/* Tuning knob for prompt batches (more than 256 rows): the LM-head kernel cuts the vocabulary into `chunks`
+ * ranges and deals (row block, range) units to the SMs round-robin; every range costs one partial (m, s, t2) per
+ * row and column half (Eq. 2 is merged from them).  0 (default) lets the library choose the smallest count whose
+ * rounds x tiles-per-range product is close to the best reachable (within 0.5 % for rows of up to 4 KB, 2 % for
+ * longer rows); a positive value forces that count (clamped to what the workspace holds).  Results do not depend
+ * on it beyond summation order. */
+EGTP_API int egtp_set_lmhead_chunks(egtp_ctx* ctx, int32_t chunks);
+
 /* Failure-detection self-test.  Every wait inside the pipeline kernels (on an mbarrier fed by TMA, by the
  * tensor core or by another warp) is bounded: when its limit runs out the kernel writes
  * EGTP_ERR_DEVICE_TIMEOUT to the status word, releases its tensor memory and returns, so a protocol

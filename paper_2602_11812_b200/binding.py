@@ -38,7 +38,7 @@ EXPORTED_SYMBOLS = [
     "egtp_launch_count", "egtp_lmhead_plan", "egtp_head_forward_static", "egtp_set_lmhead_mode",
     "egtp_entropy_from_logits", "plp_step_from_logits", "egtp_pool_baseline",
     "egtp_entropy_partials", "egtp_entropy_from_partials", "plp_step_from_partials", "egtp_selftest_wait_timeout",
-    "plp_state_bind_head",
+    "plp_state_bind_head", "egtp_set_lmhead_chunks",
 ]
 
 
@@ -86,6 +86,7 @@ def load() -> C.CDLL:
     lib.egtp_lmhead_plan.argtypes = [vp, i64, i32, i32, i32, P(i32)]
     lib.egtp_profile_enable.argtypes = [vp, C.c_int]
     lib.egtp_set_lmhead_mode.argtypes = [vp, C.c_int]
+    lib.egtp_set_lmhead_chunks.argtypes = [vp, i32]
     lib.egtp_selftest_wait_timeout.argtypes = [vp, i32, vp, vp]
     lib.egtp_entropy_partials.argtypes = [vp, P(egtp_lm_head), vp, i64, i64, vp, vp, vp]
     lib.egtp_entropy_from_partials.argtypes = [vp, vp, i32, i64, vp, vp, vp]
@@ -201,6 +202,11 @@ def egtp_lmhead_plan(ctx: int, T: int, d: int, V: int, dtype: int) -> dict:
 
 def egtp_set_lmhead_mode(ctx: int, mode: int):
     _check(load().egtp_set_lmhead_mode(ctx, mode), "egtp_set_lmhead_mode")
+
+
+def egtp_set_lmhead_chunks(ctx: int, chunks: int):
+    """Forces the number of vocabulary chunks of prompt batches (0 = chosen by the library)."""
+    _check(load().egtp_set_lmhead_chunks(ctx, chunks), "egtp_set_lmhead_chunks")
 
 
 def egtp_profile_enable(ctx: int, on: bool):

@@ -51,6 +51,7 @@ struct egtp_ctx {
 
   // bookkeeping
   int lmhead_mode = EGTP_LMHEAD_AUTO;
+  int lmhead_chunks = 0;          // 0 = chosen by the planner
   // host-buffer entry points: copies run on their own stream, one event per piece of the batch
   static constexpr int kMaxPieces = 4;
   cudaStream_t copy_stream = nullptr;
@@ -203,7 +204,7 @@ int run_lmhead(egtp_ctx* c, const egtp_lm_head* lm, const void* hidden, int64_t 
                float* head_g = nullptr) {
   const bool fuse = fuse_W1 != nullptr;
   const LmheadPlan plan = make_lmhead_plan(rows, lm->d, lm->V, elem_bytes(lm->dtype), c->num_sms, c->slot_row_capacity,
-                                           c->lmhead_mode, fuse ? fuse_m_h : 0);
+                                           c->lmhead_mode, fuse ? fuse_m_h : 0, c->lmhead_chunks);
   if (plan.rows_pad * plan.slots > c->slot_row_capacity) return EGTP_ERR_CAPACITY;
   CUtensorMap map_a, map_b, map_b_tile, map_c, map_c_tile;
   LmheadMaps maps;
@@ -492,10 +493,12 @@ int egtp_create(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_batc
 
   const int64_t rows_cap = std::max<int64_t>(max_tokens, max_batch);
   const int64_t rows_pad = (rows_cap + kTileM - 1) / kTileM * kTileM;
-  // room for 24 vocabulary chunks (two partial slots each) at the largest token count, and for one
-  // chunk per SM on decode-sized batches
-  c->slot_row_capacity = std::max<int64_t>(rows_pad * 24 * kEpiSplit,
-                                           static_cast<int64_t>(2 * kTileM) * c->num_sms * kEpiSplit);
+  // room for 24 vocabulary chunks (two partial slots each) at the largest token count, for one chunk per SM
+  // on decode-sized batches, and never less than 2 M slot rows (24 MB): batches of a few dozen row blocks need
+  // 30 to 60 chunks before (row blocks x chunks) fills whole rounds of the SMs
+  c->slot_row_capacity = std::max<int64_t>(
+      std::max<int64_t>(rows_pad * 24 * kEpiSplit, static_cast<int64_t>(2 * kTileM) * c->num_sms * kEpiSplit),
+      int64_t{1} << 21);
   const int64_t pool_chunks = (max_tokens + kPoolChunkTokens - 1) / kPoolChunkTokens + 1;
   c->head_partial_floats = std::max<int64_t>(8ll << 20, static_cast<int64_t>(max_batch) * 8192);
 
@@ -541,7 +544,7 @@ int64_t egtp_launch_count(const egtp_ctx* c) { return c ? c->launches : 0; }
 
 int egtp_lmhead_plan(const egtp_ctx* c, int64_t T, int32_t d, int32_t V, int32_t dtype, int32_t info[8]) {
   if (!c || !info || T <= 0 || d <= 0 || V <= 0) return EGTP_ERR_INVALID_ARG;
-  const LmheadPlan p = make_lmhead_plan(T, d, V, elem_bytes(dtype), c->num_sms, c->slot_row_capacity, c->lmhead_mode);
+  const LmheadPlan p = make_lmhead_plan(T, d, V, elem_bytes(dtype), c->num_sms, c->slot_row_capacity, c->lmhead_mode, 0, c->lmhead_chunks);
   info[0] = p.grid; info[1] = p.row_blocks; info[2] = p.rows_per_block; info[3] = p.chunks;
   info[4] = p.slots; info[5] = p.tile_cols; info[6] = p.k_blocks; info[7] = p.smem_bytes;
   return EGTP_OK;
@@ -551,6 +554,12 @@ int egtp_set_lmhead_mode(egtp_ctx* c, int mode) {
   if (!c || (mode != EGTP_LMHEAD_AUTO && mode != EGTP_LMHEAD_CTA_PAIRS && mode != EGTP_LMHEAD_SINGLE_CTA))
     return EGTP_ERR_INVALID_ARG;
   c->lmhead_mode = mode;
+  return EGTP_OK;
+}
+
+int egtp_set_lmhead_chunks(egtp_ctx* c, int32_t chunks) {
+  if (!c || chunks < 0) return EGTP_ERR_INVALID_ARG;
+  c->lmhead_chunks = chunks;
   return EGTP_OK;
 }
 

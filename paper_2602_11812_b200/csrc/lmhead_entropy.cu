@@ -758,7 +758,7 @@ static_assert(kShapeDecode2.mt == 2 && kShapeDecode2.bn == 256 && kShapeDecode2.
 }  // namespace
 
 LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity,
-                            int mode, int head_cols) {
+                            int mode, int head_cols, int force_chunks) {
   LmheadPlan pl{};
   // decode batches of 129..256 rows run as CTA pairs on 256 x 512 tiles unless single CTAs are asked for or the
   // device cannot co-schedule the pairs; prompt batches run as pairs only on request (and never with head columns)
@@ -794,20 +794,28 @@ LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms
   if (!one_block) {
     workers = static_cast<int>(std::min<int64_t>(workers_max, static_cast<int64_t>(pl.row_blocks) * pl.n_groups));
     // Units are dealt round-robin to the workers, so the step takes ceil(units / workers) rounds of
-    // ceil(n_tiles / S) tiles.  Take the smallest S whose makespan is within 2 % of the best
-    // reachable one (fewer chunks = fewer partials to write and merge).
+    // ceil(n_tiles / S) tiles.  Take the smallest S whose makespan is close to the best reachable one (fewer
+    // chunks = fewer partials to write and merge).  How close, measured with interleaved runs on B200:
+    // rows of up to 4 KB sweep the vocabulary as one group, W tiles are shared by all row blocks whatever S is,
+    // and the product alone decides (T = 9555, d = 2048: S = 33 at 4.22 ms against 4.31 ms with S = 17), so 0.5 %;
+    // with longer rows only a few row blocks sweep together and every extra chunk leaves fewer groups in step on
+    // the same W tiles (T = 25629, d = 4096: S = 8 at 23.7 ms, S = 11 at 24.3 ms, S = 22 at 25.7 ms although
+    // the product falls), so 2 %.
     auto makespan = [&](int S) {
       const int64_t units = static_cast<int64_t>(pl.row_blocks) * S;
       const int64_t rounds = (units + workers - 1) / workers;
       return rounds * ((pl.n_groups + S - 1) / S);
     };
+    const bool one_group = static_cast<int64_t>(d) * elem_bytes <= 4096;
+    const int64_t tol_num = one_group ? 201 : 102, tol_den = one_group ? 200 : 100;
+    const int s_lim = std::min(s_max, 64);     // more chunks only add partials to write and merge
     int64_t best = makespan(1);
-    for (int S = 2; S <= s_max; ++S) best = std::min(best, makespan(S));
+    for (int S = 2; S <= s_lim; ++S) best = std::min(best, makespan(S));
     int pick = 1;
-    for (int S = 1; S <= s_max; ++S) {
-      if (makespan(S) * 100 <= best * 102) { pick = S; break; }
+    for (int S = 1; S <= s_lim; ++S) {
+      if (makespan(S) * tol_den <= best * tol_num) { pick = S; break; }
     }
-    pl.chunks = pick;
+    pl.chunks = force_chunks > 0 ? std::min(force_chunks, s_max) : pick;
   } else {
     // One row block: one vocabulary range per worker, ranges differ by at most col_gran columns.
     pl.chunks = std::max(1, std::min(s_max, workers_max));

@@ -102,6 +102,20 @@ def test_mid_config_scaled(ctx):
     res = gu.run_egtp(ctx, wl)
     _check_all(res, ref, wl)
     assert ref["H"].std() > 0.05                                        # weights are genuinely non-uniform
+    # the number of vocabulary chunks is a tuning knob: one chunk, an odd count and more chunks than tiles (clamped)
+    # give the same result up to summation order
+    T, planned = wl.T, egtp.egtp_lmhead_plan(ctx, wl.T, wl.d, wl.V, egtp.EGTP_BF16)["chunks"]
+    try:
+        for chunks in (1, 7, 500):
+            egtp.egtp_set_lmhead_chunks(ctx, chunks)
+            got = egtp.egtp_lmhead_plan(ctx, T, wl.d, wl.V, egtp.EGTP_BF16)["chunks"]
+            assert got == min(chunks, got) and (chunks > 79 or got == chunks)      # 20072 columns = 79 tiles
+            res_c = gu.run_egtp(ctx, wl)
+            _check_all(res_c, ref, wl)
+            assert np.abs(res_c["H"] - res["H"]).max() < 1e-4
+    finally:
+        egtp.egtp_set_lmhead_chunks(ctx, 0)
+    assert egtp.egtp_lmhead_plan(ctx, T, wl.d, wl.V, egtp.EGTP_BF16)["chunks"] == planned
 
 
 def test_segment_edge_cases(ctx):
