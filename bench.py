@@ -415,6 +415,27 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     plp.update(measure_steps(st))
     plp["plan"] = egtp.egtp_lmhead_plan(ctx, slots, d, V, egtp.EGTP_BF16)
     plp["unbound_state"] = plain
+    # ---- the same bound step end to end: the step's hidden rows come from pinned host memory, the predictions go back
+    try:
+        n_e2e = min(plp_steps, 32)
+        hs_host = [gu.host_tensor(wl.hidden_steps[warm + t], "bf16") for t in range(n_e2e)]
+        rs_host = [torch.from_numpy(wl.reset_src[warm + t].copy()).pin_memory() for t in range(n_e2e)]
+        y_host = torch.empty(slots, dtype=torch.float32).pin_memory()
+        st_host = torch.zeros(1, dtype=torch.int32).pin_memory()
+        egtp.egtp_profile_enable(ctx, False)
+        for t in range(3):
+            egtp.plp_step_host(ctx, st, lm, head.c, hs_host[t], rs_host[t], None, None, None, 0, slots, 1.0, y_host, st_host)
+        t0 = time.perf_counter()
+        for t in range(n_e2e):
+            egtp.plp_step_host(ctx, st, lm, head.c, hs_host[t], rs_host[t], None, None, None, 0, slots, 1.0, y_host, st_host)
+        t1 = time.perf_counter()          # plp_step_host synchronises its stream before it returns
+        assert int(st_host.item()) == 0
+        plp["e2e"] = dict(us_per_step=(t1 - t0) / n_e2e * 1e6, steps=n_e2e, api="plp_step_host",
+                          h2d_bytes_per_step=slots * d * 2 + slots * 4, d2h_bytes_per_step=slots * 4 + 4)
+        egtp.egtp_profile_enable(ctx, True)
+    except Exception as exc:
+        plp["e2e"] = dict(error=str(exc)[:200])
+
     # ---- context only: a library GEMM of the decode shape (writes the [256, V] logits, no entropy)
     try:
         lg = torch.empty(slots, V, device="cuda", dtype=torch.bfloat16)
