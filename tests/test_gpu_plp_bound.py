@@ -155,3 +155,39 @@ def test_bind_rejects_fp32_heads(ctx):
     head32 = gu.DeviceHead(gen.make_head(5, 128, 32, 1, "f32"), "f32")
     assert egtp.plp_state_bind_head(st, head32.c, check=False) == egtp.EGTP_ERR_UNSUPPORTED
     egtp.plp_state_destroy(st)
+
+
+def test_bound_step_replayed_from_a_cuda_graph_equals_eager_steps(ctx):
+    # the decode step is two launches (the second one with programmatic stream serialization); captured once and
+    # replayed with new tokens copied into fixed buffers it must give bit for bit what eager calls give
+    wl = gen.config_plp_decode(slots=150, steps=7, d=256, V=5000, m_h=64, mu=3.0, sigma=0.3)
+    W = gu.dev_tensor(wl.W, "bf16"); lm = egtp.make_lm_head(W)
+    head = gu.DeviceHead(wl.head, "bf16")
+    hs = gu.dev_tensor(wl.hidden_steps.reshape(-1, 256), "bf16").reshape(wl.steps, 150, 256)
+    reset = torch.from_numpy(wl.reset_src).cuda()
+    st_e, st_g = egtp.plp_state_create(ctx, 150, 256), egtp.plp_state_create(ctx, 150, 256)
+    egtp.plp_state_bind_head(st_e, head.c); egtp.plp_state_bind_head(st_g, head.c)
+    y_e = torch.zeros(wl.steps, 150, device="cuda"); y_g = torch.zeros(wl.steps, 150, device="cuda")
+    status = torch.zeros(1, device="cuda", dtype=torch.int32)
+    for t in range(wl.steps):
+        egtp.plp_step(ctx, st_e, lm, head.c, hs[t], reset_src=reset[t], yrem_out=y_e[t], status_dev=status)
+    # step 0 eagerly (it also projects the empty state, which is not part of the steady-state graph)
+    h_buf, r_buf, y_buf = hs[0].clone(), reset[0].clone(), torch.zeros(150, device="cuda")
+    egtp.plp_step(ctx, st_g, lm, head.c, h_buf, reset_src=r_buf, yrem_out=y_buf, status_dev=status)
+    y_g[0].copy_(y_buf)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        egtp.plp_step(ctx, st_g, lm, head.c, h_buf, reset_src=r_buf, yrem_out=y_buf, status_dev=status,
+                      stream=torch.cuda.current_stream().cuda_stream)
+    for t in range(1, wl.steps):
+        h_buf.copy_(hs[t]); r_buf.copy_(reset[t])
+        graph.replay()
+        y_g[t].copy_(y_buf)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(y_e, y_g)
+    ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=[0, 149])
+    gu.assert_length_close(y_g.cpu().numpy().astype(np.float64)[:, [0, 149]].ravel(), ref["yrem"].ravel())
+    egtp.plp_state_destroy(st_e); egtp.plp_state_destroy(st_g)
