@@ -201,8 +201,8 @@ EGTP_API int plp_step(egtp_ctx* ctx, plp_state* st, const egtp_lm_head* lm, cons
  * result equals the unbound plp_step up to floating-point summation order.
  *   head   host struct with device pointers; wdtype must be EGTP_BF16 (EGTP_ERR_UNSUPPORTED otherwise).  The
  *          struct is copied; the weights it points at must stay in place and unchanged while bound.
- * Allocates num_slots * m_h + max_batch * m_h + (padded rows) * (padded m_h) floats and synchronises the device
- * (a create-time call, not for the decode loop).  Binding again replaces the previous binding.
+ * Allocates num_slots * m_h + max_batch * m_h floats and up to 16 slices (64 MB at most) of (padded rows) x (padded
+ * m_h) floats, and synchronises the device (a create-time call, not for the decode loop).  Binding again replaces the previous binding.
  * plp_step, plp_step_from_logits and plp_step_from_partials take the bound route when they are given the same
  * head (same W1 pointer, m_h, d, dtype) with yrem_out != NULL, bf16 hidden states (and LM head), and n_src <= the
  * context's max_batch; the two that run no LM-head GEMM get W1 h' from a launch of the LM-head kernel over the
