@@ -191,3 +191,19 @@ def test_bound_step_replayed_from_a_cuda_graph_equals_eager_steps(ctx):
     ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=[0, 149])
     gu.assert_length_close(y_g.cpu().numpy().astype(np.float64)[:, [0, 149]].ravel(), ref["yrem"].ravel())
     egtp.plp_state_destroy(st_e); egtp.plp_state_destroy(st_g)
+
+
+def test_bound_projection_does_not_drift_over_a_long_sequence(ctx):
+    # 400 steps without a restart: P = W1 acc is advanced incrementally all the way; the oracle recomputes the pool
+    # and the head from the whole token list at every step
+    wl = gen.config_plp_decode(slots=8, steps=400, d=128, V=2000, m_h=48, mu=12.0, sigma=0.1)
+    assert (wl.reset_src[1:] == gen.RESET_KEEP).all()
+    st, H, z, y, _ = _run(ctx, wl)
+    follow = [0, 7]
+    ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=follow)
+    err = np.abs(y[:, follow] - ref["yrem"])
+    assert err.max() <= 1e-3 * max(1.0, np.abs(ref["yrem"]).max()), err.max()
+    assert err[-50:].max() <= 2.0 * max(err[:50].max(), 1e-5) + 1e-4       # no growth along the sequence
+    for t in (0, 199, 399):
+        gu.assert_pooled_close(z[t, follow], ref["z"][t])
+    egtp.plp_state_destroy(st)
