@@ -57,6 +57,7 @@ struct egtp_ctx {
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t piece_ready[kMaxPieces] = {};
   cudaEvent_t stage_free = nullptr;
+  cudaEvent_t fork_ev = nullptr, join_ev = nullptr;   // side work that runs next to the main stream inside one call
   int64_t launches = 0;
   bool profiling = false;
   std::vector<EventPair> pending;
@@ -103,6 +104,8 @@ void free_ctx_memory(egtp_ctx* c) {
   if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   for (auto& e : c->piece_ready) if (e) cudaEventDestroy(e);
   if (c->stage_free) cudaEventDestroy(c->stage_free);
+  if (c->fork_ev) cudaEventDestroy(c->fork_ev);
+  if (c->join_ev) cudaEventDestroy(c->join_ev);
   for (auto& e : c->pending) { cudaEventDestroy(e.start); cudaEventDestroy(e.stop); }
   for (auto& e : c->free_events) { cudaEventDestroy(e.start); cudaEventDestroy(e.stop); }
 }
@@ -314,39 +317,66 @@ bool plp_fused_route(const egtp_ctx* c, const plp_state* st, int hidden_dtype, c
   return rows_pad <= st->g_rows;
 }
 
+// --- steps on a state bound to its head whose entropies do not come from an LM-head launch -----------------------
+bool plp_bound_tail_route(const egtp_ctx* c, const plp_state* st, int hidden_dtype, const egtp_head* head, int B_live,
+                          int n_src, const float* yrem_out, const void* hidden_step, int64_t ldh) {
+  return plp_fused_route(c, st, hidden_dtype, head, B_live, n_src, yrem_out) &&
+         reinterpret_cast<uintptr_t>(hidden_step) % 16 == 0 && (ldh * 2) % 16 == 0;
+}
+
+// P = W1 acc if it is stale, and W1 src_pooled for rows that restart from EGTP rows
+int plp_bound_prepare(egtp_ctx* c, plp_state* st, const egtp_head* head, const int32_t* reset_src,
+                      const float* src_pooled, int n_src, const int32_t* status, cudaStream_t stream) {
+  if (!st->proj_valid) {
+    int rc = project_rows(c, head, st->acc, st->d, st->num_slots, st->proj, head->m_h, status, stream);
+    if (rc != EGTP_OK) return rc;
+    st->proj_valid = true;
+  }
+  if (reset_src && n_src > 0) {
+    int rc = project_rows(c, head, src_pooled, st->d, n_src, st->src_proj, head->m_h, status, stream);
+    if (rc != EGTP_OK) return rc;
+  }
+  return EGTP_OK;
+}
+
+// W1 h' for the step's rows: the LM-head kernel over the head columns alone, K split over the SMs, into the
+// slices of st->head_g.  Independent of the step's entropies, so it may run on another stream next to them.
+int plp_bound_project(egtp_ctx* c, plp_state* st, const egtp_head* head, const void* hidden_step, int64_t ldh,
+                      int B_live, int32_t* status, cudaStream_t stream, LmheadPlan* plan_out) {
+  const LmheadPlan plan = make_headproj_plan(B_live, st->d, head->m_h, 2, c->num_sms, st->g_max_splits);
+  if (plan.rows_pad > st->g_rows || plan.head_cols_pad > st->ldg_max) return EGTP_ERR_CAPACITY;
+  CUtensorMap map_a, map_c;
+  int rc = make_tensor_map(c, &map_a, hidden_step, EGTP_BF16, B_live, st->d, ldh, plan.a_box_rows);
+  if (rc != EGTP_OK) return rc;
+  rc = make_tensor_map(c, &map_c, head->W1, EGTP_BF16, head->m_h, st->d, st->d, plan.b_box_rows);
+  if (rc != EGTP_OK) return rc;
+  LmheadMaps maps;
+  maps.hidden = &map_a;
+  maps.w = maps.w_tile = maps.w1 = maps.w1_tile = &map_c;
+  LaunchScope ls(c, EGTP_K_HEAD_HIDDEN, stream);
+  EGTP_CUDA_TRY(launch_lmhead_entropy(plan, false, maps, B_live, 0, nullptr, status, stream, st->head_g));
+  *plan_out = plan;
+  return EGTP_OK;
+}
+
 // Second half of a PLP step: merge the entropy partials, update the slots (Eq. 8), run the head.
+// projected != NULL: the caller has already taken the bound route's first two steps (plp_bound_prepare,
+// plp_bound_project with this plan) and ordered them before `stream`'s next work.
 int plp_update_and_head(egtp_ctx* c, plp_state* st, const egtp_head* head, const void* hidden_step, int64_t ldh,
                         int hidden_dtype, const float* partials, int slots, int64_t row_stride, int64_t slot_stride,
                         const int32_t* slot_ids, const int32_t* reset_src,
                         const float* src_m, const float* src_s, const float* src_pooled, int n_src, int B_live,
                         float alpha, float* Hstep_out, float* z_out, float* yrem_out, int32_t* status,
-                        cudaStream_t stream) {
-  if (plp_fused_route(c, st, hidden_dtype, head, B_live, n_src, yrem_out) &&
-      reinterpret_cast<uintptr_t>(hidden_step) % 16 == 0 && (ldh * 2) % 16 == 0) {
-    // State bound to this head, entropies from elsewhere (logits in memory, gathered shard partials): W1 h' comes
-    // from a launch of the LM-head kernel over the head columns alone (K split over the SMs), then the bound update.
-    if (!st->proj_valid) {
-      int rc = project_rows(c, head, st->acc, st->d, st->num_slots, st->proj, head->m_h, status, stream);
+                        cudaStream_t stream, const LmheadPlan* projected = nullptr) {
+  if (projected != nullptr || plp_bound_tail_route(c, st, hidden_dtype, head, B_live, n_src, yrem_out, hidden_step, ldh)) {
+    LmheadPlan plan;
+    if (projected != nullptr) {
+      plan = *projected;
+    } else {
+      int rc = plp_bound_prepare(c, st, head, reset_src, src_pooled, n_src, status, stream);
       if (rc != EGTP_OK) return rc;
-      st->proj_valid = true;
-    }
-    if (reset_src && n_src > 0) {
-      int rc = project_rows(c, head, src_pooled, st->d, n_src, st->src_proj, head->m_h, status, stream);
+      rc = plp_bound_project(c, st, head, hidden_step, ldh, B_live, status, stream, &plan);
       if (rc != EGTP_OK) return rc;
-    }
-    const LmheadPlan plan = make_headproj_plan(B_live, st->d, head->m_h, 2, c->num_sms, st->g_max_splits);
-    if (plan.rows_pad > st->g_rows || plan.head_cols_pad > st->ldg_max) return EGTP_ERR_CAPACITY;
-    CUtensorMap map_a, map_c;
-    int rc = make_tensor_map(c, &map_a, hidden_step, EGTP_BF16, B_live, st->d, ldh, plan.a_box_rows);
-    if (rc != EGTP_OK) return rc;
-    rc = make_tensor_map(c, &map_c, head->W1, EGTP_BF16, head->m_h, st->d, st->d, plan.b_box_rows);
-    if (rc != EGTP_OK) return rc;
-    LmheadMaps maps;
-    maps.hidden = &map_a;
-    maps.w = maps.w_tile = maps.w1 = maps.w1_tile = &map_c;
-    {
-      LaunchScope ls(c, EGTP_K_HEAD_HIDDEN, stream);
-      EGTP_CUDA_TRY(launch_lmhead_entropy(plan, false, maps, B_live, 0, nullptr, status, stream, st->head_g));
     }
     LaunchScope ls(c, EGTP_K_PLP_UPDATE, stream);
     EGTP_CUDA_TRY(launch_plp_update_bound(hidden_step, ldh, partials, slots, row_stride, slot_stride, Hstep_out, slot_ids,
@@ -521,6 +551,8 @@ int egtp_create(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_batc
   ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
   for (auto& e : c->piece_ready) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&c->stage_free, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&c->fork_ev, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&c->join_ev, cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     free_ctx_memory(c);
@@ -871,11 +903,27 @@ int plp_step_from_logits(egtp_ctx* c, plp_state* st, const void* logits, int64_t
   if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
   int32_t* status = status_dev ? status_dev : c->status;
   if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
+  // State bound to this head: W1 h' does not depend on the logits, so its launch goes to the context's side stream
+  // and runs next to the pass over the logits; the update waits for both.
+  LmheadPlan proj_plan;
+  const bool bound = plp_bound_tail_route(c, st, hidden_dtype, head, B_live, n_src, yrem_out, hidden_step, ldh);
+  if (bound) {
+    rc = plp_bound_prepare(c, st, head, reset_src, src_pooled, n_src, status, stream);
+    if (rc != EGTP_OK) return rc;
+    EGTP_CUDA_TRY(cudaEventRecord(c->fork_ev, stream));
+    EGTP_CUDA_TRY(cudaStreamWaitEvent(c->copy_stream, c->fork_ev, 0));
+    rc = plp_bound_project(c, st, head, hidden_step, ldh, B_live, status, c->copy_stream, &proj_plan);
+    if (cudaEventRecord(c->join_ev, c->copy_stream) != cudaSuccess) return EGTP_ERR_CUDA;
+  }
   int slots = 0;
-  rc = run_logits_entropy(c, logits, ldl, logits_dtype, B_live, V, status, stream, &slots);
+  const int rc_entropy = run_logits_entropy(c, logits, ldl, logits_dtype, B_live, V, status, stream, &slots);
+  // the side stream always rejoins, whatever failed (a stream capture in progress must not be left forked)
+  if (bound && cudaStreamWaitEvent(stream, c->join_ev, 0) != cudaSuccess) return EGTP_ERR_CUDA;
   if (rc != EGTP_OK) return rc;
+  if (rc_entropy != EGTP_OK) return rc_entropy;
   return plp_update_and_head(c, st, head, hidden_step, ldh, hidden_dtype, c->partials, slots, slots * 3, 3, slot_ids, reset_src, src_m, src_s,
-                             src_pooled, n_src, B_live, alpha, Hstep_out, z_out, yrem_out, status, stream);
+                             src_pooled, n_src, B_live, alpha, Hstep_out, z_out, yrem_out, status, stream,
+                             bound ? &proj_plan : nullptr);
 }
 
 int egtp_entropy_partials(egtp_ctx* c, const egtp_lm_head* lm_shard, const void* hidden, int64_t ldh, int64_t rows,
