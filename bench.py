@@ -213,9 +213,9 @@ def run_mine(args):
     sync_all()
     assert int(status.item()) == 0, egtp.status_string(int(status.item()))
 
-    # ---- timed region: K steps, device-timed, per-kernel events on the launching stream
-    egtp.egtp_profile_enable(ctx, True)
-    egtp.egtp_profile_read(ctx)
+    # ---- timed region: K steps, device-timed on the launching stream (no per-kernel events in it: they cost a
+    # few microseconds per launch)
+    egtp.egtp_profile_enable(ctx, False)
     launches0 = egtp.egtp_launch_count(ctx)
     sampler = ClockSampler(int(os.environ.get("CUDA_VISIBLE_DEVICES", "0").split(",")[local_rank]) if os.environ.get("CUDA_VISIBLE_DEVICES") else local_rank)
     sampler.start()
@@ -232,6 +232,13 @@ def run_mine(args):
     ms = ev0.elapsed_time(ev1)
     clocks = sampler.stop(t_wall0, t_wall1)
     launches = egtp.egtp_launch_count(ctx) - launches0
+    assert int(status.item()) == 0, egtp.status_string(int(status.item()))
+    # ---- the same K steps once more with every kernel bracketed by events: per-kernel times for the roofline
+    egtp.egtp_profile_enable(ctx, True)
+    egtp.egtp_profile_read(ctx)
+    for _ in range(steps):
+        step()
+    torch.cuda.synchronize()
     prof = egtp.egtp_profile_read(ctx)
     egtp.egtp_profile_enable(ctx, False)
     assert int(status.item()) == 0, egtp.status_string(int(status.item()))
