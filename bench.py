@@ -680,6 +680,20 @@ def bench_rl_group(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     return out
 
 
+def ensure_library():
+    """Builds the CUDA library if it is missing or older than its sources (a no-op otherwise).  Under torchrun
+    only local rank 0 compiles; the other ranks wait for the finished file."""
+    from paper_2602_11812_b200 import build as _build
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        _build.build()
+        return
+    deadline = time.time() + 600
+    while not _build.up_to_date():
+        if time.time() > deadline:
+            raise SystemExit("bench.py: the CUDA library was not built in time")
+        time.sleep(1.0)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -696,6 +710,8 @@ def main():
     ap.add_argument("--only-rl-group", action="store_true",
                     help="run only the RL group-sampling sizes (d = 5120, V = 152064, 1024 streams) and print one JSON line")
     args = ap.parse_args()
+    if args.impl != "reference":
+        ensure_library()
     if args.only_rl_group:
         import torch
         torch.cuda.set_device(0)

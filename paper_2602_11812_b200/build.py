@@ -68,10 +68,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
     with ThreadPoolExecutor(max_workers=6) as ex:
         objs = list(ex.map(compile_one, sources()))
-    cmd = [nvcc, "-shared", "-cudart", "static", "-o", LIB_PATH, *objs]
+    tmp_path = LIB_PATH + f".tmp{os.getpid()}"     # linked aside and renamed: nobody ever sees half a library
+    cmd = [nvcc, "-shared", "-cudart", "static", "-o", tmp_path, *objs]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
+    os.replace(tmp_path, LIB_PATH)
     return LIB_PATH
 
 
