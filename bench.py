@@ -685,7 +685,7 @@ def ensure_library():
     only local rank 0 compiles; the other ranks wait for the finished file."""
     from paper_2602_11812_b200 import build as _build
     if int(os.environ.get("LOCAL_RANK", "0")) == 0:
-        _build.build()
+        _build.ensure()
         return
     deadline = time.time() + 600
     while not _build.up_to_date():

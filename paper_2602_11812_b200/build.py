@@ -77,5 +77,17 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB_PATH
 
 
+def ensure() -> str:
+    """build() for callers that only want a usable library: when compiling is impossible here (no nvcc) but a
+    library file exists, that file is used as it is; every other failure is raised."""
+    try:
+        return build()
+    except RuntimeError as exc:
+        if "nvcc not found" in str(exc) and os.path.exists(LIB_PATH):
+            sys.stderr.write(f"warning: {exc}; using the existing {LIB_PATH}\n")
+            return LIB_PATH
+        raise
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

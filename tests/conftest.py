@@ -31,4 +31,4 @@ def _library_is_built():
     """Builds the CUDA library when it is missing or older than its sources (nvcc cross-compiles without a GPU);
     a no-op otherwise.  The tests then load exactly what the sources in the tree describe."""
     from paper_2602_11812_b200 import build
-    build.build()
+    build.ensure()
