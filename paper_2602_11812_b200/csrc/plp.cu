@@ -228,6 +228,20 @@ plp_update_bound_kernel(const T* __restrict__ hidden_step, int64_t ldh, const fl
 
 }  // namespace
 
+// One block per row, eight channels per thread and pass.  A row is a chain of dependent round trips (partials ->
+// entropy -> update), so the kernel wants every block resident at once: with more rows than fit at d / 8 threads
+// per block, blocks shrink (down to 128 threads, several passes over the row) until one wave holds them all.
+int update_threads(int rows, int d, int min_threads) {
+  int threads = std::min(kPlpMaxThreads, std::max(min_threads, (d / 8 + 31) / 32 * 32));
+  int device = 0, sms = 0;
+  if (cudaGetDevice(&device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms <= 0)
+    return threads;
+  while (threads > 128 && static_cast<int64_t>(rows) > static_cast<int64_t>(sms) * (2048 / threads))
+    threads = std::max(128, (threads / 2 + 31) / 32 * 32);
+  return threads;
+}
+
 cudaError_t launch_plp_update_bound(const void* hidden_step, int64_t ldh, const float* partials, int slots,
                                     int64_t row_stride, int64_t slot_stride, float* Hstep_out, const int32_t* slot_ids,
                                     const int32_t* reset_src, const float* src_m, const float* src_s,
@@ -236,7 +250,7 @@ cudaError_t launch_plp_update_bound(const void* hidden_step, int64_t ldh, const 
                                     float* st_proj, float* z, int64_t ldz, const float* g, int64_t ldg, int g_splits,
                                     int64_t g_split_stride, const HeadArgs& h, float* y, int32_t* status,
                                     cudaStream_t stream, bool overlap_previous) {
-  const int threads = std::min(kPlpMaxThreads, std::max(64, (d / 8 + 31) / 32 * 32));
+  const int threads = update_threads(rows, d, 64);
   const size_t smem = static_cast<size_t>(h.m_h + h.d_out) * sizeof(float);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(rows);
@@ -262,7 +276,7 @@ cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, c
                               const float* src_s, const float* src_pooled, int n_src, int rows, int d, int num_slots,
                               float inv_alpha, float* st_m, float* st_s, float* st_acc, float* z, int64_t ldz,
                               int32_t* status, cudaStream_t stream) {
-  const int threads = std::min(kPlpMaxThreads, std::max(32, (d / 8 + 31) / 32 * 32));
+  const int threads = update_threads(rows, d, 32);
   if (bf16) {
     plp_update_kernel<__nv_bfloat16><<<rows, threads, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(hidden_step), ldh, partials, slots, row_stride, slot_stride, Hstep_out, slot_ids, reset_src, src_m, src_s, src_pooled,
