@@ -41,6 +41,7 @@ struct egtp_ctx {
   float* piece_a = nullptr;       // [chunks][max_d]
   float* piece_b = nullptr;       // [chunks][max_d]
   float* head_partial = nullptr;  int64_t head_partial_floats = 0;
+  void* zcat = nullptr;           // [max_batch][2 * max_d] bf16: head inputs as [hi | lo] halves (tensor-core layer 1)
   float* yhat = nullptr;          // [max_batch]
   int32_t* status = nullptr;      // [1]
   // staging for the *_host entry points (device)
@@ -99,7 +100,7 @@ cudaError_t dev_alloc(egtp_ctx* c, T** p, int64_t count) {
 
 void free_ctx_memory(egtp_ctx* c) {
   cudaFree(c->partials); cudaFree(c->H); cudaFree(c->weights); cudaFree(c->seg_m); cudaFree(c->seg_s);
-  cudaFree(c->pooled); cudaFree(c->piece_a); cudaFree(c->piece_b); cudaFree(c->head_partial); cudaFree(c->yhat);
+  cudaFree(c->pooled); cudaFree(c->piece_a); cudaFree(c->piece_b); cudaFree(c->head_partial); cudaFree(c->zcat); cudaFree(c->yhat);
   cudaFree(c->status); cudaFree(c->hidden_stage); cudaFree(c->offsets_stage); cudaFree(c->reset_stage);
   if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   for (auto& e : c->piece_ready) if (e) cudaEventDestroy(e);
@@ -240,8 +241,54 @@ int run_lmhead(egtp_ctx* c, const egtp_lm_head* lm, const void* hidden, int64_t 
   return EGTP_OK;
 }
 
+// Layer 1 of the head on the tensor cores: possible when the weights are bf16 and the rows fit the context's
+// [hi | lo] staging buffer.  The fp32 input rows are split into two bf16 halves (16 significant bits together),
+// the LM-head kernel multiplies [x_hi | x_lo] against W1 twice over (head columns only, K split over the SMs) and
+// head_out adds the slices up.
+bool head_on_tensor_cores(const egtp_ctx* c, const egtp_head* head, int rows) {
+  return head->wdtype == EGTP_BF16 && head->d % 64 == 0 && head->d <= c->max_d && rows <= c->max_batch &&
+         reinterpret_cast<uintptr_t>(head->W1) % 16 == 0;
+}
+
+// y = head(x) for rows already staged in c->zcat as [hi | lo] halves
+int run_head_staged(egtp_ctx* c, const egtp_head* head, int rows, float* y, float* phat, int32_t* status,
+                    cudaStream_t stream) {
+  const HeadArgs ha = head_args(head);
+  const int64_t rows_pad = (static_cast<int64_t>(rows) + kTileM - 1) / kTileM * kTileM;
+  const int64_t cols_pad = (static_cast<int64_t>(ha.m_h) + 255) / 256 * 256;
+  const int max_splits = static_cast<int>(std::min<int64_t>(16, c->head_partial_floats / (rows_pad * cols_pad)));
+  if (max_splits < 1) return EGTP_ERR_CAPACITY;
+  const LmheadPlan plan = make_headproj_plan(rows, ha.d, ha.m_h, 2, c->num_sms, max_splits, /*a_repeats=*/2);
+  CUtensorMap map_a, map_c;
+  int rc = make_tensor_map(c, &map_a, c->zcat, EGTP_BF16, rows, 2 * ha.d, 2 * static_cast<int64_t>(ha.d), plan.a_box_rows);
+  if (rc != EGTP_OK) return rc;
+  rc = make_tensor_map(c, &map_c, ha.W1, EGTP_BF16, ha.m_h, ha.d, ha.d, plan.b_box_rows);
+  if (rc != EGTP_OK) return rc;
+  LmheadMaps maps;
+  maps.hidden = &map_a;
+  maps.w = maps.w_tile = maps.w1 = maps.w1_tile = &map_c;
+  {
+    LaunchScope ls(c, EGTP_K_HEAD_HIDDEN, stream);
+    EGTP_CUDA_TRY(launch_lmhead_entropy(plan, false, maps, rows, 0, nullptr, status, stream, c->head_partial));
+  }
+  {
+    LaunchScope ls(c, EGTP_K_HEAD_OUT, stream);
+    EGTP_CUDA_TRY(launch_head_out(ha, c->head_partial, rows, plan.k_splits, y, phat, status, stream,
+                                  plan.rows_pad * static_cast<int64_t>(plan.head_cols_pad), plan.head_cols_pad));
+  }
+  return EGTP_OK;
+}
+
 int run_head(egtp_ctx* c, const egtp_head* head, const float* z, int64_t ldz, int rows, float* y, float* phat,
-             const int32_t* status, cudaStream_t stream) {
+             int32_t* status, cudaStream_t stream) {
+  if (head_on_tensor_cores(c, head, rows) && ldz % 4 == 0 && reinterpret_cast<uintptr_t>(z) % 16 == 0) {
+    {
+      LaunchScope ls(c, EGTP_K_HEAD_HIDDEN, stream);
+      EGTP_CUDA_TRY(launch_split_hi_lo(z, ldz, rows, head->d, c->zcat, status, stream));
+    }
+    return run_head_staged(c, head, rows, y, phat, status, stream);
+  }
+  // fp32 weights or odd sizes: layer 1 on the CUDA cores
   const HeadArgs ha = head_args(head);
   const int splits = head_pick_splits(rows, ha.d, ha.m_h, c->num_sms, c->head_partial_floats);
   if (splits <= 0) return EGTP_ERR_CAPACITY;
@@ -387,16 +434,22 @@ int plp_update_and_head(egtp_ctx* c, plp_state* st, const egtp_head* head, const
                                           yrem_out, status, stream, /*overlap_previous=*/false));
     return EGTP_OK;
   }
-  float* z = z_out ? z_out : c->pooled;
   st->proj_valid = false;   // acc moves on without the projection a bound state keeps
+  const bool want_head = head && yrem_out;
+  // with the head's first layer on the tensor cores the update writes z straight into the [hi | lo] staging
+  // buffer (and as fp32 only if the caller asked for z)
+  const bool staged = want_head && head_on_tensor_cores(c, head, B_live);
+  float* z = z_out ? z_out : (staged ? nullptr : c->pooled);
   {
     LaunchScope ls(c, EGTP_K_PLP_UPDATE, stream);
     EGTP_CUDA_TRY(launch_plp_update(hidden_step, ldh, hidden_dtype == EGTP_BF16, partials, slots, row_stride, slot_stride, Hstep_out,
                                     slot_ids,
                                     reset_src, src_m, src_s, src_pooled, n_src, B_live, st->d, st->num_slots,
-                                    1.f / alpha, st->m, st->s, st->acc, z, st->d, status, stream));
+                                    1.f / alpha, st->m, st->s, st->acc, z, st->d, status, stream,
+                                    staged ? c->zcat : nullptr));
   }
-  if (head && yrem_out) return run_head(c, head, z, st->d, B_live, yrem_out, nullptr, status, stream);
+  if (staged) return run_head_staged(c, head, B_live, yrem_out, nullptr, status, stream);
+  if (want_head) return run_head(c, head, z, st->d, B_live, yrem_out, nullptr, status, stream);
   return EGTP_OK;
 }
 
@@ -542,6 +595,7 @@ int egtp_create(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_batc
   ok = ok && dev_alloc(c, &c->piece_a, pool_chunks * max_d) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->piece_b, pool_chunks * max_d) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->head_partial, c->head_partial_floats) == cudaSuccess;
+  ok = ok && dev_alloc(c, reinterpret_cast<float**>(&c->zcat), static_cast<int64_t>(max_batch) * max_d) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->yhat, max_batch) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->status, 1) == cudaSuccess;
   ok = ok && dev_alloc(c, reinterpret_cast<float**>(&c->hidden_stage), rows_cap * max_d) == cudaSuccess;

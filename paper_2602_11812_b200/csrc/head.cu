@@ -123,7 +123,7 @@ head_hidden_kernel(const float* __restrict__ z, int64_t ldz, const TW* __restric
 // (one warp per output, lanes stride the hidden units), then the output mode.
 template <typename TW>
 __global__ void __launch_bounds__(kHOutThreads)
-head_out_kernel(const float* __restrict__ partial, int rows, int splits, int m_h, int d_out,
+head_out_kernel(const float* __restrict__ partial, int64_t split_stride, int64_t row_stride, int splits, int m_h, int d_out,
                 const float* __restrict__ b1, const TW* __restrict__ W2, const float* __restrict__ b2,
                 const float* __restrict__ centres, int mode, float* __restrict__ y, float* __restrict__ phat,
                 const int32_t* __restrict__ status) {
@@ -133,8 +133,8 @@ head_out_kernel(const float* __restrict__ partial, int rows, int splits, int m_h
   float* o = smem + m_h;      // [d_out]
   const int r = blockIdx.x, tid = threadIdx.x;
   for (int j = tid; j < m_h; j += blockDim.x) {
-    const float* pj = partial + static_cast<int64_t>(r) * m_h + j;
-    const int64_t stride = static_cast<int64_t>(rows) * m_h;
+    const float* pj = partial + static_cast<int64_t>(r) * row_stride + j;
+    const int64_t stride = split_stride;
     float v = 0.f;
     int s = 0;
     for (; s + 4 <= splits; s += 4) {     // four loads in flight; the additions keep split order
@@ -161,6 +161,31 @@ head_partial_sum_kernel(const float* __restrict__ partial, int rows, int splits,
     for (int s = 0; s < splits; ++s) v += __ldg(partial + s * n + i);
     const int64_t r = i / m_h;
     out[r * ld_out + (i - r * m_h)] = v;
+  }
+}
+
+// xcat[r][0..d) = bf16(x[r]), xcat[r][d..2d) = bf16(x[r] - bf16(x[r])); 8 elements per thread
+__global__ void __launch_bounds__(256)
+split_hi_lo_kernel(const float* __restrict__ x, int64_t ldx, int rows, int d, __nv_bfloat16* __restrict__ xcat,
+                   const int32_t* __restrict__ status) {
+  if (*status != 0) return;
+  const int per_row = d / 8;
+  const int64_t n = static_cast<int64_t>(rows) * per_row;
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int64_t r = i / per_row;
+    const int col = static_cast<int>(i - r * per_row) * 8;
+    float v[8];
+    load8w<float>(x + r * ldx + col, v);
+    __align__(16) __nv_bfloat16 hi[8], lo[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      hi[k] = __float2bfloat16_rn(v[k]);
+      lo[k] = __float2bfloat16_rn(v[k] - __bfloat162float(hi[k]));
+    }
+    __nv_bfloat16* dst = xcat + r * (2 * static_cast<int64_t>(d)) + col;
+    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(hi);
+    *reinterpret_cast<uint4*>(dst + d) = *reinterpret_cast<const uint4*>(lo);
   }
 }
 
@@ -192,14 +217,16 @@ cudaError_t launch_head_hidden(const HeadArgs& h, const float* z, int64_t ldz, i
 }
 
 cudaError_t launch_head_out(const HeadArgs& h, const float* partial, int rows, int splits, float* y, float* phat,
-                            const int32_t* status, cudaStream_t stream) {
+                            const int32_t* status, cudaStream_t stream, int64_t split_stride, int64_t row_stride) {
   const size_t smem = static_cast<size_t>(h.m_h + h.d_out) * sizeof(float);
+  if (row_stride == 0) row_stride = h.m_h;
+  if (split_stride == 0) split_stride = static_cast<int64_t>(rows) * h.m_h;
   if (h.bf16) {
-    head_out_kernel<__nv_bfloat16><<<rows, kHOutThreads, smem, stream>>>(partial, rows, splits, h.m_h, h.d_out, h.b1,
+    head_out_kernel<__nv_bfloat16><<<rows, kHOutThreads, smem, stream>>>(partial, split_stride, row_stride, splits, h.m_h, h.d_out, h.b1,
                                                                static_cast<const __nv_bfloat16*>(h.W2), h.b2,
                                                                h.centres, h.mode, y, phat, status);
   } else {
-    head_out_kernel<float><<<rows, kHOutThreads, smem, stream>>>(partial, rows, splits, h.m_h, h.d_out, h.b1,
+    head_out_kernel<float><<<rows, kHOutThreads, smem, stream>>>(partial, split_stride, row_stride, splits, h.m_h, h.d_out, h.b1,
                                                        static_cast<const float*>(h.W2), h.b2, h.centres, h.mode, y,
                                                        phat, status);
   }
@@ -211,6 +238,14 @@ cudaError_t launch_head_partial_sum(const float* partial, int rows, int splits, 
   const int64_t n = static_cast<int64_t>(rows) * m_h;
   const int blocks = static_cast<int>(std::min<int64_t>(1184, (n + 255) / 256));
   head_partial_sum_kernel<<<std::max(1, blocks), 256, 0, stream>>>(partial, rows, splits, m_h, out, ld_out, status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_split_hi_lo(const float* x, int64_t ldx, int rows, int d, void* xcat, const int32_t* status,
+                               cudaStream_t stream) {
+  const int64_t n = static_cast<int64_t>(rows) * (d / 8);
+  const int blocks = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(1184, (n + 255) / 256)));
+  split_hi_lo_kernel<<<blocks, 256, 0, stream>>>(x, ldx, rows, d, static_cast<__nv_bfloat16*>(xcat), status);
   return cudaGetLastError();
 }
 

@@ -32,6 +32,7 @@ struct LmheadPlan {
   int slots;          // partial slots per row
   int group_rb;       // row blocks that sweep the vocabulary together (L2 reuse of W tiles)
   int k_blocks;       // ceil(d * elem / 128)
+  int b_k_blocks;     // > 0: W1 has this many k blocks and is read again from its start for every further segment of A
   int k_splits;       // > 1: K is split over that many units per (row block, chunk); head projection launches only
   int smem_bytes;     // dynamic shared memory
   int64_t rows_pad;   // row_blocks * rows_per_block: rows of the partial buffer
@@ -47,7 +48,10 @@ LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms
 
 // Launch shape for W1 hidden[i] alone (no vocabulary): the head columns of the prompt shape with K split over
 // up to max_splits units, each writing its own slice head_g[split][rows_pad][head_cols_pad].
-LmheadPlan make_headproj_plan(int64_t T, int d, int m_h, int elem_bytes, int num_sms, int max_splits);
+// a_repeats > 1: the rows of A are a_repeats segments of d elements (d * elem_bytes a multiple of 128) that are all
+// multiplied against the same W1 and summed, e.g. the high and low bf16 halves of fp32 vectors.
+LmheadPlan make_headproj_plan(int64_t T, int d, int m_h, int elem_bytes, int num_sms, int max_splits,
+                              int a_repeats = 1);
 
 // Opts the kernels into their dynamic shared-memory size on the current device (once per device).
 cudaError_t lmhead_prepare_device();
@@ -121,8 +125,14 @@ int head_pick_splits(int rows, int d, int m_h, int num_sms, int64_t partial_capa
 cudaError_t launch_head_hidden(const HeadArgs& h, const float* z, int64_t ldz, int rows, int splits,
                                float* partial, const int32_t* status, cudaStream_t stream);
 
+// partial[s * split_stride + r * row_stride + j]; strides 0 = the dense [splits][rows][m_h] layout
 cudaError_t launch_head_out(const HeadArgs& h, const float* partial, int rows, int splits, float* y, float* phat,
-                            const int32_t* status, cudaStream_t stream);
+                            const int32_t* status, cudaStream_t stream, int64_t split_stride = 0,
+                            int64_t row_stride = 0);
+
+// xcat[r] = [bf16(x[r]) | bf16(x[r] - bf16(x[r]))]: fp32 rows as two bf16 halves (16 significant bits together)
+cudaError_t launch_split_hi_lo(const float* x, int64_t ldx, int rows, int d, void* xcat, const int32_t* status,
+                               cudaStream_t stream);
 
 // out[r][j] = sum_s partial[s][r][j] (split order): W1 x for rows x that are not pooled vectors
 cudaError_t launch_head_partial_sum(const float* partial, int rows, int splits, int m_h, float* out, int64_t ld_out,
@@ -138,7 +148,7 @@ cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, c
                               const int32_t* slot_ids, const int32_t* reset_src, const float* src_m,
                               const float* src_s, const float* src_pooled, int n_src, int rows, int d, int num_slots,
                               float inv_alpha, float* st_m, float* st_s, float* st_acc, float* z, int64_t ldz,
-                              int32_t* status, cudaStream_t stream);
+                              int32_t* status, cudaStream_t stream, void* zcat = nullptr);
 
 // The update for a state bound to a head (bf16 hidden states and head weights): also advances the slot's
 // projection st_proj = W1 acc with g = W1 h' from the LM-head kernel and finishes the head for the row.

@@ -62,6 +62,9 @@ struct KParams {
   // [(u % k_splits) * kb_per_split, ...) of the unit u / k_splits and writes its own slice of head_g
   int k_splits, kb_per_split;
   int64_t g_split_stride;
+  // > 0: the matrices behind map_b / map_c have only this many k blocks and are read again from their start
+  // after that (A = [x_hi | x_lo], two bf16 halves of fp32 rows, multiplied against the same W1 twice)
+  int b_k_blocks;
 };
 
 __device__ __forceinline__ UnitCoord unit_coord(int u_in, const KParams& p) {
@@ -264,18 +267,19 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
               const uint32_t a_dst = smem_base + stage * kStageBytes;
               const uint32_t b_dst = a_dst + kABytes;
               const int kx = kb * kElemsPerStage;
+              const int kxb = (kFuse && p.b_k_blocks > 0) ? (kb % p.b_k_blocks) * kElemsPerStage : kx;
               mbar_arrive_expect_tx(full_bar(stage), tx_bytes);
               tma_load_2d(a_dst, &map_a, kx, uc.row_block * (kMT * kTileM), full_bar(stage));
               if constexpr (kSource == 0) {
-                tma_load_2d(b_dst, &map_b_tile, kx, n0, full_bar(stage));
+                tma_load_2d(b_dst, &map_b_tile, kxb, n0, full_bar(stage));
               } else if constexpr (kSource == 1) {
-                tma_load_2d(b_dst, &map_c_tile, kx, n0 - p.v_pad, full_bar(stage));
+                tma_load_2d(b_dst, &map_c_tile, kxb, n0 - p.v_pad, full_bar(stage));
               } else {
                 for (int i = 0; i < b_loads_w; ++i)
-                  tma_load_2d(b_dst + i * (kBBox * kRowBytes), &map_b, kx, n0 + i * kBBox, full_bar(stage));
+                  tma_load_2d(b_dst + i * (kBBox * kRowBytes), &map_b, kxb, n0 + i * kBBox, full_bar(stage));
                 if constexpr (kFuse) {
                   for (int i = b_loads_w; i < b_loads; ++i)
-                    tma_load_2d(b_dst + i * (kBBox * kRowBytes), &map_c, kx, n0 + i * kBBox - p.v_pad, full_bar(stage));
+                    tma_load_2d(b_dst + i * (kBBox * kRowBytes), &map_c, kxb, n0 + i * kBBox - p.v_pad, full_bar(stage));
                 }
               }
               if (++stage == kNumStages) { stage = 0; phase ^= 1u; }
@@ -844,7 +848,7 @@ LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms
   return pl;
 }
 
-LmheadPlan make_headproj_plan(int64_t T, int d, int m_h, int elem_bytes, int num_sms, int max_splits) {
+LmheadPlan make_headproj_plan(int64_t T, int d, int m_h, int elem_bytes, int num_sms, int max_splits, int a_repeats) {
   // The prompt shape (128-row blocks, 256-column tiles) over the head columns alone, K split so that the grid
   // fills the GPU while every split still streams several k blocks.
   LmheadPlan pl{};
@@ -861,6 +865,10 @@ LmheadPlan make_headproj_plan(int64_t T, int d, int m_h, int elem_bytes, int num
   pl.n_groups = pl.head_cols_pad / sh.col_gran;
   pl.rows_pad = static_cast<int64_t>(pl.row_blocks) * kTileM;
   pl.k_blocks = static_cast<int>((static_cast<int64_t>(d) * elem_bytes + kRowBytes - 1) / kRowBytes);
+  if (a_repeats > 1) {               // A rows are a_repeats segments of d elements, each against the same W1
+    pl.b_k_blocks = pl.k_blocks;
+    pl.k_blocks *= a_repeats;
+  }
   pl.smem_bytes = smem_bytes_for(sh.mt, sh.bn, sh.stages);
   pl.chunks = pl.n_groups;           // one 256-column tile per unit
   pl.slots = pl.chunks * kEpiSplit;  // unused: no entropy partials are written
@@ -910,6 +918,7 @@ cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const Lmhea
   p.k_splits = std::max(1, plan.k_splits);
   p.kb_per_split = (plan.k_blocks + p.k_splits - 1) / p.k_splits;
   p.g_split_stride = plan.rows_pad * static_cast<int64_t>(plan.head_cols_pad);
+  p.b_k_blocks = plan.b_k_blocks;
   p.total_units = plan.row_blocks * plan.chunks * p.k_splits;
   p.V = V;
   p.slots = plan.slots;

@@ -49,7 +49,8 @@ plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* _
                   const int32_t* __restrict__ reset_src, const float* __restrict__ src_m,
                   const float* __restrict__ src_s, const float* __restrict__ src_pooled, int n_src, int d,
                   int num_slots, float inv_alpha, float* __restrict__ st_m, float* __restrict__ st_s,
-                  float* __restrict__ st_acc, float* __restrict__ z, int64_t ldz, int32_t* status) {
+                  float* __restrict__ st_acc, float* __restrict__ z, int64_t ldz, __nv_bfloat16* __restrict__ zcat,
+                  int32_t* status) {
   if (*status != 0) return;
   const int i = blockIdx.x;
   const int slot = slot_ids ? slot_ids[i] : i;
@@ -74,7 +75,9 @@ plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* _
   if (!(s_old > 0.f)) acc_src = nullptr;    // an empty sequence carries nothing over
   float* acc_dst = st_acc + static_cast<int64_t>(slot) * d;
   const T* hrow = hidden_step + static_cast<int64_t>(i) * ldh;
-  float* zrow = z + static_cast<int64_t>(i) * ldz;
+  float* zrow = z ? z + static_cast<int64_t>(i) * ldz : nullptr;
+  // zcat (optional): z as two bf16 halves [hi | lo] per row, the operand of the head's tensor-core layer 1
+  __nv_bfloat16* zc = zcat ? zcat + static_cast<int64_t>(i) * (2 * static_cast<int64_t>(d)) : nullptr;
 
   // first pass of loads is issued before the entropy merge so that both latencies overlap
   int col = threadIdx.x * 8;
@@ -109,8 +112,21 @@ plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* _
     }
     reinterpret_cast<float4*>(acc_dst + col)[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
     reinterpret_cast<float4*>(acc_dst + col)[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
-    reinterpret_cast<float4*>(zrow + col)[0] = make_float4(acc[0] * inv_s, acc[1] * inv_s, acc[2] * inv_s, acc[3] * inv_s);
-    reinterpret_cast<float4*>(zrow + col)[1] = make_float4(acc[4] * inv_s, acc[5] * inv_s, acc[6] * inv_s, acc[7] * inv_s);
+    if (zrow != nullptr) {
+      reinterpret_cast<float4*>(zrow + col)[0] = make_float4(acc[0] * inv_s, acc[1] * inv_s, acc[2] * inv_s, acc[3] * inv_s);
+      reinterpret_cast<float4*>(zrow + col)[1] = make_float4(acc[4] * inv_s, acc[5] * inv_s, acc[6] * inv_s, acc[7] * inv_s);
+    }
+    if (zc != nullptr) {
+      __align__(16) __nv_bfloat16 hi[8], lo[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const float zv = acc[k] * inv_s;
+        hi[k] = __float2bfloat16_rn(zv);
+        lo[k] = __float2bfloat16_rn(zv - __bfloat162float(hi[k]));
+      }
+      *reinterpret_cast<uint4*>(zc + col) = *reinterpret_cast<const uint4*>(hi);
+      *reinterpret_cast<uint4*>(zc + d + col) = *reinterpret_cast<const uint4*>(lo);
+    }
   }
   if (threadIdx.x == 0) {
     st_m[slot] = m_new;
@@ -275,16 +291,16 @@ cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, c
                               int64_t row_stride, int64_t slot_stride, float* Hstep_out, const int32_t* slot_ids, const int32_t* reset_src, const float* src_m,
                               const float* src_s, const float* src_pooled, int n_src, int rows, int d, int num_slots,
                               float inv_alpha, float* st_m, float* st_s, float* st_acc, float* z, int64_t ldz,
-                              int32_t* status, cudaStream_t stream) {
+                              int32_t* status, cudaStream_t stream, void* zcat) {
   const int threads = update_threads(rows, d, 32);
   if (bf16) {
     plp_update_kernel<__nv_bfloat16><<<rows, threads, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(hidden_step), ldh, partials, slots, row_stride, slot_stride, Hstep_out, slot_ids, reset_src, src_m, src_s, src_pooled,
-        n_src, d, num_slots, inv_alpha, st_m, st_s, st_acc, z, ldz, status);
+        n_src, d, num_slots, inv_alpha, st_m, st_s, st_acc, z, ldz, static_cast<__nv_bfloat16*>(zcat), status);
   } else {
     plp_update_kernel<float><<<rows, threads, 0, stream>>>(static_cast<const float*>(hidden_step), ldh, partials, slots, row_stride, slot_stride, Hstep_out, slot_ids,
                                                        reset_src, src_m, src_s, src_pooled, n_src, d, num_slots,
-                                                       inv_alpha, st_m, st_s, st_acc, z, ldz, status);
+                                                       inv_alpha, st_m, st_s, st_acc, z, ldz, static_cast<__nv_bfloat16*>(zcat), status);
   }
   return cudaGetLastError();
 }
