@@ -118,6 +118,29 @@ def test_mid_config_scaled(ctx):
     assert egtp.egtp_lmhead_plan(ctx, T, wl.d, wl.V, egtp.EGTP_BF16)["chunks"] == planned
 
 
+def test_head_on_tensor_cores_keeps_fp32_accuracy(ctx):
+    # bf16 head weights: layer 1 runs on the tensor cores with every fp32 input row split into two bf16 halves.
+    # Fed the device's own pooled vectors, the oracle's head must agree to ~1e-5, far inside the 0.5-token bar
+    # (a single bf16 rounding of the inputs would be off by ~1e-3 relative).
+    wl = gen.config_mid(V=4096 + 8, d=512, m_h=264, B=40, max_len=120)
+    big = gen.make_head(21, 512, 264, 1, "bf16")
+    big.W2 *= 64.0; big.b2 += 300.0                      # predictions of a few hundred tokens
+    big.W2[:] = gen.round_to_bf16(big.W2)
+    wl.head = big
+    res = gu.run_egtp(ctx, wl)
+    assert res["status"] == 0
+    y_ref, _ = orc.head_forward(res["pooled"], big.W1, big.b1, big.W2, big.b2)
+    assert np.abs(y_ref).max() > 100
+    err = np.abs(res["yhat"] - y_ref)
+    assert err.max() <= 1e-4 * np.abs(y_ref).max(), err.max()
+    # bins head (K = 20) through the same route
+    bins = gen.make_head(22, 512, 264, 20, "bf16", mode=gen.HEAD_BINS)
+    wl.head = bins
+    res = gu.run_egtp(ctx, wl, want_phat=True)
+    y_ref, p_ref = orc.head_forward(res["pooled"], bins.W1, bins.b1, bins.W2, bins.b2, mode=bins.mode, centres=bins.centres)
+    assert np.abs(res["phat"] - p_ref).max() <= 1e-5 and np.abs(res["yhat"] - y_ref).max() <= 0.05
+
+
 def test_segment_edge_cases(ctx):
     # leading / trailing tokens outside every prompt, empty prompts, boundaries on and next to a 128-row tile
     # edge and a 64-token pooling chunk edge, a one-token prompt
