@@ -159,3 +159,42 @@ def test_rl_group_configuration_full_size():
         # streams of one group that were fed different tokens differ; all are finite
         assert np.all(np.isfinite(y)) and not np.array_equal(z[-1, follow[0]], z[-1, follow[1]])
     gu.assert_length_close(runs[1][2].ravel(), runs[0][2].ravel())
+
+
+def test_wide_model_d8192_llama_sized_vocabulary():
+    # hidden size 8192 (128 k blocks per tile pass, 16 KB rows) against a 128256-entry vocabulary: a prompt batch
+    # (three row blocks) and bound decode steps of 200 streams; the oracle follows sampled tokens and two streams
+    d, V, m_h = 8192, 128256, 512
+    lengths = [5, 170, 131]
+    wl = gen.make_egtp("wide", 9, lengths, d=d, V=V, dtype="bf16", m_h=m_h)
+    ctx = egtp.egtp_create(0, max_tokens=1024, max_batch=256, max_d=d, max_V=V)
+    try:
+        W_dev = gu.dev_tensor(wl.W, "bf16")
+        res = gu.run_egtp(ctx, wl, W_dev=W_dev)
+        assert res["status"] == 0
+        off = wl.offsets.astype(np.int64)
+        assert np.array_equal(res["seg_id"], orc.segment_ids(off, wl.T))
+        idx = np.array([0, 4, 5, 127, 128, 174, 175, 305])
+        gu.assert_entropy_close(res["H"][idx], orc.token_entropy(wl.hidden[idx], wl.W))
+        ref0 = orc.egtp_predict(wl.hidden[:5], np.array([0, 5]), wl.W, wl.head)        # the 5-token prompt in full
+        gu.assert_pooled_close(res["pooled"][[0]], ref0["pooled"])
+        gu.assert_length_close(res["yhat"][[0]], ref0["yhat"])
+        for b in (1, 2):
+            w = orc.entropy_weights(res["H"][off[b]:off[b + 1]])
+            gu.assert_pooled_close(res["pooled"][[b]], orc.pool(wl.hidden[off[b]:off[b + 1]], w)[None, :])
+        y_ref, _ = orc.head_forward(res["pooled"], wl.head.W1, wl.head.b1, wl.head.W2, wl.head.b2)
+        gu.assert_length_close(res["yhat"], y_ref)
+        # decode: 200 streams, 3 steps, state bound to the head
+        rng = np.random.Generator(np.random.PCG64(909))
+        hs = gen.round_to_bf16(rng.standard_normal((3, 200, d)).astype(np.float32))
+        reset = np.full((3, 200), gen.RESET_KEEP, np.int32); reset[0] = gen.RESET_EMPTY
+        pw = gen.PlpWorkload("wide_decode", "bf16", hs, reset, wl.W, wl.head)
+        H, z, y = _run_plp_steps(ctx, pw, W_dev, gu.DeviceHead(wl.head, "bf16"), bind=True)
+    finally:
+        egtp.egtp_destroy(ctx)
+    follow = [0, 199]
+    ref = orc.plp_run(hs, reset, wl.W, wl.head, slots=follow)
+    gu.assert_entropy_close(H[:, follow].ravel(), ref["H"].ravel())
+    for t in range(3):
+        gu.assert_pooled_close(z[t, follow], ref["z"][t])
+    gu.assert_length_close(y[:, follow].ravel(), ref["yrem"].ravel())
