@@ -356,6 +356,7 @@ enum {
   EGTP_K_HEAD_OUT,          /* head layer 2 + output mode */
   EGTP_K_PLP_UPDATE,        /* PLP running-state update */
   EGTP_K_LOGITS_ENTROPY,    /* Eq. 2 from logits already in memory */
+  EGTP_K_STAGE_ROWS,        /* batches of fewer than 16 rows copied into a zero-padded 16-row buffer */
   EGTP_NUM_KERNELS
 };
 EGTP_API int egtp_profile_enable(egtp_ctx* ctx, int on);

@@ -27,7 +27,7 @@ PLP_RESET_KEEP, PLP_RESET_EMPTY = -2, -1
 EGTP_LMHEAD_AUTO, EGTP_LMHEAD_CTA_PAIRS, EGTP_LMHEAD_SINGLE_CTA = 0, 1, 2
 EGTP_POOL_MEAN, EGTP_POOL_MAX, EGTP_POOL_LAST = 1, 2, 3
 KERNEL_IDS = ["validate_offsets", "lmhead_entropy", "entropy_merge", "segment_weights", "pool",
-              "pool_combine", "head_hidden", "head_out", "plp_update", "logits_entropy"]
+              "pool_combine", "head_hidden", "head_out", "plp_update", "logits_entropy", "stage_rows"]
 EGTP_NUM_KERNELS = len(KERNEL_IDS)
 EGTP_K_LMHEAD_ENTROPY = 1
 

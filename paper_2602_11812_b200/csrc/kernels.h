@@ -103,6 +103,11 @@ cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, bool take_ma
 cudaError_t launch_pool_combine(const int32_t* offsets, int B, int d, bool take_max, const float* piece_a,
                                 const float* piece_b, float* pooled, const int32_t* status, cudaStream_t stream);
 
+// dst [dst_rows][row_bytes] <- the first src_rows rows of src (ld_bytes apart), the other rows zero.
+// row_bytes and ld_bytes are multiples of 16, both pointers 16-byte aligned.
+cudaError_t launch_pad_rows(const void* src, int64_t ld_bytes, int src_rows, int64_t row_bytes, void* dst,
+                            int dst_rows, const int32_t* status, cudaStream_t stream);
+
 // ---- Eq. 2 from logits already in memory -------------------------------------------------------
 int logits_entropy_pick_splits(int64_t rows, int V, int num_sms);
 // partials [rows][splits][3] in the layout of the LM-head kernel's partials

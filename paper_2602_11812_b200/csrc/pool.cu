@@ -360,4 +360,33 @@ cudaError_t launch_pool_combine(const int32_t* offsets, int B, int d, bool take_
   return cudaGetLastError();
 }
 
+namespace {
+
+// dst [dst_rows][row_bytes] <- src rows (src_rows of them, ld_bytes apart), remaining rows zero; 16 bytes per thread
+__global__ void __launch_bounds__(256)
+pad_rows_kernel(const uint8_t* __restrict__ src, int64_t ld_bytes, int src_rows, int64_t row_bytes,
+                uint8_t* __restrict__ dst, int dst_rows, const int32_t* __restrict__ status) {
+  if (*status != 0) return;
+  const int64_t per_row = row_bytes / 16;
+  const int64_t n = per_row * dst_rows;
+  for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n;
+       i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int64_t r = i / per_row, c = (i - r * per_row) * 16;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (r < src_rows) v = *reinterpret_cast<const uint4*>(src + r * ld_bytes + c);
+    *reinterpret_cast<uint4*>(dst + r * row_bytes + c) = v;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_pad_rows(const void* src, int64_t ld_bytes, int src_rows, int64_t row_bytes, void* dst,
+                            int dst_rows, const int32_t* status, cudaStream_t stream) {
+  const int64_t n = row_bytes / 16 * dst_rows;
+  const int blocks = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(296, (n + 255) / 256)));
+  pad_rows_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint8_t*>(src), ld_bytes, src_rows, row_bytes,
+                                              static_cast<uint8_t*>(dst), dst_rows, status);
+  return cudaGetLastError();
+}
+
 }  // namespace egtp
