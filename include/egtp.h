@@ -372,6 +372,15 @@ EGTP_API int64_t egtp_launch_count(const egtp_ctx* ctx);
  * [7] = dynamic shared memory bytes.  Host pointer; nothing is launched. */
 EGTP_API int egtp_lmhead_plan(const egtp_ctx* ctx, int64_t T, int32_t d, int32_t V, int32_t dtype, int32_t info[8]);
 
+/* The same plan without a context or a GPU: for a device with num_sms SMs that can co-schedule pair_workers
+ * clusters of two CTAs (0 = none; a B200 has 148 SMs and 74 pairs), a context sized for exactly T rows, and
+ * head_cols head columns riding along (0 = none; the m_h of a bound state, Sec. 3.2-3.3).  info[0..7] as above,
+ * [8] = kernel form (0 prompt shape, 1 / 2 one-CTA decode shapes for <= 128 / <= 256 rows, 4 / 5 CTA pairs for
+ * prompts / decode), [9] = row blocks that sweep the vocabulary together, [10] = column granularity of the
+ * vocabulary split, [11] = number of such column groups (head columns included).  Pure host arithmetic. */
+EGTP_API int egtp_lmhead_plan_for(int32_t num_sms, int32_t pair_workers, int64_t T, int32_t d, int32_t V, int32_t dtype,
+                                  int32_t mode, int32_t head_cols, int32_t info[12]);
+
 #ifdef __cplusplus
 }
 #endif

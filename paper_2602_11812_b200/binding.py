@@ -38,7 +38,7 @@ EXPORTED_SYMBOLS = [
     "egtp_launch_count", "egtp_lmhead_plan", "egtp_head_forward_static", "egtp_set_lmhead_mode",
     "egtp_entropy_from_logits", "plp_step_from_logits", "egtp_pool_baseline",
     "egtp_entropy_partials", "egtp_entropy_from_partials", "plp_step_from_partials", "egtp_selftest_wait_timeout",
-    "plp_state_bind_head", "egtp_set_lmhead_chunks",
+    "plp_state_bind_head", "egtp_set_lmhead_chunks", "egtp_lmhead_plan_for",
 ]
 
 
@@ -87,6 +87,7 @@ def load() -> C.CDLL:
     lib.egtp_profile_enable.argtypes = [vp, C.c_int]
     lib.egtp_set_lmhead_mode.argtypes = [vp, C.c_int]
     lib.egtp_set_lmhead_chunks.argtypes = [vp, i32]
+    lib.egtp_lmhead_plan_for.argtypes = [i32, i32, i64, i32, i32, i32, i32, i32, P(i32)]
     lib.egtp_selftest_wait_timeout.argtypes = [vp, i32, vp, vp]
     lib.egtp_entropy_partials.argtypes = [vp, P(egtp_lm_head), vp, i64, i64, vp, vp, vp]
     lib.egtp_entropy_from_partials.argtypes = [vp, vp, i32, i64, vp, vp, vp]
@@ -197,6 +198,16 @@ def egtp_lmhead_plan(ctx: int, T: int, d: int, V: int, dtype: int) -> dict:
     info = (C.c_int32 * 8)()
     _check(load().egtp_lmhead_plan(ctx, T, d, V, dtype, info), "egtp_lmhead_plan")
     keys = ["grid", "row_blocks", "rows_per_block", "chunks", "slots", "tile_cols", "k_blocks", "smem_bytes"]
+    return dict(zip(keys, list(info)))
+
+
+def egtp_lmhead_plan_for(num_sms: int, pair_workers: int, T: int, d: int, V: int, dtype: int = EGTP_BF16,
+                         mode: int = EGTP_LMHEAD_AUTO, head_cols: int = 0) -> dict:
+    """Launch plan of the LM-head kernel for a device described by its SM count (no GPU needed)."""
+    info = (C.c_int32 * 12)()
+    _check(load().egtp_lmhead_plan_for(num_sms, pair_workers, T, d, V, dtype, mode, head_cols, info), "egtp_lmhead_plan_for")
+    keys = ["grid", "row_blocks", "rows_per_block", "chunks", "slots", "tile_cols", "k_blocks", "smem_bytes",
+            "variant", "group_rb", "col_gran", "n_groups"]
     return dict(zip(keys, list(info)))
 
 

@@ -656,6 +656,22 @@ int egtp_lmhead_plan(const egtp_ctx* c, int64_t T, int32_t d, int32_t V, int32_t
   return EGTP_OK;
 }
 
+int egtp_lmhead_plan_for(int32_t num_sms, int32_t pair_workers, int64_t T, int32_t d, int32_t V, int32_t dtype,
+                         int32_t mode, int32_t head_cols, int32_t info[12]) {
+  if (!info || num_sms <= 0 || pair_workers < 0 || T <= 0 || d <= 0 || V <= 0 || head_cols < 0) return EGTP_ERR_INVALID_ARG;
+  if (dtype != EGTP_F32 && dtype != EGTP_BF16) return EGTP_ERR_UNSUPPORTED;
+  if (mode != EGTP_LMHEAD_AUTO && mode != EGTP_LMHEAD_CTA_PAIRS && mode != EGTP_LMHEAD_SINGLE_CTA) return EGTP_ERR_INVALID_ARG;
+  // the workspace rule of egtp_create for a context sized for exactly T rows
+  const int64_t rows_pad = (T + kTileM - 1) / kTileM * kTileM;
+  const int64_t capacity = std::max<int64_t>(
+      std::max<int64_t>(rows_pad * 24 * kEpiSplit, static_cast<int64_t>(2 * kTileM) * num_sms * kEpiSplit), int64_t{1} << 21);
+  const LmheadPlan p = make_lmhead_plan(T, d, V, elem_bytes(dtype), num_sms, capacity, mode, head_cols, 0, pair_workers);
+  info[0] = p.grid; info[1] = p.row_blocks; info[2] = p.rows_per_block; info[3] = p.chunks;
+  info[4] = p.slots; info[5] = p.tile_cols; info[6] = p.k_blocks; info[7] = p.smem_bytes;
+  info[8] = p.variant; info[9] = p.group_rb; info[10] = p.col_gran; info[11] = p.n_groups;
+  return EGTP_OK;
+}
+
 int egtp_set_lmhead_mode(egtp_ctx* c, int mode) {
   if (!c || (mode != EGTP_LMHEAD_AUTO && mode != EGTP_LMHEAD_CTA_PAIRS && mode != EGTP_LMHEAD_SINGLE_CTA))
     return EGTP_ERR_INVALID_ARG;

@@ -40,11 +40,12 @@ struct LmheadPlan {
 
 // Picks chunks / grouping for T rows; slot_limit bounds chunks * kEpiSplit * rows_pad by the
 // partial buffer's capacity (in rows x slots).
-// force_chunks > 0 overrides the number of vocabulary chunks of prompt batches (clamped to the workspace).
+// pair_workers >= 0 states how many CTA pairs the device can co-schedule (default: what was measured on the
+// current device).  force_chunks > 0 overrides the number of vocabulary chunks of prompt batches (clamped to the workspace).
 // head_cols > 0: that many rows of a second matrix (the head's W1) are appended to the vocabulary as
 // extra columns whose raw products the kernel writes out (bf16, one-CTA shapes only).
 LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity,
-                            int mode, int head_cols = 0, int force_chunks = 0);
+                            int mode, int head_cols = 0, int force_chunks = 0, int pair_workers = -1);
 
 // Launch shape for W1 hidden[i] alone (no vocabulary): the head columns of the prompt shape with K split over
 // up to max_splits units, each writing its own slice head_g[split][rows_pad][head_cols_pad].

@@ -762,12 +762,15 @@ static_assert(kShapeDecode2.mt == 2 && kShapeDecode2.bn == 256 && kShapeDecode2.
 }  // namespace
 
 LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity,
-                            int mode, int head_cols, int force_chunks) {
+                            int mode, int head_cols, int force_chunks, int pair_workers) {
+  // CTA pairs the device can co-schedule: what lmhead_prepare_device found, unless the caller states a number
+  // (planning for a device that is not present)
+  const int pair_cap = pair_workers >= 0 ? pair_workers : g_pair_workers_max;
   LmheadPlan pl{};
   // decode batches of 129..256 rows run as CTA pairs on 256 x 512 tiles unless single CTAs are asked for or the
   // device cannot co-schedule the pairs; prompt batches run as pairs only on request (and never with head columns)
   pl.variant = T <= kTileM ? 1 : (T <= 2 * kTileM ? 2 : 0);
-  const bool pairs_ok = g_pair_workers_max > 0 && mode != EGTP_LMHEAD_SINGLE_CTA;
+  const bool pairs_ok = pair_cap > 0 && mode != EGTP_LMHEAD_SINGLE_CTA;
   if (pl.variant == 2 && pairs_ok) pl.variant = 5;
   if (pl.variant == 0 && pairs_ok && mode == EGTP_LMHEAD_CTA_PAIRS && head_cols == 0) pl.variant = 4;
   const bool pair = pl.variant >= 4;
@@ -790,7 +793,7 @@ LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms
   // warps unless the two warps serve two different row tiles
   const int slots_per_chunk = pl.variant == 2 ? 1 : kEpiSplit;
   // CTAs, or CTA pairs that fit on the device at once
-  const int workers_max = pair ? std::max(1, g_pair_workers_max > 0 ? std::min(g_pair_workers_max, num_sms / 2) : num_sms / 2)
+  const int workers_max = pair ? std::max(1, pair_cap > 0 ? std::min(pair_cap, num_sms / 2) : num_sms / 2)
                                : num_sms;
   const int64_t s_cap = std::max<int64_t>(1, slot_row_capacity / (pl.rows_pad * slots_per_chunk));
   const int s_max = static_cast<int>(std::min<int64_t>(pl.n_groups, s_cap));
