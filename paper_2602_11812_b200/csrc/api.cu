@@ -269,9 +269,10 @@ bool head_on_tensor_cores(const egtp_ctx* c, const egtp_head* head, int rows) {
          reinterpret_cast<uintptr_t>(head->W1) % 16 == 0;
 }
 
-// y = head(x) for rows already staged in c->zcat as [hi | lo] halves
-int run_head_staged(egtp_ctx* c, const egtp_head* head, int rows, float* y, float* phat, int32_t* status,
-                    cudaStream_t stream) {
+// W1 x for rows already staged in c->zcat as [hi | lo] halves: slices [plan.k_splits][rows_pad][head_cols_pad] in
+// c->head_partial
+int run_projection_staged(egtp_ctx* c, const egtp_head* head, int rows, int32_t* status, cudaStream_t stream,
+                          LmheadPlan* plan_out) {
   const HeadArgs ha = head_args(head);
   const int64_t rows_pad = (static_cast<int64_t>(rows) + kTileM - 1) / kTileM * kTileM;
   const int64_t cols_pad = (static_cast<int64_t>(ha.m_h) + 255) / 256 * 256;
@@ -286,15 +287,21 @@ int run_head_staged(egtp_ctx* c, const egtp_head* head, int rows, float* y, floa
   LmheadMaps maps;
   maps.hidden = &map_a;
   maps.w = maps.w_tile = maps.w1 = maps.w1_tile = &map_c;
-  {
-    LaunchScope ls(c, EGTP_K_HEAD_HIDDEN, stream);
-    EGTP_CUDA_TRY(launch_lmhead_entropy(plan, false, maps, rows, 0, nullptr, status, stream, c->head_partial));
-  }
-  {
-    LaunchScope ls(c, EGTP_K_HEAD_OUT, stream);
-    EGTP_CUDA_TRY(launch_head_out(ha, c->head_partial, rows, plan.k_splits, y, phat, status, stream,
-                                  plan.rows_pad * static_cast<int64_t>(plan.head_cols_pad), plan.head_cols_pad));
-  }
+  LaunchScope ls(c, EGTP_K_HEAD_HIDDEN, stream);
+  EGTP_CUDA_TRY(launch_lmhead_entropy(plan, false, maps, rows, 0, nullptr, status, stream, c->head_partial));
+  *plan_out = plan;
+  return EGTP_OK;
+}
+
+// y = head(x) for rows already staged in c->zcat
+int run_head_staged(egtp_ctx* c, const egtp_head* head, int rows, float* y, float* phat, int32_t* status,
+                    cudaStream_t stream) {
+  LmheadPlan plan;
+  int rc = run_projection_staged(c, head, rows, status, stream, &plan);
+  if (rc != EGTP_OK) return rc;
+  LaunchScope ls(c, EGTP_K_HEAD_OUT, stream);
+  EGTP_CUDA_TRY(launch_head_out(head_args(head), c->head_partial, rows, plan.k_splits, y, phat, status, stream,
+                                plan.rows_pad * static_cast<int64_t>(plan.head_cols_pad), plan.head_cols_pad));
   return EGTP_OK;
 }
 
@@ -351,8 +358,26 @@ int check_plp_common(const egtp_ctx* c, const plp_state* st, const egtp_head* he
 // out[r] = W1 x[r] for rows of fp32 vectors x (layer 1 of the head without bias and ReLU), in row chunks that fit
 // the split-K workspace.
 int project_rows(egtp_ctx* c, const egtp_head* head, const float* x, int64_t ldx, int rows, float* out, int64_t ld_out,
-                 const int32_t* status, cudaStream_t stream) {
+                 int32_t* status, cudaStream_t stream) {
   const HeadArgs ha = head_args(head);
+  if (head_on_tensor_cores(c, head, 1) && ldx % 4 == 0 && reinterpret_cast<uintptr_t>(x) % 16 == 0) {
+    // tensor cores, max_batch rows at a time through the [hi | lo] staging buffer
+    for (int r0 = 0; r0 < rows; r0 += c->max_batch) {
+      const int n = std::min<int>(c->max_batch, rows - r0);
+      {
+        LaunchScope ls(c, EGTP_K_HEAD_HIDDEN, stream);
+        EGTP_CUDA_TRY(launch_split_hi_lo(x + static_cast<int64_t>(r0) * ldx, ldx, n, ha.d, c->zcat, status, stream));
+      }
+      LmheadPlan plan;
+      int rc = run_projection_staged(c, head, n, status, stream, &plan);
+      if (rc != EGTP_OK) return rc;
+      LaunchScope ls(c, EGTP_K_HEAD_OUT, stream);
+      EGTP_CUDA_TRY(launch_head_partial_sum(c->head_partial, n, plan.k_splits, ha.m_h, out + static_cast<int64_t>(r0) * ld_out,
+                                            ld_out, status, stream,
+                                            plan.rows_pad * static_cast<int64_t>(plan.head_cols_pad), plan.head_cols_pad));
+    }
+    return EGTP_OK;
+  }
   const int chunk = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(rows, c->head_partial_floats / ha.m_h)));
   for (int r0 = 0; r0 < rows; r0 += chunk) {
     const int n = std::min(chunk, rows - r0);
@@ -360,11 +385,11 @@ int project_rows(egtp_ctx* c, const egtp_head* head, const float* x, int64_t ldx
     if (splits <= 0) return EGTP_ERR_CAPACITY;
     {
       LaunchScope ls(c, EGTP_K_HEAD_HIDDEN, stream);
-      EGTP_CUDA_TRY(launch_head_hidden(ha, x + r0 * ldx, ldx, n, splits, c->head_partial, status, stream));
+      EGTP_CUDA_TRY(launch_head_hidden(ha, x + static_cast<int64_t>(r0) * ldx, ldx, n, splits, c->head_partial, status, stream));
     }
     {
       LaunchScope ls(c, EGTP_K_HEAD_OUT, stream);
-      EGTP_CUDA_TRY(launch_head_partial_sum(c->head_partial, n, splits, ha.m_h, out + r0 * ld_out, ld_out, status, stream));
+      EGTP_CUDA_TRY(launch_head_partial_sum(c->head_partial, n, splits, ha.m_h, out + static_cast<int64_t>(r0) * ld_out, ld_out, status, stream));
     }
   }
   return EGTP_OK;
@@ -392,7 +417,7 @@ bool plp_bound_tail_route(const egtp_ctx* c, const plp_state* st, int hidden_dty
 
 // P = W1 acc if it is stale, and W1 src_pooled for rows that restart from EGTP rows
 int plp_bound_prepare(egtp_ctx* c, plp_state* st, const egtp_head* head, const int32_t* reset_src,
-                      const float* src_pooled, int n_src, const int32_t* status, cudaStream_t stream) {
+                      const float* src_pooled, int n_src, int32_t* status, cudaStream_t stream) {
   if (!st->proj_valid) {
     int rc = project_rows(c, head, st->acc, st->d, st->num_slots, st->proj, head->m_h, status, stream);
     if (rc != EGTP_OK) return rc;

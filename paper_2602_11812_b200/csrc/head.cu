@@ -151,16 +151,19 @@ head_out_kernel(const float* __restrict__ partial, int64_t split_stride, int64_t
 // out[r][j] = sum over splits of partial[split][r][j], added in split order: the projection W1 x of rows x
 // that are not pooled vectors (the running sums of a PLP state bound to a head).
 __global__ void __launch_bounds__(256)
-head_partial_sum_kernel(const float* __restrict__ partial, int rows, int splits, int m_h, float* __restrict__ out,
-                        int64_t ld_out, const int32_t* __restrict__ status) {
+head_partial_sum_kernel(const float* __restrict__ partial, int64_t split_stride, int64_t row_stride, int rows,
+                        int splits, int m_h, float* __restrict__ out, int64_t ld_out,
+                        const int32_t* __restrict__ status) {
   if (*status != 0) return;
   const int64_t n = static_cast<int64_t>(rows) * m_h;
   for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < n;
        i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
-    float v = 0.f;
-    for (int s = 0; s < splits; ++s) v += __ldg(partial + s * n + i);
     const int64_t r = i / m_h;
-    out[r * ld_out + (i - r * m_h)] = v;
+    const int64_t j = i - r * m_h;
+    const float* pj = partial + r * row_stride + j;
+    float v = 0.f;
+    for (int s = 0; s < splits; ++s) v += __ldg(pj + s * split_stride);
+    out[r * ld_out + j] = v;
   }
 }
 
@@ -234,10 +237,14 @@ cudaError_t launch_head_out(const HeadArgs& h, const float* partial, int rows, i
 }
 
 cudaError_t launch_head_partial_sum(const float* partial, int rows, int splits, int m_h, float* out, int64_t ld_out,
-                                    const int32_t* status, cudaStream_t stream) {
+                                    const int32_t* status, cudaStream_t stream, int64_t split_stride,
+                                    int64_t row_stride) {
+  if (row_stride == 0) row_stride = m_h;
+  if (split_stride == 0) split_stride = static_cast<int64_t>(rows) * m_h;
   const int64_t n = static_cast<int64_t>(rows) * m_h;
   const int blocks = static_cast<int>(std::min<int64_t>(1184, (n + 255) / 256));
-  head_partial_sum_kernel<<<std::max(1, blocks), 256, 0, stream>>>(partial, rows, splits, m_h, out, ld_out, status);
+  head_partial_sum_kernel<<<std::max(1, blocks), 256, 0, stream>>>(partial, split_stride, row_stride, rows, splits, m_h, out,
+                                                                  ld_out, status);
   return cudaGetLastError();
 }
 

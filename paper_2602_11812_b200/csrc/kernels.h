@@ -141,8 +141,10 @@ cudaError_t launch_split_hi_lo(const float* x, int64_t ldx, int rows, int d, voi
                                cudaStream_t stream);
 
 // out[r][j] = sum_s partial[s][r][j] (split order): W1 x for rows x that are not pooled vectors
+// (strides as in launch_head_out)
 cudaError_t launch_head_partial_sum(const float* partial, int rows, int splits, int m_h, float* out, int64_t ld_out,
-                                    const int32_t* status, cudaStream_t stream);
+                                    const int32_t* status, cudaStream_t stream, int64_t split_stride = 0,
+                                    int64_t row_stride = 0);
 
 // ---- self-test of the bounded wait (a wait on a barrier nobody signals must end with an error status)
 cudaError_t launch_wait_timeout_selftest(uint64_t limit_ns, int32_t* status, cudaStream_t stream);

@@ -86,8 +86,8 @@ def test_plp_step_from_logits_matches_oracle_and_plp_step(ctx, bind, slots, m_h)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     # per step: entropy from logits + update + head layer 1 + head output, and the 4 kernels of plp_step; bound:
-    # entropy from logits + projection + fused update (and 2 launches once for the projection of the empty state)
-    assert egtp.egtp_launch_count(ctx) - n0 == ((3 + 4) * steps + 2 if bind else (4 + 4) * steps)
+    # entropy from logits + projection + fused update (and 3 launches once for the projection of the empty state: halves, GEMM, sum)
+    assert egtp.egtp_launch_count(ctx) - n0 == ((3 + 4) * steps + 3 if bind else (4 + 4) * steps)
     # oracle on exactly the logits the kernel read (bf16-rounded), followed through the token lists
     H_ref = np.stack([orc.entropy_from_logits(x.astype(np.float64)) for x in logits_all])
     follow = [0, 64, slots - 1]

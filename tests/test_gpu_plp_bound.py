@@ -61,8 +61,8 @@ def test_bound_decode_loop_matches_oracle(ctx, slots, V, m_h):
     wl = gen.config_plp_decode(slots=slots, steps=12, d=256, V=V, m_h=m_h, mu=1.5, sigma=0.8)
     assert (wl.reset_src[1:] == gen.RESET_EMPTY).sum() > 10
     st, H, z, y, launches = _run(ctx, wl)
-    # first step projects the (empty) state: 2 launches; then 2 launches per step (LM head, fused update + head)
-    assert launches == 2 + 2 * wl.steps
+    # first step projects the (empty) state: 3 launches (halves, GEMM, sum); then 2 launches per step (LM head, fused update + head)
+    assert launches == 3 + 2 * wl.steps
     follow = sorted({0, 1, slots // 2, slots - 2, slots - 1})
     ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=follow)
     _compare(H, z, y, ref, follow)
@@ -85,7 +85,7 @@ def test_bound_decode_loop_in_single_cta_mode(ctx):
         st, H, z, y, launches = _run(ctx, wl)
     finally:
         egtp.egtp_set_lmhead_mode(ctx, egtp.EGTP_LMHEAD_AUTO)
-    assert launches == 2 + 2 * wl.steps
+    assert launches == 3 + 2 * wl.steps
     follow = [0, 127, 128, 189]
     ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=follow)
     _compare(H, z, y, ref, follow)
