@@ -207,3 +207,41 @@ def test_bound_projection_does_not_drift_over_a_long_sequence(ctx):
     for t in (0, 199, 399):
         gu.assert_pooled_close(z[t, follow], ref["z"][t])
     egtp.plp_state_destroy(st)
+
+
+def test_two_contexts_on_two_streams_do_not_disturb_each_other():
+    # two contexts (each with its own workspace) driven from two CUDA streams at the same time give bit for bit
+    # what each gives alone: the library keeps no per-call state outside the context
+    wl = gen.config_plp_decode(slots=140, steps=6, d=256, V=6000, m_h=64, mu=2.0, sigma=0.5)
+    W = gu.dev_tensor(wl.W, "bf16"); lm = egtp.make_lm_head(W)
+    head = gu.DeviceHead(wl.head, "bf16")
+    hs = gu.dev_tensor(wl.hidden_steps.reshape(-1, 256), "bf16").reshape(wl.steps, 140, 256)
+    reset = torch.from_numpy(wl.reset_src).cuda()
+
+    def run(ctxs, streams):
+        ys, sts, stat = [], [], []
+        for c in ctxs:
+            st = egtp.plp_state_create(c, 140, 256)
+            egtp.plp_state_bind_head(st, head.c)
+            sts.append(st); ys.append(torch.zeros(wl.steps, 140, device="cuda"))
+            stat.append(torch.zeros(1, device="cuda", dtype=torch.int32))
+        torch.cuda.synchronize()
+        for t in range(wl.steps):
+            for k, c in enumerate(ctxs):
+                with torch.cuda.stream(streams[k]):
+                    egtp.plp_step(c, sts[k], lm, head.c, hs[t], reset_src=reset[t], yrem_out=ys[k][t], status_dev=stat[k])
+        torch.cuda.synchronize()
+        for st in sts:
+            egtp.plp_state_destroy(st)
+        assert all(int(s.item()) == 0 for s in stat)
+        return ys
+
+    c1 = egtp.egtp_create(0, max_tokens=1024, max_batch=256, max_d=256, max_V=8192)
+    c2 = egtp.egtp_create(0, max_tokens=1024, max_batch=256, max_d=256, max_V=8192)
+    try:
+        alone = run([c1], [torch.cuda.current_stream()])[0]
+        s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+        both = run([c1, c2], [s1, s2])
+    finally:
+        egtp.egtp_destroy(c1); egtp.egtp_destroy(c2)
+    assert torch.equal(both[0], alone) and torch.equal(both[1], alone)
