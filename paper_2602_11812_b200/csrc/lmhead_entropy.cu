@@ -16,10 +16,16 @@
 //               one row per thread, 128 columns per tile, tcgen05.ld in 32-column pieces
 // A work unit is (row block, vocabulary chunk); units are ordered so that CTAs running at the
 // same time share W tiles (same chunk, neighbouring row blocks) and hidden tiles stay in L2.
-// Three tile shapes: prompts (128 rows x 256 columns per tile, tensor-bound), and two decode shapes
+// One-CTA tile shapes: prompts (128 rows x 256 columns per tile, tensor-bound), and two decode shapes
 // for <= 128 and <= 256 rows, where the step is bound by streaming W from HBM once: every SM
 // gets its own vocabulary range (equal to within 32 columns) and, for 129..256 rows, multiplies
-// both row tiles against each W tile it loads.
+// both row tiles against each W tile it loads.  The CTA-pair kernel further down (tcgen05.mma.cta_group::2)
+// is the default for 129..256 rows (256 x 512 tiles) and an option for prompts (256 x 256 tiles).
+//
+// Two more uses of the same machinery (prediction head, Sec. 3.2; PLP, Sec. 3.3): with kFuse the column space
+// continues past the vocabulary with the rows of the head's W1, whose products are written out instead of
+// entering the entropy; and a launch over those head columns alone, with K split over the SMs, is layer 1 of
+// the head for any batch of input rows (bf16 rows, or fp32 rows given as two bf16 halves along K).
 #include "kernels.h"
 #include "sm100_ptx.cuh"
 #include "../../include/egtp.h"
