@@ -1,7 +1,10 @@
 // Prediction head (paper Sec. 3.2, Eq. 6): u = ReLU(W1 z + b1), o = W2 u + b2, then either the
-// scalar o[0] or the expectation of softmax(o) over the bin centres.  A few MB of weights and
-// at most a few thousand rows: plain fp32 FMA on the CUDA cores, register-tiled, split along d
-// so that small batches still fill the GPU; the split partials are added in a fixed order.
+// scalar o[0] or the expectation of softmax(o) over the bin centres.
+// Layer 1 has two forms.  With bf16 weights it runs on the tensor cores: split_hi_lo_kernel writes every fp32
+// input row as two bf16 halves and the LM-head kernel multiplies them against W1 (a launch over the head
+// columns alone, K split over the SMs).  head_hidden_kernel is the CUDA-core form (fp32 weights, and the entry
+// point that works without a context): plain fp32 FMA, register-tiled, split along d so that small batches
+// still fill the GPU.  Either way the split partials are added in a fixed order by head_out_kernel.
 #include "kernels.h"
 #include "head_out.cuh"
 #include "../../include/egtp.h"
