@@ -276,7 +276,7 @@ int run_projection_staged(egtp_ctx* c, const egtp_head* head, int rows, int32_t*
   const HeadArgs ha = head_args(head);
   const int64_t rows_pad = (static_cast<int64_t>(rows) + kTileM - 1) / kTileM * kTileM;
   const int64_t cols_pad = (static_cast<int64_t>(ha.m_h) + 255) / 256 * 256;
-  const int max_splits = static_cast<int>(std::min<int64_t>(16, c->head_partial_floats / (rows_pad * cols_pad)));
+  const int max_splits = static_cast<int>(std::min<int64_t>(8, c->head_partial_floats / (rows_pad * cols_pad)));
   if (max_splits < 1) return EGTP_ERR_CAPACITY;
   const LmheadPlan plan = make_headproj_plan(rows, ha.d, ha.m_h, 2, c->num_sms, max_splits, /*a_repeats=*/2);
   CUtensorMap map_a, map_c;
