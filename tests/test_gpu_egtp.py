@@ -272,6 +272,38 @@ def test_many_tokens_small_model_64bit_indexing():
     gu.assert_length_close(res["yhat"], y_ref)
 
 
+def test_fewer_than_16_rows_in_fp32_and_with_a_row_stride(ctx):
+    # batches of fewer than 16 rows go through a zero-padded 16-row staging buffer: fp32 rows (tf32 tensor-core path),
+    # and bf16 rows that are 3 * d elements apart in memory
+    rng = np.random.default_rng(77)
+    d, V = 64, 500
+    hidden = (rng.standard_normal((7, d)) * 1.5).astype(np.float32)
+    W = (rng.standard_normal((V, d)) * 0.3).astype(np.float32)
+    head = gen.make_head(6, d, 24, 1, "f32")
+    wl = gen.EgtpWorkload("few_f32", "f32", hidden, gen.offsets_from_lengths([3, 4]), W, head)
+    res = gu.run_egtp(ctx, wl)
+    # fp32 operands enter the tensor core as tf32 (mantissa cut to 10 bits); these logits are large enough for
+    # that to show, so the oracle gets the cut operands and must then agree to the usual tolerance
+    cut = lambda a: (a.view(np.uint32) & np.uint32(0xFFFFE000)).view(np.float32)
+    ref = orc.egtp_predict(hidden, wl.offsets, W, head)
+    assert res["status"] == 0 and np.array_equal(res["seg_id"], ref["seg_id"])
+    gu.assert_entropy_close(res["H"], orc.token_entropy(cut(hidden), cut(W)))
+    assert np.abs(res["H"] - ref["H"]).max() <= 5e-3
+    gu.assert_length_close(res["yhat"], ref["yhat"])
+    hb = gen.round_to_bf16(hidden); Wb = gen.round_to_bf16(W)
+    wide = torch.zeros(7, 3 * d, device="cuda", dtype=torch.bfloat16)
+    wide[:, :d] = gu.dev_tensor(hb, "bf16")
+    wide[:, d:] = 9.0                                            # poison beside the rows
+    H = torch.zeros(7, device="cuda")
+    status = torch.zeros(1, device="cuda", dtype=torch.int32)
+    lm = egtp.make_lm_head(gu.dev_tensor(Wb, "bf16"))
+    off = torch.tensor([0, 7], dtype=torch.int32, device="cuda")
+    egtp.egtp_predict(ctx, lm, None, wide[:, :d], off, 1, 7, 1.0, H_out=H, status_dev=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    gu.assert_entropy_close(H.cpu().numpy().astype(np.float64), orc.token_entropy(hb, Wb))
+
+
 @pytest.mark.parametrize("T,d,V", [(3, 16, 40), (129, 32, 300), (256, 48, 1000), (257, 80, 1000), (128, 272, 31), (1, 2048, 9)])
 def test_small_and_boundary_shapes(ctx, T, d, V):
     # row counts on both sides of the 128 / 256-row launch shapes, hidden sizes that are not multiples of
