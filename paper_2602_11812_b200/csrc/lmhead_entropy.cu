@@ -183,7 +183,8 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   // one copy; the same maps when kBBox == kBN)
   constexpr int kABytes = kMT * kTileM * kRowBytes;
   constexpr int kBBytes = kBN * kRowBytes;
-  constexpr int kStageBytes = kABytes + kBBytes;
+  // fp32 operands: a stage holds the tiles twice, as loaded (turned into their high parts in place) and their low parts
+  constexpr int kStageBytes = (kTf32 ? 2 : 1) * (kABytes + kBBytes);
   constexpr int kAccCols = kMT * kBN;                 // TMEM columns of one accumulator set
   constexpr int kNumAcc = kTmemCols / kAccCols;       // 2: epilogue of tile j overlaps MMAs of tile j+1; 1 for 256 x 256 tiles
   constexpr int kSpan = kAccCols / kEpiSplit;         // TMEM columns one epilogue warp reads per tile
@@ -299,7 +300,76 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if constexpr (kTf32) {
+      // fp32 operands.  kind::tf32 keeps 10 mantissa bits of each operand, which alone would cost the entropy
+      // its 1e-3 tolerance once the logits are a few units large.  So every operand x is taken apart as
+      // x = hi + lo, hi = x with its 13 low mantissa bits cleared (exact in tf32), lo = x - hi (exact in fp32, then
+      // cut to tf32 as well), and each k step issues three MMAs: hi.hi + hi.lo + lo.hi (the dropped lo.lo term is
+      // 2^-22 of the product).  The whole warp splits a stage in shared memory once its copy has landed: the high
+      // parts replace the loaded values in place, the low parts go to the second half of the stage, same swizzled
+      // layout, so the same descriptors (plus an offset) address them.  Conversion of stage s+1 overlaps the MMAs of
+      // stage s; this path serves the small fp32 configuration, not the throughput workloads (those are bf16).
+      constexpr int kHalfBytes = kABytes + kBBytes;
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < p.total_units && ok; u += gridDim.x) {
+        const UnitCoord uc = unit_coord(u, p);
+        for (int n0 = uc.col_begin; n0 < uc.col_end && ok; n0 += kBN) {
+          const int ncols = min(kBN, uc.col_end - n0);
+          const uint32_t idesc = kIdescNoN | (static_cast<uint32_t>(ncols >> 3) << 17);
+          ok = __all_sync(0xffffffffu, mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag));
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kAccCols);
+          for (int kb = uc.kb_begin; kb < uc.kb_end; ++kb) {
+            ok = __all_sync(0xffffffffu, mbar_wait(full_bar(stage), phase, abort_flag));
+            if (!ok) break;
+            uint4* hi_p = reinterpret_cast<uint4*>(smem_gen + stage * kStageBytes);
+            uint4* lo_p = reinterpret_cast<uint4*>(smem_gen + stage * kStageBytes + kHalfBytes);
+            for (int i = lane; i < kHalfBytes / 16; i += 32) {
+              const uint4 v = hi_p[i];
+              const uint32_t x[4] = {v.x, v.y, v.z, v.w};
+              uint32_t h[4], l[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                h[q] = x[q] & 0xFFFFE000u;
+                l[q] = __float_as_uint(__uint_as_float(x[q]) - __uint_as_float(h[q])) & 0xFFFFE000u;
+              }
+              hi_p[i] = make_uint4(h[0], h[1], h[2], h[3]);
+              lo_p[i] = make_uint4(l[0], l[1], l[2], l[3]);
+            }
+            fence_proxy_async_shared();      // the MMAs read shared memory through the async proxy
+            __syncwarp();
+            if (lane == 0) {
+              tc_fence_after_sync();
+              const uint32_t a_src = smem_base + stage * kStageBytes;
+              const uint64_t b_hi = umma_desc_k_major_sw128(a_src + kABytes);
+              const uint64_t b_lo = umma_desc_k_major_sw128(a_src + kHalfBytes + kABytes);
+#pragma unroll
+              for (int mt = 0; mt < kMT; ++mt) {
+                const uint64_t a_hi = umma_desc_k_major_sw128(a_src + mt * (kTileM * kRowBytes));
+                const uint64_t a_lo = umma_desc_k_major_sw128(a_src + kHalfBytes + mt * (kTileM * kRowBytes));
+#pragma unroll
+                for (int k = 0; k < kMmaPerStage; ++k) {
+                  umma_ss<true>(d_tmem + mt * kBN, a_lo + 2u * k, b_hi + 2u * k, idesc, (kb != uc.kb_begin || k != 0) ? 1u : 0u);
+                  umma_ss<true>(d_tmem + mt * kBN, a_hi + 2u * k, b_lo + 2u * k, idesc, 1u);
+                  umma_ss<true>(d_tmem + mt * kBN, a_hi + 2u * k, b_hi + 2u * k, idesc, 1u);
+                }
+              }
+              umma_commit(empty_bar(stage));
+            }
+            __syncwarp();
+            if (++stage == kNumStages) { stage = 0; phase ^= 1u; }
+          }
+          if (ok && lane == 0) umma_commit(acc_full_bar(acc));
+          __syncwarp();
+          if (++acc == kNumAcc) { acc = 0; acc_phase ^= 1u; }
+        }
+      }
+    } else if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -683,8 +753,10 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
   }
 }
 
-constexpr int smem_bytes_for(int mt, int bn, int stages) {
-  return stages * (mt * kTileM * kRowBytes + bn * kRowBytes) + kBarrierBytes + 1024;   // + slack for alignment
+// fp32 operands: two stages, each holding its tiles twice (high and low parts)
+constexpr int kF32Stages = 2;
+constexpr int smem_bytes_for(int mt, int bn, int stages, bool f32 = false) {
+  return (f32 ? 2 * kF32Stages : stages) * (mt * kTileM * kRowBytes + bn * kRowBytes) + kBarrierBytes + 1024;   // + slack for alignment
 }
 
 // The three shapes the host chooses from.
@@ -711,8 +783,8 @@ cudaError_t launch_shape(const LmheadPlan& plan, const LmheadMaps& m, const KPar
   auto kernel = lmhead_entropy_kernel<kTf32, kMT, kBN, kBBox, kNumStages, kFuse>;
   const CUtensorMap* c = kFuse ? m.w1 : m.w;
   const CUtensorMap* c_tile = kFuse ? m.w1_tile : m.w_tile;
-  kernel<<<plan.grid, kLmheadThreads, smem_bytes_for(kMT, kBN, kNumStages), stream>>>(*m.hidden, *m.w, *m.w_tile, *c,
-                                                                                     *c_tile, p);
+  kernel<<<plan.grid, kLmheadThreads, smem_bytes_for(kMT, kBN, kNumStages, kTf32), stream>>>(*m.hidden, *m.w, *m.w_tile,
+                                                                                            *c, *c_tile, p);
   return cudaGetLastError();
 }
 
@@ -720,7 +792,7 @@ template <bool kTf32, int kMT, int kBN, int kBBox, int kNumStages, bool kFuse = 
 cudaError_t prepare_shape() {
   auto kernel = lmhead_entropy_kernel<kTf32, kMT, kBN, kBBox, kNumStages, kFuse>;
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              smem_bytes_for(kMT, kBN, kNumStages));
+                              smem_bytes_for(kMT, kBN, kNumStages, kTf32));
 }
 
 // kBBox 128: 256 x 256 tiles (prompt batches); 32: 256 x 512 tiles (decode batches), optionally with head columns
@@ -761,6 +833,8 @@ cudaError_t prepare_pair(int num_sms) {
 #define EGTP_SHAPE_PROMPT 1, 256, 256, 4
 #define EGTP_SHAPE_DECODE1 1, 256, 32, 4
 #define EGTP_SHAPE_DECODE2 2, 256, 32, 3
+#define EGTP_SHAPE_PROMPT_F32 1, 256, 256, kF32Stages
+#define EGTP_SHAPE_DECODE1_F32 1, 256, 32, kF32Stages
 static_assert(kShapePrompt.mt == 1 && kShapePrompt.bn == 256 && kShapePrompt.bbox == 256 && kShapePrompt.stages == 4, "");
 static_assert(kShapeDecode1.mt == 1 && kShapeDecode1.bn == 256 && kShapeDecode1.bbox == 32 && kShapeDecode1.stages == 4, "");
 static_assert(kShapeDecode2.mt == 2 && kShapeDecode2.bn == 256 && kShapeDecode2.bbox == 32 && kShapeDecode2.stages == 3, "");
@@ -775,8 +849,11 @@ LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms
   LmheadPlan pl{};
   // decode batches of 129..256 rows run as CTA pairs on 256 x 512 tiles unless single CTAs are asked for or the
   // device cannot co-schedule the pairs; prompt batches run as pairs only on request (and never with head columns)
-  pl.variant = T <= kTileM ? 1 : (T <= 2 * kTileM ? 2 : 0);
-  const bool pairs_ok = pair_cap > 0 && mode != EGTP_LMHEAD_SINGLE_CTA;
+  // fp32 rows (three tf32 MMAs per k step on operands split in shared memory) have the prompt shape and the
+  // one-row-tile decode shape only, always one CTA per SM
+  const bool f32 = elem_bytes == 4;
+  pl.variant = T <= kTileM ? 1 : ((T <= 2 * kTileM && !f32) ? 2 : 0);
+  const bool pairs_ok = pair_cap > 0 && mode != EGTP_LMHEAD_SINGLE_CTA && !f32;
   if (pl.variant == 2 && pairs_ok) pl.variant = 5;
   if (pl.variant == 0 && pairs_ok && mode == EGTP_LMHEAD_CTA_PAIRS && head_cols == 0) pl.variant = 4;
   const bool pair = pl.variant >= 4;
@@ -794,7 +871,7 @@ LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms
   pl.n_groups += pl.head_cols_pad / sh.col_gran;     // head columns follow the (padded) vocabulary
   pl.rows_pad = static_cast<int64_t>(pl.row_blocks) * pl.rows_per_block;
   pl.k_blocks = static_cast<int>((static_cast<int64_t>(d) * elem_bytes + kRowBytes - 1) / kRowBytes);
-  pl.smem_bytes = pair ? kPairSmemBytes : smem_bytes_for(sh.mt, sh.bn, sh.stages);
+  pl.smem_bytes = pair ? kPairSmemBytes : smem_bytes_for(sh.mt, sh.bn, sh.stages, f32);
   // partial slots a row gets per vocabulary chunk: its tile columns are split over two epilogue
   // warps unless the two warps serve two different row tiles
   const int slots_per_chunk = pl.variant == 2 ? 1 : kEpiSplit;
@@ -897,9 +974,8 @@ cudaError_t lmhead_prepare_device() {
   if ((e = prepare_shape<false, EGTP_SHAPE_PROMPT>()) != cudaSuccess) return e;
   if ((e = prepare_shape<false, EGTP_SHAPE_DECODE1>()) != cudaSuccess) return e;
   if ((e = prepare_shape<false, EGTP_SHAPE_DECODE2>()) != cudaSuccess) return e;
-  if ((e = prepare_shape<true, EGTP_SHAPE_PROMPT>()) != cudaSuccess) return e;
-  if ((e = prepare_shape<true, EGTP_SHAPE_DECODE1>()) != cudaSuccess) return e;
-  if ((e = prepare_shape<true, EGTP_SHAPE_DECODE2>()) != cudaSuccess) return e;
+  if ((e = prepare_shape<true, EGTP_SHAPE_PROMPT_F32>()) != cudaSuccess) return e;
+  if ((e = prepare_shape<true, EGTP_SHAPE_DECODE1_F32>()) != cudaSuccess) return e;
   if ((e = prepare_shape<false, EGTP_SHAPE_PROMPT, true>()) != cudaSuccess) return e;
   if ((e = prepare_shape<false, EGTP_SHAPE_DECODE1, true>()) != cudaSuccess) return e;
   if ((e = prepare_shape<false, EGTP_SHAPE_DECODE2, true>()) != cudaSuccess) return e;
@@ -909,9 +985,7 @@ cudaError_t lmhead_prepare_device() {
   g_pair_workers_max = 0;
   if ((e = prepare_pair<false, 128>(num_sms)) != cudaSuccess) return e;
   if ((e = prepare_pair<false, 32>(num_sms)) != cudaSuccess) return e;
-  if ((e = prepare_pair<true, 128>(num_sms)) != cudaSuccess) return e;
-  if ((e = prepare_pair<false, 32, true>(num_sms)) != cudaSuccess) return e;
-  return prepare_pair<true, 32>(num_sms);
+  return prepare_pair<false, 32, true>(num_sms);
 }
 
 cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const LmheadMaps& maps, int64_t T, int V,
@@ -951,11 +1025,9 @@ cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const Lmhea
   }
   if (tf32) {
     switch (plan.variant) {
-      case 1: return launch_shape<true, EGTP_SHAPE_DECODE1>(plan, maps, p, stream);
-      case 2: return launch_shape<true, EGTP_SHAPE_DECODE2>(plan, maps, p, stream);
-      case 4: return launch_pair<true, 128>(plan, maps, p, stream);
-      case 5: return launch_pair<true, 32>(plan, maps, p, stream);
-      default: return launch_shape<true, EGTP_SHAPE_PROMPT>(plan, maps, p, stream);
+      case 0: return launch_shape<true, EGTP_SHAPE_PROMPT_F32>(plan, maps, p, stream);
+      case 1: return launch_shape<true, EGTP_SHAPE_DECODE1_F32>(plan, maps, p, stream);
+      default: return cudaErrorInvalidValue;     // the planner gives fp32 rows no other shape
     }
   }
   switch (plan.variant) {

@@ -18,7 +18,53 @@ namespace egtp {
 namespace {
 
 constexpr int kLogitsThreads = 128;
+constexpr int kLogitsBlocksPerSm = 7;   // 72 registers per thread at most: 28 warps per SM
 constexpr float kLog2e = 1.4426950408889634f;
+
+// Eight consecutive logits as they come out of memory.  bf16 values stay packed until they are consumed: the
+// maximum of the eight is taken on the packed pairs (exact: the maximum of bf16 numbers is one of them), and
+// a value is widened to fp32 (a shift or a mask) only where the exponential needs it.
+template <typename T>
+struct Vec8;
+template <>
+struct Vec8<__nv_bfloat16> {
+  uint4 q;
+  __device__ __forceinline__ void load(const __nv_bfloat16* p) { q = __ldcs(reinterpret_cast<const uint4*>(p)); }   // streamed once
+  __device__ __forceinline__ float vmax() const {
+    const __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&q.x), *reinterpret_cast<const __nv_bfloat162*>(&q.y));
+    const __nv_bfloat162 b = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&q.z), *reinterpret_cast<const __nv_bfloat162*>(&q.w));
+    const __nv_bfloat162 c = __hmax2(a, b);
+    const uint32_t w = *reinterpret_cast<const uint32_t*>(&c);
+    return fmaxf(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+  }
+  __device__ __forceinline__ void get(float (&v)[8]) const {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  }
+};
+template <>
+struct Vec8<float> {
+  float4 a, b;
+  __device__ __forceinline__ void load(const float* p) {
+    a = __ldcs(reinterpret_cast<const float4*>(p));
+    b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+  }
+  __device__ __forceinline__ float vmax() const {
+    return fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w)));
+  }
+  __device__ __forceinline__ void get(float (&v)[8]) const {
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  }
+};
+
+// vectors of eight logits a thread has in flight while it folds the previous ones: 64 bytes either way
+template <typename T>
+constexpr int kVecPerBatch = sizeof(T) == 2 ? 4 : 2;
 
 // Running state of one thread: max m and four independent (s, t2) accumulators (short dependency chains).
 struct ThreadState {
@@ -30,8 +76,7 @@ struct ThreadState {
 #pragma unroll
     for (int i = 0; i < 4; ++i) { s[i] = 0.f; t[i] = 0.f; }
   }
-  __device__ __forceinline__ void fold8(const float (&x)[8]) {
-    const float cmax = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])), fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
+  __device__ __forceinline__ void raise_max(float cmax) {
     if (cmax > m) {
       const float dm = (m - cmax) * kLog2e;
       const float r = ex2_approx(dm);
@@ -41,43 +86,27 @@ struct ThreadState {
         s[i] *= r;
       }
       m = cmax;
-    }
-    const float neg_m_l2 = -m * kLog2e;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float y = fmaf(x[j], kLog2e, neg_m_l2);
-      const float e = ex2_approx(y);
-      s[j & 3] += e;
-      t[j & 3] = fmaf(e, y, t[j & 3]);
     }
   }
-  // 32 values at once: one running-max update, then 32 independent exponentials (more work in flight)
-  __device__ __forceinline__ void fold32(const float (&a)[8], const float (&b)[8], const float (&c)[8],
-                                         const float (&d)[8]) {
-    float ma = a[0], mb = b[0], mc = c[0], md = d[0];
+  // kN vectors of eight values at once: one running-max update, then 8 kN independent exponentials
+  template <typename T, int kN>
+  __device__ __forceinline__ void fold(const Vec8<T> (&x)[kN]) {
+    float cmax = x[0].vmax();
 #pragma unroll
-    for (int j = 1; j < 8; ++j) {
-      ma = fmaxf(ma, a[j]); mb = fmaxf(mb, b[j]); mc = fmaxf(mc, c[j]); md = fmaxf(md, d[j]);
-    }
-    const float cmax = fmaxf(fmaxf(ma, mb), fmaxf(mc, md));
-    if (cmax > m) {
-      const float dm = (m - cmax) * kLog2e;
-      const float r = ex2_approx(dm);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        t[i] = r * fmaf(dm, s[i], t[i]);
-        s[i] *= r;
-      }
-      m = cmax;
-    }
+    for (int u = 1; u < kN; ++u) cmax = fmaxf(cmax, x[u].vmax());
+    raise_max(cmax);
     const float neg_m_l2 = -m * kLog2e;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float ya = fmaf(a[j], kLog2e, neg_m_l2), yb = fmaf(b[j], kLog2e, neg_m_l2);
-      const float yc = fmaf(c[j], kLog2e, neg_m_l2), yd = fmaf(d[j], kLog2e, neg_m_l2);
-      const float ea = ex2_approx(ya), eb = ex2_approx(yb), ec = ex2_approx(yc), ed = ex2_approx(yd);
-      s[0] += ea; s[1] += eb; s[2] += ec; s[3] += ed;
-      t[0] = fmaf(ea, ya, t[0]); t[1] = fmaf(eb, yb, t[1]); t[2] = fmaf(ec, yc, t[2]); t[3] = fmaf(ed, yd, t[3]);
+    for (int u = 0; u < kN; ++u) {
+      float v[8];
+      x[u].get(v);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float y = fmaf(v[j], kLog2e, neg_m_l2);
+        const float e = ex2_approx(y);
+        s[(u + j) & 3] += e;
+        t[(u + j) & 3] = fmaf(e, y, t[(u + j) & 3]);
+      }
     }
   }
   __device__ __forceinline__ EntropyPartial total() const {
@@ -86,34 +115,18 @@ struct ThreadState {
 };
 
 template <typename T>
-__device__ __forceinline__ void load8_logits(const T* p, float (&v)[8]);
-template <>
-__device__ __forceinline__ void load8_logits<__nv_bfloat16>(const __nv_bfloat16* p, float (&v)[8]) {
-  const uint4 q = __ldcs(reinterpret_cast<const uint4*>(p));   // streamed once: do not keep in cache
-  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    v[2 * i] = __uint_as_float(w[i] << 16);
-    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-  }
-}
-template <>
-__device__ __forceinline__ void load8_logits<float>(const float* p, float (&v)[8]) {
-  const float4 a = __ldcs(reinterpret_cast<const float4*>(p));
-  const float4 b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
-  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
-  v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
-}
-template <typename T>
 __device__ __forceinline__ float to_float(T v);
 template <>
 __device__ __forceinline__ float to_float<float>(float v) { return v; }
 template <>
 __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
 
-// block (split, row): columns [split * cols_per_split, ...) of one row
+// block (split, row): columns [split * cols_per_split, ...) of one row.  The loads of the next batch of vectors are
+// issued before the current batch is folded, so that every warp keeps memory requests in flight while it computes
+// (one ex2 and about five other instructions per logit: the arithmetic alone takes most of the time the memory
+// system needs to deliver the row).
 template <typename T>
-__global__ void __launch_bounds__(kLogitsThreads)
+__global__ void __launch_bounds__(kLogitsThreads, kLogitsBlocksPerSm)
 logits_entropy_kernel(const T* __restrict__ logits, int64_t ldl, int V, int cols_per_split, int splits,
                       float* __restrict__ partials, const int32_t* __restrict__ status) {
   if (*status != 0) return;
@@ -122,29 +135,39 @@ logits_entropy_kernel(const T* __restrict__ logits, int64_t ldl, int V, int cols
   const int64_t row = blockIdx.y;
   const int c0 = split * cols_per_split;
   const int c1 = min(V, c0 + cols_per_split);
-  const T* base = logits + row * ldl;
+  const T* base = logits + row * ldl + c0;
   ThreadState ts;
   ts.init();
   const int n_vec = max(0, c1 - c0) >> 3;                       // cols_per_split is a multiple of 8
-  int v = threadIdx.x;
-  for (; v + 3 * kLogitsThreads < n_vec; v += 4 * kLogitsThreads) {   // four 16-byte loads in flight
-    float x0[8], x1[8], x2[8], x3[8];
-    load8_logits<T>(base + c0 + 8 * v, x0);
-    load8_logits<T>(base + c0 + 8 * (v + kLogitsThreads), x1);
-    load8_logits<T>(base + c0 + 8 * (v + 2 * kLogitsThreads), x2);
-    load8_logits<T>(base + c0 + 8 * (v + 3 * kLogitsThreads), x3);
-    ts.fold32(x0, x1, x2, x3);
+  constexpr int kN = kVecPerBatch<T>;
+  constexpr int kBatch = kN * kLogitsThreads;                    // vectors per block and batch
+  const int n_batches = n_vec / kBatch;
+  const T* p = base + 8 * threadIdx.x;
+  Vec8<T> cur[kN], nxt[kN];
+  if (n_batches > 0) {
+#pragma unroll
+    for (int u = 0; u < kN; ++u) cur[u].load(p + 8 * u * kLogitsThreads);
   }
-  for (; v < n_vec; v += kLogitsThreads) {
-    float x0[8];
-    load8_logits<T>(base + c0 + 8 * v, x0);
-    ts.fold8(x0);
+  for (int b = 0; b < n_batches; ++b) {
+    p += 8 * kBatch;
+    if (b + 1 < n_batches) {
+#pragma unroll
+      for (int u = 0; u < kN; ++u) nxt[u].load(p + 8 * u * kLogitsThreads);
+    }
+    ts.fold<T, kN>(cur);
+#pragma unroll
+    for (int u = 0; u < kN; ++u) cur[u] = nxt[u];
+  }
+  for (int v = n_batches * kBatch + threadIdx.x; v < n_vec; v += kLogitsThreads) {
+    Vec8<T> one[1];
+    one[0].load(base + 8 * v);
+    ts.fold<T, 1>(one);
   }
   EntropyPartial st = ts.total();
   // ragged tail of the row (fewer than 8 columns), handled by one thread
   if (threadIdx.x == 0) {
     for (int c = c0 + 8 * n_vec; c < c1; ++c) {
-      const EntropyPartial one = {to_float<T>(base[c]), 1.f, 0.f};
+      const EntropyPartial one = {to_float<T>(logits[row * ldl + c]), 1.f, 0.f};
       st = combine_partials(st, one);
     }
   }
@@ -163,9 +186,9 @@ logits_entropy_kernel(const T* __restrict__ logits, int64_t ldl, int V, int cols
 }  // namespace
 
 int logits_entropy_pick_splits(int64_t rows, int V, int num_sms) {
-  // One wave of blocks: about seven 128-thread blocks per SM fit at once, and every thread should see a few
+  // One wave of blocks: seven 128-thread blocks per SM fit at once (kLogitsBlocksPerSm), and every thread should see a few
   // hundred logits so that the per-block combine is amortised; never less than 2K columns per block.
-  int64_t splits = std::max<int64_t>(1, (7ll * num_sms) / std::max<int64_t>(rows, 1));
+  int64_t splits = std::max<int64_t>(1, (static_cast<int64_t>(kLogitsBlocksPerSm) * num_sms) / std::max<int64_t>(rows, 1));
   splits = std::min<int64_t>(splits, std::max(1, V / 2048));
   return static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(splits, 128)));
 }

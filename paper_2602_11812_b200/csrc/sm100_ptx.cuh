@@ -83,6 +83,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const void* tenso
       : "memory");
 }
 
+// Orders this thread's ordinary (generic-proxy) writes to shared memory before later reads of that memory through
+// the async proxy (TMA, tcgen05.mma operands).
+__device__ __forceinline__ void fence_proxy_async_shared() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
 __device__ __forceinline__ void tma_prefetch_descriptor(const void* tensor_map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tensor_map)) : "memory");
 }

@@ -236,6 +236,19 @@ def make_head(seed: int, d: int, m_h: int, d_out: int, dtype: str, mode: int = H
     return HeadParams(W1=W1, b1=b1, W2=W2, b2=b2, mode=mode, centres=centres)
 
 
+def scaled_head(head: HeadParams, dtype: str, gain: float = 64.0, shift: float = 300.0) -> HeadParams:
+    """The same scalar head with its output layer rescaled: W2 * gain (kept representable in `dtype`), b2 + shift.
+
+    A Xavier-initialised head predicts a fraction of a token, so an absolute tolerance of half a token says
+    nothing about it; rescaled like this it predicts a few hundred tokens, the range real lengths live in.
+    """
+    if head.mode != HEAD_SCALAR:
+        raise ValueError("only scalar heads are rescaled (a bins head already predicts in token units)")
+    W2 = _maybe_round(head.W2 * np.float32(gain), dtype)
+    b2 = (head.b2 + np.float32(shift)).astype(np.float32)
+    return HeadParams(W1=head.W1, b1=head.b1, W2=W2, b2=b2, mode=head.mode, centres=head.centres)
+
+
 def make_egtp(name: str, seed: int, lengths, d: int, V: int, dtype: str, m_h: int, d_out: int = 1,
               mode: int = HEAD_SCALAR, outlier_frac: float = 0.0, outlier_gain: float = 1.0,
               alpha: float = 1.0, W: Optional[np.ndarray] = None) -> EgtpWorkload:

@@ -99,5 +99,7 @@ def test_plp_step_from_logits_matches_oracle_and_plp_step(ctx, bind, slots, m_h)
     gu.assert_length_close(ya_n[:, follow].ravel(), ref["yrem"].ravel())
     # and against the GEMM-fused path: bf16 rounding of the logits moves the entropy by well under the tolerance
     assert np.abs(Ha_n - Hb.cpu().numpy()).max() < 5e-3
-    gu.assert_length_close(ya_n.ravel(), yb.cpu().numpy().astype(np.float64).ravel())
+    # (the two paths read different inputs, rounded and unrounded logits: close, not equal to tolerance)
+    yb_n = yb.cpu().numpy().astype(np.float64)
+    assert np.abs(ya_n - yb_n).max() <= 2e-3 * max(1.0, np.abs(yb_n).max())
     egtp.plp_state_destroy(st_a); egtp.plp_state_destroy(st_b)

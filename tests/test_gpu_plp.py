@@ -18,11 +18,11 @@ def ctx():
     egtp.egtp_destroy(c)
 
 
-def _run_plp(ctx, wl: gen.PlpWorkload, src=None, slot_ids=None, num_slots=None):
+def _run_plp(ctx, wl: gen.PlpWorkload, src=None, slot_ids=None, num_slots=None, head=None):
     """All steps of a PLP workload through plp_step; returns H, z, yrem as float64 arrays [steps, slots(, d)]."""
     steps, slots, d = wl.steps, wl.slots, wl.d
     W = gu.dev_tensor(wl.W, wl.dtype)
-    head = gu.DeviceHead(wl.head, wl.dtype)
+    head = gu.DeviceHead(wl.head if head is None else head, wl.dtype)
     hs = gu.dev_tensor(wl.hidden_steps.reshape(-1, d), wl.dtype).reshape(steps, slots, d)
     reset = torch.from_numpy(wl.reset_src).cuda()
     st = egtp.plp_state_create(ctx, num_slots or slots, d)
@@ -56,6 +56,13 @@ def test_decode_loop_with_retirement_matches_oracle(ctx):
     follow = [0, 1, 57, 128, 129]
     ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=follow)
     _compare(H, z, y, ref, follow)
+    # the same loop with the head rescaled to predict hundreds of tokens (the first one predicts fractions of one)
+    big = gen.scaled_head(wl.head, "bf16")
+    st_b, H_b, z_b, y_b = _run_plp(ctx, wl, head=big)
+    ref_b = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, big, slots=follow, H_steps=ref["H"])
+    assert np.abs(ref_b["yrem"]).min() > 100
+    _compare(H_b, z_b, y_b, ref_b, follow)
+    egtp.plp_state_destroy(st_b)
     # a slot that was just reset holds exactly its one token: z == h'
     t, s = np.argwhere(wl.reset_src[1:] == gen.RESET_EMPTY)[0]
     assert np.array_equal(z[t + 1, s], wl.hidden_steps[t + 1, s].astype(np.float64))
@@ -104,6 +111,13 @@ def test_rl_group_sampling_continues_from_egtp_state(ctx):
     ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=follow,
                       prompts=dict(hidden=eg.hidden, offsets=eg.offsets, H=ref_eg["H"]))
     _compare(H, z, y, ref, follow)
+    big = gen.scaled_head(wl.head, "bf16")                     # the same streams with a head that predicts hundreds of tokens
+    st_b, H_b, z_b, y_b = _run_plp(ctx, wl, src=src, head=big)
+    ref_b = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, big, slots=follow, H_steps=ref["H"],
+                        prompts=dict(hidden=eg.hidden, offsets=eg.offsets, H=ref_eg["H"]))
+    assert np.abs(ref_b["yrem"]).min() > 100
+    _compare(H_b, z_b, y_b, ref_b, follow)
+    egtp.plp_state_destroy(st_b)
     # streaming state == batch EGTP over the concatenation [prompt 0 ; generated tokens 1..12] of slot 0
     cat = np.concatenate([eg.hidden[eg.offsets[0]:eg.offsets[1]], wl.hidden_steps[:, 0, :]])
     both = orc.egtp_predict(cat, np.array([0, cat.shape[0]]), wl.W, wl.head)

@@ -67,6 +67,13 @@ def test_bound_decode_loop_matches_oracle(ctx, slots, V, m_h):
     ref = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, wl.head, slots=follow)
     _compare(H, z, y, ref, follow)
     egtp.plp_state_destroy(st)
+    # the same loop bound to a head that predicts hundreds of tokens (the configuration's own predicts fractions of one)
+    big = gen.scaled_head(wl.head, "bf16")
+    st_b, H_b, z_b, y_b, _ = _run(ctx, wl, head=gu.DeviceHead(big, "bf16"))
+    ref_b = orc.plp_run(wl.hidden_steps, wl.reset_src, wl.W, big, slots=follow, H_steps=ref["H"])
+    assert np.abs(ref_b["yrem"]).min() > 100
+    _compare(H_b, z_b, y_b, ref_b, follow)
+    egtp.plp_state_destroy(st_b)
     # the unbound route on the same inputs: same entropies bit for bit (same vocabulary columns per tile only when
     # the column split is the same, so compare within tolerance), same lengths within tolerance
     st2, H2, z2, y2, launches2 = _run(ctx, wl, bind=False)
