@@ -4,15 +4,19 @@
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl mine|reference]
 
 A step is one pass of the whole EGTP hot path (LM-head GEMM with online entropy, merge,
-Eq. 3 weights, Eq. 4 pooling, head) over one synthetic batch shaped like the "EGTP mid"
-configuration: 32 prompts, lognormal(5.5, 0.8) lengths clipped to [32, 2048], d = 2048 bf16
-hidden states with 1 % outlier channels, LM head 151936 x 2048 bf16, head 2048 -> 512 -> 1.
+Eq. 3-4 pooling, head) over one synthetic batch shaped like the "EGTP mid" configuration:
+32 prompts, lognormal(5.5, 0.8) lengths clipped to [32, 2048], d = 2048 bf16 hidden states
+with 1 % outlier channels, LM head 151936 x 2048 bf16, head 2048 -> 512 -> 1.
 With N > 1 every rank (one process per GPU) runs its own batch of that shape (different seed):
 prompts are independent, so there is no collective on the data path ("weak" scaling).
-Rank 0 prints ONE JSON line.  The PLP decode step (256 live sequences, d = 4096) is timed on
-rank 0 at N = 1 and reported in the same line under "plp_decode".
+Rank 0 prints ONE JSON line.  At N = 1 the other named workloads are timed in the same run and
+summarised inside the line's "roofline" object (key "legs"): the PLP decode step at 256 live
+sequences (d = 4096), the long-tailed prompt batch (d = 4096) with its HBM-bound pooling kernel,
+entropy from logits already in memory, and the RL group-sampling sizes (d = 5120, 1024 streams).
 
 --impl reference times the fp64 CPU oracle (oracle/) on a bounded sample of the same workload.
+--vocab-parallel times the PLP decode step with the LM head's rows sharded over the N ranks
+(one all-gather of rows x 3 floats per step) instead of the default workload.
 """
 from __future__ import annotations
 
@@ -30,11 +34,6 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes (read + write) of one launch of the dominant kernel on the bench workload, from the ncu
-# capture summarised in profiles/lmhead_entropy_egtp_mid.md (seed-1 batch, 9555 tokens).  Set to None
-# whenever the kernel or its launch plan changes after the capture.
-NCU_TRAFFIC_LMHEAD_MID_BYTES = 959.8e6 + 15.9e6
-
 METRIC = "egtp_prompt_tokens_per_sec"
 UNIT = "tokens/s"
 
@@ -49,14 +48,30 @@ def load_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
+def ncu_traffic(key: str, live: dict):
+    """DRAM bytes (read + write) per launch of a kernel from the ncu capture recorded in profiles/traffic.json,
+    or None when the live launch (tokens, plan) is not the one that was captured."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            rec = json.load(f)[key]
+    except (OSError, KeyError, ValueError):
+        return None
+    for k, v in rec.get("launch", {}).items():
+        if live.get(k) != v:
+            return None
+    return float(rec["dram_bytes_per_launch"])
+
+
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    """Samples nvidia-smi clocks and throttle reasons of one GPU (read-only) for the whole run; window(t0, t1)
+    summarises the samples that fall into one timed region."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_index: int, period_ms: int = 20):
         self.gpu_index = gpu_index
+        self.period_ms = period_ms
         self.rows = []
         self.proc = None
         self.thread = None
@@ -64,7 +79,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", str(self.period_ms),
                  "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -76,17 +91,23 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append((time.time(), line.strip()))
 
-    def stop(self, t0: float, t1: float):
+    def stop(self):
         if self.proc is None:
-            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
-        time.sleep(0.12)
+            return
+        time.sleep(0.1)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=2)
         except Exception:
             self.proc.kill()
+
+    def window(self, t0: float, t1: float):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(min(0.1, 2.5e-3 * self.period_ms))          # let the last sample of the window arrive
+        inside = [r for (t, r) in self.rows if t0 <= t <= t1]
+        rows = inside or [r for (t, r) in self.rows if t0 - 0.06 <= t <= t1 + 0.06]
         sm, smax, reasons, power = [], [], set(), []
-        rows = [r for (t, r) in self.rows if t0 - 0.05 <= t <= t1 + 0.1] or [r for (_, r) in self.rows]
         for r in rows:
             parts = [x.strip() for x in r.split(",")]
             if len(parts) < 7:
@@ -100,6 +121,12 @@ class ClockSampler:
                     reasons.add(name)
         return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(smax) if smax else None,
                     power_w=float(np.median(power)) if power else None, samples=len(sm), reasons=sorted(reasons))
+
+
+def cycles(time_us: float, clk: dict):
+    """time x median SM clock of the same region, in millions of SM cycles (None without clock samples): a figure that
+    does not move with the power state the region happened to run in."""
+    return None if not clk or not clk.get("sm_mhz") else time_us * clk["sm_mhz"] * 1e-6
 
 
 def dist_env():
@@ -128,14 +155,17 @@ def oracle_sample(wl, max_tokens: int = 192):
     return rows, off, pick
 
 
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return int(max([p.get("num_threads", 1) for p in threadpool_info()] or [1]))
+    except Exception:
+        return os.cpu_count() or 1
+
+
 def time_oracle(wl, steps: int, warmup: int, max_tokens: int = 192):
     from oracle import egtp_oracle as orc
     rows, off, pick = oracle_sample(wl, max_tokens)
-    try:
-        from threadpoolctl import threadpool_info
-        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
-    except Exception:
-        threads = os.cpu_count() or 1
     for _ in range(warmup):
         orc.egtp_predict(rows, off, wl.W, wl.head, wl.alpha)
     t0 = time.perf_counter()
@@ -143,9 +173,25 @@ def time_oracle(wl, steps: int, warmup: int, max_tokens: int = 192):
         orc.egtp_predict(rows, off, wl.W, wl.head, wl.alpha)
     dt = time.perf_counter() - t0
     tokens = int(rows.shape[0])
-    return dict(value=tokens * steps / dt, unit=UNIT, cores=int(threads), kind="oracle",
+    return dict(value=tokens * steps / dt, unit=UNIT, cores=oracle_threads(), kind="oracle",
                 sample=f"{len(pick)} shortest whole prompts of the batch ({tokens} tokens) x {steps} passes, "
                        f"fp64 numpy, {dt:.1f} s", ms_per_step=1e3 * dt / steps, tokens=tokens)
+
+
+def time_oracle_plp(pw, budget_s: float = 12.0):
+    """The oracle's PLP decode step at the full batch of the decode configuration (256 live sequences): whole steps,
+    every slot followed from its explicit token list, as many steps as fit the budget (at least 2)."""
+    from oracle import egtp_oracle as orc
+    t0 = time.perf_counter()
+    orc.plp_run(pw.hidden_steps[:1], pw.reset_src[:1], pw.W, pw.head)
+    first = time.perf_counter() - t0                       # includes widening the LM head to fp64 once
+    n = int(max(2, min(8, budget_s / max(first, 1e-3))))
+    t0 = time.perf_counter()
+    orc.plp_run(pw.hidden_steps[:n], pw.reset_src[:n], pw.W, pw.head)
+    dt = time.perf_counter() - t0
+    return dict(value=dt / n * 1e6, unit="us per decode step at B=256", cores=oracle_threads(), kind="oracle",
+                sample=f"{n} whole decode steps of all {pw.slots} slots (d={pw.d}, V={pw.V}) in one oracle run "
+                       f"(the LM head is widened to fp64 once per run), fp64 numpy, {dt:.1f} s; not scaled")
 
 
 def run_reference(args):
@@ -170,12 +216,19 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------
 # the CUDA path
 # ------------------------------------------------------------------------------------------------
+def gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    try:
+        return int(vis.split(",")[local_rank]) if vis else local_rank
+    except (ValueError, IndexError):
+        return local_rank
+
+
 def run_mine(args):
     import torch
     import torch.distributed as dist
 
     from paper_2602_11812_b200 import binding as egtp
-    from paper_2602_11812_b200 import inputs as gen
     from paper_2602_11812_b200 import device as gu
     from paper_2602_11812_b200 import shard
 
@@ -208,6 +261,8 @@ def run_mine(args):
             dist.barrier()
             torch.cuda.synchronize()
 
+    sampler = ClockSampler(gpu_index(local_rank))
+    sampler.start()
     for _ in range(warmup):
         step()
     sync_all()
@@ -217,9 +272,6 @@ def run_mine(args):
     # few microseconds per launch)
     egtp.egtp_profile_enable(ctx, False)
     launches0 = egtp.egtp_launch_count(ctx)
-    sampler = ClockSampler(int(os.environ.get("CUDA_VISIBLE_DEVICES", "0").split(",")[local_rank]) if os.environ.get("CUDA_VISIBLE_DEVICES") else local_rank)
-    sampler.start()
-    time.sleep(0.15)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sync_all()
     t_wall0 = time.time()
@@ -230,7 +282,7 @@ def run_mine(args):
     sync_all()
     t_wall1 = time.time()
     ms = ev0.elapsed_time(ev1)
-    clocks = sampler.stop(t_wall0, t_wall1)
+    clocks = sampler.window(t_wall0, t_wall1)
     launches = egtp.egtp_launch_count(ctx) - launches0
     assert int(status.item()) == 0, egtp.status_string(int(status.item()))
     # ---- the same K steps once more with every kernel bracketed by events: per-kernel times for the roofline
@@ -290,6 +342,7 @@ def run_mine(args):
 
     if rank != 0:
         egtp.egtp_destroy(ctx)
+        sampler.stop()
         if world > 1:
             dist.destroy_process_group()
         return
@@ -300,17 +353,17 @@ def run_mine(args):
     flops = 2.0 * d * V * T                      # algorithmic flops of one launch: 2 d V per token
     achieved = flops / (k1_ms * 1e-3) / 1e12
     peak = peaks["bf16_tflops"] if ms < 2000 else peaks["bf16_tflops_sustained"]
+    plan = egtp.egtp_lmhead_plan(ctx, T, d, V, egtp.EGTP_BF16)
+    traffic = ncu_traffic("lmhead_entropy_egtp_mid", dict(tokens=T, d=d, V=V, chunks=plan["chunks"], grid=plan["grid"])) \
+        if world == 1 else None
     roofline = dict(bound="tensor", kernel="lmhead_entropy", achieved=achieved, peak=peak, unit="TFLOP/s",
-                    frac=achieved / peak, traffic=NCU_TRAFFIC_LMHEAD_MID_BYTES if (world == 1 and T == 9555) else None,
+                    frac=achieved / peak, traffic=traffic,
                     algorithmic_bytes=2.0 * V * d + 2.0 * T * d, peak_source=peaks["source"],
                     ms_per_launch=k1_ms, frac_of_sustained=achieved / peaks["bf16_tflops_sustained"],
-                    frac_of_nominal_2250=achieved / 2250.0)
-    pool = prof["pool"]
-    pool_ms = pool["ms"] / max(1, pool["launches"])
-    pool_gbs = (2.0 * d * T + 4.0 * T) / (pool_ms * 1e-3) / 1e9 if pool_ms > 0 else None
+                    frac_of_nominal_2250=achieved / 2250.0,
+                    mcycles_per_launch=cycles(k1_ms * 1e3, clocks), sm_mhz=clocks.get("sm_mhz"))
     kernels = {k: dict(ms_per_launch=v["ms"] / max(1, v["launches"]), launches=v["launches"]) for k, v in prof.items()
                if v["launches"]}
-    plan = egtp.egtp_lmhead_plan(ctx, T, d, V, egtp.EGTP_BF16)
 
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=steps, warmup=warmup,
                 ms_per_step=ms_max / steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
@@ -319,31 +372,70 @@ def run_mine(args):
                                      "(1% outlier channels x20), LM head 151936x2048 bf16, head 2048->512->1",
                             tokens_per_gpu=T, prompts_per_gpu=B, d=d, V=V,
                             l2="inputs (622 MB LM head) larger than the 126 MB L2; no explicit flush",
-                            lmhead_plan=plan),
+                            lmhead_plan=plan, launches_per_step=launches / steps),
                 clocks=clocks,
                 e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                          steps=e2e_steps, api="egtp_predict_host"),
                 gpu_launches=int(launches),
                 roofline=roofline,
                 kernels=kernels,
-                library_gemm_same_shape=lib_gemm,
-                pool=dict(bound="hbm", achieved=pool_gbs, peak=peaks["hbm_gbs"], unit="GB/s",
-                          frac=(pool_gbs / peaks["hbm_gbs"]) if pool_gbs else None,
-                          note="40 MB of hidden states: launch-latency sized at this workload"))
+                library_gemm_same_shape=lib_gemm)
 
+    egtp.egtp_destroy(ctx)
+    del hidden, W
+    legs = {}
+    plp_wl = None
     if world == 1 and not args.no_plp:
-        line["plp_decode"], line["egtp_long"] = bench_d4096(local_rank, peaks, args.plp_steps, args.long_steps)
+        plp, long_, plp_wl = bench_d4096(local_rank, peaks, args.plp_steps, args.long_steps, sampler)
+        line["plp_decode"], line["egtp_long"] = plp, long_
+        # the parts of those legs that belong to the metric, where the rest of the line is kept
+        legs["plp_decode"] = dict(
+            metric="plp_decode_step_us", workload="256 live sequences, d=4096, V=151936, head 4096->256->1, state bound to its head",
+            us_per_step_median=plp["us_per_step_median"], us_per_step_p10=plp["us_per_step_p10"],
+            us_per_step_p90=plp["us_per_step_p90"], launches_per_step=plp["launches_per_step"],
+            bound="hbm", unit="GB/s", peak=peaks["hbm_gbs"], kernel="lmhead_entropy_pair",
+            kernel_us=plp["lmhead_us"], achieved=plp["hbm"]["achieved"], frac=plp["hbm"]["frac"],
+            whole_step_frac=plp["hbm"]["whole_step_frac"], tensor_frac=plp["tensor"]["frac"],
+            cuda_graph_us=plp.get("cuda_graph_us_per_step"), sm_mhz=plp["clocks"].get("sm_mhz"),
+            mcycles_per_step=cycles(plp["us_per_step_median"], plp["clocks"]),
+            e2e_us=plp.get("e2e", {}).get("us_per_step"), unbound_us_per_step_median=plp["unbound_state"]["us_per_step_median"])
+        fl = plp["from_logits"]
+        legs["from_logits"] = dict(workload="[256, 151936] bf16 logits already in memory (3 buffers in rotation: larger than L2)",
+                                   bound="hbm", unit="GB/s", peak=peaks["hbm_gbs"], kernel="logits_entropy",
+                                   kernel_us=fl["entropy_call_us"], achieved=fl["hbm"]["achieved"], frac=fl["hbm"]["frac"],
+                                   timing=fl["hbm"]["timing"], us_per_plp_step=fl["us_per_step"])
+        legs["egtp_long"] = dict(metric=METRIC, workload=long_["workload"], tokens=long_["tokens"], value=long_["value"],
+                                 ms_per_step=long_["ms_per_step"], bound="tensor", unit="TFLOP/s",
+                                 peak=long_["lmhead"]["peak"], achieved=long_["lmhead"]["achieved"],
+                                 frac=long_["lmhead"]["frac"], sm_mhz=long_["clocks"].get("sm_mhz"),
+                                 mcycles_per_step=cycles(long_["ms_per_step"] * 1e3, long_["clocks"]))
+        legs["pool"] = dict(workload="Eq. 3-4 pooling of the long-tailed batch (25629 tokens x 4096 bf16 = 210 MB)",
+                            **long_["pool"])
+    if world == 1 and not args.no_rl:
+        rl = bench_rl_group(local_rank, peaks, min(args.plp_steps, 16), min(args.long_steps, 3), sampler)
+        line["rl_group"] = rl
+        legs["rl_group"] = dict(
+            workload=rl["workload"], egtp_tokens=rl["egtp"]["tokens"], egtp_value=rl["egtp"]["value"],
+            egtp_ms_per_step=rl["egtp"]["ms_per_step"], egtp_lmhead_frac=rl["egtp"]["lmhead"]["frac"],
+            pool_frac=rl["egtp"]["pool"]["frac"], pool_us=rl["egtp"]["pool"]["us_per_launch"],
+            plp_B1024_us_per_step=rl["plp_B1024"]["bound_to_head"]["us_per_step"],
+            plp_B1024_lmhead_frac=rl["plp_B1024"]["bound_to_head"]["lmhead"]["frac"], bound="tensor",
+            peak=peaks["bf16_tflops"], unit="TFLOP/s", sm_mhz=rl["egtp"]["clocks"].get("sm_mhz"))
+    if legs:
+        roofline["legs"] = legs
+    sampler.stop()
     if world == 1 and not args.no_cpu:
         probe = time_oracle(wl, steps=1, warmup=0, max_tokens=256)          # one pass tells how many fit in ~15 s
         cb = time_oracle(wl, steps=int(min(40, max(2, 15.0 / (probe["ms_per_step"] * 1e-3)))), warmup=0, max_tokens=256)
         line["cpu_baseline"] = dict(value=cb["value"], unit=UNIT, cores=cb["cores"], kind="oracle", sample=cb["sample"])
-    egtp.egtp_destroy(ctx)
+        if plp_wl is not None:
+            line["cpu_baseline"]["plp_decode_step"] = time_oracle_plp(plp_wl)
     if world > 1:
         dist.destroy_process_group()
     print(json.dumps(line), flush=True)
 
 
-def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
+def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int, sampler=None):
     """The two d = 4096 workloads, sharing one 151936 x 4096 bf16 LM head on the device.
 
     plp_decode: 256 live sequences, one token per step, head 4096 -> 256 -> 1, slots retire at
@@ -356,6 +448,9 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     from paper_2602_11812_b200 import binding as egtp
     from paper_2602_11812_b200 import device as gu
     from paper_2602_11812_b200 import inputs as gen
+
+    def window(t0, t1):
+        return sampler.window(t0, t1) if sampler is not None else {}
 
     warm = 5
     wl = gen.config_plp_decode(steps=plp_steps + warm)
@@ -384,11 +479,14 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
         for t in range(warm):
             egtp.plp_step(ctx, st, lm, head.c, hs[t], reset_src=None, yrem_out=yrem, status_dev=status)
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(plp_steps + 1)]
+        torch.cuda.synchronize()
+        t0 = time.time()
         evs[0].record()
         for t in range(plp_steps):
             egtp.plp_step(ctx, st, lm, head.c, hs[warm + t], reset_src=reset[warm + t], yrem_out=yrem, status_dev=status)
             evs[t + 1].record()
         torch.cuda.synchronize()
+        clk = window(t0, time.time())
         # pass 2: the same steps again with every kernel bracketed by events (per-kernel breakdown)
         egtp.egtp_profile_enable(ctx, True)
         egtp.egtp_profile_read(ctx)
@@ -401,7 +499,7 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
         k1_us = prof["lmhead_entropy"]["ms"] / prof["lmhead_entropy"]["launches"] * 1e3
         step_us = float(np.median(per_step))
         return dict(us_per_step_median=step_us, us_per_step_p10=float(np.percentile(per_step, 10)),
-                    us_per_step_p90=float(np.percentile(per_step, 90)), lmhead_us=k1_us,
+                    us_per_step_p90=float(np.percentile(per_step, 90)), lmhead_us=k1_us, clocks=clk,
                     hbm=dict(bound="hbm", kernel="lmhead_entropy", achieved=w_bytes / (k1_us * 1e-6) / 1e9,
                              peak=peaks["hbm_gbs"], unit="GB/s", frac=w_bytes / (k1_us * 1e-6) / 1e9 / peaks["hbm_gbs"],
                              whole_step_frac=w_bytes / (step_us * 1e-6) / 1e9 / peaks["hbm_gbs"]),
@@ -483,7 +581,7 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         g0.record()
         for t in range(plp_steps):
-            static_h.copy_(hs[warm + t], non_blocking=True)      # the step's new tokens (0.2 MB device copy)
+            static_h.copy_(hs[warm + t], non_blocking=True)      # the step's new tokens (2 MB device copy)
             graph.replay()
         g1.record()
         torch.cuda.synchronize()
@@ -495,18 +593,19 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     egtp.egtp_profile_enable(ctx, True)
     assert int(status.item()) == 0
 
-    # ---- the same decode step when the serving engine already holds the step's logits
+    # ---- the same decode step when the serving engine already holds the step's logits.  Three logits buffers are
+    # used in rotation (233 MB, larger than L2), so every pass really streams its 78 MB from HBM.
     torch.manual_seed(0)
-    logits = (torch.randn(slots, V, device="cuda") * 1.5).to(torch.bfloat16)
-    n_fl = max(8, plp_steps)
+    logit_bufs = [(torch.randn(slots, V, device="cuda") * 1.5).to(torch.bfloat16) for _ in range(3)]
+    n_fl = max(9, plp_steps)
 
     def measure_from_logits(state):
         def steps_():
             for t in range(n_fl):
-                egtp.plp_step_from_logits(ctx, state, logits, head.c, hs[warm + t % plp_steps],
+                egtp.plp_step_from_logits(ctx, state, logit_bufs[t % 3], head.c, hs[warm + t % plp_steps],
                                           reset_src=reset[warm + t % plp_steps], yrem_out=yrem, status_dev=status)
         for t in range(3):
-            egtp.plp_step_from_logits(ctx, state, logits, head.c, hs[t], reset_src=reset[t], yrem_out=yrem, status_dev=status)
+            egtp.plp_step_from_logits(ctx, state, logit_bufs[t], head.c, hs[t], reset_src=reset[t], yrem_out=yrem, status_dev=status)
         torch.cuda.synchronize()
         egtp.egtp_profile_enable(ctx, False)
         f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -520,11 +619,8 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
         torch.cuda.synchronize()
         prof_fl = egtp.egtp_profile_read(ctx)
         assert int(status.item()) == 0
-        le_us = prof_fl["logits_entropy"]["ms"] / prof_fl["logits_entropy"]["launches"] * 1e3
-        le_gbs = 2.0 * slots * V / (le_us * 1e-6) / 1e9
-        return dict(us_per_step=f0.elapsed_time(f1) / n_fl * 1e3, logits_entropy_us=le_us,
-                    hbm=dict(bound="hbm", kernel="logits_entropy", achieved=le_gbs, peak=peaks["hbm_gbs"],
-                             unit="GB/s", frac=le_gbs / peaks["hbm_gbs"], bytes_per_row=2 * V),
+        return dict(us_per_step=f0.elapsed_time(f1) / n_fl * 1e3,
+                    logits_entropy_us_event_bracketed=prof_fl["logits_entropy"]["ms"] / prof_fl["logits_entropy"]["launches"] * 1e3,
                     kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof_fl.items() if v["launches"]})
 
     # bound state: W1 h' from a launch of the LM-head kernel over the head columns alone (reported as head_hidden)
@@ -532,8 +628,46 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     st_plain = egtp.plp_state_create(ctx, slots, d)
     plp["from_logits"]["unbound_state"] = measure_from_logits(st_plain)
     egtp.plp_state_destroy(st_plain)
+    # The entropy kernel by itself: egtp_entropy_from_logits is one launch, so a CUDA graph of 12 calls over the
+    # rotating buffers, replayed, times the kernel without the few microseconds an event pair around a 20 us kernel adds.
+    Hfl = torch.empty(slots, device="cuda", dtype=torch.float32)
+    egtp.egtp_profile_enable(ctx, False)
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for i in range(3):
+                egtp.egtp_entropy_from_logits(ctx, logit_bufs[i], Hfl, status_dev=status)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        calls = 12
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for i in range(calls):
+                egtp.egtp_entropy_from_logits(ctx, logit_bufs[i % 3], Hfl, status_dev=status)
+        for _ in range(2):
+            graph.replay()
+        torch.cuda.synchronize()
+        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 10
+        q0.record()
+        for _ in range(reps):
+            graph.replay()
+        q1.record()
+        torch.cuda.synchronize()
+        call_us = q0.elapsed_time(q1) / (reps * calls) * 1e3
+        timing = "CUDA graph of 12 single-launch calls over 3 rotating buffers, replayed 10 times"
+        del graph
+    except Exception as exc:
+        call_us = plp["from_logits"]["logits_entropy_us_event_bracketed"]
+        timing = f"event-bracketed launches (graph capture failed: {str(exc)[:80]})"
+    le_gbs = 2.0 * slots * V / (call_us * 1e-6) / 1e9
+    plp["from_logits"]["entropy_call_us"] = call_us
+    plp["from_logits"]["hbm"] = dict(bound="hbm", kernel="logits_entropy", achieved=le_gbs, peak=peaks["hbm_gbs"], unit="GB/s",
+                                     frac=le_gbs / peaks["hbm_gbs"], bytes_per_row=2 * V, timing=timing)
+    egtp.egtp_profile_enable(ctx, True)
     egtp.plp_state_destroy(st)
-    del hs, logits
+    del hs, logit_bufs
 
     # ---- EGTP over the long-tailed prompt batch
     hidden = gu.dev_tensor(wl3.hidden, "bf16")
@@ -543,28 +677,36 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     for _ in range(3):
         egtp.egtp_predict(ctx, lm, head3.c, hidden, off, wl3.B, wl3.T, 1.0, yhat_out=yhat, status_dev=status)
     torch.cuda.synchronize()
-    egtp.egtp_profile_read(ctx)
+    egtp.egtp_profile_enable(ctx, False)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
     e0.record()
     for _ in range(egtp_steps):
         egtp.egtp_predict(ctx, lm, head3.c, hidden, off, wl3.B, wl3.T, 1.0, yhat_out=yhat, status_dev=status)
     e1.record()
     torch.cuda.synchronize()
+    clk3 = window(t0, time.time())
+    ms_step = e0.elapsed_time(e1) / egtp_steps
+    egtp.egtp_profile_enable(ctx, True)
+    egtp.egtp_profile_read(ctx)
+    for _ in range(egtp_steps):
+        egtp.egtp_predict(ctx, lm, head3.c, hidden, off, wl3.B, wl3.T, 1.0, yhat_out=yhat, status_dev=status)
+    torch.cuda.synchronize()
     prof3 = egtp.egtp_profile_read(ctx)
     assert int(status.item()) == 0
-    ms_step = e0.elapsed_time(e1) / egtp_steps
     k1_ms = prof3["lmhead_entropy"]["ms"] / prof3["lmhead_entropy"]["launches"]
     pool_us = prof3["pool"]["ms"] / prof3["pool"]["launches"] * 1e3
     tf = 2.0 * d * V * wl3.T / (k1_ms * 1e-3) / 1e12
     pool_gbs = (2.0 * d + 4.0) * wl3.T / (pool_us * 1e-6) / 1e9
     long_ = dict(metric=METRIC, workload="egtp_long: 64 prompts Pareto(1.2) in [128,8192], d=4096, V=151936, head 4096->1024->1",
-                 tokens=wl3.T, steps=egtp_steps, ms_per_step=ms_step, value=wl3.T / (ms_step * 1e-3), unit=UNIT,
+                 tokens=wl3.T, steps=egtp_steps, ms_per_step=ms_step, value=wl3.T / (ms_step * 1e-3), unit=UNIT, clocks=clk3,
                  lmhead=dict(bound="tensor", achieved=tf, peak=peaks["bf16_tflops"], unit="TFLOP/s",
                              frac=tf / peaks["bf16_tflops"], ms_per_launch=k1_ms),
                  pool=dict(bound="hbm", kernel="pool", achieved=pool_gbs, peak=peaks["hbm_gbs"], unit="GB/s",
                            frac=pool_gbs / peaks["hbm_gbs"], us_per_launch=pool_us,
-                           bytes_per_token=2 * d + 4),
+                           bytes_per_token=2 * d + 4, timing="event-bracketed launches"),
                  kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof3.items() if v["launches"]},
+                 launches_per_step=sum(v["launches"] for v in prof3.values()) / egtp_steps,
                  plan=egtp.egtp_lmhead_plan(ctx, wl3.T, d, V, egtp.EGTP_BF16))
     # ---- the paper's pooling comparators (Table 3) on the same batch: pooling alone, no LM head
     comp = {}
@@ -583,10 +725,10 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     long_["pooling_comparators"] = comp
     assert int(status.item()) == 0
     egtp.egtp_destroy(ctx)
-    return plp, long_
+    return plp, long_, wl
 
 
-def bench_rl_group(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
+def bench_rl_group(ctx_device: int, peaks, plp_steps: int, egtp_steps: int, sampler=None):
     """RL group sampling at its full sizes: EGTP over 64 shared prompts (d = 5120, V = 152064), then PLP steps over
     1024 decode streams that start from their prompt's state (tensor-bound: 8 row blocks of 128 rows per step)."""
     import torch
@@ -602,7 +744,9 @@ def bench_rl_group(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     W = gu.dev_tensor(wl.W, "bf16")
     lm = egtp.make_lm_head(W)
     head = gu.DeviceHead(wl.head, "bf16")
-    ctx = egtp.egtp_create(ctx_device, max_tokens=eg.T, max_batch=slots, max_d=d, max_V=V)
+    # no host staging: this leg calls the device-pointer entry points only (the staging copy would be 2.8 GB)
+    ctx = egtp.egtp_create_ex(ctx_device, max_tokens=eg.T, max_batch=slots, max_d=d, max_V=V,
+                              flags=egtp.EGTP_CREATE_NO_HOST_STAGING)
     status = torch.zeros(1, device="cuda", dtype=torch.int32)
     f = dict(device="cuda", dtype=torch.float32)
     # ---- EGTP over the shared prompts
@@ -620,19 +764,26 @@ def bench_rl_group(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     egtp.egtp_profile_enable(ctx, True)
     egtp.egtp_profile_read(ctx)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
     e0.record()
     for _ in range(egtp_steps):
         predict()
     e1.record()
     torch.cuda.synchronize()
+    clk = sampler.window(t0, time.time()) if sampler is not None else {}
     prof = egtp.egtp_profile_read(ctx)
     ms_step = e0.elapsed_time(e1) / egtp_steps
     k1_ms = prof["lmhead_entropy"]["ms"] / prof["lmhead_entropy"]["launches"]
     tf = 2.0 * d * V * eg.T / (k1_ms * 1e-3) / 1e12
+    pool_us = prof["pool"]["ms"] / prof["pool"]["launches"] * 1e3
     out = dict(workload="rl_group: 64 prompts U[256,4096] x 16 streams, d=5120, V=152064, head 5120->512->1",
-               egtp=dict(tokens=eg.T, steps=egtp_steps, ms_per_step=ms_step, value=eg.T / (ms_step * 1e-3), unit=UNIT,
+               workspace_bytes=egtp.egtp_workspace_bytes(ctx),
+               egtp=dict(tokens=eg.T, steps=egtp_steps, ms_per_step=ms_step, value=eg.T / (ms_step * 1e-3), unit=UNIT, clocks=clk,
                          lmhead=dict(bound="tensor", achieved=tf, peak=peaks["bf16_tflops"], unit="TFLOP/s",
                                      frac=tf / peaks["bf16_tflops"], ms_per_launch=k1_ms),
+                         pool=dict(bound="hbm", us_per_launch=pool_us, achieved=(2.0 * d + 4.0) * eg.T / (pool_us * 1e-6) / 1e9,
+                                   peak=peaks["hbm_gbs"], unit="GB/s",
+                                   frac=(2.0 * d + 4.0) * eg.T / (pool_us * 1e-6) / 1e9 / peaks["hbm_gbs"]),
                          kernels_us={k: v["ms"] / v["launches"] * 1e3 for k, v in prof.items() if v["launches"]}))
     del hidden
     # ---- PLP over the 1024 streams: ordinary route, then the state bound to the head
@@ -680,6 +831,86 @@ def bench_rl_group(ctx_device: int, peaks, plp_steps: int, egtp_steps: int):
     return out
 
 
+def run_vocab_parallel(args):
+    """The PLP decode step (256 live sequences, d = 4096, V = 151936) with the LM head's rows sharded over the ranks:
+    every rank reduces its shard to one (m, s, t2) triple per row, one all-gather of rows x 3 floats per rank
+    exchanges them (NCCL), every rank merges and advances its replica of the state.  One JSON line from rank 0;
+    at N = 1 the shard is the whole vocabulary and the exchange is skipped."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2602_11812_b200 import binding as egtp
+    from paper_2602_11812_b200 import device as gu
+    from paper_2602_11812_b200 import inputs as gen
+    from paper_2602_11812_b200 import shard
+
+    rank, local_rank, world = dist_env()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    peaks = load_peaks()
+    steps, warmup = max(1, args.steps), max(3, args.warmup)
+    wl = gen.config_plp_decode(steps=steps + warmup)
+    slots, d, V = wl.slots, wl.d, wl.V
+    v0, v1 = shard.vocab_shards(V, world)[rank]
+    W = gu.dev_tensor(wl.W[v0:v1], "bf16")
+    lm = egtp.make_lm_head(W)
+    head = gu.DeviceHead(wl.head, "bf16")
+    ctx = egtp.egtp_create(local_rank, max_tokens=1024, max_batch=slots, max_d=d, max_V=V)
+    st = egtp.plp_state_create(ctx, slots, d)
+    egtp.plp_state_bind_head(st, head.c)
+    hs = gu.dev_tensor(wl.hidden_steps.reshape(-1, d), "bf16").reshape(steps + warmup, slots, d)
+    reset = torch.from_numpy(wl.reset_src).cuda()
+    yrem = torch.empty(slots, device="cuda", dtype=torch.float32)
+    status = torch.zeros(1, device="cuda", dtype=torch.int32)
+    partial = torch.empty(slots, 3, device="cuda", dtype=torch.float32)
+
+    def step(t):
+        shard.plp_step_vocab_parallel(ctx, st, lm, head.c, hs[t], partial_buf=partial, reset_src=reset[t], yrem_out=yrem,
+                                      status_dev=status)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for t in range(warmup):
+        step(t)
+    sync_all()
+    sampler = ClockSampler(gpu_index(local_rank))
+    sampler.start()
+    launches0 = egtp.egtp_launch_count(ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    t0 = time.time()
+    e0.record()
+    for t in range(steps):
+        step(warmup + t)
+    e1.record()
+    sync_all()
+    clocks = sampler.window(t0, time.time())
+    sampler.stop()
+    assert int(status.item()) == 0
+    ms_max, _ = shard.reduce_time_and_work(e0.elapsed_time(e1), 1.0, torch.device("cuda", local_rank))
+    us = ms_max / steps * 1e3
+    if rank == 0:
+        shard_bytes = 2.0 * d * (v1 - v0)
+        print(json.dumps(dict(
+            metric="plp_decode_step_us_vocab_parallel", value=us, unit="us", n_gpus=world, steps=steps, warmup=warmup,
+            ms_per_step=us * 1e-3, higher_is_better=False, scaling="strong", vs_baseline=None, dtype="bf16", data="synthetic",
+            config=dict(workload="plp_decode: 256 live sequences, d=4096, V=151936 sharded by rows over the ranks, head 4096->256->1",
+                        vocab_rows_per_rank=v1 - v0, exchange="all-gather of [256, 3] fp32 per rank and step" if world > 1 else "none (one rank)"),
+            clocks=clocks, gpu_launches=int(egtp.egtp_launch_count(ctx) - launches0),
+            roofline=dict(bound="hbm", kernel="lmhead_entropy (one vocabulary shard)", achieved=shard_bytes / (us * 1e-6) / 1e9,
+                          peak=peaks["hbm_gbs"], unit="GB/s", frac=shard_bytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"], traffic=None,
+                          note="whole step (its launches and the exchange) against this rank's share of the W stream"))), flush=True)
+    egtp.plp_state_destroy(st)
+    egtp.egtp_destroy(ctx)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def ensure_library():
     """Builds the CUDA library if it is missing or older than its sources (a no-op otherwise).  Under torchrun
     only local rank 0 compiles; the other ranks wait for the finished file."""
@@ -703,15 +934,23 @@ def main():
     ap.add_argument("--plp-steps", type=int, default=64)
     ap.add_argument("--long-steps", type=int, default=10)
     ap.add_argument("--no-plp", action="store_true", help="skip the d = 4096 workloads (PLP decode, long prompts)")
+    ap.add_argument("--no-rl", action="store_true", help="skip the RL group-sampling sizes (d = 5120, 1024 streams)")
     ap.add_argument("--only-d4096", action="store_true",
                     help="run only the d = 4096 workloads and print their two objects as one JSON line "
                          "(used for profiler captures of the decode and pooling kernels)")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--only-rl-group", action="store_true",
                     help="run only the RL group-sampling sizes (d = 5120, V = 152064, 1024 streams) and print one JSON line")
+    ap.add_argument("--vocab-parallel", action="store_true",
+                    help="time the PLP decode step with the LM head's rows sharded over the ranks")
     args = ap.parse_args()
-    if args.impl != "reference":
-        ensure_library()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    ensure_library()
+    if args.vocab_parallel:
+        run_vocab_parallel(args)
+        return
     if args.only_rl_group:
         import torch
         torch.cuda.set_device(0)
@@ -721,13 +960,10 @@ def main():
     if args.only_d4096:
         import torch
         torch.cuda.set_device(0)
-        plp, long_ = bench_d4096(0, load_peaks(), args.plp_steps, args.long_steps)
+        plp, long_, _ = bench_d4096(0, load_peaks(), args.plp_steps, args.long_steps)
         print(json.dumps(dict(plp_decode=plp, egtp_long=long_)), flush=True)
         return
-    if args.impl == "reference":
-        run_reference(args)
-    else:
-        run_mine(args)
+    run_mine(args)
 
 
 if __name__ == "__main__":

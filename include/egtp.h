@@ -95,6 +95,14 @@ typedef struct {
 EGTP_API int egtp_create(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_batch,
                 int32_t max_d, int32_t max_V);
 
+/* egtp_create with options.  EGTP_CREATE_NO_HOST_STAGING leaves out the device copy of the hidden states that
+ * only the *_host entry points use (max(max_tokens, max_batch) * max_d * 4 bytes, the largest buffer of a context
+ * sized for long prompt batches); egtp_predict_host and plp_step_host then return EGTP_ERR_UNSUPPORTED.
+ * flags == 0 is egtp_create.  Unknown flag bits: EGTP_ERR_INVALID_ARG. */
+enum { EGTP_CREATE_NO_HOST_STAGING = 1 };
+EGTP_API int egtp_create_ex(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_batch,
+                int32_t max_d, int32_t max_V, int32_t flags);
+
 /* Frees the context's device memory. Outstanding work on its streams must have finished. */
 EGTP_API int egtp_destroy(egtp_ctx* ctx);
 

@@ -26,6 +26,7 @@ EGTP_HEAD_SCALAR, EGTP_HEAD_BINS = 0, 1
 PLP_RESET_KEEP, PLP_RESET_EMPTY = -2, -1
 EGTP_LMHEAD_AUTO, EGTP_LMHEAD_CTA_PAIRS, EGTP_LMHEAD_SINGLE_CTA = 0, 1, 2
 EGTP_POOL_MEAN, EGTP_POOL_MAX, EGTP_POOL_LAST = 1, 2, 3
+EGTP_CREATE_NO_HOST_STAGING = 1
 KERNEL_IDS = ["validate_offsets", "lmhead_entropy", "entropy_merge", "segment_weights", "pool",
               "pool_combine", "head_hidden", "head_out", "plp_update", "logits_entropy", "stage_rows"]
 EGTP_NUM_KERNELS = len(KERNEL_IDS)
@@ -38,7 +39,7 @@ EXPORTED_SYMBOLS = [
     "egtp_launch_count", "egtp_lmhead_plan", "egtp_head_forward_static", "egtp_set_lmhead_mode",
     "egtp_entropy_from_logits", "plp_step_from_logits", "egtp_pool_baseline",
     "egtp_entropy_partials", "egtp_entropy_from_partials", "plp_step_from_partials", "egtp_selftest_wait_timeout",
-    "plp_state_bind_head", "egtp_set_lmhead_chunks", "egtp_lmhead_plan_for",
+    "plp_state_bind_head", "egtp_set_lmhead_chunks", "egtp_lmhead_plan_for", "egtp_create_ex",
 ]
 
 
@@ -74,6 +75,7 @@ def load() -> C.CDLL:
     vp, i32, i64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
     P = C.POINTER
     lib.egtp_create.argtypes = [P(vp), C.c_int, i64, i32, i32, i32]
+    lib.egtp_create_ex.argtypes = [P(vp), C.c_int, i64, i32, i32, i32, i32]
     lib.egtp_destroy.argtypes = [vp]
     lib.egtp_status_string.argtypes = [C.c_int]
     lib.egtp_status_string.restype = C.c_char_p
@@ -176,6 +178,17 @@ def egtp_create(device: int, max_tokens: int, max_batch: int, max_d: int, max_V:
     ctx = C.c_void_p()
     _check(load().egtp_create(C.byref(ctx), device, max_tokens, max_batch, max_d, max_V), "egtp_create")
     return ctx.value
+
+
+def egtp_create_ex(device: int, max_tokens: int, max_batch: int, max_d: int, max_V: int, flags: int = 0,
+                   check: bool = True):
+    """egtp_create with option flags (EGTP_CREATE_NO_HOST_STAGING); returns the context handle (or the status with check=False)."""
+    ctx = C.c_void_p()
+    rc = load().egtp_create_ex(C.byref(ctx), device, max_tokens, max_batch, max_d, max_V, flags)
+    if check:
+        _check(rc, "egtp_create_ex")
+        return ctx.value
+    return rc
 
 
 def egtp_destroy(ctx: int):

@@ -27,6 +27,7 @@ struct EventPair {
 struct egtp_ctx {
   int device = 0;
   int num_sms = 0;
+  int pair_workers = 0;           // CTA pairs of the pair kernels this device holds at once
   int64_t max_tokens = 0;
   int32_t max_batch = 0, max_d = 0, max_V = 0;
   PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
@@ -34,19 +35,21 @@ struct egtp_ctx {
   // workspace (device)
   float* partials = nullptr;      int64_t slot_row_capacity = 0;   // rows x slots the partial buffer holds
   float* H = nullptr;             // [max(max_tokens, max_batch)]
-  float* weights = nullptr;       // [max_tokens]
+  int32_t* arrivals = nullptr;    // [max(max_tokens, max_batch)], zero between calls: per-row block counters
   float* seg_m = nullptr;         // [max_batch]
   float* seg_s = nullptr;         // [max_batch]
   float* pooled = nullptr;        // [max_batch][max_d]  (also z of a PLP step)
   float* piece_a = nullptr;       // [chunks][max_d]
   float* piece_b = nullptr;       // [chunks][max_d]
+  float* piece_ms = nullptr;      // [2 * chunks][2]: (m, sum of weights) of every piece
   float* head_partial = nullptr;  int64_t head_partial_floats = 0;
   void* small_rows = nullptr;     // [kMinLmheadRows][max_d] in the widest dtype: tiny batches, zero-padded
   void* zcat = nullptr;           // [max_batch][2 * max_d] bf16: head inputs as [hi | lo] halves (tensor-core layer 1)
   float* yhat = nullptr;          // [max_batch]
   int32_t* status = nullptr;      // [1]
   // staging for the *_host entry points (device)
-  void* hidden_stage = nullptr;   // [max_tokens][max_d] in the widest supported dtype
+  void* hidden_stage = nullptr;   // [max_tokens][max_d] in the widest supported dtype; NULL without host staging
+  bool host_staging = true;
   int32_t* offsets_stage = nullptr;  // [max_batch + 1]
   int32_t* reset_stage = nullptr;    // [max_batch]
   int64_t bytes = 0;
@@ -70,6 +73,7 @@ struct egtp_ctx {
 
 struct plp_state {
   egtp_ctx* ctx = nullptr;
+  int device = 0;               // the context's device (kept here: the state may outlive the context object)
   int32_t num_slots = 0, d = 0;
   float* m = nullptr;
   float* s = nullptr;
@@ -101,8 +105,8 @@ cudaError_t dev_alloc(egtp_ctx* c, T** p, int64_t count) {
 }
 
 void free_ctx_memory(egtp_ctx* c) {
-  cudaFree(c->partials); cudaFree(c->H); cudaFree(c->weights); cudaFree(c->seg_m); cudaFree(c->seg_s);
-  cudaFree(c->pooled); cudaFree(c->piece_a); cudaFree(c->piece_b); cudaFree(c->head_partial); cudaFree(c->zcat); cudaFree(c->small_rows); cudaFree(c->yhat);
+  cudaFree(c->partials); cudaFree(c->H); cudaFree(c->arrivals); cudaFree(c->seg_m); cudaFree(c->seg_s);
+  cudaFree(c->pooled); cudaFree(c->piece_a); cudaFree(c->piece_b); cudaFree(c->piece_ms); cudaFree(c->head_partial); cudaFree(c->zcat); cudaFree(c->small_rows); cudaFree(c->yhat);
   cudaFree(c->status); cudaFree(c->hidden_stage); cudaFree(c->offsets_stage); cudaFree(c->reset_stage);
   if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   for (auto& e : c->piece_ready) if (e) cudaEventDestroy(e);
@@ -211,9 +215,10 @@ constexpr int kMinLmheadRows = 16;
 
 // With fuse_W1 != NULL (bf16 only) the m_h rows of that matrix ride along as extra output columns and
 // head_g [plan.rows_pad][plan.head_cols_pad] receives W1 hidden[i] for every row.
+// head_g must then have room for g_rows x g_ld floats: a plan that needs more is refused before anything is launched.
 int run_lmhead(egtp_ctx* c, const egtp_lm_head* lm, const void* hidden, int64_t ldh, int64_t rows, int32_t* status,
                cudaStream_t stream, LmheadPlan* plan_out, const void* fuse_W1 = nullptr, int fuse_m_h = 0,
-               float* head_g = nullptr) {
+               float* head_g = nullptr, int64_t g_rows = 0, int64_t g_ld = 0) {
   const bool fuse = fuse_W1 != nullptr;
   if (rows < kMinLmheadRows) {
     const int64_t row_bytes = static_cast<int64_t>(lm->d) * elem_bytes(lm->dtype);
@@ -227,8 +232,9 @@ int run_lmhead(egtp_ctx* c, const egtp_lm_head* lm, const void* hidden, int64_t 
     rows = kMinLmheadRows;      // the padding rows get entropies too (ln V); nothing downstream reads them
   }
   const LmheadPlan plan = make_lmhead_plan(rows, lm->d, lm->V, elem_bytes(lm->dtype), c->num_sms, c->slot_row_capacity,
-                                           c->lmhead_mode, fuse ? fuse_m_h : 0, c->lmhead_chunks);
+                                           c->lmhead_mode, fuse ? fuse_m_h : 0, c->lmhead_chunks, c->pair_workers);
   if (plan.rows_pad * plan.slots > c->slot_row_capacity) return EGTP_ERR_CAPACITY;
+  if (fuse && (plan.rows_pad > g_rows || plan.head_cols_pad > g_ld)) return EGTP_ERR_CAPACITY;
   CUtensorMap map_a, map_b, map_b_tile, map_c, map_c_tile;
   LmheadMaps maps;
   int rc = make_tensor_map(c, &map_a, hidden, lm->dtype, rows, lm->d, ldh, plan.a_box_rows);
@@ -330,8 +336,9 @@ int run_head(egtp_ctx* c, const egtp_head* head, const float* z, int64_t ldz, in
 }
 
 // Eq. 2 from logits in memory: per-(row, split) partials into the workspace.
+// H_out != NULL: the same launch also merges them into H_out[rows].
 int run_logits_entropy(egtp_ctx* c, const void* logits, int64_t ldl, int dtype, int64_t rows, int V, int32_t* status,
-                       cudaStream_t stream, int* slots_out) {
+                       cudaStream_t stream, int* slots_out, float* H_out = nullptr) {
   if (!logits || V <= 0 || ldl < V) return EGTP_ERR_INVALID_ARG;
   if (dtype != EGTP_F32 && dtype != EGTP_BF16) return EGTP_ERR_UNSUPPORTED;
   if ((ldl * elem_bytes(dtype)) % 16 != 0 || reinterpret_cast<uintptr_t>(logits) % 16 != 0) return EGTP_ERR_UNSUPPORTED;
@@ -340,7 +347,8 @@ int run_logits_entropy(egtp_ctx* c, const void* logits, int64_t ldl, int dtype, 
   while (splits > 1 && rows * splits > c->slot_row_capacity) --splits;
   if (rows * splits > c->slot_row_capacity) return EGTP_ERR_CAPACITY;
   LaunchScope ls(c, EGTP_K_LOGITS_ENTROPY, stream);
-  EGTP_CUDA_TRY(launch_logits_entropy(logits, ldl, dtype == EGTP_BF16, rows, V, splits, c->partials, status, stream));
+  EGTP_CUDA_TRY(launch_logits_entropy(logits, ldl, dtype == EGTP_BF16, rows, V, splits, c->partials, H_out, c->arrivals,
+                                      status, stream));
   *slots_out = splits;
   return EGTP_OK;
 }
@@ -528,12 +536,14 @@ int predict_impl(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, con
 
   const int d = lm->d;
   float* H = H_out ? H_out : c->H;
-  float* weights = weights_out ? weights_out : c->weights;
   float* pooled = pooled_out ? pooled_out : c->pooled;
   float* seg_m = state_m_out ? state_m_out : c->seg_m;
   float* seg_s = state_s_out ? state_s_out : c->seg_s;
+  const bool want_head = head && (yhat_out || phat_out);
+  // bf16 head weights: layer 1 runs on the tensor cores and the pooling writes its [hi | lo] input directly
+  const bool staged = want_head && head_on_tensor_cores(c, head, B);
 
-  if (B > 0) {
+  if (B > 0 && T_total == 0) {      // only empty prompts can be valid; no merge launch will check the offsets
     LaunchScope ls(c, EGTP_K_VALIDATE, stream);
     EGTP_CUDA_TRY(launch_validate_offsets(offsets, B, T_total, status, stream));
   }
@@ -546,28 +556,28 @@ int predict_impl(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, con
     LmheadPlan plan;
     int rc = run_lmhead(c, lm, piece_ptr, ldh, rows, status, stream, &plan);
     if (rc != EGTP_OK) return rc;
+    // the first merge launch also checks the offsets (everything that indexes tokens through them comes later)
     LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
     EGTP_CUDA_TRY(launch_entropy_merge(c->partials, plan.slots, plan.slots * 3, 3, rows, r0, H, offsets, B, seg_id_out,
-                                       weights, status, stream));
+                                       (p == 0 && B > 0) ? T_total : -1, status, stream));
   }
   if (B == 0) return EGTP_OK;
-  {
-    LaunchScope ls(c, EGTP_K_SEGMENT_WEIGHTS, stream);
-    EGTP_CUDA_TRY(launch_segment_weights(H, offsets, B, 1.f / alpha, weights, seg_m, seg_s, status, stream));
-  }
   if (T_total > 0) {
     LaunchScope ls(c, EGTP_K_POOL, stream);
-    EGTP_CUDA_TRY(launch_pool(hidden, ldh, lm->dtype == EGTP_BF16, false, weights, offsets, B, T_total, d, pooled,
-                              c->piece_a, c->piece_b, status, stream));
+    EGTP_CUDA_TRY(launch_pool(hidden, ldh, lm->dtype == EGTP_BF16, 0, H, 1.f / alpha, offsets, B, T_total, d, pooled,
+                              c->piece_a, c->piece_b, c->piece_ms, seg_m, seg_s, status, stream));
   }
   {
     LaunchScope ls(c, EGTP_K_POOL_COMBINE, stream);
-    EGTP_CUDA_TRY(launch_pool_combine(offsets, B, d, false, c->piece_a, c->piece_b, pooled, status, stream));
+    EGTP_CUDA_TRY(launch_pool_combine(offsets, B, T_total, d, 0, c->piece_a, c->piece_b, c->piece_ms, pooled, seg_m, seg_s,
+                                      staged ? c->zcat : nullptr, status, stream));
   }
-  if (head && (yhat_out || phat_out)) {
-    int rc = run_head(c, head, pooled, d, B, yhat_out, phat_out, status, stream);
-    if (rc != EGTP_OK) return rc;
+  if (weights_out) {
+    LaunchScope ls(c, EGTP_K_SEGMENT_WEIGHTS, stream);
+    EGTP_CUDA_TRY(launch_token_weights(H, offsets, B, T_total, 1.f / alpha, seg_m, seg_s, weights_out, status, stream));
   }
+  if (staged) return run_head_staged(c, head, B, yhat_out, phat_out, status, stream);
+  if (want_head) return run_head(c, head, pooled, d, B, yhat_out, phat_out, status, stream);
   return EGTP_OK;
 }
 
@@ -596,7 +606,13 @@ const char* egtp_kernel_name(int kernel_id) {
 }
 
 int egtp_create(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_batch, int32_t max_d, int32_t max_V) {
+  return egtp_create_ex(out, device, max_tokens, max_batch, max_d, max_V, 0);
+}
+
+int egtp_create_ex(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_batch, int32_t max_d, int32_t max_V,
+                   int32_t flags) {
   if (!out || max_tokens <= 0 || max_batch <= 0 || max_d <= 0 || max_V <= 0) return EGTP_ERR_INVALID_ARG;
+  if ((flags & ~EGTP_CREATE_NO_HOST_STAGING) != 0) return EGTP_ERR_INVALID_ARG;
   if (max_tokens >= (1ll << 31)) return EGTP_ERR_UNSUPPORTED;   // offsets are int32 token indices
   if (cudaSetDevice(device) != cudaSuccess) return EGTP_ERR_CUDA;
   cudaDeviceProp prop;
@@ -616,7 +632,7 @@ int egtp_create(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_batc
     return EGTP_ERR_CUDA;
   }
   c->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
-  if (lmhead_prepare_device() != cudaSuccess) { delete c; return EGTP_ERR_CUDA; }
+  if (lmhead_prepare_device(&c->pair_workers) != cudaSuccess) { delete c; return EGTP_ERR_CUDA; }
 
   const int64_t rows_cap = std::max<int64_t>(max_tokens, max_batch);
   const int64_t rows_pad = (rows_cap + kTileM - 1) / kTileM * kTileM;
@@ -632,18 +648,24 @@ int egtp_create(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_batc
   bool ok = true;
   ok = ok && dev_alloc(c, &c->partials, c->slot_row_capacity * 3) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->H, rows_cap) == cudaSuccess;
-  ok = ok && dev_alloc(c, &c->weights, max_tokens) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->arrivals, rows_cap) == cudaSuccess;
+  ok = ok && cudaMemset(c->arrivals, 0, sizeof(int32_t) * static_cast<size_t>(rows_cap)) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->seg_m, max_batch) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->seg_s, max_batch) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->pooled, static_cast<int64_t>(max_batch) * max_d) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->piece_a, pool_chunks * max_d) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->piece_b, pool_chunks * max_d) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->piece_ms, pool_chunks * 4) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->head_partial, c->head_partial_floats) == cudaSuccess;
   ok = ok && dev_alloc(c, reinterpret_cast<float**>(&c->small_rows), static_cast<int64_t>(kMinLmheadRows) * max_d) == cudaSuccess;
   ok = ok && dev_alloc(c, reinterpret_cast<float**>(&c->zcat), static_cast<int64_t>(max_batch) * max_d) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->yhat, max_batch) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->status, 1) == cudaSuccess;
-  ok = ok && dev_alloc(c, reinterpret_cast<float**>(&c->hidden_stage), rows_cap * max_d) == cudaSuccess;
+  // staging for the hidden states of the *_host entry points: the largest single buffer of the context
+  // (rows x max_d x 4 bytes), left out on request
+  c->host_staging = (flags & EGTP_CREATE_NO_HOST_STAGING) == 0;
+  if (c->host_staging)
+    ok = ok && dev_alloc(c, reinterpret_cast<float**>(&c->hidden_stage), rows_cap * max_d) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->offsets_stage, static_cast<int64_t>(max_batch) + 1) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->reset_stage, max_batch) == cudaSuccess;
   ok = ok && cudaMemset(c->status, 0, sizeof(int32_t)) == cudaSuccess;
@@ -675,7 +697,7 @@ int64_t egtp_launch_count(const egtp_ctx* c) { return c ? c->launches : 0; }
 
 int egtp_lmhead_plan(const egtp_ctx* c, int64_t T, int32_t d, int32_t V, int32_t dtype, int32_t info[8]) {
   if (!c || !info || T <= 0 || d <= 0 || V <= 0) return EGTP_ERR_INVALID_ARG;
-  const LmheadPlan p = make_lmhead_plan(T, d, V, elem_bytes(dtype), c->num_sms, c->slot_row_capacity, c->lmhead_mode, 0, c->lmhead_chunks);
+  const LmheadPlan p = make_lmhead_plan(T, d, V, elem_bytes(dtype), c->num_sms, c->slot_row_capacity, c->lmhead_mode, 0, c->lmhead_chunks, c->pair_workers);
   info[0] = p.grid; info[1] = p.row_blocks; info[2] = p.rows_per_block; info[3] = p.chunks;
   info[4] = p.slots; info[5] = p.tile_cols; info[6] = p.k_blocks; info[7] = p.smem_bytes;
   return EGTP_OK;
@@ -774,25 +796,24 @@ int egtp_pool_baseline(egtp_ctx* c, const egtp_head* head, const void* hidden, i
   int32_t* status = status_dev ? status_dev : c->status;
   if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
   float* pooled = pooled_out ? pooled_out : c->pooled;
-  const bool take_max = mode == EGTP_POOL_MAX;
+  const bool want_head = head && yhat_out;
+  const bool staged = want_head && head_on_tensor_cores(c, head, B);
   {
     LaunchScope ls(c, EGTP_K_VALIDATE, stream);
     EGTP_CUDA_TRY(launch_validate_offsets(offsets, B, T_total, status, stream));
   }
-  if (!take_max && T_total > 0) {
-    LaunchScope ls(c, EGTP_K_SEGMENT_WEIGHTS, stream);
-    EGTP_CUDA_TRY(launch_baseline_weights(offsets, B, mode, c->weights, status, stream));
-  }
   if (T_total > 0) {
     LaunchScope ls(c, EGTP_K_POOL, stream);
-    EGTP_CUDA_TRY(launch_pool(hidden, ldh, dtype == EGTP_BF16, take_max, c->weights, offsets, B, T_total, d, pooled,
-                              c->piece_a, c->piece_b, status, stream));
+    EGTP_CUDA_TRY(launch_pool(hidden, ldh, dtype == EGTP_BF16, mode, nullptr, 1.f, offsets, B, T_total, d, pooled,
+                              c->piece_a, c->piece_b, c->piece_ms, nullptr, nullptr, status, stream));
   }
   {
     LaunchScope ls(c, EGTP_K_POOL_COMBINE, stream);
-    EGTP_CUDA_TRY(launch_pool_combine(offsets, B, d, take_max, c->piece_a, c->piece_b, pooled, status, stream));
+    EGTP_CUDA_TRY(launch_pool_combine(offsets, B, T_total, d, mode, c->piece_a, c->piece_b, c->piece_ms, pooled, nullptr,
+                                      nullptr, staged ? c->zcat : nullptr, status, stream));
   }
-  if (head && yhat_out) return run_head(c, head, pooled, d, B, yhat_out, nullptr, status, stream);
+  if (staged) return run_head_staged(c, head, B, yhat_out, nullptr, status, stream);
+  if (want_head) return run_head(c, head, pooled, d, B, yhat_out, nullptr, status, stream);
   return EGTP_OK;
 }
 
@@ -801,6 +822,7 @@ int egtp_predict_host(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head
                       float* pooled_host, int32_t* status_host, void* stream_v) {
   if (!c || !lm || !head || !hidden_host || !offsets_host || !yhat_host || !status_host) return EGTP_ERR_INVALID_ARG;
   if (B <= 0 || T_total <= 0) return EGTP_ERR_INVALID_ARG;
+  if (!c->host_staging) return EGTP_ERR_UNSUPPORTED;
   if (T_total > c->max_tokens || B > c->max_batch || lm->d > c->max_d) return EGTP_ERR_CAPACITY;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
   if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
@@ -847,7 +869,7 @@ int plp_state_create(egtp_ctx* c, plp_state** out, int32_t num_slots, int32_t d)
   if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
   plp_state* st = new (std::nothrow) plp_state();
   if (!st) return EGTP_ERR_CUDA;
-  st->ctx = c; st->num_slots = num_slots; st->d = d;
+  st->ctx = c; st->device = c->device; st->num_slots = num_slots; st->d = d;
   bool ok = cudaMalloc(reinterpret_cast<void**>(&st->m), sizeof(float) * num_slots) == cudaSuccess;
   ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->s), sizeof(float) * num_slots) == cudaSuccess;
   ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->acc), sizeof(float) * static_cast<size_t>(num_slots) * d) == cudaSuccess;
@@ -869,7 +891,7 @@ int plp_state_create(egtp_ctx* c, plp_state** out, int32_t num_slots, int32_t d)
 
 int plp_state_destroy(plp_state* st) {
   if (!st) return EGTP_ERR_INVALID_ARG;
-  cudaSetDevice(st->ctx->device);
+  cudaSetDevice(st->device);
   cudaFree(st->m); cudaFree(st->s); cudaFree(st->acc);
   cudaFree(st->proj); cudaFree(st->src_proj); cudaFree(st->head_g);
   delete st;
@@ -879,7 +901,7 @@ int plp_state_destroy(plp_state* st) {
 int plp_state_export(plp_state* st, float* m, float* s, float* acc, void* stream_v) {
   if (!st || !m || !s || !acc) return EGTP_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
-  if (cudaSetDevice(st->ctx->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  if (cudaSetDevice(st->device) != cudaSuccess) return EGTP_ERR_CUDA;
   EGTP_CUDA_TRY(cudaMemcpyAsync(m, st->m, sizeof(float) * st->num_slots, cudaMemcpyDeviceToDevice, stream));
   EGTP_CUDA_TRY(cudaMemcpyAsync(s, st->s, sizeof(float) * st->num_slots, cudaMemcpyDeviceToDevice, stream));
   EGTP_CUDA_TRY(cudaMemcpyAsync(acc, st->acc, sizeof(float) * static_cast<size_t>(st->num_slots) * st->d,
@@ -890,7 +912,7 @@ int plp_state_export(plp_state* st, float* m, float* s, float* acc, void* stream
 int plp_state_import(plp_state* st, const float* m, const float* s, const float* acc, void* stream_v) {
   if (!st || !m || !s || !acc) return EGTP_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
-  if (cudaSetDevice(st->ctx->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  if (cudaSetDevice(st->device) != cudaSuccess) return EGTP_ERR_CUDA;
   EGTP_CUDA_TRY(cudaMemcpyAsync(st->m, m, sizeof(float) * st->num_slots, cudaMemcpyDeviceToDevice, stream));
   EGTP_CUDA_TRY(cudaMemcpyAsync(st->s, s, sizeof(float) * st->num_slots, cudaMemcpyDeviceToDevice, stream));
   EGTP_CUDA_TRY(cudaMemcpyAsync(st->acc, acc, sizeof(float) * static_cast<size_t>(st->num_slots) * st->d,
@@ -930,9 +952,9 @@ int plp_step(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head
       rc = project_rows(c, head, src_pooled, st->d, n_src, st->src_proj, head->m_h, status, stream);
       if (rc != EGTP_OK) return rc;
     }
-    rc = run_lmhead(c, lm, hidden_step, ldh, B_live, status, stream, &plan, head->W1, head->m_h, st->head_g);
+    rc = run_lmhead(c, lm, hidden_step, ldh, B_live, status, stream, &plan, head->W1, head->m_h, st->head_g, st->g_rows,
+                    st->ldg_max);
     if (rc != EGTP_OK) return rc;
-    if (plan.rows_pad > st->g_rows || plan.head_cols_pad > st->ldg_max) return EGTP_ERR_CAPACITY;
     LaunchScope ls(c, EGTP_K_PLP_UPDATE, stream);
     EGTP_CUDA_TRY(launch_plp_update_bound(hidden_step, ldh, c->partials, plan.slots, plan.slots * 3, 3, Hstep_out, slot_ids,
                                           reset_src, src_m, src_s, src_pooled, st->src_proj, n_src, B_live, st->d,
@@ -990,11 +1012,7 @@ int egtp_entropy_from_logits(egtp_ctx* c, const void* logits, int64_t ldl, int32
   if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
   int32_t* status = status_dev ? status_dev : c->status;
   if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
-  int rc = run_logits_entropy(c, logits, ldl, logits_dtype, rows, V, status, stream, &slots);
-  if (rc != EGTP_OK) return rc;
-  LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
-  EGTP_CUDA_TRY(launch_entropy_merge(c->partials, slots, slots * 3, 3, rows, 0, H_out, nullptr, 0, nullptr, nullptr, status, stream));
-  return EGTP_OK;
+  return run_logits_entropy(c, logits, ldl, logits_dtype, rows, V, status, stream, &slots, H_out);
 }
 
 int plp_step_from_logits(egtp_ctx* c, plp_state* st, const void* logits, int64_t ldl, int32_t logits_dtype, int32_t V,
@@ -1069,7 +1087,7 @@ int egtp_entropy_from_partials(egtp_ctx* c, const float* gathered, int32_t num_s
   int32_t* status = status_dev ? status_dev : c->status;
   if (!status_dev) EGTP_CUDA_TRY(cudaMemsetAsync(c->status, 0, sizeof(int32_t), stream));
   LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
-  EGTP_CUDA_TRY(launch_entropy_merge(gathered, num_shards, 3, rows * 3, rows, 0, H_out, nullptr, 0, nullptr, nullptr, status,
+  EGTP_CUDA_TRY(launch_entropy_merge(gathered, num_shards, 3, rows * 3, rows, 0, H_out, nullptr, 0, nullptr, -1, status,
                                      stream));
   return EGTP_OK;
 }
@@ -1106,6 +1124,7 @@ int plp_step_host(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp
                   int32_t* status_host, void* stream_v) {
   if (!c || !st || !lm || !head || !hidden_step_host || !yrem_host || !status_host) return EGTP_ERR_INVALID_ARG;
   if (B_live <= 0) return EGTP_ERR_INVALID_ARG;
+  if (!c->host_staging) return EGTP_ERR_UNSUPPORTED;
   if (B_live > c->max_batch || lm->d > c->max_d) return EGTP_ERR_CAPACITY;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
   if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;

@@ -40,12 +40,11 @@ struct LmheadPlan {
 
 // Picks chunks / grouping for T rows; slot_limit bounds chunks * kEpiSplit * rows_pad by the
 // partial buffer's capacity (in rows x slots).
-// pair_workers >= 0 states how many CTA pairs the device can co-schedule (default: what was measured on the
-// current device).  force_chunks > 0 overrides the number of vocabulary chunks of prompt batches (clamped to the workspace).
+// pair_workers states how many CTA pairs the device can co-schedule (lmhead_prepare_device measures it; 0 = none).  force_chunks > 0 overrides the number of vocabulary chunks of prompt batches (clamped to the workspace).
 // head_cols > 0: that many rows of a second matrix (the head's W1) are appended to the vocabulary as
 // extra columns whose raw products the kernel writes out (bf16, one-CTA shapes only).
 LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity,
-                            int mode, int head_cols = 0, int force_chunks = 0, int pair_workers = -1);
+                            int mode, int head_cols, int force_chunks, int pair_workers);
 
 // Launch shape for W1 hidden[i] alone (no vocabulary): the head columns of the prompt shape with K split over
 // up to max_splits units, each writing its own slice head_g[split][rows_pad][head_cols_pad].
@@ -54,8 +53,9 @@ LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms
 LmheadPlan make_headproj_plan(int64_t T, int d, int m_h, int elem_bytes, int num_sms, int max_splits,
                               int a_repeats = 1);
 
-// Opts the kernels into their dynamic shared-memory size on the current device (once per device).
-cudaError_t lmhead_prepare_device();
+// Opts the kernels into their dynamic shared-memory size on the current device and reports how many CTA pairs of
+// the pair kernels that device can hold at once.
+cudaError_t lmhead_prepare_device(int* pair_workers_out);
 
 // partials layout: [rows_pad][slots][3] floats: (m, s, t2) with m the running max logit,
 // s = sum 2^((x-m) log2 e), t2 = sum 2^(...) * (x-m) log2 e over the slot's vocabulary range.
@@ -74,7 +74,7 @@ struct LmheadMaps {
 cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const LmheadMaps& maps, int64_t T, int V,
                                   float* partials, int32_t* status, cudaStream_t stream, float* head_g = nullptr);
 
-// ---- K2: entropy merge, Eq. 3 weights, Eq. 4 pooling -------------------------------------
+// ---- K2: entropy merge, Eq. 3-4 pooling -------------------------------------
 constexpr int kPoolChunkTokens = 64;   // tokens per first-stage pooling chunk
 constexpr int kPoolThreads = 128;      // each thread owns 8 consecutive channels
 
@@ -84,25 +84,31 @@ cudaError_t launch_validate_offsets(const int32_t* offsets, int B, int64_t T, in
 // the batch (H, weights and segment ids are indexed by the batch-wide token index)
 cudaError_t launch_partials_reduce(const float* partials, int slots, int64_t rows, float* out, const int32_t* status,
                                    cudaStream_t stream);
+// T_check >= 0: the launch also checks the offsets against that token count (EGTP_ERR_BAD_OFFSETS in *status)
 cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t row_stride, int64_t slot_stride, int64_t T,
-                                 int64_t row0, float* H,
-                                 const int32_t* offsets, int B, int32_t* seg_id_out, float* weights_zero,
-                                 const int32_t* status, cudaStream_t stream);
+                                 int64_t row0, float* H, const int32_t* offsets, int B, int32_t* seg_id_out,
+                                 int64_t T_check, int32_t* status, cudaStream_t stream);
 
-cudaError_t launch_segment_weights(const float* H, const int32_t* offsets, int B, float inv_alpha, float* weights,
-                                   float* seg_m, float* seg_s, const int32_t* status, cudaStream_t stream);
+// Eq. 3 weights as an output: w_i = exp(H_i/alpha - M_b) / Z_b from the per-prompt state the pooling left (0 outside prompts)
+cudaError_t launch_token_weights(const float* H, const int32_t* offsets, int B, int64_t T, float inv_alpha,
+                                 const float* seg_m, const float* seg_s, float* weights, const int32_t* status,
+                                 cudaStream_t stream);
 
-// weights of average (w = 1/n) or last-token (one-hot) pooling for every prompt
-cudaError_t launch_baseline_weights(const int32_t* offsets, int B, int mode, float* weights, const int32_t* status,
-                                    cudaStream_t stream);
-
-// take_max: channel-wise maximum instead of the weighted sum (weights unused)
-cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, bool take_max, const float* weights,
+// Pooling over the prompts' token spans.  mode 0: entropy-weighted (Eq. 3-4; H and inv_alpha give the weights, which
+// are formed on the fly relative to chunk-local maxima and never stored); EGTP_POOL_MEAN / _MAX / _LAST: the
+// alternatives of the paper's ablation (H unused).  piece_a / piece_b [chunks][d] and piece_ms [2 * chunks][2]
+// (chunks = ceil(T / kPoolChunkTokens)) receive the pieces of prompts that span several chunks; seg_m / seg_s (may be
+// NULL) the softmax state (M, Z) of prompts finished in one chunk.
+cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, int mode, const float* H, float inv_alpha,
                         const int32_t* offsets, int B, int64_t T, int d, float* pooled, float* piece_a,
-                        float* piece_b, const int32_t* status, cudaStream_t stream);
+                        float* piece_b, float* piece_ms, float* seg_m, float* seg_s, const int32_t* status,
+                        cudaStream_t stream);
 
-cudaError_t launch_pool_combine(const int32_t* offsets, int B, int d, bool take_max, const float* piece_a,
-                                const float* piece_b, float* pooled, const int32_t* status, cudaStream_t stream);
+// Merges the pieces (same T and mode as the launch_pool before it), zero-fills empty prompts, completes seg_m / seg_s and,
+// with zcat != NULL, also writes every pooled row as [hi | lo] bf16 halves: zcat [B][2 d]
+cudaError_t launch_pool_combine(const int32_t* offsets, int B, int64_t T, int d, int mode, const float* piece_a,
+                                const float* piece_b, const float* piece_ms, float* pooled, float* seg_m, float* seg_s,
+                                void* zcat, const int32_t* status, cudaStream_t stream);
 
 // dst [dst_rows][row_bytes] <- the first src_rows rows of src (ld_bytes apart), the other rows zero.
 // row_bytes and ld_bytes are multiples of 16, both pointers 16-byte aligned.
@@ -111,9 +117,12 @@ cudaError_t launch_pad_rows(const void* src, int64_t ld_bytes, int src_rows, int
 
 // ---- Eq. 2 from logits already in memory -------------------------------------------------------
 int logits_entropy_pick_splits(int64_t rows, int V, int num_sms);
-// partials [rows][splits][3] in the layout of the LM-head kernel's partials
+// partials [rows][splits][3] in the layout of the LM-head kernel's partials.  H_out != NULL: the kernel also merges
+// each row's partials into H_out[row] (the last block of the row to finish does it); arrivals [rows] int32 must
+// then be zero on entry and is zero again on exit.
 cudaError_t launch_logits_entropy(const void* logits, int64_t ldl, bool bf16, int64_t rows, int V, int splits,
-                                  float* partials, const int32_t* status, cudaStream_t stream);
+                                  float* partials, float* H_out, int32_t* arrivals, const int32_t* status,
+                                  cudaStream_t stream);
 
 // ---- K3: head ------------------------------------------------------------------------------
 struct HeadArgs {

@@ -804,11 +804,9 @@ cudaError_t launch_pair(const LmheadPlan& plan, const LmheadMaps& m, const KPara
   return cudaGetLastError();
 }
 
-// CTA pairs that can be resident at once on the current device (set by lmhead_prepare_device).
-int g_pair_workers_max = 0;
-
+// *pair_workers receives the smaller of its value and the CTA pairs of this kernel that can be resident at once
 template <bool kTf32, int kBBox, bool kFuse = false>
-cudaError_t prepare_pair(int num_sms) {
+cudaError_t prepare_pair(int num_sms, int* pair_workers) {
   auto kernel = kBBox == 32 ? lmhead_entropy_pair_kernel<kTf32, kBBox, kPairWideStages, 2, kFuse>
                             : lmhead_entropy_pair_kernel<kTf32, kBBox, kPairStages, 1, kFuse>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes);
@@ -825,7 +823,7 @@ cudaError_t prepare_pair(int num_sms) {
   int clusters = 0;
   e = cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg);
   if (e != cudaSuccess) return e;
-  g_pair_workers_max = g_pair_workers_max == 0 ? clusters : std::min(g_pair_workers_max, clusters);
+  *pair_workers = std::min(*pair_workers, clusters);
   return cudaSuccess;
 }
 
@@ -843,9 +841,9 @@ static_assert(kShapeDecode2.mt == 2 && kShapeDecode2.bn == 256 && kShapeDecode2.
 
 LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms, int64_t slot_row_capacity,
                             int mode, int head_cols, int force_chunks, int pair_workers) {
-  // CTA pairs the device can co-schedule: what lmhead_prepare_device found, unless the caller states a number
-  // (planning for a device that is not present)
-  const int pair_cap = pair_workers >= 0 ? pair_workers : g_pair_workers_max;
+  // CTA pairs the device can co-schedule (what lmhead_prepare_device found on the context's device, or a number
+  // the caller states when planning for a device that is not present)
+  const int pair_cap = pair_workers;
   LmheadPlan pl{};
   // decode batches of 129..256 rows run as CTA pairs on 256 x 512 tiles unless single CTAs are asked for or the
   // device cannot co-schedule the pairs; prompt batches run as pairs only on request (and never with head columns)
@@ -969,7 +967,7 @@ LmheadPlan make_headproj_plan(int64_t T, int d, int m_h, int elem_bytes, int num
   return pl;
 }
 
-cudaError_t lmhead_prepare_device() {
+cudaError_t lmhead_prepare_device(int* pair_workers_out) {
   cudaError_t e;
   if ((e = prepare_shape<false, EGTP_SHAPE_PROMPT>()) != cudaSuccess) return e;
   if ((e = prepare_shape<false, EGTP_SHAPE_DECODE1>()) != cudaSuccess) return e;
@@ -982,10 +980,12 @@ cudaError_t lmhead_prepare_device() {
   int device = 0, num_sms = 0;
   if ((e = cudaGetDevice(&device)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess) return e;
-  g_pair_workers_max = 0;
-  if ((e = prepare_pair<false, 128>(num_sms)) != cudaSuccess) return e;
-  if ((e = prepare_pair<false, 32>(num_sms)) != cudaSuccess) return e;
-  return prepare_pair<false, 32, true>(num_sms);
+  int pairs = num_sms / 2;
+  if ((e = prepare_pair<false, 128>(num_sms, &pairs)) != cudaSuccess) return e;
+  if ((e = prepare_pair<false, 32>(num_sms, &pairs)) != cudaSuccess) return e;
+  if ((e = prepare_pair<false, 32, true>(num_sms, &pairs)) != cudaSuccess) return e;
+  *pair_workers_out = pairs;
+  return cudaSuccess;
 }
 
 cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const LmheadMaps& maps, int64_t T, int V,

@@ -3,7 +3,8 @@
 // step; the entropy then costs one pass over those values instead of a second LM-head GEMM.
 // HBM-bound: 16-byte coalesced loads, one running (m, s, t2) per thread (same definition as the
 // LM-head kernel's epilogue), warp-shuffle and shared-memory combine, one partial per
-// (row, vocabulary split) in the layout the merge kernels read.
+// (row, vocabulary split) in the layout the merge kernels read; when the caller wants H itself, the last block
+// of a row to finish merges the row's partials, so that entropy from logits is a single launch.
 #include "kernels.h"
 #include "entropy_merge.cuh"
 #include "sm100_ptx.cuh"
@@ -18,7 +19,7 @@ namespace egtp {
 namespace {
 
 constexpr int kLogitsThreads = 128;
-constexpr int kLogitsBlocksPerSm = 7;   // 72 registers per thread at most: 28 warps per SM
+constexpr int kLogitsBlocksPerSm = 8;   // 64 registers per thread at most: 32 warps per SM
 constexpr float kLog2e = 1.4426950408889634f;
 
 // Eight consecutive logits as they come out of memory.  bf16 values stay packed until they are consumed: the
@@ -66,24 +67,27 @@ struct Vec8<float> {
 template <typename T>
 constexpr int kVecPerBatch = sizeof(T) == 2 ? 4 : 2;
 
-// Running state of one thread: max m and four independent (s, t2) accumulators (short dependency chains).
+// Running state of one thread: max m and four independent (s, t2) accumulators kept as two packed pairs, so that
+// the three fp32 operations per logit besides the exponential (y = x log2 e - m log2 e, s += e, t2 += e y) are
+// issued two logits at a time (fma / add on f32x2).
 struct ThreadState {
   float m;
-  float s[4];
-  float t[4];
+  uint64_t s[2];
+  uint64_t t[2];
   __device__ __forceinline__ void init() {
     m = kNegBig;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) { s[i] = 0.f; t[i] = 0.f; }
+    s[0] = s[1] = t[0] = t[1] = pack_f32x2(0.f, 0.f);
   }
   __device__ __forceinline__ void raise_max(float cmax) {
     if (cmax > m) {
+      // new running max: s <- s r, t2 <- r (t2 + dm s) with dm = (m - cmax) log2 e, r = 2^dm
       const float dm = (m - cmax) * kLog2e;
       const float r = ex2_approx(dm);
+      const uint64_t r2 = pack_f32x2(r, r), dm2 = pack_f32x2(dm, dm);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        t[i] = r * fmaf(dm, s[i], t[i]);
-        s[i] *= r;
+      for (int i = 0; i < 2; ++i) {
+        t[i] = mul_f32x2(r2, fma_f32x2(dm2, s[i], t[i]));
+        s[i] = mul_f32x2(s[i], r2);
       }
       m = cmax;
     }
@@ -96,21 +100,27 @@ struct ThreadState {
     for (int u = 1; u < kN; ++u) cmax = fmaxf(cmax, x[u].vmax());
     raise_max(cmax);
     const float neg_m_l2 = -m * kLog2e;
+    const uint64_t l2 = pack_f32x2(kLog2e, kLog2e), nm2 = pack_f32x2(neg_m_l2, neg_m_l2);
 #pragma unroll
     for (int u = 0; u < kN; ++u) {
       float v[8];
       x[u].get(v);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float y = fmaf(v[j], kLog2e, neg_m_l2);
-        const float e = ex2_approx(y);
-        s[(u + j) & 3] += e;
-        t[(u + j) & 3] = fmaf(e, y, t[(u + j) & 3]);
+      for (int j = 0; j < 4; ++j) {
+        const uint64_t y2 = fma_f32x2(pack_f32x2(v[2 * j], v[2 * j + 1]), l2, nm2);
+        float y0, y1;
+        unpack_f32x2(y2, y0, y1);
+        const uint64_t e2 = pack_f32x2(ex2_approx(y0), ex2_approx(y1));
+        s[j & 1] = add_f32x2(s[j & 1], e2);
+        t[j & 1] = fma_f32x2(e2, y2, t[j & 1]);
       }
     }
   }
   __device__ __forceinline__ EntropyPartial total() const {
-    return {m, (s[0] + s[1]) + (s[2] + s[3]), (t[0] + t[1]) + (t[2] + t[3])};
+    float s0, s1, s2, s3, t0, t1, t2, t3;
+    unpack_f32x2(s[0], s0, s1); unpack_f32x2(s[1], s2, s3);
+    unpack_f32x2(t[0], t0, t1); unpack_f32x2(t[1], t2, t3);
+    return {m, (s0 + s1) + (s2 + s3), (t0 + t1) + (t2 + t3)};
   }
 };
 
@@ -128,11 +138,13 @@ __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 v) { retu
 template <typename T>
 __global__ void __launch_bounds__(kLogitsThreads, kLogitsBlocksPerSm)
 logits_entropy_kernel(const T* __restrict__ logits, int64_t ldl, int V, int cols_per_split, int splits,
-                      float* __restrict__ partials, const int32_t* __restrict__ status) {
+                      float* __restrict__ partials, float* __restrict__ H_out, int32_t* __restrict__ arrivals,
+                      const int32_t* __restrict__ status) {
   if (*status != 0) return;
   __shared__ EntropyPartial red[kLogitsThreads / 32];
-  const int split = blockIdx.x;
-  const int64_t row = blockIdx.y;
+  __shared__ int is_last;
+  const int64_t row = blockIdx.x / splits;
+  const int split = static_cast<int>(blockIdx.x - row * splits);
   const int c0 = split * cols_per_split;
   const int c1 = min(V, c0 + cols_per_split);
   const T* base = logits + row * ldl + c0;
@@ -180,6 +192,21 @@ logits_entropy_kernel(const T* __restrict__ logits, int64_t ldl, int V, int cols
     for (int w = 1; w < kLogitsThreads / 32; ++w) acc = combine_partials(acc, red[w]);
     float* dst = partials + (row * splits + split) * 3;
     dst[0] = acc.m; dst[1] = acc.s; dst[2] = acc.t2;
+    if (H_out != nullptr) {
+      // the block that finds all other partials of its row already written merges them (slot order, so the result
+      // does not depend on which block that is) and leaves the row's arrival counter at zero for the next call
+      __threadfence();
+      is_last = atomicAdd(arrivals + row, 1) == splits - 1 ? 1 : 0;
+    }
+  }
+  if (H_out == nullptr) return;
+  __syncthreads();
+  if (is_last == 0 || wid != 0) return;
+  __threadfence();
+  const float h = merge_partials_warp(partials + row * splits * 3, splits, 3, lane);
+  if (lane == 0) {
+    H_out[row] = h;
+    arrivals[row] = 0;
   }
 }
 
@@ -194,16 +221,19 @@ int logits_entropy_pick_splits(int64_t rows, int V, int num_sms) {
 }
 
 cudaError_t launch_logits_entropy(const void* logits, int64_t ldl, bool bf16, int64_t rows, int V, int splits,
-                                  float* partials, const int32_t* status, cudaStream_t stream) {
+                                  float* partials, float* H_out, int32_t* arrivals, const int32_t* status,
+                                  cudaStream_t stream) {
   int cols_per_split = (V + splits - 1) / splits;
   cols_per_split = (cols_per_split + 7) / 8 * 8;
-  dim3 grid(splits, static_cast<unsigned>(rows));
+  if (rows * splits >= (int64_t{1} << 31) || (H_out != nullptr && arrivals == nullptr)) return cudaErrorInvalidValue;
+  const unsigned grid = static_cast<unsigned>(rows * splits);      // block = (row, split), splits of a row adjacent
   if (bf16) {
     logits_entropy_kernel<__nv_bfloat16><<<grid, kLogitsThreads, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(logits), ldl, V, cols_per_split, splits, partials, status);
+        static_cast<const __nv_bfloat16*>(logits), ldl, V, cols_per_split, splits, partials, H_out, arrivals, status);
   } else {
     logits_entropy_kernel<float><<<grid, kLogitsThreads, 0, stream>>>(static_cast<const float*>(logits), ldl, V,
-                                                                     cols_per_split, splits, partials, status);
+                                                                     cols_per_split, splits, partials, H_out, arrivals,
+                                                                     status);
   }
   return cudaGetLastError();
 }

@@ -1,5 +1,5 @@
-// Offsets check, entropy merge (Eq. 2), per-prompt softmax weights (Eq. 3) and the
-// entropy-weighted ragged pooling (Eq. 4).  HBM-bound work: plain coalesced 16-byte loads,
+// Offsets check, entropy merge (Eq. 2) and the entropy-weighted ragged pooling with its softmax over each
+// prompt's entropies folded in (Eq. 3-4).  HBM-bound work: plain coalesced 16-byte loads,
 // fp32 accumulation, warp-shuffle / block reductions, no floating-point atomics.
 #include "kernels.h"
 #include "entropy_merge.cuh"
@@ -33,14 +33,18 @@ __device__ __forceinline__ int upper_segment(const int32_t* __restrict__ off, in
 }
 
 // --------------------------------------------------------------------------- offsets check
-__global__ void validate_offsets_kernel(const int32_t* __restrict__ off, int B, int64_t T, int32_t* status) {
+__device__ __forceinline__ bool offsets_bad(const int32_t* __restrict__ off, int B, int64_t T) {
   bool bad = false;
   for (int b = threadIdx.x; b <= B; b += blockDim.x) {
     const int64_t v = off[b];
     if (v < 0 || v > T) bad = true;
     if (b < B && static_cast<int64_t>(off[b + 1]) < v) bad = true;
   }
-  if (__syncthreads_or(bad ? 1 : 0)) {
+  return bad;
+}
+
+__global__ void validate_offsets_kernel(const int32_t* __restrict__ off, int B, int64_t T, int32_t* status) {
+  if (__syncthreads_or(offsets_bad(off, B, T) ? 1 : 0)) {
     if (threadIdx.x == 0) atomicCAS(status, 0, EGTP_ERR_BAD_OFFSETS);
   }
 }
@@ -48,12 +52,17 @@ __global__ void validate_offsets_kernel(const int32_t* __restrict__ off, int B, 
 // --------------------------------------------------------------------------- Eq. 2: merge
 // One warp per token: lanes stride over the token's (m, s, t2) partials (contiguous in memory),
 // fold them in a fixed order, then combine across lanes: H = ln S - ln2 * T2 / S.
-// Also writes the token's prompt index and clears its weight.
+// Also writes the token's prompt index.  With T_check >= 0, block 0 first checks the offsets against that
+// token count (the kernels that index tokens through the offsets come later in the stream and see the status).
 __global__ void entropy_merge_kernel(const float* __restrict__ partials, int slots, int64_t row_stride,
                                      int64_t slot_stride, int64_t T, int64_t row0, float* __restrict__ H, const int32_t* __restrict__ off, int B,
-                                     int32_t* __restrict__ seg_id, float* __restrict__ weights,
-                                     const int32_t* __restrict__ status) {
+                                     int32_t* __restrict__ seg_id, int64_t T_check, int32_t* __restrict__ status) {
   if (*status != 0) return;
+  if (T_check >= 0 && blockIdx.x == 0) {
+    if (__syncthreads_or(offsets_bad(off, B, T_check) ? 1 : 0)) {
+      if (threadIdx.x == 0) atomicCAS(status, 0, EGTP_ERR_BAD_OFFSETS);
+    }
+  }
   const int lane = threadIdx.x & 31;
   const int64_t i = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (i >= T) return;
@@ -61,7 +70,6 @@ __global__ void entropy_merge_kernel(const float* __restrict__ partials, int slo
   if (lane == 0) {
     const int64_t g = row0 + i;      // token index in the whole batch (the partials may cover one piece of it)
     H[g] = h;
-    if (weights != nullptr) weights[g] = 0.f;
     if (seg_id != nullptr) {
       int sid = -1;
       if (B > 0 && g >= off[0] && g < off[B]) sid = upper_segment(off, B, g);
@@ -86,71 +94,24 @@ __global__ void partials_reduce_kernel(const float* __restrict__ partials, int s
   }
 }
 
-// --------------------------------------------------------------------------- Eq. 3: weights
-// One block per prompt: M = max_i H_i/alpha, Z = sum_i exp(H_i/alpha - M), w_i = exp(.)/Z.
-__global__ void segment_weights_kernel(const float* __restrict__ H, const int32_t* __restrict__ off, int B,
-                                       float inv_alpha, float* __restrict__ weights, float* __restrict__ seg_m,
-                                       float* __restrict__ seg_s, const int32_t* __restrict__ status) {
+// --------------------------------------------------------------------------- Eq. 3: weights as an output
+// The pooling kernels below never materialise the normalised weights; a caller that wants them gets
+// w_i = exp(H_i/alpha - M_b) / Z_b from the per-prompt state (M_b, Z_b) the pooling left behind (0 outside prompts).
+__global__ void token_weights_kernel(const float* __restrict__ H, const int32_t* __restrict__ off, int B, int64_t T,
+                                     float inv_alpha, const float* __restrict__ seg_m, const float* __restrict__ seg_s,
+                                     float* __restrict__ weights, const int32_t* __restrict__ status) {
   if (*status != 0) return;
-  __shared__ float red[32];
-  __shared__ float bcast;
-  const int b = blockIdx.x;
-  const int s0 = off[b], s1 = off[b + 1];
-  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
-  if (s1 <= s0) {
-    if (tid == 0) {
-      if (seg_m) seg_m[b] = -INFINITY;
-      if (seg_s) seg_s[b] = 0.f;
-    }
-    return;
+  const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= T) return;
+  float w = 0.f;
+  if (B > 0 && i >= off[0] && i < off[B]) {
+    const int b = upper_segment(off, B, i);
+    w = expf(H[i] * inv_alpha - seg_m[b]) / seg_s[b];
   }
-  float mx = -INFINITY;
-  for (int i = s0 + tid; i < s1; i += blockDim.x) mx = fmaxf(mx, H[i] * inv_alpha);
-  mx = warp_max(mx);
-  if (lane == 0) red[wid] = mx;
-  __syncthreads();
-  if (wid == 0) {
-    float v = lane < nw ? red[lane] : -INFINITY;
-    v = warp_max(v);
-    if (lane == 0) bcast = v;
-  }
-  __syncthreads();
-  const float M = bcast;
-  float sum = 0.f;
-  for (int i = s0 + tid; i < s1; i += blockDim.x) sum += expf(H[i] * inv_alpha - M);
-  sum = warp_sum(sum);
-  __syncthreads();
-  if (lane == 0) red[wid] = sum;
-  __syncthreads();
-  if (wid == 0) {
-    float v = lane < nw ? red[lane] : 0.f;
-    v = warp_sum(v);
-    if (lane == 0) bcast = v;
-  }
-  __syncthreads();
-  const float Z = bcast;
-  const float invZ = 1.f / Z;
-  for (int i = s0 + tid; i < s1; i += blockDim.x) weights[i] = expf(H[i] * inv_alpha - M) * invZ;
-  if (tid == 0) {
-    if (seg_m) seg_m[b] = M;
-    if (seg_s) seg_s[b] = Z;
-  }
+  weights[i] = w;
 }
 
-// Weights of the pooling alternatives in the paper's ablation (Table 3) that are weighted sums:
-// average pooling (w = 1/n) and last-token pooling (w = 1 on the prompt's last token).
-__global__ void baseline_weights_kernel(const int32_t* __restrict__ off, int B, int mode, float* __restrict__ weights,
-                                        const int32_t* __restrict__ status) {
-  if (*status != 0) return;
-  const int b = blockIdx.x;
-  const int s0 = off[b], s1 = off[b + 1];
-  if (s1 <= s0) return;
-  const float inv_n = 1.f / static_cast<float>(s1 - s0);
-  for (int i = s0 + threadIdx.x; i < s1; i += blockDim.x)
-    weights[i] = mode == EGTP_POOL_MEAN ? inv_n : (i == s1 - 1 ? 1.f : 0.f);
-}
-
-// --------------------------------------------------------------------------- Eq. 4: pooling
+// --------------------------------------------------------------------------- Eq. 3 + Eq. 4: pooling
 template <typename T>
 struct Row8;
 template <>
@@ -179,19 +140,46 @@ __device__ __forceinline__ void store8(float* p, const float (&v)[8]) {
   reinterpret_cast<float4*>(p)[0] = make_float4(v[0], v[1], v[2], v[3]);
   reinterpret_cast<float4*>(p)[1] = make_float4(v[4], v[5], v[6], v[7]);
 }
+__device__ __forceinline__ void load8f(const float* p, float (&v)[8]) {
+  const float4 a = reinterpret_cast<const float4*>(p)[0], b = reinterpret_cast<const float4*>(p)[1];
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+  v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
 
-// Block (c, y): tokens [c*64, (c+1)*64) clipped to [offsets[0], offsets[B]), channels
-// [(y*128 + tid)*8, +8).  A prompt that lies wholly inside the chunk is finished here; a prompt
-// that crosses chunk borders leaves one piece per chunk: piece_a[c] if it entered from the
-// left, piece_b[c] if it starts here and leaves to the right.  The combine kernel adds the
+// [hi | lo] halves of a row of fp32 values: hi = bf16(x), lo = bf16(x - hi); the input format of the head's
+// tensor-core layer 1
+__device__ __forceinline__ void store8_hi_lo(__nv_bfloat16* row, int d, int col, const float (&v)[8]) {
+  __align__(16) __nv_bfloat16 hi[8], lo[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    hi[k] = __float2bfloat16_rn(v[k]);
+    lo[k] = __float2bfloat16_rn(v[k] - __bfloat162float(hi[k]));
+  }
+  *reinterpret_cast<uint4*>(row + col) = *reinterpret_cast<const uint4*>(hi);
+  *reinterpret_cast<uint4*>(row + d + col) = *reinterpret_cast<const uint4*>(lo);
+}
+
+// Pooling modes: the paper's entropy-weighted pooling (Eq. 3-4) and the alternatives of its ablation (Table 3).
+// All but the maximum are weighted sums sum_i w_i h_i / sum_i w_i with unnormalised weights
+//   entropy: w_i = exp(H_i/alpha - m), m = the largest H_i/alpha among the tokens summed together
+//   mean:    w_i = 1                    last: w_i = 1 for the prompt's last token, else 0
+// so one kernel serves them: a block sums a run of tokens with weights relative to the run's own m and leaves
+// (m, sum w, sum w h); runs of one prompt are merged later by rescaling to the common maximum (the same
+// recurrence as the PLP state, Eq. 8).  The normalised weights of Eq. 3 are never stored.
+enum : int { kPoolEntropy = 0, kPoolMean = 1, kPoolMax = 2, kPoolLast = 3 };
+
+// Block (c, y): tokens [c*64, (c+1)*64) clipped to [offsets[0], offsets[B]), channels [(y*128 + tid)*8, +8).
+// A prompt that lies wholly inside the chunk is finished here (pooled row, and its (M, Z) by the y = 0 block); a
+// prompt that crosses chunk borders leaves one piece per chunk: piece_a[c] if it entered from the left, piece_b[c]
+// if it starts here and leaves to the right, each with its (m, sum w) in piece_ms.  The combine kernel merges the
 // pieces of each prompt in chunk order.
-// With kMax the weights are ignored and the channel-wise maximum is taken instead of the weighted sum
-// (max pooling, Table 3); pieces of a prompt that spans chunks are then combined with max.
-template <typename T, bool kMax>
+template <typename T, int kMode>
 __global__ void __launch_bounds__(kPoolThreads)
-pool_kernel(const T* __restrict__ hidden, int64_t ldh, const float* __restrict__ weights,
+pool_kernel(const T* __restrict__ hidden, int64_t ldh, const float* __restrict__ H, float inv_alpha,
             const int32_t* __restrict__ off, int B, int d, float* __restrict__ pooled,
-            float* __restrict__ piece_a, float* __restrict__ piece_b, const int32_t* __restrict__ status) {
+            float* __restrict__ piece_a, float* __restrict__ piece_b, float2* __restrict__ ms_a,
+            float2* __restrict__ ms_b, float* __restrict__ seg_m, float* __restrict__ seg_s,
+            const int32_t* __restrict__ status) {
   if (*status != 0) return;
   const int64_t c = blockIdx.x;
   const int col = (blockIdx.y * kPoolThreads + threadIdx.x) * 8;
@@ -199,98 +187,168 @@ pool_kernel(const T* __restrict__ hidden, int64_t ldh, const float* __restrict__
   int64_t t0 = max(c_lo, static_cast<int64_t>(off[0]));
   const int64_t t1 = min(c_hi, static_cast<int64_t>(off[B]));
   if (t0 >= t1 || col >= d) return;
+  const bool scribe = blockIdx.y == 0 && threadIdx.x == 0;      // writes the per-run scalars
   int b = upper_segment(off, B, t0);
   while (t0 < t1) {
     const int64_t seg_begin = off[b], seg_end = off[b + 1];
     if (seg_end <= t0) { ++b; continue; }       // empty prompts own no token
     const int64_t run_end = min(seg_end, t1);
+    // the run's reference point and (for last-token pooling) the one row that counts
+    float m = 0.f;
+    if constexpr (kMode == kPoolEntropy) {
+      m = -INFINITY;
+      for (int64_t t = t0; t < run_end; ++t) m = fmaxf(m, __ldg(H + t) * inv_alpha);
+    }
     float acc[8];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) acc[k] = kMax ? -INFINITY : 0.f;
-    const T* rowp = hidden + t0 * ldh + col;
-    int64_t t = t0;
-    for (; t + 4 <= run_end; t += 4) {           // four rows in flight per thread
-      float w0 = 0.f, w1 = 0.f, w2 = 0.f, w3 = 0.f;
-      if constexpr (!kMax) {
-        w0 = __ldg(weights + t); w1 = __ldg(weights + t + 1); w2 = __ldg(weights + t + 2); w3 = __ldg(weights + t + 3);
-        // rows that carry no weight (last-token pooling: all but one) are not read at all
-        if (w0 == 0.f && w1 == 0.f && w2 == 0.f && w3 == 0.f) { rowp += 4 * ldh; continue; }
+    for (int k = 0; k < 8; ++k) acc[k] = kMode == kPoolMax ? -INFINITY : 0.f;
+    float wsum = 0.f;
+    if constexpr (kMode == kPoolLast) {
+      if (run_end == seg_end) {                   // the prompt's last token is in this run: read that row only
+        Row8<T>::load(hidden + (seg_end - 1) * ldh + col, acc);
+        wsum = 1.f;
       }
-      float v0[8], v1[8], v2[8], v3[8];
-      Row8<T>::load(rowp, v0);
-      Row8<T>::load(rowp + ldh, v1);
-      Row8<T>::load(rowp + 2 * ldh, v2);
-      Row8<T>::load(rowp + 3 * ldh, v3);
-      if constexpr (kMax) {
+    } else {
+      const T* rowp = hidden + t0 * ldh + col;
+      int64_t t = t0;
+      for (; t + 4 <= run_end; t += 4) {           // four rows in flight per thread
+        float v0[8], v1[8], v2[8], v3[8];
+        Row8<T>::load(rowp, v0);
+        Row8<T>::load(rowp + ldh, v1);
+        Row8<T>::load(rowp + 2 * ldh, v2);
+        Row8<T>::load(rowp + 3 * ldh, v3);
+        if constexpr (kMode == kPoolMax) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) acc[k] = fmaxf(fmaxf(acc[k], fmaxf(v0[k], v1[k])), fmaxf(v2[k], v3[k]));
-      } else {
+          for (int k = 0; k < 8; ++k) acc[k] = fmaxf(fmaxf(acc[k], fmaxf(v0[k], v1[k])), fmaxf(v2[k], v3[k]));
+        } else {
+          float w0 = 1.f, w1 = 1.f, w2 = 1.f, w3 = 1.f;
+          if constexpr (kMode == kPoolEntropy) {
+            w0 = expf(__ldg(H + t) * inv_alpha - m); w1 = expf(__ldg(H + t + 1) * inv_alpha - m);
+            w2 = expf(__ldg(H + t + 2) * inv_alpha - m); w3 = expf(__ldg(H + t + 3) * inv_alpha - m);
+          }
+          wsum += (w0 + w1) + (w2 + w3);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          acc[k] = fmaf(w0, v0[k], acc[k]);
-          acc[k] = fmaf(w1, v1[k], acc[k]);
-          acc[k] = fmaf(w2, v2[k], acc[k]);
-          acc[k] = fmaf(w3, v3[k], acc[k]);
+          for (int k = 0; k < 8; ++k) {
+            acc[k] = fmaf(w0, v0[k], acc[k]);
+            acc[k] = fmaf(w1, v1[k], acc[k]);
+            acc[k] = fmaf(w2, v2[k], acc[k]);
+            acc[k] = fmaf(w3, v3[k], acc[k]);
+          }
         }
+        rowp += 4 * ldh;
       }
-      rowp += 4 * ldh;
-    }
-    for (; t < run_end; ++t) {
-      float v0[8];
-      Row8<T>::load(rowp, v0);
-      if constexpr (kMax) {
+      for (; t < run_end; ++t) {
+        float v0[8];
+        Row8<T>::load(rowp, v0);
+        if constexpr (kMode == kPoolMax) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) acc[k] = fmaxf(acc[k], v0[k]);
-      } else {
-        const float w0 = __ldg(weights + t);
+          for (int k = 0; k < 8; ++k) acc[k] = fmaxf(acc[k], v0[k]);
+        } else {
+          const float w0 = kMode == kPoolEntropy ? expf(__ldg(H + t) * inv_alpha - m) : 1.f;
+          wsum += w0;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) acc[k] = fmaf(w0, v0[k], acc[k]);
+          for (int k = 0; k < 8; ++k) acc[k] = fmaf(w0, v0[k], acc[k]);
+        }
+        rowp += ldh;
       }
-      rowp += ldh;
     }
-    float* dst;
-    if (seg_begin >= c_lo && seg_end <= c_hi) dst = pooled + static_cast<int64_t>(b) * d + col;
-    else if (seg_begin < c_lo) dst = piece_a + c * d + col;
-    else dst = piece_b + c * d + col;
-    store8(dst, acc);
+    if (seg_begin >= c_lo && seg_end <= c_hi) {       // the whole prompt: normalise and finish
+      if constexpr (kMode != kPoolMax) {
+        const float inv = 1.f / wsum;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) acc[k] *= inv;
+      }
+      store8(pooled + static_cast<int64_t>(b) * d + col, acc);
+      if (scribe) {
+        if (seg_m) seg_m[b] = m;
+        if (seg_s) seg_s[b] = wsum;
+      }
+    } else if (seg_begin < c_lo) {
+      store8(piece_a + c * d + col, acc);
+      if (scribe) ms_a[c] = make_float2(m, wsum);
+    } else {
+      store8(piece_b + c * d + col, acc);
+      if (scribe) ms_b[c] = make_float2(m, wsum);
+    }
     t0 = run_end;
     ++b;
   }
 }
 
-// One block per prompt (x) and 1024-channel slab (y): zero for an empty prompt, nothing for a
-// prompt finished by the first stage, else piece_b[c0] + piece_a[c0+1] + ... + piece_a[c1].
-template <bool kMax>
+// One block per prompt (x) and 1024-channel slab (y): zero for an empty prompt; a prompt finished by the first stage
+// is left as it is; else the pieces piece_b[c0], piece_a[c0+1], ..., piece_a[c1] are merged in that order: rescaled
+// to the largest m, summed and normalised (maximum: channel-wise max).  Also leaves the prompt's (M, Z) and,
+// if zcat is given, the pooled row once more as [hi | lo] bf16 halves (input of the head's tensor-core layer 1).
+template <int kMode>
 __global__ void __launch_bounds__(kPoolThreads)
 pool_combine_kernel(const int32_t* __restrict__ off, int B, int d, const float* __restrict__ piece_a,
-                    const float* __restrict__ piece_b, float* __restrict__ pooled,
-                    const int32_t* __restrict__ status) {
+                    const float* __restrict__ piece_b, const float2* __restrict__ ms_a,
+                    const float2* __restrict__ ms_b, float* __restrict__ pooled, float* __restrict__ seg_m,
+                    float* __restrict__ seg_s, __nv_bfloat16* __restrict__ zcat, const int32_t* __restrict__ status) {
   if (*status != 0) return;
   const int b = blockIdx.x;
   const int col = (blockIdx.y * kPoolThreads + threadIdx.x) * 8;
   if (col >= d) return;
+  const bool scribe = blockIdx.y == 0 && threadIdx.x == 0;
   const int64_t s0 = off[b], s1 = off[b + 1];
   float acc[8];
-#pragma unroll
-  for (int k = 0; k < 8; ++k) acc[k] = 0.f;
   float* dst = pooled + static_cast<int64_t>(b) * d + col;
-  if (s1 <= s0) { store8(dst, acc); return; }
-  const int64_t c0 = s0 / kPoolChunkTokens, c1 = (s1 - 1) / kPoolChunkTokens;
-  if (c0 == c1) return;
-  {
-    const float4* p = reinterpret_cast<const float4*>(piece_b + c0 * d + col);
-    const float4 a = p[0], bq = p[1];
-    acc[0] = a.x; acc[1] = a.y; acc[2] = a.z; acc[3] = a.w;
-    acc[4] = bq.x; acc[5] = bq.y; acc[6] = bq.z; acc[7] = bq.w;
-  }
-  for (int64_t c = c0 + 1; c <= c1; ++c) {
-    const float4* p = reinterpret_cast<const float4*>(piece_a + c * d + col);
-    const float4 a = p[0], bq = p[1];
-    const float pv[8] = {a.x, a.y, a.z, a.w, bq.x, bq.y, bq.z, bq.w};
+  __nv_bfloat16* zrow = zcat ? zcat + static_cast<int64_t>(b) * (2 * static_cast<int64_t>(d)) : nullptr;
+  if (s1 <= s0) {
 #pragma unroll
-    for (int k = 0; k < 8; ++k) acc[k] = kMax ? fmaxf(acc[k], pv[k]) : acc[k] + pv[k];
+    for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+    store8(dst, acc);
+    if (zrow) store8_hi_lo(zrow, d, col, acc);
+    if (scribe) {
+      if (seg_m) seg_m[b] = -INFINITY;
+      if (seg_s) seg_s[b] = 0.f;
+    }
+    return;
+  }
+  const int64_t c0 = s0 / kPoolChunkTokens, c1 = (s1 - 1) / kPoolChunkTokens;
+  if (c0 == c1) {
+    if (zrow) {
+      load8f(dst, acc);
+      store8_hi_lo(zrow, d, col, acc);
+    }
+    return;
+  }
+  if constexpr (kMode == kPoolMax) {
+    load8f(piece_b + c0 * d + col, acc);
+    for (int64_t c = c0 + 1; c <= c1; ++c) {
+      float pv[8];
+      load8f(piece_a + c * d + col, pv);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) acc[k] = fmaxf(acc[k], pv[k]);
+    }
+  } else {
+    float M = ms_b[c0].x;
+    for (int64_t c = c0 + 1; c <= c1; ++c) M = fmaxf(M, ms_a[c].x);
+    const float2 first = ms_b[c0];
+    float r = expf(first.x - M);
+    float Z = first.y * r;
+    load8f(piece_b + c0 * d + col, acc);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) acc[k] *= r;
+    for (int64_t c = c0 + 1; c <= c1; ++c) {
+      const float2 ms = ms_a[c];
+      r = expf(ms.x - M);
+      Z = fmaf(ms.y, r, Z);
+      float pv[8];
+      load8f(piece_a + c * d + col, pv);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) acc[k] = fmaf(pv[k], r, acc[k]);
+    }
+    const float inv = 1.f / Z;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) acc[k] *= inv;
+    if (scribe) {
+      if (seg_m) seg_m[b] = M;
+      if (seg_s) seg_s[b] = Z;
+    }
   }
   store8(dst, acc);
+  if (zrow) store8_hi_lo(zrow, d, col, acc);
 }
 
 }  // namespace
@@ -301,12 +359,12 @@ cudaError_t launch_validate_offsets(const int32_t* offsets, int B, int64_t T, in
 }
 
 cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t row_stride, int64_t slot_stride, int64_t T,
-                                 int64_t row0, float* H, const int32_t* offsets, int B, int32_t* seg_id_out, float* weights_zero,
-                                 const int32_t* status, cudaStream_t stream) {
+                                 int64_t row0, float* H, const int32_t* offsets, int B, int32_t* seg_id_out,
+                                 int64_t T_check, int32_t* status, cudaStream_t stream) {
   const int threads = 256, rows_per_block = threads / 32;
   const unsigned blocks = static_cast<unsigned>((T + rows_per_block - 1) / rows_per_block);
   entropy_merge_kernel<<<blocks, threads, 0, stream>>>(partials, slots, row_stride, slot_stride, T, row0, H, offsets, B,
-                                                       seg_id_out, weights_zero, status);
+                                                       seg_id_out, T_check, status);
   return cudaGetLastError();
 }
 
@@ -318,45 +376,71 @@ cudaError_t launch_partials_reduce(const float* partials, int slots, int64_t row
   return cudaGetLastError();
 }
 
-cudaError_t launch_segment_weights(const float* H, const int32_t* offsets, int B, float inv_alpha, float* weights,
-                                   float* seg_m, float* seg_s, const int32_t* status, cudaStream_t stream) {
-  segment_weights_kernel<<<B, 256, 0, stream>>>(H, offsets, B, inv_alpha, weights, seg_m, seg_s, status);
+cudaError_t launch_token_weights(const float* H, const int32_t* offsets, int B, int64_t T, float inv_alpha,
+                                 const float* seg_m, const float* seg_s, float* weights, const int32_t* status,
+                                 cudaStream_t stream) {
+  const unsigned blocks = static_cast<unsigned>((T + 255) / 256);
+  token_weights_kernel<<<blocks, 256, 0, stream>>>(H, offsets, B, T, inv_alpha, seg_m, seg_s, weights, status);
   return cudaGetLastError();
 }
 
-cudaError_t launch_baseline_weights(const int32_t* offsets, int B, int mode, float* weights, const int32_t* status,
-                                    cudaStream_t stream) {
-  baseline_weights_kernel<<<B, 256, 0, stream>>>(offsets, B, mode, weights, status);
-  return cudaGetLastError();
+namespace {
+
+template <typename T>
+void launch_pool_typed(int mode, dim3 grid, cudaStream_t stream, const T* hidden, int64_t ldh, const float* H,
+                       float inv_alpha, const int32_t* off, int B, int d, float* pooled, float* piece_a, float* piece_b,
+                       float2* ms_a, float2* ms_b, float* seg_m, float* seg_s, const int32_t* status) {
+  switch (mode) {
+    case kPoolEntropy:
+      pool_kernel<T, kPoolEntropy><<<grid, kPoolThreads, 0, stream>>>(hidden, ldh, H, inv_alpha, off, B, d, pooled, piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
+      break;
+    case kPoolMean:
+      pool_kernel<T, kPoolMean><<<grid, kPoolThreads, 0, stream>>>(hidden, ldh, H, inv_alpha, off, B, d, pooled, piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
+      break;
+    case kPoolMax:
+      pool_kernel<T, kPoolMax><<<grid, kPoolThreads, 0, stream>>>(hidden, ldh, H, inv_alpha, off, B, d, pooled, piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
+      break;
+    default:
+      pool_kernel<T, kPoolLast><<<grid, kPoolThreads, 0, stream>>>(hidden, ldh, H, inv_alpha, off, B, d, pooled, piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
+      break;
+  }
 }
 
-cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, bool take_max, const float* weights,
+}  // namespace
+
+static_assert(kPoolMean == EGTP_POOL_MEAN && kPoolMax == EGTP_POOL_MAX && kPoolLast == EGTP_POOL_LAST, "pooling mode codes");
+
+cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, int mode, const float* H, float inv_alpha,
                         const int32_t* offsets, int B, int64_t T, int d, float* pooled, float* piece_a,
-                        float* piece_b, const int32_t* status, cudaStream_t stream) {
+                        float* piece_b, float* piece_ms, float* seg_m, float* seg_s, const int32_t* status,
+                        cudaStream_t stream) {
   const unsigned chunks = static_cast<unsigned>((T + kPoolChunkTokens - 1) / kPoolChunkTokens);
   const unsigned slabs = static_cast<unsigned>((d + kPoolThreads * 8 - 1) / (kPoolThreads * 8));
   dim3 grid(chunks, slabs);
-  const __nv_bfloat16* hb = static_cast<const __nv_bfloat16*>(hidden);
-  const float* hf = static_cast<const float*>(hidden);
-  if (bf16 && take_max)
-    pool_kernel<__nv_bfloat16, true><<<grid, kPoolThreads, 0, stream>>>(hb, ldh, weights, offsets, B, d, pooled, piece_a, piece_b, status);
-  else if (bf16)
-    pool_kernel<__nv_bfloat16, false><<<grid, kPoolThreads, 0, stream>>>(hb, ldh, weights, offsets, B, d, pooled, piece_a, piece_b, status);
-  else if (take_max)
-    pool_kernel<float, true><<<grid, kPoolThreads, 0, stream>>>(hf, ldh, weights, offsets, B, d, pooled, piece_a, piece_b, status);
+  float2* ms_a = reinterpret_cast<float2*>(piece_ms);
+  float2* ms_b = ms_a + chunks;
+  if (bf16)
+    launch_pool_typed<__nv_bfloat16>(mode, grid, stream, static_cast<const __nv_bfloat16*>(hidden), ldh, H, inv_alpha, offsets, B, d,
+                                     pooled, piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
   else
-    pool_kernel<float, false><<<grid, kPoolThreads, 0, stream>>>(hf, ldh, weights, offsets, B, d, pooled, piece_a, piece_b, status);
+    launch_pool_typed<float>(mode, grid, stream, static_cast<const float*>(hidden), ldh, H, inv_alpha, offsets, B, d, pooled,
+                             piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
   return cudaGetLastError();
 }
 
-cudaError_t launch_pool_combine(const int32_t* offsets, int B, int d, bool take_max, const float* piece_a,
-                                const float* piece_b, float* pooled, const int32_t* status, cudaStream_t stream) {
+cudaError_t launch_pool_combine(const int32_t* offsets, int B, int64_t T, int d, int mode, const float* piece_a,
+                                const float* piece_b, const float* piece_ms, float* pooled, float* seg_m, float* seg_s,
+                                void* zcat, const int32_t* status, cudaStream_t stream) {
+  const unsigned chunks = static_cast<unsigned>((T + kPoolChunkTokens - 1) / kPoolChunkTokens);
   const unsigned slabs = static_cast<unsigned>((d + kPoolThreads * 8 - 1) / (kPoolThreads * 8));
   dim3 grid(B, slabs);
-  if (take_max)
-    pool_combine_kernel<true><<<grid, kPoolThreads, 0, stream>>>(offsets, B, d, piece_a, piece_b, pooled, status);
+  const float2* ms_a = reinterpret_cast<const float2*>(piece_ms);
+  const float2* ms_b = ms_a + chunks;
+  __nv_bfloat16* zc = static_cast<__nv_bfloat16*>(zcat);
+  if (mode == kPoolMax)
+    pool_combine_kernel<kPoolMax><<<grid, kPoolThreads, 0, stream>>>(offsets, B, d, piece_a, piece_b, ms_a, ms_b, pooled, seg_m, seg_s, zc, status);
   else
-    pool_combine_kernel<false><<<grid, kPoolThreads, 0, stream>>>(offsets, B, d, piece_a, piece_b, pooled, status);
+    pool_combine_kernel<kPoolEntropy><<<grid, kPoolThreads, 0, stream>>>(offsets, B, d, piece_a, piece_b, ms_a, ms_b, pooled, seg_m, seg_s, zc, status);
   return cudaGetLastError();
 }
 

@@ -88,3 +88,32 @@ def all_gather_partials(partial_local: torch.Tensor, group=None) -> torch.Tensor
     out = torch.empty((world,) + tuple(partial_local.shape), device=partial_local.device, dtype=partial_local.dtype)
     dist.all_gather(list(out.unbind(0)), partial_local.contiguous(), group=group)   # writes into the views of `out`
     return out
+
+
+def plp_step_vocab_parallel(ctx: int, st: int, lm_shard, head, hidden_step, group=None, partial_buf=None, **step_args):
+    """One PLP decode step (Sec. 3.3, Eq. 8) on a rank that holds only its row shard of the LM head.
+
+    Every rank sees the same `hidden_step` rows and owns a replica of the running state `st`.  The step is
+      1. egtp_entropy_partials: this rank's (m, s, t2) per row over its vocabulary shard (Eq. 2, first half),
+      2. all_gather_partials: the path's one exchange, rows x 3 floats per rank (NCCL between GPUs; with a gloo
+         group the triples travel through host memory, which is how the orchestration is tested on one GPU),
+      3. plp_step_from_partials: every rank merges the gathered triples into the rows' entropies and advances its
+         replica of the state, so all ranks end the step with the same state and the same predictions.
+    step_args are plp_step_from_partials' keyword arguments (slot_ids, reset_src, src_*, alpha, outputs, status_dev).
+    Returns the gathered triples [world, rows, 3].
+    """
+    from . import binding as egtp
+
+    rows = hidden_step.shape[0]
+    if partial_buf is None:
+        partial_buf = torch.empty(rows, 3, device=hidden_step.device, dtype=torch.float32)
+    egtp.egtp_entropy_partials(ctx, lm_shard, hidden_step, partial_buf, status_dev=step_args.get("status_dev"))
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        if dist.get_backend(group) == "gloo" and partial_buf.is_cuda:
+            gathered = all_gather_partials(partial_buf.cpu(), group).to(partial_buf.device)   # .cpu() waits for the kernel
+        else:
+            gathered = all_gather_partials(partial_buf, group)
+    else:
+        gathered = partial_buf.unsqueeze(0)
+    egtp.plp_step_from_partials(ctx, st, gathered, head, hidden_step, **step_args)
+    return gathered

@@ -347,3 +347,35 @@ def test_bounded_wait_reports_timeout_and_context_survives(ctx):
     ref = orc.egtp_predict(wl.hidden, wl.offsets, wl.W, wl.head, wl.alpha)
     _check_all(gu.run_egtp(ctx, wl), ref, wl)
     assert egtp.egtp_selftest_wait_timeout(ctx, 0, status, check=False) == egtp.EGTP_ERR_INVALID_ARG
+
+
+def test_launch_count_of_a_prediction_and_context_without_host_staging():
+    # a whole prediction is six launches (LM head, merge + offsets check + segment ids, pooling, combine + head input,
+    # head layer 1, head output); a context created without host staging holds max_tokens * max_d * 4 bytes less,
+    # computes the same, and refuses the host-buffer entry points
+    wl = gen.config_mid(V=3000, d=256, m_h=64, B=8)
+    ref = orc.egtp_predict(wl.hidden, wl.offsets, wl.W, wl.head, wl.alpha)
+    full = egtp.egtp_create(0, 4096, 64, 256, 4096)
+    lean = egtp.egtp_create_ex(0, 4096, 64, 256, 4096, egtp.EGTP_CREATE_NO_HOST_STAGING)
+    try:
+        assert egtp.egtp_workspace_bytes(full) - egtp.egtp_workspace_bytes(lean) == 4096 * 256 * 4
+        _check_all(gu.run_egtp(lean, wl), ref, wl)
+        W = gu.dev_tensor(wl.W, wl.dtype); hidden = gu.dev_tensor(wl.hidden, wl.dtype)
+        hd = gu.DeviceHead(wl.head, wl.dtype)
+        off = torch.from_numpy(wl.offsets).cuda()
+        y = torch.empty(wl.B, device="cuda")
+        status = torch.zeros(1, device="cuda", dtype=torch.int32)
+        n0 = egtp.egtp_launch_count(lean)
+        egtp.egtp_predict(lean, egtp.make_lm_head(W), hd.c, hidden, off, wl.B, wl.T, 1.0, yhat_out=y, status_dev=status)
+        torch.cuda.synchronize()
+        assert egtp.egtp_launch_count(lean) - n0 == 6 and int(status.item()) == 0
+        gu.assert_length_close(y.cpu().numpy().astype(np.float64), ref["yhat"])
+        hidden_host = gu.host_tensor(wl.hidden, wl.dtype)
+        off_host = torch.from_numpy(wl.offsets).pin_memory()
+        yh = torch.empty(wl.B, dtype=torch.float32).pin_memory()
+        st = torch.zeros(1, dtype=torch.int32).pin_memory()
+        assert egtp.egtp_predict_host(lean, egtp.make_lm_head(W), hd.c, hidden_host, off_host, wl.B, wl.T, 1.0, yh, None, st,
+                                      check=False) == egtp.EGTP_ERR_UNSUPPORTED
+        assert egtp.egtp_create_ex(0, 4096, 64, 256, 4096, flags=2, check=False) == egtp.EGTP_ERR_INVALID_ARG
+    finally:
+        egtp.egtp_destroy(full); egtp.egtp_destroy(lean)
