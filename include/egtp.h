@@ -328,8 +328,11 @@ EGTP_API int egtp_pool_baseline(egtp_ctx* ctx, const egtp_head* head, const void
  *   EGTP_LMHEAD_CTA_PAIRS: CTA pairs for prompt batches too (256 x 256 tiles).  On a power-capped B200 this
  *     measured equal or slower than AUTO for prompts, so it is an option.
  *   EGTP_LMHEAD_SINGLE_CTA: never use CTA pairs (129..256 rows then run both row tiles in one CTA).
+ *   EGTP_LMHEAD_CTA_PAIRS_WIDE: CTA pairs on 256 x 512 tiles for prompt batches too (the decode tile shape): half
+ *     the operand bytes an SM pulls in per flop, one accumulator set (the epilogue of a tile does not overlap the next
+ *     tile's MMAs).
  * All modes give the same entropies up to summation order. */
-enum { EGTP_LMHEAD_AUTO = 0, EGTP_LMHEAD_CTA_PAIRS = 1, EGTP_LMHEAD_SINGLE_CTA = 2 };
+enum { EGTP_LMHEAD_AUTO = 0, EGTP_LMHEAD_CTA_PAIRS = 1, EGTP_LMHEAD_SINGLE_CTA = 2, EGTP_LMHEAD_CTA_PAIRS_WIDE = 3 };
 EGTP_API int egtp_set_lmhead_mode(egtp_ctx* ctx, int mode);
 
 /* Tuning knob for prompt batches (more than 256 rows): the LM-head kernel cuts the vocabulary into `chunks`
@@ -339,6 +342,14 @@ EGTP_API int egtp_set_lmhead_mode(egtp_ctx* ctx, int mode);
  * longer rows); a positive value forces that count (clamped to what the workspace holds).  Results do not depend
  * on it beyond summation order. */
 EGTP_API int egtp_set_lmhead_chunks(egtp_ctx* ctx, int32_t chunks);
+
+/* Launch overlap (on by default).  The LM-head kernel and the kernel that finishes a PLP step on a state bound to
+ * its head are launched with programmatic stream serialization: their blocks are set up (barriers, tensor memory,
+ * state rows read ahead) while the kernel before them in the stream is still finishing, and each waits for that
+ * kernel's end before it reads anything the stream wrote earlier or writes anything the stream may still read.
+ * Results are identical either way; on = 0 launches them plainly (per-kernel event timing does the same while it
+ * is enabled, because an overlapped start would be charged to the kernel before). */
+EGTP_API int egtp_set_launch_overlap(egtp_ctx* ctx, int on);
 
 /* Failure-detection self-test.  Every wait inside the pipeline kernels (on an mbarrier fed by TMA, by the
  * tensor core or by another warp) is bounded: when its limit runs out the kernel writes

@@ -24,7 +24,7 @@ EGTP_ERR_BAD_SLOT = -7
 EGTP_F32, EGTP_BF16 = 0, 1
 EGTP_HEAD_SCALAR, EGTP_HEAD_BINS = 0, 1
 PLP_RESET_KEEP, PLP_RESET_EMPTY = -2, -1
-EGTP_LMHEAD_AUTO, EGTP_LMHEAD_CTA_PAIRS, EGTP_LMHEAD_SINGLE_CTA = 0, 1, 2
+EGTP_LMHEAD_AUTO, EGTP_LMHEAD_CTA_PAIRS, EGTP_LMHEAD_SINGLE_CTA, EGTP_LMHEAD_CTA_PAIRS_WIDE = 0, 1, 2, 3
 EGTP_POOL_MEAN, EGTP_POOL_MAX, EGTP_POOL_LAST = 1, 2, 3
 EGTP_CREATE_NO_HOST_STAGING = 1
 KERNEL_IDS = ["validate_offsets", "lmhead_entropy", "entropy_merge", "segment_weights", "pool",
@@ -39,7 +39,7 @@ EXPORTED_SYMBOLS = [
     "egtp_launch_count", "egtp_lmhead_plan", "egtp_head_forward_static", "egtp_set_lmhead_mode",
     "egtp_entropy_from_logits", "plp_step_from_logits", "egtp_pool_baseline",
     "egtp_entropy_partials", "egtp_entropy_from_partials", "plp_step_from_partials", "egtp_selftest_wait_timeout",
-    "plp_state_bind_head", "egtp_set_lmhead_chunks", "egtp_lmhead_plan_for", "egtp_create_ex",
+    "plp_state_bind_head", "egtp_set_lmhead_chunks", "egtp_lmhead_plan_for", "egtp_create_ex", "egtp_set_launch_overlap",
 ]
 
 
@@ -89,6 +89,7 @@ def load() -> C.CDLL:
     lib.egtp_profile_enable.argtypes = [vp, C.c_int]
     lib.egtp_set_lmhead_mode.argtypes = [vp, C.c_int]
     lib.egtp_set_lmhead_chunks.argtypes = [vp, i32]
+    lib.egtp_set_launch_overlap.argtypes = [vp, C.c_int]
     lib.egtp_lmhead_plan_for.argtypes = [i32, i32, i64, i32, i32, i32, i32, i32, P(i32)]
     lib.egtp_selftest_wait_timeout.argtypes = [vp, i32, vp, vp]
     lib.egtp_entropy_partials.argtypes = [vp, P(egtp_lm_head), vp, i64, i64, vp, vp, vp]
@@ -231,6 +232,10 @@ def egtp_set_lmhead_mode(ctx: int, mode: int):
 def egtp_set_lmhead_chunks(ctx: int, chunks: int):
     """Forces the number of vocabulary chunks of prompt batches (0 = chosen by the library)."""
     _check(load().egtp_set_lmhead_chunks(ctx, chunks), "egtp_set_lmhead_chunks")
+
+
+def egtp_set_launch_overlap(ctx: int, on: bool):
+    _check(load().egtp_set_launch_overlap(ctx, 1 if on else 0), "egtp_set_launch_overlap")
 
 
 def egtp_profile_enable(ctx: int, on: bool):

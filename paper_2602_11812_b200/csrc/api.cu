@@ -36,6 +36,7 @@ struct egtp_ctx {
   float* partials = nullptr;      int64_t slot_row_capacity = 0;   // rows x slots the partial buffer holds
   float* H = nullptr;             // [max(max_tokens, max_batch)]
   int32_t* arrivals = nullptr;    // [max(max_tokens, max_batch)], zero between calls: per-row block counters
+  float* weights = nullptr;       // [max_tokens]: unnormalised Eq. 3 weights, chunk-local reference
   float* seg_m = nullptr;         // [max_batch]
   float* seg_s = nullptr;         // [max_batch]
   float* pooled = nullptr;        // [max_batch][max_d]  (also z of a PLP step)
@@ -57,6 +58,7 @@ struct egtp_ctx {
   // bookkeeping
   int lmhead_mode = EGTP_LMHEAD_AUTO;
   int lmhead_chunks = 0;          // 0 = chosen by the planner
+  bool launch_overlap = true;     // programmatic dependent launch of the LM-head and bound-update kernels
   // host-buffer entry points: copies run on their own stream, one event per piece of the batch
   static constexpr int kMaxPieces = 4;
   cudaStream_t copy_stream = nullptr;
@@ -78,6 +80,8 @@ struct plp_state {
   float* m = nullptr;
   float* s = nullptr;
   float* acc = nullptr;
+  int32_t* owner = nullptr;     // [num_slots]: stamp of the last step that touched the slot (duplicate slot ids)
+  int32_t* epoch = nullptr;     // [2]: stamp of the next step, blocks of the running step that have left
   // binding to one prediction head (plp_state_bind_head)
   bool bound = false;
   egtp_head bound_head{};
@@ -105,7 +109,7 @@ cudaError_t dev_alloc(egtp_ctx* c, T** p, int64_t count) {
 }
 
 void free_ctx_memory(egtp_ctx* c) {
-  cudaFree(c->partials); cudaFree(c->H); cudaFree(c->arrivals); cudaFree(c->seg_m); cudaFree(c->seg_s);
+  cudaFree(c->partials); cudaFree(c->H); cudaFree(c->arrivals); cudaFree(c->weights); cudaFree(c->seg_m); cudaFree(c->seg_s);
   cudaFree(c->pooled); cudaFree(c->piece_a); cudaFree(c->piece_b); cudaFree(c->piece_ms); cudaFree(c->head_partial); cudaFree(c->zcat); cudaFree(c->small_rows); cudaFree(c->yhat);
   cudaFree(c->status); cudaFree(c->hidden_stage); cudaFree(c->offsets_stage); cudaFree(c->reset_stage);
   if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
@@ -260,8 +264,9 @@ int run_lmhead(egtp_ctx* c, const egtp_lm_head* lm, const void* hidden, int64_t 
     }
   }
   LaunchScope ls(c, EGTP_K_LMHEAD_ENTROPY, stream);
+  // (per-kernel event timing would charge an overlapped start to the kernel before)
   EGTP_CUDA_TRY(launch_lmhead_entropy(plan, lm->dtype == EGTP_F32, maps, rows, lm->V, c->partials, status, stream,
-                                      head_g));
+                                      head_g, /*overlap_previous=*/c->launch_overlap && !c->profiling));
   *plan_out = plan;
   return EGTP_OK;
 }
@@ -483,7 +488,7 @@ int plp_update_and_head(egtp_ctx* c, plp_state* st, const egtp_head* head, const
                                           st->num_slots, 1.f / alpha, st->m, st->s, st->acc, st->proj, z_out, st->d,
                                           st->head_g, plan.head_cols_pad, plan.k_splits,
                                           plan.rows_pad * static_cast<int64_t>(plan.head_cols_pad), head_args(head),
-                                          yrem_out, status, stream, /*overlap_previous=*/false));
+                                          yrem_out, st->owner, st->epoch, status, stream, /*overlap_previous=*/false));
     return EGTP_OK;
   }
   st->proj_valid = false;   // acc moves on without the projection a bound state keeps
@@ -497,7 +502,7 @@ int plp_update_and_head(egtp_ctx* c, plp_state* st, const egtp_head* head, const
     EGTP_CUDA_TRY(launch_plp_update(hidden_step, ldh, hidden_dtype == EGTP_BF16, partials, slots, row_stride, slot_stride, Hstep_out,
                                     slot_ids,
                                     reset_src, src_m, src_s, src_pooled, n_src, B_live, st->d, st->num_slots,
-                                    1.f / alpha, st->m, st->s, st->acc, z, st->d, status, stream,
+                                    1.f / alpha, st->m, st->s, st->acc, z, st->d, st->owner, st->epoch, status, stream,
                                     staged ? c->zcat : nullptr));
   }
   if (staged) return run_head_staged(c, head, B_live, yrem_out, nullptr, status, stream);
@@ -556,15 +561,18 @@ int predict_impl(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, con
     LmheadPlan plan;
     int rc = run_lmhead(c, lm, piece_ptr, ldh, rows, status, stream, &plan);
     if (rc != EGTP_OK) return rc;
-    // the first merge launch also checks the offsets (everything that indexes tokens through them comes later)
+    // the first merge launch also checks the offsets (everything that indexes tokens through them comes later);
+    // every merge launch prepares the pooling of its tokens (unnormalised Eq. 3 weights per 64-token chunk)
+    const PoolPrep prep{1.f / alpha, c->weights, c->piece_ms,
+                        (T_total + kPoolChunkTokens - 1) / kPoolChunkTokens, seg_m, seg_s};
     LaunchScope ls(c, EGTP_K_ENTROPY_MERGE, stream);
     EGTP_CUDA_TRY(launch_entropy_merge(c->partials, plan.slots, plan.slots * 3, 3, rows, r0, H, offsets, B, seg_id_out,
-                                       (p == 0 && B > 0) ? T_total : -1, status, stream));
+                                       (p == 0 && B > 0) ? T_total : -1, status, stream, B > 0 ? &prep : nullptr));
   }
   if (B == 0) return EGTP_OK;
   if (T_total > 0) {
     LaunchScope ls(c, EGTP_K_POOL, stream);
-    EGTP_CUDA_TRY(launch_pool(hidden, ldh, lm->dtype == EGTP_BF16, 0, H, 1.f / alpha, offsets, B, T_total, d, pooled,
+    EGTP_CUDA_TRY(launch_pool(hidden, ldh, lm->dtype == EGTP_BF16, 0, c->weights, offsets, B, T_total, d, pooled,
                               c->piece_a, c->piece_b, c->piece_ms, seg_m, seg_s, status, stream));
   }
   {
@@ -650,6 +658,7 @@ int egtp_create_ex(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_b
   ok = ok && dev_alloc(c, &c->H, rows_cap) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->arrivals, rows_cap) == cudaSuccess;
   ok = ok && cudaMemset(c->arrivals, 0, sizeof(int32_t) * static_cast<size_t>(rows_cap)) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->weights, max_tokens) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->seg_m, max_batch) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->seg_s, max_batch) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->pooled, static_cast<int64_t>(max_batch) * max_d) == cudaSuccess;
@@ -707,7 +716,7 @@ int egtp_lmhead_plan_for(int32_t num_sms, int32_t pair_workers, int64_t T, int32
                          int32_t mode, int32_t head_cols, int32_t info[12]) {
   if (!info || num_sms <= 0 || pair_workers < 0 || T <= 0 || d <= 0 || V <= 0 || head_cols < 0) return EGTP_ERR_INVALID_ARG;
   if (dtype != EGTP_F32 && dtype != EGTP_BF16) return EGTP_ERR_UNSUPPORTED;
-  if (mode != EGTP_LMHEAD_AUTO && mode != EGTP_LMHEAD_CTA_PAIRS && mode != EGTP_LMHEAD_SINGLE_CTA) return EGTP_ERR_INVALID_ARG;
+  if (mode < EGTP_LMHEAD_AUTO || mode > EGTP_LMHEAD_CTA_PAIRS_WIDE) return EGTP_ERR_INVALID_ARG;
   // the workspace rule of egtp_create for a context sized for exactly T rows
   const int64_t rows_pad = (T + kTileM - 1) / kTileM * kTileM;
   const int64_t capacity = std::max<int64_t>(
@@ -720,7 +729,7 @@ int egtp_lmhead_plan_for(int32_t num_sms, int32_t pair_workers, int64_t T, int32
 }
 
 int egtp_set_lmhead_mode(egtp_ctx* c, int mode) {
-  if (!c || (mode != EGTP_LMHEAD_AUTO && mode != EGTP_LMHEAD_CTA_PAIRS && mode != EGTP_LMHEAD_SINGLE_CTA))
+  if (!c || mode < EGTP_LMHEAD_AUTO || mode > EGTP_LMHEAD_CTA_PAIRS_WIDE)
     return EGTP_ERR_INVALID_ARG;
   c->lmhead_mode = mode;
   return EGTP_OK;
@@ -729,6 +738,12 @@ int egtp_set_lmhead_mode(egtp_ctx* c, int mode) {
 int egtp_set_lmhead_chunks(egtp_ctx* c, int32_t chunks) {
   if (!c || chunks < 0) return EGTP_ERR_INVALID_ARG;
   c->lmhead_chunks = chunks;
+  return EGTP_OK;
+}
+
+int egtp_set_launch_overlap(egtp_ctx* c, int on) {
+  if (!c) return EGTP_ERR_INVALID_ARG;
+  c->launch_overlap = on != 0;
   return EGTP_OK;
 }
 
@@ -804,7 +819,7 @@ int egtp_pool_baseline(egtp_ctx* c, const egtp_head* head, const void* hidden, i
   }
   if (T_total > 0) {
     LaunchScope ls(c, EGTP_K_POOL, stream);
-    EGTP_CUDA_TRY(launch_pool(hidden, ldh, dtype == EGTP_BF16, mode, nullptr, 1.f, offsets, B, T_total, d, pooled,
+    EGTP_CUDA_TRY(launch_pool(hidden, ldh, dtype == EGTP_BF16, mode, nullptr, offsets, B, T_total, d, pooled,
                               c->piece_a, c->piece_b, c->piece_ms, nullptr, nullptr, status, stream));
   }
   {
@@ -873,6 +888,13 @@ int plp_state_create(egtp_ctx* c, plp_state** out, int32_t num_slots, int32_t d)
   bool ok = cudaMalloc(reinterpret_cast<void**>(&st->m), sizeof(float) * num_slots) == cudaSuccess;
   ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->s), sizeof(float) * num_slots) == cudaSuccess;
   ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->acc), sizeof(float) * static_cast<size_t>(num_slots) * d) == cudaSuccess;
+  ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->owner), sizeof(int32_t) * num_slots) == cudaSuccess;
+  ok = ok && cudaMalloc(reinterpret_cast<void**>(&st->epoch), sizeof(int32_t) * 2) == cudaSuccess;
+  if (ok) {
+    const int32_t epoch0[2] = {1, 0};
+    ok = cudaMemset(st->owner, 0, sizeof(int32_t) * num_slots) == cudaSuccess &&
+         cudaMemcpy(st->epoch, epoch0, sizeof(epoch0), cudaMemcpyHostToDevice) == cudaSuccess;
+  }
   if (ok) {
     std::vector<float> neg(num_slots, -INFINITY);
     ok = cudaMemcpy(st->m, neg.data(), sizeof(float) * num_slots, cudaMemcpyHostToDevice) == cudaSuccess;
@@ -881,7 +903,7 @@ int plp_state_create(egtp_ctx* c, plp_state** out, int32_t num_slots, int32_t d)
   }
   if (!ok) {
     cudaGetLastError();
-    cudaFree(st->m); cudaFree(st->s); cudaFree(st->acc);
+    cudaFree(st->m); cudaFree(st->s); cudaFree(st->acc); cudaFree(st->owner); cudaFree(st->epoch);
     delete st;
     return EGTP_ERR_CUDA;
   }
@@ -892,7 +914,7 @@ int plp_state_create(egtp_ctx* c, plp_state** out, int32_t num_slots, int32_t d)
 int plp_state_destroy(plp_state* st) {
   if (!st) return EGTP_ERR_INVALID_ARG;
   cudaSetDevice(st->device);
-  cudaFree(st->m); cudaFree(st->s); cudaFree(st->acc);
+  cudaFree(st->m); cudaFree(st->s); cudaFree(st->acc); cudaFree(st->owner); cudaFree(st->epoch);
   cudaFree(st->proj); cudaFree(st->src_proj); cudaFree(st->head_g);
   delete st;
   return EGTP_OK;
@@ -959,8 +981,8 @@ int plp_step(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head
     EGTP_CUDA_TRY(launch_plp_update_bound(hidden_step, ldh, c->partials, plan.slots, plan.slots * 3, 3, Hstep_out, slot_ids,
                                           reset_src, src_m, src_s, src_pooled, st->src_proj, n_src, B_live, st->d,
                                           st->num_slots, 1.f / alpha, st->m, st->s, st->acc, st->proj, z_out, st->d,
-                                          st->head_g, plan.head_cols_pad, 1, 0, head_args(head), yrem_out, status, stream,
-                                          /*overlap_previous=*/!c->profiling));
+                                          st->head_g, plan.head_cols_pad, 1, 0, head_args(head), yrem_out, st->owner, st->epoch, status, stream,
+                                          /*overlap_previous=*/c->launch_overlap && !c->profiling));
     return EGTP_OK;
   }
   rc = run_lmhead(c, lm, hidden_step, ldh, B_live, status, stream, &plan);

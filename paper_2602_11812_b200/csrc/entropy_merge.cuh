@@ -58,6 +58,33 @@ __device__ __forceinline__ EntropyPartial merge_partials_warp_raw(const float* _
   return warp_combine_partials(acc);
 }
 
+// The same merge by a group of kLanes consecutive lanes (kLanes a power of two): 32 / kLanes rows per warp at
+// once.  Every lane of the group returns the row's (m, s, t2).
+template <int kLanes>
+__device__ __forceinline__ EntropyPartial merge_partials_group_raw(const float* __restrict__ row, int slots,
+                                                                   int64_t slot_stride, int lane_in_group) {
+  constexpr float kLog2e = 1.4426950408889634f;
+  EntropyPartial acc = {kNegBig, 0.f, 0.f};
+  for (int j = lane_in_group; j < slots; j += kLanes) {
+    const float* pj = row + j * slot_stride;
+    const EntropyPartial q = {pj[0], pj[1], pj[2]};
+    acc = combine_partials(acc, q);
+  }
+  float M = acc.m;
+#pragma unroll
+  for (int o = kLanes / 2; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  const float dm = (acc.m - M) * kLog2e;
+  const float r = exp2f(dm);
+  float s = acc.s * r;
+  float t2 = r * fmaf(dm, acc.s, acc.t2);
+#pragma unroll
+  for (int o = kLanes / 2; o > 0; o >>= 1) {
+    s += __shfl_xor_sync(0xffffffffu, s, o);
+    t2 += __shfl_xor_sync(0xffffffffu, t2, o);
+  }
+  return {M, s, t2};
+}
+
 __device__ __forceinline__ float entropy_of(const EntropyPartial& p) {
   constexpr float kLn2 = 0.6931471805599453f;
   return logf(p.s) - kLn2 * p.t2 / p.s;

@@ -71,8 +71,11 @@ struct LmheadMaps {
   const CUtensorMap* w1 = nullptr;
   const CUtensorMap* w1_tile = nullptr;
 };
+// overlap_previous: launch with programmatic stream serialization: the blocks set themselves up while the kernel
+// before this one in the stream is still finishing and wait for its end before they touch global memory.
 cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const LmheadMaps& maps, int64_t T, int V,
-                                  float* partials, int32_t* status, cudaStream_t stream, float* head_g = nullptr);
+                                  float* partials, int32_t* status, cudaStream_t stream, float* head_g = nullptr,
+                                  bool overlap_previous = false);
 
 // ---- K2: entropy merge, Eq. 3-4 pooling -------------------------------------
 constexpr int kPoolChunkTokens = 64;   // tokens per first-stage pooling chunk
@@ -84,22 +87,34 @@ cudaError_t launch_validate_offsets(const int32_t* offsets, int B, int64_t T, in
 // the batch (H, weights and segment ids are indexed by the batch-wide token index)
 cudaError_t launch_partials_reduce(const float* partials, int slots, int64_t rows, float* out, const int32_t* status,
                                    cudaStream_t stream);
-// T_check >= 0: the launch also checks the offsets against that token count (EGTP_ERR_BAD_OFFSETS in *status)
+// What the merge kernel leaves for the entropy-weighted pooling of the same tokens (Eq. 3 up to its normaliser): per
+// token the unnormalised weight exp(H/alpha - m) relative to the maximum m of its prompt's run inside its 64-token
+// chunk, and (m, sum of weights) per run: in seg_m / seg_s for prompts inside one chunk, else in piece_ms
+// ([2 * chunks][2], chunks = ceil(T_total / kPoolChunkTokens) of the whole batch).
+struct PoolPrep {
+  float inv_alpha;
+  float* weights;      // [T_total]
+  float* piece_ms;
+  int64_t chunks;
+  float* seg_m;        // [B]
+  float* seg_s;        // [B]
+};
+// T_check >= 0: the launch also checks the offsets against that token count (EGTP_ERR_BAD_OFFSETS in *status).
+// prep != NULL needs offsets and row0 a multiple of kPoolChunkTokens.
 cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t row_stride, int64_t slot_stride, int64_t T,
                                  int64_t row0, float* H, const int32_t* offsets, int B, int32_t* seg_id_out,
-                                 int64_t T_check, int32_t* status, cudaStream_t stream);
+                                 int64_t T_check, int32_t* status, cudaStream_t stream, const PoolPrep* prep = nullptr);
 
 // Eq. 3 weights as an output: w_i = exp(H_i/alpha - M_b) / Z_b from the per-prompt state the pooling left (0 outside prompts)
 cudaError_t launch_token_weights(const float* H, const int32_t* offsets, int B, int64_t T, float inv_alpha,
                                  const float* seg_m, const float* seg_s, float* weights, const int32_t* status,
                                  cudaStream_t stream);
 
-// Pooling over the prompts' token spans.  mode 0: entropy-weighted (Eq. 3-4; H and inv_alpha give the weights, which
-// are formed on the fly relative to chunk-local maxima and never stored); EGTP_POOL_MEAN / _MAX / _LAST: the
-// alternatives of the paper's ablation (H unused).  piece_a / piece_b [chunks][d] and piece_ms [2 * chunks][2]
-// (chunks = ceil(T / kPoolChunkTokens)) receive the pieces of prompts that span several chunks; seg_m / seg_s (may be
-// NULL) the softmax state (M, Z) of prompts finished in one chunk.
-cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, int mode, const float* H, float inv_alpha,
+// Pooling over the prompts' token spans.  mode 0: entropy-weighted (Eq. 3-4) with the unnormalised weights, seg_s and
+// piece_ms a merge launch with a PoolPrep left; EGTP_POOL_MEAN / _MAX / _LAST: the alternatives of the paper's
+// ablation (weights unused; the kernel fills seg_m / seg_s / piece_ms itself).  piece_a / piece_b [chunks][d] and
+// piece_ms [2 * chunks][2] (chunks = ceil(T / kPoolChunkTokens)) hold the pieces of prompts that span several chunks.
+cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, int mode, const float* weights,
                         const int32_t* offsets, int B, int64_t T, int d, float* pooled, float* piece_a,
                         float* piece_b, float* piece_ms, float* seg_m, float* seg_s, const int32_t* status,
                         cudaStream_t stream);
@@ -160,12 +175,14 @@ cudaError_t launch_wait_timeout_selftest(uint64_t limit_ns, int32_t* status, cud
 
 // ---- K4: PLP running-state update ---------------------------------------------------------
 // Merges the row's entropy partials itself (Eq. 2), optionally writes H' to Hstep_out, then updates the slot.
+// owner [num_slots] (zero-initialised) and epoch [2] (initialised to {1, 0}) belong to the state: with them the kernels
+// refuse a second row of one step on the same slot (EGTP_ERR_BAD_SLOT).
 cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, const float* partials, int slots,
                               int64_t row_stride, int64_t slot_stride, float* Hstep_out,
                               const int32_t* slot_ids, const int32_t* reset_src, const float* src_m,
                               const float* src_s, const float* src_pooled, int n_src, int rows, int d, int num_slots,
                               float inv_alpha, float* st_m, float* st_s, float* st_acc, float* z, int64_t ldz,
-                              int32_t* status, cudaStream_t stream, void* zcat = nullptr);
+                              int32_t* owner, int32_t* epoch, int32_t* status, cudaStream_t stream, void* zcat = nullptr);
 
 // The update for a state bound to a head (bf16 hidden states and head weights): also advances the slot's
 // projection st_proj = W1 acc with g = W1 h' from the LM-head kernel and finishes the head for the row.
@@ -178,7 +195,7 @@ cudaError_t launch_plp_update_bound(const void* hidden_step, int64_t ldh, const 
                                     const float* src_pooled, const float* src_proj, int n_src, int rows, int d,
                                     int num_slots, float inv_alpha, float* st_m, float* st_s, float* st_acc,
                                     float* st_proj, float* z, int64_t ldz, const float* g, int64_t ldg, int g_splits,
-                                    int64_t g_split_stride, const HeadArgs& h, float* y, int32_t* status,
-                                    cudaStream_t stream, bool overlap_previous);
+                                    int64_t g_split_stride, const HeadArgs& h, float* y, int32_t* owner, int32_t* epoch,
+                                    int32_t* status, cudaStream_t stream, bool overlap_previous);
 
 }  // namespace egtp

@@ -204,19 +204,14 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   volatile uint32_t* tmem_slot =
       reinterpret_cast<volatile uint32_t*>(smem_gen + kNumStages * kStageBytes + 8 * (2 * kMaxStages + 4));
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  volatile uint32_t* skip_flag = tmem_slot + 2;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
-  // An earlier step of this call failed: do nothing.  One thread reads the word so that the
-  // whole block takes the same decision.
-  if (threadIdx.x == 0) *abort_flag = (*p.status != 0) ? 1u : 0u;
-  __syncthreads();
-  if (*abort_flag != 0u) return;
-  __syncthreads();
-  // the kernel that consumes the partials may be staged on SMs this grid has left (it waits for the grid's end
-  // before it reads anything written here)
-  pdl_launch_dependents();
+  // This kernel may have been started (programmatic dependent launch) while the kernel before it in the stream is
+  // still finishing: everything up to pdl_wait() below touches only this block's shared and tensor memory and the
+  // kernel's own parameters.
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kNumStages; ++s) {
@@ -242,12 +237,26 @@ lmhead_entropy_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // From here on the kernel reads what earlier work in the stream wrote (hidden rows, the status word) and writes
+  // what that work may still be reading (the partials).
+  pdl_wait();
+  // Only now may the kernel after this one be staged on SMs this grid has left (it waits for this grid's end before it
+  // reads anything written here, but it reads its own state rows ahead: those must be final, which they are once
+  // the work before this kernel has completed).
+  pdl_launch_dependents();
+  // An earlier step of this call failed: do nothing.  One thread reads the word so that the
+  // whole block takes the same decision.
+  if (threadIdx.x == 0) *skip_flag = (*p.status != 0) ? 1u : 0u;
+  __syncthreads();
+  const bool skip = *skip_flag != 0u;
 
   constexpr int kElemsPerStage = kTf32 ? kRowBytes / 4 : kRowBytes / 2;   // K elements per stage
   constexpr int kMmaPerStage = 4;                                         // 32 bytes of K per MMA
   constexpr uint32_t kIdescNoN = umma_idesc(kTf32 ? 2u : 1u, kTileM, 0);  // N is filled in per tile
 
-  if (warp == 0) {
+  if (skip) {
+    // nothing to do
+  } else if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int stage = 0;
@@ -523,10 +532,8 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
   constexpr int kStageBytes = kABytes + kBBytes;
   constexpr int kAccCols = kBN;
   constexpr int kNumAcc = kTmemCols / kAccCols;
-  constexpr int kSpan = kAccCols / kEpiSplit;
   static_assert(kNumStages <= kMaxStages && (kSubN / 2) % kBBox == 0 && kBBox % 8 == 0, "bad tile configuration");
-  static_assert((kNT == 1 && kNumAcc == 2 && kSpan == 128) || (kNT == 2 && kNumAcc == 1 && kSpan == 256),
-                "two 256-column accumulators or one of 512 columns");
+  static_assert((kNT == 1 && kNumAcc == 2) || (kNT == 2 && kNumAcc == 1), "two 256-column accumulators or one of 512 columns");
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -553,12 +560,14 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
       mbar_init(full_bar(s), 1);            // leader: its own arrive.expect_tx (bytes of both CTAs)
       mbar_init(empty_bar(s), 1);           // one commit arrival, delivered to both CTAs
     }
-    for (int a = 0; a < kNumAcc; ++a) {
+    // 256 x 256 tiles: two accumulator sets, each with its "full" and "empty" barrier.  256 x 512 tiles: one set, one
+    // "full" barrier, but an "empty" barrier per 256-column subtile, so that the next tile's MMAs into the first
+    // subtile can start while the epilogue is still reading the second
+    for (int a = 0; a < 2; ++a) {
       mbar_init(acc_full_bar(a), 1);                    // commit arrival, delivered to both CTAs
       mbar_init(acc_empty_bar(a), 2 * 4 * kEpiSplit);   // leader: the epilogue warps of both CTAs
     }
     *abort_flag = 0u;
-    *skip_flag = (*p.status != 0) ? 1u : 0u;            // an earlier step of this call failed
     mbar_fence_init();
     tma_prefetch_descriptor(&map_a);
     tma_prefetch_descriptor(&map_b);
@@ -570,10 +579,12 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
   }
   tc_fence_before_sync();
   __syncthreads();
+  pdl_wait();                   // see the one-CTA kernel: nothing before this line touched global memory
+  pdl_launch_dependents();
+  if (threadIdx.x == 0) *skip_flag = (*p.status != 0) ? 1u : 0u;            // an earlier step of this call failed
   cluster_sync_all();           // barriers of both CTAs are initialised before anyone signals across
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_launch_dependents();      // see the one-CTA kernel
   // both CTAs follow the leader's reading of the status word
   const bool skip = ld_shared_cluster_u32(map_to_cta(smem_u32(const_cast<uint32_t*>(skip_flag)), 0)) != 0u;
 
@@ -640,6 +651,15 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
+      // MMAs of k block `stg` of the current tile into subtile t
+      auto issue = [&](int stg, int t, const uint32_t (&idesc)[kNT], uint32_t d_tmem, bool first_kb) {
+        const uint32_t a_src = smem_base + stg * kStageBytes;
+        const uint64_t a_desc = umma_desc_k_major_sw128(a_src);
+        const uint64_t b_desc = umma_desc_k_major_sw128(a_src + kABytes + t * kSubBBytes);
+#pragma unroll
+        for (int k = 0; k < kMmaPerStage; ++k)
+          umma_ss_pair<kTf32>(d_tmem + t * kSubN, a_desc + 2u * k, b_desc + 2u * k, idesc[t], (!first_kb || k != 0) ? 1u : 0u);
+      };
       for (int u = pair; u < p.total_units && ok; u += num_pairs) {
         const UnitCoord uc = unit_coord(u, p);
         for (int n0 = uc.col_begin; n0 < uc.col_end && ok; n0 += kBN) {
@@ -648,27 +668,54 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
 #pragma unroll
           for (int t = 0; t < kNT; ++t)
             idesc[t] = kIdescNoN | (static_cast<uint32_t>(max(0, min(kSubN, ncols - t * kSubN)) >> 3) << 17);
-          if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
-          tc_fence_after_sync();
-          const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kAccCols);
-          for (int kb = 0; kb < p.k_blocks; ++kb) {
-            if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          if constexpr (kNT == 1) {
+            if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
-            const uint32_t a_src = smem_base + stage * kStageBytes;
-            const uint64_t a_desc = umma_desc_k_major_sw128(a_src);
-#pragma unroll
-            for (int t = 0; t < kNT; ++t) {
-              if (ncols <= t * kSubN) break;                // ragged tile without this subtile
-              const uint64_t b_desc = umma_desc_k_major_sw128(a_src + kABytes + t * kSubBBytes);
-#pragma unroll
-              for (int k = 0; k < kMmaPerStage; ++k)
-                umma_ss_pair<kTf32>(d_tmem + t * kSubN, a_desc + 2u * k, b_desc + 2u * k, idesc[t], (kb | k) != 0 ? 1u : 0u);
+            const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kAccCols);
+            for (int kb = 0; kb < p.k_blocks; ++kb) {
+              if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+              tc_fence_after_sync();
+              issue(stage, 0, idesc, d_tmem, kb == 0);
+              umma_commit_pair(empty_bar(stage), 0x3);        // frees the stage in both CTAs
+              if (++stage == kNumStages) { stage = 0; phase ^= 1u; }
             }
-            umma_commit_pair(empty_bar(stage), 0x3);        // frees the stage in both CTAs
-            if (++stage == kNumStages) { stage = 0; phase ^= 1u; }
+            if (ok) umma_commit_pair(acc_full_bar(acc), 0x3); // accumulator complete in both CTAs
+            if (++acc == kNumAcc) { acc = 0; acc_phase ^= 1u; }
+          } else {
+            // One 512-column accumulator set.  The epilogue hands back the first subtile when it is half way through,
+            // so the first kLag k blocks are multiplied into the first subtile alone (their stages stay held), then,
+            // once the second subtile is free as well, into the second; from there on both per k block.
+            constexpr int kLag = kNumStages - 1;
+            const bool two = ncols > kSubN;                     // ragged tiles may have no second subtile
+            const int lag = min(kLag, p.k_blocks);
+            if (!mbar_wait(acc_empty_bar(0), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            int held = stage;                                   // first of the stages held back
+            for (int kb = 0; kb < lag && ok; ++kb) {
+              if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+              tc_fence_after_sync();
+              issue(stage, 0, idesc, tmem_base, kb == 0);
+              if (++stage == kNumStages) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) break;
+            if (!mbar_wait(acc_empty_bar(1), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            for (int kb = 0; kb < lag; ++kb) {
+              if (two) issue(held, 1, idesc, tmem_base, kb == 0);
+              umma_commit_pair(empty_bar(held), 0x3);
+              if (++held == kNumStages) held = 0;
+            }
+            for (int kb = lag; kb < p.k_blocks; ++kb) {
+              if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+              tc_fence_after_sync();
+              issue(stage, 0, idesc, tmem_base, kb == 0);
+              if (two) issue(stage, 1, idesc, tmem_base, kb == 0);
+              umma_commit_pair(empty_bar(stage), 0x3);
+              if (++stage == kNumStages) { stage = 0; phase ^= 1u; }
+            }
+            if (ok) umma_commit_pair(acc_full_bar(0), 0x3);
+            acc_phase ^= 1u;
           }
-          if (ok) umma_commit_pair(acc_full_bar(acc), 0x3); // accumulator complete in both CTAs
-          if (++acc == kNumAcc) { acc = 0; acc_phase ^= 1u; }
         }
       }
     }
@@ -690,36 +737,43 @@ lmhead_entropy_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         tc_fence_after_sync();
         const int tile_cols = min(kBN, uc.col_end - n0);
         const int ncols = kFuse ? tile_cols : min(tile_cols, p.V - n0);
-        const int cols_valid = min(kSpan, ncols - half * kSpan);
-        const int npieces = cols_valid > 0 ? (cols_valid + 31) >> 5 : 0;
-        const int c_base = n0 + half * kSpan;
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
-                               static_cast<uint32_t>(acc * kAccCols + half * kSpan);
-        const uint32_t acc_empty_leader = map_to_cta(acc_empty_bar(acc), 0);
-        auto release = [&]() {
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
-        };
-        auto consume = [&](const uint32_t (&buf)[32], int pc) {
-          consume_piece<kFuse>(st, buf, c_base + pc * 32, cols_valid - pc * 32, p, row);
-        };
-        uint32_t bufA[32], bufB[32];
-        if (npieces == 0) {
-          release();
-        } else {
-          tmem_ld_32(taddr, bufA);
-          tmem_ld_wait(bufA);
-          for (int pc = 0; pc < npieces; pc += 2) {
-            const bool has1 = pc + 1 < npieces;
-            if (has1) tmem_ld_32(taddr + (pc + 1) * 32, bufB); else release();
-            consume(bufA, pc);
-            if (has1) {
-              tmem_ld_wait(bufB);
-              const bool has2 = pc + 2 < npieces;
-              if (has2) tmem_ld_32(taddr + (pc + 2) * 32, bufA); else release();
-              consume(bufB, pc + 1);
-              if (has2) tmem_ld_wait(bufA);
+        // This warp reads 128 columns of every 256-column subtile (column half `half`) and hands each subtile back
+        // as soon as it has read it: with 256 x 512 tiles the first subtile is free again when the epilogue is half way.
+        constexpr int kSubSpan = kSubN / kEpiSplit;
+#pragma unroll
+        for (int sub = 0; sub < kNT; ++sub) {
+          const int co = sub * kSubN + half * kSubSpan;             // first column of the span inside the tile
+          const int cols_valid = min(kSubSpan, ncols - co);
+          const int npieces = cols_valid > 0 ? (cols_valid + 31) >> 5 : 0;
+          const int c_base = n0 + co;
+          const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
+                                 static_cast<uint32_t>(acc * kAccCols + co);
+          const uint32_t acc_empty_leader = map_to_cta(acc_empty_bar(kNT == 1 ? acc : sub), 0);
+          auto release = [&]() {
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+          };
+          auto consume = [&](const uint32_t (&buf)[32], int pc) {
+            consume_piece<kFuse>(st, buf, c_base + pc * 32, cols_valid - pc * 32, p, row);
+          };
+          uint32_t bufA[32], bufB[32];
+          if (npieces == 0) {
+            release();
+          } else {
+            tmem_ld_32(taddr, bufA);
+            tmem_ld_wait(bufA);
+            for (int pc = 0; pc < npieces; pc += 2) {
+              const bool has1 = pc + 1 < npieces;
+              if (has1) tmem_ld_32(taddr + (pc + 1) * 32, bufB); else release();
+              consume(bufA, pc);
+              if (has1) {
+                tmem_ld_wait(bufB);
+                const bool has2 = pc + 2 < npieces;
+                if (has2) tmem_ld_32(taddr + (pc + 2) * 32, bufA); else release();
+                consume(bufB, pc + 1);
+                if (has2) tmem_ld_wait(bufA);
+              }
             }
           }
         }
@@ -767,6 +821,7 @@ constexpr Shape kShapeDecode2 = {2, 256, 32, 3, 32};    // 129..256 rows: both r
 
 constexpr Shape kShapePairPrompt = {2, 256, 128, 6, 256};  // CTA pairs, 256 x 256 tiles
 constexpr Shape kShapePairDecode = {2, 512, 32, 4, 64};    // CTA pairs, 256 x 512 tiles, one vocabulary range per pair
+constexpr Shape kShapePairWide = {2, 512, 32, 4, 512};     // CTA pairs, 256 x 512 tiles, prompt batches
 constexpr int kPairStages = 6;         // 256 x 256 tiles: 6 x 32 KB
 constexpr int kPairWideStages = 4;     // 256 x 512 tiles: 4 x 48 KB
 constexpr int kPairSmemBytes = kPairStages * (kTileM * kRowBytes + 128 * kRowBytes) + kBarrierBytes + 1024;
@@ -775,17 +830,35 @@ static_assert(kPairWideStages * (kTileM * kRowBytes + 2 * 128 * kRowBytes) + kBa
 const Shape& shape_of(int variant) {
   if (variant == 4) return kShapePairPrompt;
   if (variant == 5) return kShapePairDecode;
+  if (variant == 6) return kShapePairWide;
   return variant == 1 ? kShapeDecode1 : (variant == 2 ? kShapeDecode2 : kShapePrompt);
 }
 
+// overlap: launch with programmatic stream serialization, so that the blocks may be set up (barriers, tensor memory)
+// while the kernel before this one in the stream is still finishing; the kernel waits for that kernel's end before
+// it touches global memory
+struct LaunchConfig {
+  cudaLaunchConfig_t cfg{};
+  cudaLaunchAttribute attr{};
+  LaunchConfig(int grid, int smem_bytes, cudaStream_t stream, bool overlap) {
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kLmheadThreads);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+  }
+};
+
 template <bool kTf32, int kMT, int kBN, int kBBox, int kNumStages, bool kFuse = false>
-cudaError_t launch_shape(const LmheadPlan& plan, const LmheadMaps& m, const KParams& p, cudaStream_t stream) {
+cudaError_t launch_shape(const LmheadPlan& plan, const LmheadMaps& m, const KParams& p, cudaStream_t stream, bool overlap) {
   auto kernel = lmhead_entropy_kernel<kTf32, kMT, kBN, kBBox, kNumStages, kFuse>;
   const CUtensorMap* c = kFuse ? m.w1 : m.w;
   const CUtensorMap* c_tile = kFuse ? m.w1_tile : m.w_tile;
-  kernel<<<plan.grid, kLmheadThreads, smem_bytes_for(kMT, kBN, kNumStages, kTf32), stream>>>(*m.hidden, *m.w, *m.w_tile,
-                                                                                            *c, *c_tile, p);
-  return cudaGetLastError();
+  LaunchConfig lc(plan.grid, smem_bytes_for(kMT, kBN, kNumStages, kTf32), stream, overlap);
+  return cudaLaunchKernelEx(&lc.cfg, kernel, *m.hidden, *m.w, *m.w_tile, *c, *c_tile, p);
 }
 
 template <bool kTf32, int kMT, int kBN, int kBBox, int kNumStages, bool kFuse = false>
@@ -797,11 +870,11 @@ cudaError_t prepare_shape() {
 
 // kBBox 128: 256 x 256 tiles (prompt batches); 32: 256 x 512 tiles (decode batches), optionally with head columns
 template <bool kTf32, int kBBox, bool kFuse = false>
-cudaError_t launch_pair(const LmheadPlan& plan, const LmheadMaps& m, const KParams& p, cudaStream_t stream) {
+cudaError_t launch_pair(const LmheadPlan& plan, const LmheadMaps& m, const KParams& p, cudaStream_t stream, bool overlap) {
   auto kernel = kBBox == 32 ? lmhead_entropy_pair_kernel<kTf32, kBBox, kPairWideStages, 2, kFuse>
                             : lmhead_entropy_pair_kernel<kTf32, kBBox, kPairStages, 1, kFuse>;
-  kernel<<<plan.grid, kLmheadThreads, kPairSmemBytes, stream>>>(*m.hidden, *m.w, kFuse ? *m.w1 : *m.w, p);
-  return cudaGetLastError();
+  LaunchConfig lc(plan.grid, kPairSmemBytes, stream, overlap);
+  return cudaLaunchKernelEx(&lc.cfg, kernel, *m.hidden, *m.w, kFuse ? *m.w1 : *m.w, p);
 }
 
 // *pair_workers receives the smaller of its value and the CTA pairs of this kernel that can be resident at once
@@ -854,6 +927,7 @@ LmheadPlan make_lmhead_plan(int64_t T, int d, int V, int elem_bytes, int num_sms
   const bool pairs_ok = pair_cap > 0 && mode != EGTP_LMHEAD_SINGLE_CTA && !f32;
   if (pl.variant == 2 && pairs_ok) pl.variant = 5;
   if (pl.variant == 0 && pairs_ok && mode == EGTP_LMHEAD_CTA_PAIRS && head_cols == 0) pl.variant = 4;
+  if (pl.variant == 0 && pairs_ok && mode == EGTP_LMHEAD_CTA_PAIRS_WIDE && head_cols == 0) pl.variant = 6;
   const bool pair = pl.variant >= 4;
   const bool one_block = pl.variant == 1 || pl.variant == 2 || pl.variant == 5;
   const Shape& sh = shape_of(pl.variant);
@@ -989,7 +1063,8 @@ cudaError_t lmhead_prepare_device(int* pair_workers_out) {
 }
 
 cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const LmheadMaps& maps, int64_t T, int V,
-                                  float* partials, int32_t* status, cudaStream_t stream, float* head_g) {
+                                  float* partials, int32_t* status, cudaStream_t stream, float* head_g,
+                                  bool overlap_previous) {
   (void)T;
   KParams p{};
   p.row_blocks = plan.row_blocks;
@@ -1016,26 +1091,27 @@ cudaError_t launch_lmhead_entropy(const LmheadPlan& plan, bool tf32, const Lmhea
     // fused head columns: bf16, one CTA per SM only
     if (tf32 || maps.w1 == nullptr || (plan.variant < 4 && maps.w1_tile == nullptr) || head_g == nullptr) return cudaErrorInvalidValue;
     switch (plan.variant) {
-      case 0: return launch_shape<false, EGTP_SHAPE_PROMPT, true>(plan, maps, p, stream);
-      case 1: return launch_shape<false, EGTP_SHAPE_DECODE1, true>(plan, maps, p, stream);
-      case 2: return launch_shape<false, EGTP_SHAPE_DECODE2, true>(plan, maps, p, stream);
-      case 5: return launch_pair<false, 32, true>(plan, maps, p, stream);
+      case 0: return launch_shape<false, EGTP_SHAPE_PROMPT, true>(plan, maps, p, stream, overlap_previous);
+      case 1: return launch_shape<false, EGTP_SHAPE_DECODE1, true>(plan, maps, p, stream, overlap_previous);
+      case 2: return launch_shape<false, EGTP_SHAPE_DECODE2, true>(plan, maps, p, stream, overlap_previous);
+      case 5: return launch_pair<false, 32, true>(plan, maps, p, stream, overlap_previous);
       default: return cudaErrorInvalidValue;
     }
   }
   if (tf32) {
     switch (plan.variant) {
-      case 0: return launch_shape<true, EGTP_SHAPE_PROMPT_F32>(plan, maps, p, stream);
-      case 1: return launch_shape<true, EGTP_SHAPE_DECODE1_F32>(plan, maps, p, stream);
+      case 0: return launch_shape<true, EGTP_SHAPE_PROMPT_F32>(plan, maps, p, stream, overlap_previous);
+      case 1: return launch_shape<true, EGTP_SHAPE_DECODE1_F32>(plan, maps, p, stream, overlap_previous);
       default: return cudaErrorInvalidValue;     // the planner gives fp32 rows no other shape
     }
   }
   switch (plan.variant) {
-    case 1: return launch_shape<false, EGTP_SHAPE_DECODE1>(plan, maps, p, stream);
-    case 2: return launch_shape<false, EGTP_SHAPE_DECODE2>(plan, maps, p, stream);
-    case 4: return launch_pair<false, 128>(plan, maps, p, stream);
-    case 5: return launch_pair<false, 32>(plan, maps, p, stream);
-    default: return launch_shape<false, EGTP_SHAPE_PROMPT>(plan, maps, p, stream);
+    case 1: return launch_shape<false, EGTP_SHAPE_DECODE1>(plan, maps, p, stream, overlap_previous);
+    case 2: return launch_shape<false, EGTP_SHAPE_DECODE2>(plan, maps, p, stream, overlap_previous);
+    case 4: return launch_pair<false, 128>(plan, maps, p, stream, overlap_previous);
+    case 5:
+    case 6: return launch_pair<false, 32>(plan, maps, p, stream, overlap_previous);
+    default: return launch_shape<false, EGTP_SHAPE_PROMPT>(plan, maps, p, stream, overlap_previous);
   }
 }
 

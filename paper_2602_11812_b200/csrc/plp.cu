@@ -42,6 +42,23 @@ __device__ __forceinline__ void load8<float>(const float* p, float (&v)[8]) {
 
 constexpr int kPlpMaxThreads = 1024;
 
+// Two live rows of one step must not name the same slot (they would race on its state).  Every step of a state has
+// a stamp (epoch[0]); a block claims its slot by swapping the stamp into the slot's owner word and finds the stamp
+// already there if another row of the same step was first.  The last block of a launch to leave (epoch[1] counts them)
+// moves the stamp on, so every block of a launch sees the same stamp whatever the order they run in, and a step that is
+// replayed from a CUDA graph gets a fresh stamp each time.
+__device__ __forceinline__ bool claim_slot(int32_t* owner, int slot, int stamp) {
+  return atomicExch(owner + slot, stamp) != stamp;
+}
+__device__ __forceinline__ void leave_step(int32_t* epoch, int stamp) {
+  __threadfence();
+  if (atomicAdd(epoch + 1, 1) == static_cast<int>(gridDim.x) - 1) {
+    epoch[1] = 0;
+    __threadfence();
+    *reinterpret_cast<volatile int32_t*>(epoch) = stamp == 0x7fffffff ? 1 : stamp + 1;
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kPlpMaxThreads)
 plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* __restrict__ partials, int slots,
@@ -50,13 +67,23 @@ plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* _
                   const float* __restrict__ src_s, const float* __restrict__ src_pooled, int n_src, int d,
                   int num_slots, float inv_alpha, float* __restrict__ st_m, float* __restrict__ st_s,
                   float* __restrict__ st_acc, float* __restrict__ z, int64_t ldz, __nv_bfloat16* __restrict__ zcat,
-                  int32_t* status) {
-  if (*status != 0) return;
+                  int32_t* __restrict__ owner, int32_t* __restrict__ epoch, int32_t* status) {
+  __shared__ int refused;
+  const int stamp = *reinterpret_cast<volatile int32_t*>(epoch);
   const int i = blockIdx.x;
   const int slot = slot_ids ? slot_ids[i] : i;
   const int rs = reset_src ? reset_src[i] : PLP_RESET_KEEP;
-  if (slot < 0 || slot >= num_slots || rs < PLP_RESET_KEEP || rs >= n_src) {
-    if (threadIdx.x == 0) atomicCAS(status, 0, EGTP_ERR_BAD_SLOT);
+  if (threadIdx.x == 0) {
+    int r = *status != 0 ? 1 : 0;
+    if (r == 0 && (slot < 0 || slot >= num_slots || rs < PLP_RESET_KEEP || rs >= n_src || !claim_slot(owner, slot, stamp))) {
+      atomicCAS(status, 0, EGTP_ERR_BAD_SLOT);      // out of range, or a second row of this step on the same slot
+      r = 1;
+    }
+    refused = r;
+  }
+  __syncthreads();
+  if (refused != 0) {
+    if (threadIdx.x == 0) leave_step(epoch, stamp);
     return;
   }
   // state before this token
@@ -131,6 +158,7 @@ plp_update_kernel(const T* __restrict__ hidden_step, int64_t ldh, const float* _
   if (threadIdx.x == 0) {
     st_m[slot] = m_new;
     st_s[slot] = s_new;
+    leave_step(epoch, stamp);
   }
 }
 
@@ -153,20 +181,26 @@ plp_update_bound_kernel(const T* __restrict__ hidden_step, int64_t ldh, const fl
                         const float* __restrict__ g, int64_t ldg, int g_splits, int64_t g_split_stride, int m_h,
                         int d_out, const float* __restrict__ b1,
                         const TW* __restrict__ W2, const float* __restrict__ b2, const float* __restrict__ centres,
-                        int mode, float* __restrict__ y, int32_t* status) {
+                        int mode, float* __restrict__ y, int32_t* __restrict__ owner, int32_t* __restrict__ epoch,
+                        int32_t* status) {
   // Launched with programmatic stream serialization: this block may start while the LM-head kernel is still
   // running.  Its inputs and the state rows (last written by an earlier, completed kernel) are read ahead;
   // the status word, the entropy partials and g come after pdl_wait().
   extern __shared__ float smem[];
   float* u = smem;            // [m_h]
   float* o = smem + m_h;      // [d_out]
+  // the next step's LM-head kernel may set its blocks up as this grid drains (it waits for this grid's end before
+  // it reads or writes anything in global memory)
+  pdl_launch_dependents();
+  __shared__ int refused;
   const int i = blockIdx.x;
-  const int slot = slot_ids ? slot_ids[i] : i;
-  const int rs = reset_src ? reset_src[i] : PLP_RESET_KEEP;
-  if (slot < 0 || slot >= num_slots || rs < PLP_RESET_KEEP || rs >= n_src) {
-    if (threadIdx.x == 0) atomicCAS(status, 0, EGTP_ERR_BAD_SLOT);
-    return;
-  }
+  const int slot_in = slot_ids ? slot_ids[i] : i;
+  const int rs_in = reset_src ? reset_src[i] : PLP_RESET_KEEP;
+  // a row with a slot or reset source out of range reads ahead as if it were row 0 of an untouched state and is
+  // refused after the wait below (every block has to take part in the step's bookkeeping there)
+  const bool in_range = slot_in >= 0 && slot_in < num_slots && rs_in >= PLP_RESET_KEEP && rs_in < n_src;
+  const int slot = in_range ? slot_in : 0;
+  const int rs = in_range ? rs_in : PLP_RESET_KEEP;
   float m_old, s_old;
   const float* acc_src;    // nullptr = zeros
   const float* proj_src;   // W1 times the vector acc_src points at
@@ -195,7 +229,20 @@ plp_update_bound_kernel(const T* __restrict__ hidden_step, int64_t ldh, const fl
     if (acc_src != nullptr) load8<float>(acc_src + col, acc);
   }
   pdl_wait();
-  if (*status != 0) return;     // uniform over the block
+  const int stamp = *reinterpret_cast<volatile int32_t*>(epoch);
+  if (threadIdx.x == 0) {
+    int r = *status != 0 ? 1 : 0;
+    if (r == 0 && (!in_range || !claim_slot(owner, slot, stamp))) {
+      atomicCAS(status, 0, EGTP_ERR_BAD_SLOT);      // out of range, or a second row of this step on the same slot
+      r = 1;
+    }
+    refused = r;
+  }
+  __syncthreads();
+  if (refused != 0) {
+    if (threadIdx.x == 0) leave_step(epoch, stamp);
+    return;
+  }
   const float H_new = merge_partials_warp(partials + static_cast<int64_t>(i) * row_stride, slots, slot_stride, threadIdx.x & 31);
   if (threadIdx.x == 0 && Hstep_out != nullptr) Hstep_out[i] = H_new;
   const float a = H_new * inv_alpha;
@@ -238,6 +285,7 @@ plp_update_bound_kernel(const T* __restrict__ hidden_step, int64_t ldh, const fl
   if (threadIdx.x == 0) {
     st_m[slot] = m_new;
     st_s[slot] = s_new;
+    leave_step(epoch, stamp);
   }
   head_output_stage<TW>(u, o, m_h, d_out, W2, b2, centres, mode, y, nullptr, i);
 }
@@ -264,8 +312,8 @@ cudaError_t launch_plp_update_bound(const void* hidden_step, int64_t ldh, const 
                                     const float* src_pooled, const float* src_proj, int n_src, int rows, int d,
                                     int num_slots, float inv_alpha, float* st_m, float* st_s, float* st_acc,
                                     float* st_proj, float* z, int64_t ldz, const float* g, int64_t ldg, int g_splits,
-                                    int64_t g_split_stride, const HeadArgs& h, float* y, int32_t* status,
-                                    cudaStream_t stream, bool overlap_previous) {
+                                    int64_t g_split_stride, const HeadArgs& h, float* y, int32_t* owner, int32_t* epoch,
+                                    int32_t* status, cudaStream_t stream, bool overlap_previous) {
   const int threads = update_threads(rows, d, 64);
   const size_t smem = static_cast<size_t>(h.m_h + h.d_out) * sizeof(float);
   cudaLaunchConfig_t cfg{};
@@ -284,23 +332,23 @@ cudaError_t launch_plp_update_bound(const void* hidden_step, int64_t ldh, const 
                             row_stride, slot_stride, Hstep_out, slot_ids, reset_src, src_m, src_s, src_pooled, src_proj,
                             n_src, d, num_slots, inv_alpha, st_m, st_s, st_acc, st_proj, z, ldz, g, ldg, g_splits, g_split_stride,
                             h.m_h, h.d_out,
-                            h.b1, W2, h.b2, h.centres, h.mode, y, status);
+                            h.b1, W2, h.b2, h.centres, h.mode, y, owner, epoch, status);
 }
 
 cudaError_t launch_plp_update(const void* hidden_step, int64_t ldh, bool bf16, const float* partials, int slots,
                               int64_t row_stride, int64_t slot_stride, float* Hstep_out, const int32_t* slot_ids, const int32_t* reset_src, const float* src_m,
                               const float* src_s, const float* src_pooled, int n_src, int rows, int d, int num_slots,
                               float inv_alpha, float* st_m, float* st_s, float* st_acc, float* z, int64_t ldz,
-                              int32_t* status, cudaStream_t stream, void* zcat) {
+                              int32_t* owner, int32_t* epoch, int32_t* status, cudaStream_t stream, void* zcat) {
   const int threads = update_threads(rows, d, 32);
   if (bf16) {
     plp_update_kernel<__nv_bfloat16><<<rows, threads, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(hidden_step), ldh, partials, slots, row_stride, slot_stride, Hstep_out, slot_ids, reset_src, src_m, src_s, src_pooled,
-        n_src, d, num_slots, inv_alpha, st_m, st_s, st_acc, z, ldz, static_cast<__nv_bfloat16*>(zcat), status);
+        n_src, d, num_slots, inv_alpha, st_m, st_s, st_acc, z, ldz, static_cast<__nv_bfloat16*>(zcat), owner, epoch, status);
   } else {
     plp_update_kernel<float><<<rows, threads, 0, stream>>>(static_cast<const float*>(hidden_step), ldh, partials, slots, row_stride, slot_stride, Hstep_out, slot_ids,
                                                        reset_src, src_m, src_s, src_pooled, n_src, d, num_slots,
-                                                       inv_alpha, st_m, st_s, st_acc, z, ldz, static_cast<__nv_bfloat16*>(zcat), status);
+                                                       inv_alpha, st_m, st_s, st_acc, z, ldz, static_cast<__nv_bfloat16*>(zcat), owner, epoch, status);
   }
   return cudaGetLastError();
 }

@@ -11,16 +11,7 @@ namespace egtp {
 
 namespace {
 
-__device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-  return v;
-}
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
+constexpr int kMergeThreads = 256;   // four lanes for each token of a 64-token pooling chunk
 
 // Largest b in [0, B] with offsets[b] <= t (offsets non-decreasing, offsets[0] <= t assumed).
 __device__ __forceinline__ int upper_segment(const int32_t* __restrict__ off, int B, int64_t t) {
@@ -49,31 +40,78 @@ __global__ void validate_offsets_kernel(const int32_t* __restrict__ off, int B, 
   }
 }
 
-// --------------------------------------------------------------------------- Eq. 2: merge
-// One warp per token: lanes stride over the token's (m, s, t2) partials (contiguous in memory),
-// fold them in a fixed order, then combine across lanes: H = ln S - ln2 * T2 / S.
-// Also writes the token's prompt index.  With T_check >= 0, block 0 first checks the offsets against that
-// token count (the kernels that index tokens through the offsets come later in the stream and see the status).
-__global__ void entropy_merge_kernel(const float* __restrict__ partials, int slots, int64_t row_stride,
-                                     int64_t slot_stride, int64_t T, int64_t row0, float* __restrict__ H, const int32_t* __restrict__ off, int B,
-                                     int32_t* __restrict__ seg_id, int64_t T_check, int32_t* __restrict__ status) {
+// --------------------------------------------------------------------------- Eq. 2: merge (and the first half of Eq. 3)
+// One block per pooling chunk of 64 tokens, four lanes per token: the lanes stride over the token's (m, s, t2)
+// partials (contiguous in memory), fold them in a fixed order, then combine across lanes: H = ln S - ln2 * T2 / S.
+// Also writes the token's prompt index.  With T_check >= 0, block 0 first checks the offsets against that token
+// count (the kernels that index tokens through the offsets come later in the stream and see the status).
+// With `weights` given, the block then prepares the pooling of its chunk: for every run of tokens of one prompt inside
+// the chunk, m = max H_i/alpha over the run, the unnormalised weights w_i = exp(H_i/alpha - m) (Eq. 3 up to the
+// normaliser) and (m, sum w) of the run, stored where the pooling kernels expect them: seg_m / seg_s for a prompt
+// that lies wholly inside the chunk, else ms_a[c] (run entered from the left) or ms_b[c] (run leaves to the right).
+__global__ void __launch_bounds__(kMergeThreads)
+entropy_merge_kernel(const float* __restrict__ partials, int slots, int64_t row_stride, int64_t slot_stride, int64_t T,
+                     int64_t row0, float* __restrict__ H, const int32_t* __restrict__ off, int B,
+                     int32_t* __restrict__ seg_id, int64_t T_check, float inv_alpha, float* __restrict__ weights,
+                     float2* __restrict__ ms_a, float2* __restrict__ ms_b, float* __restrict__ seg_m,
+                     float* __restrict__ seg_s, int32_t* __restrict__ status) {
   if (*status != 0) return;
   if (T_check >= 0 && blockIdx.x == 0) {
     if (__syncthreads_or(offsets_bad(off, B, T_check) ? 1 : 0)) {
       if (threadIdx.x == 0) atomicCAS(status, 0, EGTP_ERR_BAD_OFFSETS);
     }
   }
-  const int lane = threadIdx.x & 31;
-  const int64_t i = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (i >= T) return;
-  const float h = merge_partials_warp(partials + i * row_stride, slots, slot_stride, lane);
-  if (lane == 0) {
-    const int64_t g = row0 + i;      // token index in the whole batch (the partials may cover one piece of it)
-    H[g] = h;
-    if (seg_id != nullptr) {
+  __shared__ float a_s[kPoolChunkTokens];
+  __shared__ int sid_s[kPoolChunkTokens];
+  // four lanes per token, eight tokens per warp at once: thread 4 idx + q works on token idx of the chunk
+  static_assert(kMergeThreads == 4 * kPoolChunkTokens, "four lanes per token of the chunk");
+  const int idx = threadIdx.x >> 2, q = threadIdx.x & 3;
+  const int64_t i0 = static_cast<int64_t>(blockIdx.x) * kPoolChunkTokens;      // first token of the chunk in this piece
+  const int64_t i = i0 + idx;
+  const bool in_range = i < T;
+  // (rows past the end take part with zero slots: the group shuffles need every lane of the warp)
+  const EntropyPartial ep = merge_partials_group_raw<4>(partials + (in_range ? i : 0) * row_stride, in_range ? slots : 0,
+                                                        slot_stride, q);
+  if (q == 0) {
+    if (!in_range) {
+      sid_s[idx] = -1;
+    } else {
+      const float h = entropy_of(ep);
+      const int64_t g = row0 + i;      // token index in the whole batch (the partials may cover one piece of it)
+      H[g] = h;
       int sid = -1;
-      if (B > 0 && g >= off[0] && g < off[B]) sid = upper_segment(off, B, g);
-      seg_id[g] = sid;
+      if (off != nullptr && B > 0 && g >= off[0] && g < off[B]) sid = upper_segment(off, B, g);
+      if (seg_id != nullptr) seg_id[g] = sid;
+      a_s[idx] = h * inv_alpha;
+      sid_s[idx] = sid;
+    }
+  }
+  if (weights == nullptr) return;
+  __syncthreads();
+  const int t = threadIdx.x;
+  if (t >= kPoolChunkTokens || i0 + t >= T) return;
+  const int64_t g = row0 + i0 + t;
+  const int sid = sid_s[t];
+  if (sid < 0) { weights[g] = 0.f; return; }
+  int lo = t, hi = t + 1;                                   // the run of this prompt inside the chunk: [lo, hi)
+  while (lo > 0 && sid_s[lo - 1] == sid) --lo;
+  while (hi < kPoolChunkTokens && sid_s[hi] == sid) ++hi;
+  float m = a_s[lo];
+  for (int j = lo + 1; j < hi; ++j) m = fmaxf(m, a_s[j]);
+  weights[g] = expf(a_s[t] - m);
+  if (t == lo) {
+    float wsum = 0.f;
+    for (int j = lo; j < hi; ++j) wsum += expf(a_s[j] - m);
+    const int64_t c = (row0 + i0) / kPoolChunkTokens;       // chunk index in the whole batch
+    const int64_t c_lo = c * kPoolChunkTokens, c_hi = c_lo + kPoolChunkTokens;
+    const int64_t seg_begin = off[sid], seg_end = off[sid + 1];
+    if (seg_begin >= c_lo && seg_end <= c_hi) {
+      if (seg_m) seg_m[sid] = m;
+      if (seg_s) seg_s[sid] = wsum;
+    } else if (seg_begin < c_lo) {
+      ms_a[c] = make_float2(m, wsum);
+    } else {
+      ms_b[c] = make_float2(m, wsum);
     }
   }
 }
@@ -112,12 +150,15 @@ __global__ void token_weights_kernel(const float* __restrict__ H, const int32_t*
 }
 
 // --------------------------------------------------------------------------- Eq. 3 + Eq. 4: pooling
+// Eight consecutive channels of one row: loaded as they are (16 bytes of bf16, or 32 bytes of fp32) and widened
+// only where they are consumed, so that four rows in flight cost a thread 16 registers in the bf16 case.
 template <typename T>
 struct Row8;
 template <>
 struct Row8<__nv_bfloat16> {
-  static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&v)[8]) {
-    const uint4 q = __ldg(reinterpret_cast<const uint4*>(p));
+  uint4 q;
+  __device__ __forceinline__ void load(const __nv_bfloat16* p) { q = __ldg(reinterpret_cast<const uint4*>(p)); }
+  __device__ __forceinline__ void get(float (&v)[8]) const {
     const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -128,13 +169,24 @@ struct Row8<__nv_bfloat16> {
 };
 template <>
 struct Row8<float> {
-  static __device__ __forceinline__ void load(const float* p, float (&v)[8]) {
-    const float4 a = __ldg(reinterpret_cast<const float4*>(p));
-    const float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+  float4 a, b;
+  __device__ __forceinline__ void load(const float* p) {
+    a = __ldg(reinterpret_cast<const float4*>(p));
+    b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+  }
+  __device__ __forceinline__ void get(float (&v)[8]) const {
     v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
     v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
   }
 };
+// acc += w * row, or acc = max(acc, row)
+template <typename T, bool kMax>
+__device__ __forceinline__ void fold_row(float (&acc)[8], const Row8<T>& row, float w) {
+  float v[8];
+  row.get(v);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) acc[k] = kMax ? fmaxf(acc[k], v[k]) : fmaf(w, v[k], acc[k]);
+}
 
 __device__ __forceinline__ void store8(float* p, const float (&v)[8]) {
   reinterpret_cast<float4*>(p)[0] = make_float4(v[0], v[1], v[2], v[3]);
@@ -163,9 +215,10 @@ __device__ __forceinline__ void store8_hi_lo(__nv_bfloat16* row, int d, int col,
 // All but the maximum are weighted sums sum_i w_i h_i / sum_i w_i with unnormalised weights
 //   entropy: w_i = exp(H_i/alpha - m), m = the largest H_i/alpha among the tokens summed together
 //   mean:    w_i = 1                    last: w_i = 1 for the prompt's last token, else 0
-// so one kernel serves them: a block sums a run of tokens with weights relative to the run's own m and leaves
-// (m, sum w, sum w h); runs of one prompt are merged later by rescaling to the common maximum (the same
-// recurrence as the PLP state, Eq. 8).  The normalised weights of Eq. 3 are never stored.
+// so one kernel serves them: a block sums a run of tokens with weights relative to the run's own m, which leaves
+// (m, sum w, sum w h) per run (in entropy mode the weights and the two scalars come prepared from the merge
+// kernel); runs of one prompt are merged later by rescaling to the common maximum (the same recurrence as the PLP
+// state, Eq. 8).  The normalised weights of Eq. 3 are never stored.
 enum : int { kPoolEntropy = 0, kPoolMean = 1, kPoolMax = 2, kPoolLast = 3 };
 
 // Block (c, y): tokens [c*64, (c+1)*64) clipped to [offsets[0], offsets[B]), channels [(y*128 + tid)*8, +8).
@@ -174,8 +227,8 @@ enum : int { kPoolEntropy = 0, kPoolMean = 1, kPoolMax = 2, kPoolLast = 3 };
 // if it starts here and leaves to the right, each with its (m, sum w) in piece_ms.  The combine kernel merges the
 // pieces of each prompt in chunk order.
 template <typename T, int kMode>
-__global__ void __launch_bounds__(kPoolThreads)
-pool_kernel(const T* __restrict__ hidden, int64_t ldh, const float* __restrict__ H, float inv_alpha,
+__global__ void __launch_bounds__(kPoolThreads, sizeof(T) == 2 ? (kMode == kPoolEntropy ? 16 : 12) : 8)   // bf16: 32 (40) registers, an SM full of warps keeps the row loads in flight
+pool_kernel(const T* __restrict__ hidden, int64_t ldh, const float* __restrict__ weights,
             const int32_t* __restrict__ off, int B, int d, float* __restrict__ pooled,
             float* __restrict__ piece_a, float* __restrict__ piece_b, float2* __restrict__ ms_a,
             float2* __restrict__ ms_b, float* __restrict__ seg_m, float* __restrict__ seg_s,
@@ -193,82 +246,63 @@ pool_kernel(const T* __restrict__ hidden, int64_t ldh, const float* __restrict__
     const int64_t seg_begin = off[b], seg_end = off[b + 1];
     if (seg_end <= t0) { ++b; continue; }       // empty prompts own no token
     const int64_t run_end = min(seg_end, t1);
-    // the run's reference point and (for last-token pooling) the one row that counts
-    float m = 0.f;
-    if constexpr (kMode == kPoolEntropy) {
-      m = -INFINITY;
-      for (int64_t t = t0; t < run_end; ++t) m = fmaxf(m, __ldg(H + t) * inv_alpha);
-    }
     float acc[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) acc[k] = kMode == kPoolMax ? -INFINITY : 0.f;
     float wsum = 0.f;
     if constexpr (kMode == kPoolLast) {
       if (run_end == seg_end) {                   // the prompt's last token is in this run: read that row only
-        Row8<T>::load(hidden + (seg_end - 1) * ldh + col, acc);
+        Row8<T> r;
+        r.load(hidden + (seg_end - 1) * ldh + col);
+        r.get(acc);
         wsum = 1.f;
       }
     } else {
+      constexpr bool kIsMax = kMode == kPoolMax;
       const T* rowp = hidden + t0 * ldh + col;
       int64_t t = t0;
       for (; t + 4 <= run_end; t += 4) {           // four rows in flight per thread
-        float v0[8], v1[8], v2[8], v3[8];
-        Row8<T>::load(rowp, v0);
-        Row8<T>::load(rowp + ldh, v1);
-        Row8<T>::load(rowp + 2 * ldh, v2);
-        Row8<T>::load(rowp + 3 * ldh, v3);
-        if constexpr (kMode == kPoolMax) {
-#pragma unroll
-          for (int k = 0; k < 8; ++k) acc[k] = fmaxf(fmaxf(acc[k], fmaxf(v0[k], v1[k])), fmaxf(v2[k], v3[k]));
-        } else {
-          float w0 = 1.f, w1 = 1.f, w2 = 1.f, w3 = 1.f;
-          if constexpr (kMode == kPoolEntropy) {
-            w0 = expf(__ldg(H + t) * inv_alpha - m); w1 = expf(__ldg(H + t + 1) * inv_alpha - m);
-            w2 = expf(__ldg(H + t + 2) * inv_alpha - m); w3 = expf(__ldg(H + t + 3) * inv_alpha - m);
-          }
-          wsum += (w0 + w1) + (w2 + w3);
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            acc[k] = fmaf(w0, v0[k], acc[k]);
-            acc[k] = fmaf(w1, v1[k], acc[k]);
-            acc[k] = fmaf(w2, v2[k], acc[k]);
-            acc[k] = fmaf(w3, v3[k], acc[k]);
-          }
+        Row8<T> r0, r1, r2, r3;
+        r0.load(rowp);
+        r1.load(rowp + ldh);
+        r2.load(rowp + 2 * ldh);
+        r3.load(rowp + 3 * ldh);
+        float w0 = 1.f, w1 = 1.f, w2 = 1.f, w3 = 1.f;
+        if constexpr (kMode == kPoolEntropy) {
+          w0 = __ldg(weights + t); w1 = __ldg(weights + t + 1); w2 = __ldg(weights + t + 2); w3 = __ldg(weights + t + 3);
         }
+        fold_row<T, kIsMax>(acc, r0, w0);
+        fold_row<T, kIsMax>(acc, r1, w1);
+        fold_row<T, kIsMax>(acc, r2, w2);
+        fold_row<T, kIsMax>(acc, r3, w3);
         rowp += 4 * ldh;
       }
       for (; t < run_end; ++t) {
-        float v0[8];
-        Row8<T>::load(rowp, v0);
-        if constexpr (kMode == kPoolMax) {
-#pragma unroll
-          for (int k = 0; k < 8; ++k) acc[k] = fmaxf(acc[k], v0[k]);
-        } else {
-          const float w0 = kMode == kPoolEntropy ? expf(__ldg(H + t) * inv_alpha - m) : 1.f;
-          wsum += w0;
-#pragma unroll
-          for (int k = 0; k < 8; ++k) acc[k] = fmaf(w0, v0[k], acc[k]);
-        }
+        Row8<T> r0;
+        r0.load(rowp);
+        fold_row<T, kIsMax>(acc, r0, kMode == kPoolEntropy ? __ldg(weights + t) : 1.f);
         rowp += ldh;
       }
+      if constexpr (kMode == kPoolMean) wsum = static_cast<float>(run_end - t0);
     }
+    // entropy mode: (m, sum w) of every run were left by the merge kernel; the other modes have m = 0 and count here
     if (seg_begin >= c_lo && seg_end <= c_hi) {       // the whole prompt: normalise and finish
       if constexpr (kMode != kPoolMax) {
-        const float inv = 1.f / wsum;
+        const float inv = 1.f / (kMode == kPoolEntropy ? seg_s[b] : wsum);
 #pragma unroll
         for (int k = 0; k < 8; ++k) acc[k] *= inv;
       }
       store8(pooled + static_cast<int64_t>(b) * d + col, acc);
-      if (scribe) {
-        if (seg_m) seg_m[b] = m;
+      if (kMode != kPoolEntropy && scribe) {
+        if (seg_m) seg_m[b] = 0.f;
         if (seg_s) seg_s[b] = wsum;
       }
     } else if (seg_begin < c_lo) {
       store8(piece_a + c * d + col, acc);
-      if (scribe) ms_a[c] = make_float2(m, wsum);
+      if (kMode != kPoolEntropy && scribe) ms_a[c] = make_float2(0.f, wsum);
     } else {
       store8(piece_b + c * d + col, acc);
-      if (scribe) ms_b[c] = make_float2(m, wsum);
+      if (kMode != kPoolEntropy && scribe) ms_b[c] = make_float2(0.f, wsum);
     }
     t0 = run_end;
     ++b;
@@ -330,7 +364,24 @@ pool_combine_kernel(const int32_t* __restrict__ off, int B, int d, const float* 
     load8f(piece_b + c0 * d + col, acc);
 #pragma unroll
     for (int k = 0; k < 8; ++k) acc[k] *= r;
-    for (int64_t c = c0 + 1; c <= c1; ++c) {
+    int64_t c = c0 + 1;
+    for (; c + 4 <= c1 + 1; c += 4) {            // four pieces in flight, added in chunk order
+      float2 ms[4];
+      float pv[4][8];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        ms[u] = ms_a[c + u];
+        load8f(piece_a + (c + u) * d + col, pv[u]);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        r = expf(ms[u].x - M);
+        Z = fmaf(ms[u].y, r, Z);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) acc[k] = fmaf(pv[u][k], r, acc[k]);
+      }
+    }
+    for (; c <= c1; ++c) {
       const float2 ms = ms_a[c];
       r = expf(ms.x - M);
       Z = fmaf(ms.y, r, Z);
@@ -360,11 +411,15 @@ cudaError_t launch_validate_offsets(const int32_t* offsets, int B, int64_t T, in
 
 cudaError_t launch_entropy_merge(const float* partials, int slots, int64_t row_stride, int64_t slot_stride, int64_t T,
                                  int64_t row0, float* H, const int32_t* offsets, int B, int32_t* seg_id_out,
-                                 int64_t T_check, int32_t* status, cudaStream_t stream) {
-  const int threads = 256, rows_per_block = threads / 32;
-  const unsigned blocks = static_cast<unsigned>((T + rows_per_block - 1) / rows_per_block);
-  entropy_merge_kernel<<<blocks, threads, 0, stream>>>(partials, slots, row_stride, slot_stride, T, row0, H, offsets, B,
-                                                       seg_id_out, T_check, status);
+                                 int64_t T_check, int32_t* status, cudaStream_t stream, const PoolPrep* prep) {
+  if (prep != nullptr && (row0 % kPoolChunkTokens != 0 || offsets == nullptr)) return cudaErrorInvalidValue;
+  const unsigned blocks = static_cast<unsigned>((T + kPoolChunkTokens - 1) / kPoolChunkTokens);
+  float2* ms_a = prep ? reinterpret_cast<float2*>(prep->piece_ms) : nullptr;
+  float2* ms_b = prep ? ms_a + prep->chunks : nullptr;
+  entropy_merge_kernel<<<blocks, kMergeThreads, 0, stream>>>(partials, slots, row_stride, slot_stride, T, row0, H, offsets, B,
+                                                             seg_id_out, T_check, prep ? prep->inv_alpha : 1.f,
+                                                             prep ? prep->weights : nullptr, ms_a, ms_b,
+                                                             prep ? prep->seg_m : nullptr, prep ? prep->seg_s : nullptr, status);
   return cudaGetLastError();
 }
 
@@ -387,30 +442,31 @@ cudaError_t launch_token_weights(const float* H, const int32_t* offsets, int B, 
 namespace {
 
 template <typename T>
-void launch_pool_typed(int mode, dim3 grid, cudaStream_t stream, const T* hidden, int64_t ldh, const float* H,
-                       float inv_alpha, const int32_t* off, int B, int d, float* pooled, float* piece_a, float* piece_b,
+void launch_pool_typed(int mode, dim3 grid, cudaStream_t stream, const T* hidden, int64_t ldh, const float* weights,
+                       const int32_t* off, int B, int d, float* pooled, float* piece_a, float* piece_b,
                        float2* ms_a, float2* ms_b, float* seg_m, float* seg_s, const int32_t* status) {
   switch (mode) {
     case kPoolEntropy:
-      pool_kernel<T, kPoolEntropy><<<grid, kPoolThreads, 0, stream>>>(hidden, ldh, H, inv_alpha, off, B, d, pooled, piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
+      pool_kernel<T, kPoolEntropy><<<grid, kPoolThreads, 0, stream>>>(hidden, ldh, weights, off, B, d, pooled, piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
       break;
     case kPoolMean:
-      pool_kernel<T, kPoolMean><<<grid, kPoolThreads, 0, stream>>>(hidden, ldh, H, inv_alpha, off, B, d, pooled, piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
+      pool_kernel<T, kPoolMean><<<grid, kPoolThreads, 0, stream>>>(hidden, ldh, weights, off, B, d, pooled, piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
       break;
     case kPoolMax:
-      pool_kernel<T, kPoolMax><<<grid, kPoolThreads, 0, stream>>>(hidden, ldh, H, inv_alpha, off, B, d, pooled, piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
+      pool_kernel<T, kPoolMax><<<grid, kPoolThreads, 0, stream>>>(hidden, ldh, weights, off, B, d, pooled, piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
       break;
     default:
-      pool_kernel<T, kPoolLast><<<grid, kPoolThreads, 0, stream>>>(hidden, ldh, H, inv_alpha, off, B, d, pooled, piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
+      pool_kernel<T, kPoolLast><<<grid, kPoolThreads, 0, stream>>>(hidden, ldh, weights, off, B, d, pooled, piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
       break;
   }
 }
 
 }  // namespace
 
-static_assert(kPoolMean == EGTP_POOL_MEAN && kPoolMax == EGTP_POOL_MAX && kPoolLast == EGTP_POOL_LAST, "pooling mode codes");
+static_assert(static_cast<int>(kPoolMean) == static_cast<int>(EGTP_POOL_MEAN) && static_cast<int>(kPoolMax) == static_cast<int>(EGTP_POOL_MAX) &&
+                  static_cast<int>(kPoolLast) == static_cast<int>(EGTP_POOL_LAST), "pooling mode codes");
 
-cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, int mode, const float* H, float inv_alpha,
+cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, int mode, const float* weights,
                         const int32_t* offsets, int B, int64_t T, int d, float* pooled, float* piece_a,
                         float* piece_b, float* piece_ms, float* seg_m, float* seg_s, const int32_t* status,
                         cudaStream_t stream) {
@@ -420,10 +476,10 @@ cudaError_t launch_pool(const void* hidden, int64_t ldh, bool bf16, int mode, co
   float2* ms_a = reinterpret_cast<float2*>(piece_ms);
   float2* ms_b = ms_a + chunks;
   if (bf16)
-    launch_pool_typed<__nv_bfloat16>(mode, grid, stream, static_cast<const __nv_bfloat16*>(hidden), ldh, H, inv_alpha, offsets, B, d,
+    launch_pool_typed<__nv_bfloat16>(mode, grid, stream, static_cast<const __nv_bfloat16*>(hidden), ldh, weights, offsets, B, d,
                                      pooled, piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
   else
-    launch_pool_typed<float>(mode, grid, stream, static_cast<const float*>(hidden), ldh, H, inv_alpha, offsets, B, d, pooled,
+    launch_pool_typed<float>(mode, grid, stream, static_cast<const float*>(hidden), ldh, weights, offsets, B, d, pooled,
                              piece_a, piece_b, ms_a, ms_b, seg_m, seg_s, status);
   return cudaGetLastError();
 }

@@ -225,11 +225,15 @@ def test_host_buffer_entry_point(ctx, B):
     gu.assert_length_close(y.numpy().astype(np.float64), ref["yhat"])
 
 
-def test_cta_pair_tile_shape_matches_oracle():
-    # the same checks with the LM-head kernel switched to clusters of two CTAs (256 x 256 tiles)
+@pytest.mark.parametrize("mode,tile_cols", [(egtp.EGTP_LMHEAD_CTA_PAIRS, 256), (egtp.EGTP_LMHEAD_CTA_PAIRS_WIDE, 512)])
+def test_cta_pair_tile_shape_matches_oracle(mode, tile_cols):
+    # the same checks with the LM-head kernel switched to clusters of two CTAs (256 x 256 tiles with two accumulator
+    # sets, or 256 x 512 tiles with one set whose two halves are handed back to the MMA warp one after the other)
     c = egtp.egtp_create(0, max_tokens=16384, max_batch=256, max_d=2048, max_V=40000)
     try:
-        egtp.egtp_set_lmhead_mode(c, egtp.EGTP_LMHEAD_CTA_PAIRS)
+        egtp.egtp_set_lmhead_mode(c, mode)
+        plan = egtp.egtp_lmhead_plan(c, 9555, 512, 20072, egtp.EGTP_BF16)
+        assert (plan["rows_per_block"], plan["tile_cols"]) == (256, tile_cols)
         wl = gen.config_mid(V=20000 + 72, d=512, m_h=128)
         ref = orc.egtp_predict(wl.hidden, wl.offsets, wl.W, wl.head, wl.alpha)
         _check_all(gu.run_egtp(c, wl), ref, wl)

@@ -177,6 +177,28 @@ def test_plp_errors_and_host_entry_point(ctx):
     egtp.plp_step(ctx, st, lm, None, hs, reset_src=bad_reset, status_dev=status)
     torch.cuda.synchronize()
     assert int(status.item()) == egtp.EGTP_ERR_BAD_SLOT
+    # two rows of one step on the same slot would race on its state: refused on the device, on both routes, and the
+    # state serves the next (valid) step as before
+    for bind in (False, True):
+        st_d = egtp.plp_state_create(ctx, 8, 128)
+        if bind:
+            egtp.plp_state_bind_head(st_d, head.c)
+        dup = torch.tensor([0, 1, 2, 3, 4, 5, 6, 3], dtype=torch.int32, device="cuda")
+        y = torch.zeros(8, device="cuda")
+        status.zero_()
+        egtp.plp_step(ctx, st_d, lm, head.c, hs, slot_ids=dup, yrem_out=y, status_dev=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == egtp.EGTP_ERR_BAD_SLOT
+        status.zero_()
+        ok_ids = torch.arange(8, dtype=torch.int32, device="cuda")
+        reset_all = torch.full((8,), gen.RESET_EMPTY, dtype=torch.int32, device="cuda")
+        z = torch.zeros(8, 128, device="cuda")
+        egtp.plp_step(ctx, st_d, lm, head.c, hs, slot_ids=ok_ids, reset_src=reset_all, z_out=z, yrem_out=y, status_dev=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert np.array_equal(z.cpu().numpy(), wl.hidden_steps[0])          # restarted empty: z is the row itself
+        egtp.plp_state_destroy(st_d)
+    status.zero_()
     assert egtp.plp_step(ctx, st, lm, None, hs, alpha=-1.0, check=False) == egtp.EGTP_ERR_INVALID_ARG
     st_small = egtp.plp_state_create(ctx, 4, 128)
     assert egtp.plp_step(ctx, st_small, lm, None, hs, check=False) == egtp.EGTP_ERR_CAPACITY
