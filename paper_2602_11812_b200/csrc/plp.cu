@@ -229,6 +229,8 @@ plp_update_bound_kernel(const T* __restrict__ hidden_step, int64_t ldh, const fl
     if (acc_src != nullptr) load8<float>(acc_src + col, acc);
   }
   pdl_wait();
+  // Thread 0 looks at the status word and claims the slot while all warps already merge the row's entropy (reads
+  // only); nothing is written before the block knows that it may go ahead.
   const int stamp = *reinterpret_cast<volatile int32_t*>(epoch);
   if (threadIdx.x == 0) {
     int r = *status != 0 ? 1 : 0;
@@ -238,13 +240,7 @@ plp_update_bound_kernel(const T* __restrict__ hidden_step, int64_t ldh, const fl
     }
     refused = r;
   }
-  __syncthreads();
-  if (refused != 0) {
-    if (threadIdx.x == 0) leave_step(epoch, stamp);
-    return;
-  }
   const float H_new = merge_partials_warp(partials + static_cast<int64_t>(i) * row_stride, slots, slot_stride, threadIdx.x & 31);
-  if (threadIdx.x == 0 && Hstep_out != nullptr) Hstep_out[i] = H_new;
   const float a = H_new * inv_alpha;
   const float m_new = fmaxf(m_old, a);
   const float carry = (s_old > 0.f) ? expf(m_old - m_new) : 0.f;
@@ -252,6 +248,12 @@ plp_update_bound_kernel(const T* __restrict__ hidden_step, int64_t ldh, const fl
   const float s_new = fmaf(s_old, carry, e);
   const float inv_s = 1.f / s_new;
   const float acc_factor = carry * acc_scale_in;
+  __syncthreads();
+  if (refused != 0) {
+    if (threadIdx.x == 0) leave_step(epoch, stamp);
+    return;
+  }
+  if (threadIdx.x == 0 && Hstep_out != nullptr) Hstep_out[i] = H_new;
   // the projected state and the head's hidden layer
   const float* grow = g + static_cast<int64_t>(i) * ldg;
   float* proj_dst = st_proj + static_cast<int64_t>(slot) * m_h;
