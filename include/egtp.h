@@ -130,7 +130,8 @@ EGTP_API int64_t egtp_workspace_bytes(const egtp_ctx* ctx);
  *                 <= T_total (checked on the device: EGTP_ERR_BAD_OFFSETS in the status word)
  *   alpha         temperature dividing the entropies in Eq. 3, > 0
  *   H_out         [T_total] or NULL      token entropies (nats)
- *   weights_out   [T_total] or NULL      w_i of Eq. 3 (0 for tokens in no prompt)
+ *   weights_out   [T_total] or NULL      w_i of Eq. 3 (0 for tokens in no prompt); the pooling itself never stores
+ *                 normalised weights, so asking for them costs one more small launch
  *   seg_id_out    int32 [T_total] or NULL  prompt index of each token, -1 if none
  *   pooled_out    [B][d] or NULL         Eq. 4
  *   state_m_out, state_s_out  [B] each or NULL: max_i H_i/alpha and sum_i exp(H_i/alpha - max),
@@ -184,7 +185,9 @@ EGTP_API int plp_state_import(plp_state* st, const float* m, const float* s, con
  *   then the new token's entropy H' (Eq. 2) enters the softmax and hidden_step[i] the pool.
  * Arguments (device unless stated):
  *   hidden_step   [B_live][ldh] rows in lm->dtype
- *   slot_ids      int32 [B_live], distinct, each in [0, num_slots); NULL = identity (row i -> slot i)
+ *   slot_ids      int32 [B_live], distinct, each in [0, num_slots); NULL = identity (row i -> slot i).  A slot out of
+ *                 range, or named by two rows of one step (they would race on its state), is refused on the device:
+ *                 EGTP_ERR_BAD_SLOT in the status word, the refused rows change nothing
  *   reset_src     int32 [B_live] or NULL (all keep)
  *   src_m, src_s  [n_src]; src_pooled [n_src][d]; may be NULL when n_src == 0
  *   Hstep_out     [B_live] or NULL   entropy of each new token
@@ -236,8 +239,11 @@ EGTP_API int plp_step_host(egtp_ctx* ctx, plp_state* st, const egtp_lm_head* lm,
  * another runtime, a process with a fixed memory budget.  Such callers cannot use egtp_create,
  * which allocates its workspace.  This call needs no context and calls neither cudaMalloc nor
  * cudaFree nor any allocating library routine: the scratch for the first layer's split-K partial
- * sums is a fixed 4 MiB (+256 B) array inside the library image, present on every GPU that has
- * loaded the library until the process exits.
+ * sums is a fixed 4 MiB (+256 B) array inside the library image, held by every GPU that has
+ * loaded the library's device code until the process exits (CUDA loads that code lazily: on a device
+ * that has not run anything of this library yet, the first call is what places the array, and it can
+ * fail with EGTP_ERR_CUDA if the device's memory is exhausted at that moment, so make one warm-up call
+ * at start-up).
  * Computes y_out[r] = head(z[r]) for r < rows exactly as egtp_predict / plp_step do for their
  * pooled vectors (Eq. 6 in bins mode), on the CURRENT device.
  *   head      host struct with device pointers, as above
@@ -328,6 +334,8 @@ EGTP_API int egtp_pool_baseline(egtp_ctx* ctx, const egtp_head* head, const void
  *   EGTP_LMHEAD_CTA_PAIRS: CTA pairs for prompt batches too (256 x 256 tiles).  On a power-capped B200 this
  *     measured equal or slower than AUTO for prompts, so it is an option.
  *   EGTP_LMHEAD_SINGLE_CTA: never use CTA pairs (129..256 rows then run both row tiles in one CTA).
+ *   fp32 inputs always run one CTA per SM, whatever the mode: each operand is split into two tf32 parts in shared
+ *   memory and every k step issues three MMAs (hi.hi + hi.lo + lo.hi), so that the logits keep fp32-level accuracy.
  *   EGTP_LMHEAD_CTA_PAIRS_WIDE: CTA pairs on 256 x 512 tiles for prompt batches too (the decode tile shape): half
  *     the operand bytes an SM pulls in per flop, one accumulator set (the epilogue of a tile does not overlap the next
  *     tile's MMAs).
