@@ -156,7 +156,8 @@ EGTP_API int egtp_predict(egtp_ctx* ctx, const egtp_lm_head* lm, const egtp_head
  * (output), status_host int32 [1] (output: final device status word).  lm and head still
  * point at device-resident parameters.  Copies in, runs, copies out, synchronises `stream`.
  * For batches of 4096 tokens or more the hidden states are copied in up to four row ranges on a stream the
- * context owns, and the LM-head kernel of one range runs while the next range is still being copied. */
+ * context owns (512 rows first, then ranges four times as long, the last one taking the rest), and the LM-head
+ * kernel of one range runs while the next range is still being copied. */
 EGTP_API int egtp_predict_host(egtp_ctx* ctx, const egtp_lm_head* lm, const egtp_head* head,
                       const void* hidden_host, const int32_t* offsets_host,
                       int32_t B, int64_t T_total, float alpha,

@@ -510,13 +510,13 @@ int plp_update_and_head(egtp_ctx* c, plp_state* st, const egtp_head* head, const
   return EGTP_OK;
 }
 
-// The whole EGTP chain.  With pieces > 1 the LM-head phase runs over row ranges of the batch one after the
-// other, each waiting for its own event (the host entry point records one when that range's copy has
-// landed), so that the copy of range i+1 overlaps the GEMM of range i.
+// The whole EGTP chain.  With pieces > 1 the LM-head phase runs over the row ranges [piece_begin[p], piece_begin[p+1])
+// of the batch one after the other (boundaries on multiples of 256 rows), each waiting for its own event (the host
+// entry point records one when that range's copy has landed), so that the copy of range i+1 overlaps the GEMM of range i.
 int predict_impl(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, const void* hidden, int64_t ldh,
                  const int32_t* offsets, int32_t B, int64_t T_total, float alpha, float* H_out, float* weights_out,
                  int32_t* seg_id_out, float* pooled_out, float* state_m_out, float* state_s_out, float* yhat_out,
-                 float* phat_out, int32_t* status_dev, void* stream_v, int pieces, int64_t piece_rows,
+                 float* phat_out, int32_t* status_dev, void* stream_v, int pieces, const int64_t* piece_begin,
                  const cudaEvent_t* piece_ready) {
   if (!c) return EGTP_ERR_INVALID_ARG;
   if (B < 0 || T_total < 0 || !(alpha > 0.f) || !std::isfinite(alpha)) return EGTP_ERR_INVALID_ARG;
@@ -553,9 +553,9 @@ int predict_impl(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, con
     EGTP_CUDA_TRY(launch_validate_offsets(offsets, B, T_total, status, stream));
   }
   for (int p = 0; p < pieces && T_total > 0; ++p) {
-    const int64_t r0 = p * piece_rows;
-    const int64_t rows = std::min<int64_t>(piece_rows, T_total - r0);
-    if (rows <= 0) break;
+    const int64_t r0 = piece_begin ? piece_begin[p] : 0;
+    const int64_t rows = (piece_begin ? piece_begin[p + 1] : T_total) - r0;
+    if (rows <= 0) continue;
     if (piece_ready) EGTP_CUDA_TRY(cudaStreamWaitEvent(stream, piece_ready[p], 0));
     const char* piece_ptr = static_cast<const char*>(hidden) + r0 * ldh * elem_bytes(lm->dtype);
     LmheadPlan plan;
@@ -788,7 +788,7 @@ int egtp_predict(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, con
                  int32_t* seg_id_out, float* pooled_out, float* state_m_out, float* state_s_out, float* yhat_out,
                  float* phat_out, int32_t* status_dev, void* stream_v) {
   return predict_impl(c, lm, head, hidden, ldh, offsets, B, T_total, alpha, H_out, weights_out, seg_id_out, pooled_out,
-                      state_m_out, state_s_out, yhat_out, phat_out, status_dev, stream_v, 1, T_total, nullptr);
+                      state_m_out, state_s_out, yhat_out, phat_out, status_dev, stream_v, 1, nullptr, nullptr);
 }
 
 int egtp_pool_baseline(egtp_ctx* c, const egtp_head* head, const void* hidden, int64_t ldh, int32_t dtype, int32_t d,
@@ -841,19 +841,30 @@ int egtp_predict_host(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head
   if (T_total > c->max_tokens || B > c->max_batch || lm->d > c->max_d) return EGTP_ERR_CAPACITY;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
   if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
-  // The hidden states travel in up to four row ranges on the context's copy stream; the LM-head kernel of
-  // range i starts when its copy has landed, while range i+1 is still on the bus.
+  // The hidden states travel in up to four row ranges on the context's copy stream; the LM-head kernel of range i
+  // starts when its copy has landed, while range i+1 is still on the bus.  A row is copied several times faster than
+  // it is multiplied against the vocabulary, so the ranges grow fourfold from a small first one (512 rows: the only
+  // copy nothing hides) and the last takes the rest: most rows run in one large, efficient launch.
   const int eb = elem_bytes(lm->dtype);
-  const int64_t min_piece = 2048;
-  int pieces = static_cast<int>(std::min<int64_t>(egtp_ctx::kMaxPieces, std::max<int64_t>(1, T_total / min_piece)));
-  const int64_t piece_rows = ((T_total + pieces - 1) / pieces + 255) / 256 * 256;
-  pieces = static_cast<int>((T_total + piece_rows - 1) / piece_rows);
+  int64_t piece_begin[egtp_ctx::kMaxPieces + 1] = {0};
+  int pieces = 0;
+  if (T_total < 4096) {
+    piece_begin[++pieces] = T_total;
+  } else {
+    int64_t next = 512;
+    while (pieces < egtp_ctx::kMaxPieces - 1 && piece_begin[pieces] + next + 1024 <= T_total) {
+      piece_begin[pieces + 1] = piece_begin[pieces] + next;
+      ++pieces;
+      next *= 4;
+    }
+    piece_begin[++pieces] = T_total;
+  }
   // the staging buffer may still be read by earlier work on `stream`
   EGTP_CUDA_TRY(cudaEventRecord(c->stage_free, stream));
   EGTP_CUDA_TRY(cudaStreamWaitEvent(c->copy_stream, c->stage_free, 0));
   for (int p = 0; p < pieces; ++p) {
-    const int64_t r0 = p * piece_rows;
-    const int64_t rows = std::min<int64_t>(piece_rows, T_total - r0);
+    const int64_t r0 = piece_begin[p];
+    const int64_t rows = piece_begin[p + 1] - r0;
     const size_t off_bytes = static_cast<size_t>(r0) * lm->d * eb;
     EGTP_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(c->hidden_stage) + off_bytes,
                                   static_cast<const char*>(hidden_host) + off_bytes,
@@ -863,7 +874,7 @@ int egtp_predict_host(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head
   EGTP_CUDA_TRY(cudaMemcpyAsync(c->offsets_stage, offsets_host, sizeof(int32_t) * (static_cast<size_t>(B) + 1),
                                 cudaMemcpyHostToDevice, stream));
   int rc = predict_impl(c, lm, head, c->hidden_stage, lm->d, c->offsets_stage, B, T_total, alpha, nullptr, nullptr,
-                        nullptr, nullptr, nullptr, nullptr, c->yhat, nullptr, nullptr, stream, pieces, piece_rows,
+                        nullptr, nullptr, nullptr, nullptr, c->yhat, nullptr, nullptr, stream, pieces, piece_begin,
                         c->piece_ready);
   if (rc != EGTP_OK) {
     cudaStreamSynchronize(c->copy_stream);

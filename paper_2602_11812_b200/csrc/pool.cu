@@ -309,30 +309,37 @@ pool_kernel(const T* __restrict__ hidden, int64_t ldh, const float* __restrict__
   }
 }
 
-// One block per prompt (x) and 1024-channel slab (y): zero for an empty prompt; a prompt finished by the first stage
-// is left as it is; else the pieces piece_b[c0], piece_a[c0+1], ..., piece_a[c1] are merged in that order: rescaled
-// to the largest m, summed and normalised (maximum: channel-wise max).  Also leaves the prompt's (M, Z) and,
-// if zcat is given, the pooled row once more as [hi | lo] bf16 halves (input of the head's tensor-core layer 1).
+// One block per prompt (x) and 256-channel slab (y): zero for an empty prompt; a prompt finished by the first stage
+// is left as it is; else the pieces piece_b[c0], piece_a[c0+1], ..., piece_a[c1] are rescaled to the largest m, summed
+// and normalised (maximum: channel-wise max).  The block's four warps take every fourth piece each (two in flight per
+// thread) and their sums are added in warp order, so the result does not depend on timing.  Also leaves the prompt's
+// (M, Z) and, if zcat is given, the pooled row once more as [hi | lo] bf16 halves (input of the head's tensor-core layer 1).
+constexpr int kCombineLanes = 4;                         // warps of a block = pieces worked on at once
+constexpr int kCombineChannels = 32 * 8;                 // channels per block: one warp, 8 per thread
 template <int kMode>
-__global__ void __launch_bounds__(kPoolThreads)
+__global__ void __launch_bounds__(32 * kCombineLanes)
 pool_combine_kernel(const int32_t* __restrict__ off, int B, int d, const float* __restrict__ piece_a,
                     const float* __restrict__ piece_b, const float2* __restrict__ ms_a,
                     const float2* __restrict__ ms_b, float* __restrict__ pooled, float* __restrict__ seg_m,
                     float* __restrict__ seg_s, __nv_bfloat16* __restrict__ zcat, const int32_t* __restrict__ status) {
   if (*status != 0) return;
+  __shared__ float part[kCombineLanes][32][9];            // per warp and thread: 8 channel sums and the weight sum
   const int b = blockIdx.x;
-  const int col = (blockIdx.y * kPoolThreads + threadIdx.x) * 8;
-  if (col >= d) return;
+  const int pl = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int col = blockIdx.y * kCombineChannels + lane * 8;
+  const bool in_d = col < d;
   const bool scribe = blockIdx.y == 0 && threadIdx.x == 0;
   const int64_t s0 = off[b], s1 = off[b + 1];
   float acc[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) acc[k] = 0.f;
   float* dst = pooled + static_cast<int64_t>(b) * d + col;
   __nv_bfloat16* zrow = zcat ? zcat + static_cast<int64_t>(b) * (2 * static_cast<int64_t>(d)) : nullptr;
   if (s1 <= s0) {
-#pragma unroll
-    for (int k = 0; k < 8; ++k) acc[k] = 0.f;
-    store8(dst, acc);
-    if (zrow) store8_hi_lo(zrow, d, col, acc);
+    if (pl == 0 && in_d) {
+      store8(dst, acc);
+      if (zrow) store8_hi_lo(zrow, d, col, acc);
+    }
     if (scribe) {
       if (seg_m) seg_m[b] = -INFINITY;
       if (seg_s) seg_s[b] = 0.f;
@@ -341,55 +348,66 @@ pool_combine_kernel(const int32_t* __restrict__ off, int B, int d, const float* 
   }
   const int64_t c0 = s0 / kPoolChunkTokens, c1 = (s1 - 1) / kPoolChunkTokens;
   if (c0 == c1) {
-    if (zrow) {
+    if (zrow && pl == 0 && in_d) {
       load8f(dst, acc);
       store8_hi_lo(zrow, d, col, acc);
     }
     return;
   }
-  if constexpr (kMode == kPoolMax) {
-    load8f(piece_b + c0 * d + col, acc);
-    for (int64_t c = c0 + 1; c <= c1; ++c) {
-      float pv[8];
-      load8f(piece_a + c * d + col, pv);
+  // pieces in order: index 0 = piece_b[c0], index j >= 1 = piece_a[c0 + j]; warp pl takes j = pl, pl + 4, ...
+  const int64_t n_pieces = c1 - c0 + 1;
+  float M = 0.f;
+  if constexpr (kMode != kPoolMax) {
+    M = ms_b[c0].x;
+    for (int64_t c = c0 + 1; c <= c1; ++c) M = fmaxf(M, ms_a[c].x);
+  } else {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) acc[k] = -INFINITY;
+  }
+  float Z = 0.f;
+  auto piece_ptr = [&](int64_t j) { return (j == 0 ? piece_b : piece_a) + (c0 + j) * d + col; };
+  auto piece_ms = [&](int64_t j) { return j == 0 ? ms_b[c0] : ms_a[c0 + j]; };
+  auto fold = [&](const float (&pv)[8], float2 ms) {
+    if constexpr (kMode == kPoolMax) {
 #pragma unroll
       for (int k = 0; k < 8; ++k) acc[k] = fmaxf(acc[k], pv[k]);
-    }
-  } else {
-    float M = ms_b[c0].x;
-    for (int64_t c = c0 + 1; c <= c1; ++c) M = fmaxf(M, ms_a[c].x);
-    const float2 first = ms_b[c0];
-    float r = expf(first.x - M);
-    float Z = first.y * r;
-    load8f(piece_b + c0 * d + col, acc);
-#pragma unroll
-    for (int k = 0; k < 8; ++k) acc[k] *= r;
-    int64_t c = c0 + 1;
-    for (; c + 4 <= c1 + 1; c += 4) {            // four pieces in flight, added in chunk order
-      float2 ms[4];
-      float pv[4][8];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        ms[u] = ms_a[c + u];
-        load8f(piece_a + (c + u) * d + col, pv[u]);
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        r = expf(ms[u].x - M);
-        Z = fmaf(ms[u].y, r, Z);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) acc[k] = fmaf(pv[u][k], r, acc[k]);
-      }
-    }
-    for (; c <= c1; ++c) {
-      const float2 ms = ms_a[c];
-      r = expf(ms.x - M);
+    } else {
+      const float r = expf(ms.x - M);
       Z = fmaf(ms.y, r, Z);
-      float pv[8];
-      load8f(piece_a + c * d + col, pv);
 #pragma unroll
       for (int k = 0; k < 8; ++k) acc[k] = fmaf(pv[k], r, acc[k]);
     }
+  };
+  if (in_d) {
+    int64_t j = pl;
+    for (; j + kCombineLanes < n_pieces; j += 2 * kCombineLanes) {     // two pieces in flight per thread
+      float p0[8], p1[8];
+      const float2 m0 = kMode == kPoolMax ? make_float2(0.f, 0.f) : piece_ms(j);
+      const float2 m1 = kMode == kPoolMax ? make_float2(0.f, 0.f) : piece_ms(j + kCombineLanes);
+      load8f(piece_ptr(j), p0);
+      load8f(piece_ptr(j + kCombineLanes), p1);
+      fold(p0, m0);
+      fold(p1, m1);
+    }
+    if (j < n_pieces) {
+      float p0[8];
+      const float2 m0 = kMode == kPoolMax ? make_float2(0.f, 0.f) : piece_ms(j);
+      load8f(piece_ptr(j), p0);
+      fold(p0, m0);
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < 8; ++k) part[pl][lane][k] = acc[k];
+  part[pl][lane][8] = Z;
+  __syncthreads();
+  if (pl != 0) return;
+#pragma unroll
+  for (int w = 1; w < kCombineLanes; ++w) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) acc[k] = kMode == kPoolMax ? fmaxf(acc[k], part[w][lane][k]) : acc[k] + part[w][lane][k];
+    Z += part[w][lane][8];
+  }
+  if constexpr (kMode != kPoolMax) {
     const float inv = 1.f / Z;
 #pragma unroll
     for (int k = 0; k < 8; ++k) acc[k] *= inv;
@@ -398,8 +416,10 @@ pool_combine_kernel(const int32_t* __restrict__ off, int B, int d, const float* 
       if (seg_s) seg_s[b] = Z;
     }
   }
-  store8(dst, acc);
-  if (zrow) store8_hi_lo(zrow, d, col, acc);
+  if (in_d) {
+    store8(dst, acc);
+    if (zrow) store8_hi_lo(zrow, d, col, acc);
+  }
 }
 
 }  // namespace
@@ -488,15 +508,16 @@ cudaError_t launch_pool_combine(const int32_t* offsets, int B, int64_t T, int d,
                                 const float* piece_b, const float* piece_ms, float* pooled, float* seg_m, float* seg_s,
                                 void* zcat, const int32_t* status, cudaStream_t stream) {
   const unsigned chunks = static_cast<unsigned>((T + kPoolChunkTokens - 1) / kPoolChunkTokens);
-  const unsigned slabs = static_cast<unsigned>((d + kPoolThreads * 8 - 1) / (kPoolThreads * 8));
+  const unsigned slabs = static_cast<unsigned>((d + kCombineChannels - 1) / kCombineChannels);
   dim3 grid(B, slabs);
   const float2* ms_a = reinterpret_cast<const float2*>(piece_ms);
   const float2* ms_b = ms_a + chunks;
   __nv_bfloat16* zc = static_cast<__nv_bfloat16*>(zcat);
+  constexpr int kThreads = 32 * kCombineLanes;
   if (mode == kPoolMax)
-    pool_combine_kernel<kPoolMax><<<grid, kPoolThreads, 0, stream>>>(offsets, B, d, piece_a, piece_b, ms_a, ms_b, pooled, seg_m, seg_s, zc, status);
+    pool_combine_kernel<kPoolMax><<<grid, kThreads, 0, stream>>>(offsets, B, d, piece_a, piece_b, ms_a, ms_b, pooled, seg_m, seg_s, zc, status);
   else
-    pool_combine_kernel<kPoolEntropy><<<grid, kPoolThreads, 0, stream>>>(offsets, B, d, piece_a, piece_b, ms_a, ms_b, pooled, seg_m, seg_s, zc, status);
+    pool_combine_kernel<kPoolEntropy><<<grid, kThreads, 0, stream>>>(offsets, B, d, piece_a, piece_b, ms_a, ms_b, pooled, seg_m, seg_s, zc, status);
   return cudaGetLastError();
 }
 

@@ -24,6 +24,14 @@ def test_kernel_form_by_row_count():
     # pairs for prompt batches only on request, and never together with head columns
     assert plan(9555, 2048, 151936, mode=egtp.EGTP_LMHEAD_CTA_PAIRS)["variant"] == 4
     assert plan(1024, 5120, 152064, mode=egtp.EGTP_LMHEAD_CTA_PAIRS, head_cols=512)["variant"] == 0
+    wide = plan(25629, 4096, 151936, mode=egtp.EGTP_LMHEAD_CTA_PAIRS_WIDE)      # 256 x 512 tiles for prompts on request
+    assert (wide["variant"], wide["rows_per_block"], wide["tile_cols"], wide["row_blocks"]) == (6, 256, 512, 101)
+    assert wide["n_groups"] == math.ceil(151936 / 512)
+    # fp32 rows: prompt shape and one-row-tile decode shape only, never pairs, two stages holding every tile twice
+    f = egtp.EGTP_F32
+    assert plan(200, 256, 4096, dtype=f)["variant"] == 0 and plan(100, 256, 4096, dtype=f)["variant"] == 1
+    assert plan(9555, 256, 4096, dtype=f, mode=egtp.EGTP_LMHEAD_CTA_PAIRS)["variant"] == 0
+    assert plan(200, 256, 4096, dtype=f)["smem_bytes"] == 2 * 2 * (128 * 128 + 256 * 128) + 256 + 1024
 
 
 def test_decode_plans_give_every_worker_one_vocabulary_range():
