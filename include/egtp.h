@@ -374,12 +374,12 @@ EGTP_API int egtp_selftest_wait_timeout(egtp_ctx* ctx, int32_t limit_ms, int32_t
  * elapsed milliseconds and launch counts per kernel since the last read and clears them.
  * Kernel ids index the two output arrays (host pointers, EGTP_NUM_KERNELS entries each). */
 enum {
-  EGTP_K_VALIDATE = 0,      /* offsets check */
+  EGTP_K_VALIDATE = 0,      /* offsets check as a kernel of its own (normally part of the merge) */
   EGTP_K_LMHEAD_ENTROPY,    /* tcgen05 LM-head GEMM with the online entropy epilogue */
-  EGTP_K_ENTROPY_MERGE,     /* merge of per-vocabulary-chunk partials into H */
-  EGTP_K_SEGMENT_WEIGHTS,   /* Eq. 3 per prompt */
+  EGTP_K_ENTROPY_MERGE,     /* merge of per-vocabulary-chunk partials into H, offsets check, unnormalised Eq. 3 weights */
+  EGTP_K_TOKEN_WEIGHTS,     /* normalised Eq. 3 weights, only when the caller asks for them */
   EGTP_K_POOL,              /* Eq. 4, first stage */
-  EGTP_K_POOL_COMBINE,      /* Eq. 4, deterministic combine of prompts that span chunks */
+  EGTP_K_POOL_COMBINE,      /* Eq. 3-4, deterministic combine of prompts that span chunks, (M, Z), head input */
   EGTP_K_HEAD_HIDDEN,       /* head layer 1 */
   EGTP_K_HEAD_OUT,          /* head layer 2 + output mode */
   EGTP_K_PLP_UPDATE,        /* PLP running-state update */

@@ -27,7 +27,7 @@ PLP_RESET_KEEP, PLP_RESET_EMPTY = -2, -1
 EGTP_LMHEAD_AUTO, EGTP_LMHEAD_CTA_PAIRS, EGTP_LMHEAD_SINGLE_CTA, EGTP_LMHEAD_CTA_PAIRS_WIDE = 0, 1, 2, 3
 EGTP_POOL_MEAN, EGTP_POOL_MAX, EGTP_POOL_LAST = 1, 2, 3
 EGTP_CREATE_NO_HOST_STAGING = 1
-KERNEL_IDS = ["validate_offsets", "lmhead_entropy", "entropy_merge", "segment_weights", "pool",
+KERNEL_IDS = ["validate_offsets", "lmhead_entropy", "entropy_merge", "token_weights", "pool",
               "pool_combine", "head_hidden", "head_out", "plp_update", "logits_entropy", "stage_rows"]
 EGTP_NUM_KERNELS = len(KERNEL_IDS)
 EGTP_K_LMHEAD_ENTROPY = 1

@@ -96,7 +96,7 @@ struct plp_state {
 namespace {
 
 const char* const kKernelNames[EGTP_NUM_KERNELS] = {
-    "validate_offsets", "lmhead_entropy", "entropy_merge", "segment_weights", "pool",
+    "validate_offsets", "lmhead_entropy", "entropy_merge", "token_weights", "pool",
     "pool_combine",     "head_hidden",    "head_out",      "plp_update",    "logits_entropy",
     "stage_rows"};
 
@@ -581,7 +581,7 @@ int predict_impl(egtp_ctx* c, const egtp_lm_head* lm, const egtp_head* head, con
                                       staged ? c->zcat : nullptr, status, stream));
   }
   if (weights_out) {
-    LaunchScope ls(c, EGTP_K_SEGMENT_WEIGHTS, stream);
+    LaunchScope ls(c, EGTP_K_TOKEN_WEIGHTS, stream);
     EGTP_CUDA_TRY(launch_token_weights(H, offsets, B, T_total, 1.f / alpha, seg_m, seg_s, weights_out, status, stream));
   }
   if (staged) return run_head_staged(c, head, B, yhat_out, phat_out, status, stream);
