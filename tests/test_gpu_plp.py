@@ -214,3 +214,24 @@ def test_plp_errors_and_host_entry_point(ctx):
         assert int(sh.item()) == 0
         gu.assert_length_close(y.numpy().astype(np.float64), ref["yrem"][t])
     egtp.plp_state_destroy(st)
+
+
+@pytest.mark.parametrize("slots", [40, 150])
+def test_decode_loop_with_fp32_inputs(ctx, slots):
+    # fp32 hidden states and weights: the LM-head kernel splits every operand into two tf32 parts (three MMAs per k
+    # step); up to 128 rows take the one-row-tile decode shape, more rows the prompt shape
+    rng = np.random.default_rng(slots)
+    d, V, steps = 64, 1500, 4
+    hs = (rng.standard_normal((steps, slots, d)) * 1.5).astype(np.float32)
+    W = (rng.standard_normal((V, d)) * 0.3).astype(np.float32)
+    reset = np.full((steps, slots), gen.RESET_KEEP, np.int32)
+    reset[0] = gen.RESET_EMPTY
+    reset[2, ::7] = gen.RESET_EMPTY
+    head = gen.scaled_head(gen.make_head(31, d, 24, 1, "f32"), "f32")
+    wl = gen.PlpWorkload("f32_decode", "f32", hs, reset, W, head)
+    st, H, z, y = _run_plp(ctx, wl)
+    follow = [0, 7, slots - 1]
+    ref = orc.plp_run(hs, reset, W, head, slots=follow)
+    assert np.abs(orc.logits(hs[0], W)).max() > 8           # logits large enough for a single tf32 rounding to show
+    _compare(H, z, y, ref, follow)
+    egtp.plp_state_destroy(st)
