@@ -398,7 +398,8 @@ def run_mine(args):
             whole_step_frac=plp["hbm"]["whole_step_frac"], tensor_frac=plp["tensor"]["frac"],
             cuda_graph_us=plp.get("cuda_graph_us_per_step"), sm_mhz=plp["clocks"].get("sm_mhz"),
             mcycles_per_step=cycles(plp["us_per_step_median"], plp["clocks"]),
-            e2e_us=plp.get("e2e", {}).get("us_per_step"), unbound_us_per_step_median=plp["unbound_state"]["us_per_step_median"])
+            e2e_us=plp.get("e2e", {}).get("us_per_step"), e2e_pipelined_us=plp.get("e2e", {}).get("pipelined_us_per_step"),
+            unbound_us_per_step_median=plp["unbound_state"]["us_per_step_median"])
         fl = plp["from_logits"]
         legs["from_logits"] = dict(workload="[256, 151936] bf16 logits already in memory (3 buffers in rotation: larger than L2)",
                                    bound="hbm", unit="GB/s", peak=peaks["hbm_gbs"], kernel="logits_entropy",
@@ -537,6 +538,25 @@ def bench_d4096(ctx_device: int, peaks, plp_steps: int, egtp_steps: int, sampler
         assert int(st_host.item()) == 0
         plp["e2e"] = dict(us_per_step=(t1 - t0) / n_e2e * 1e6, steps=n_e2e, api="plp_step_host",
                           h2d_bytes_per_step=slots * d * 2 + slots * 4, d2h_bytes_per_step=slots * 4 + 4)
+        # the same steps handed over without waiting in between (plp_step_host_async: the copy of step t + 1 runs
+        # next to the kernels of step t); every step still gets its rows from pinned host memory and returns its predictions
+        ys = [torch.empty(slots, dtype=torch.float32).pin_memory() for _ in range(n_e2e)]
+        sts = [torch.zeros(1, dtype=torch.int32).pin_memory() for _ in range(n_e2e)]
+        for t in range(3):
+            egtp.plp_step_host_async(ctx, st, lm, head.c, hs_host[t], rs_host[t], None, None, None, 0, slots, 1.0, ys[t], sts[t])
+        torch.cuda.synchronize()
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.perf_counter()
+        p0.record()
+        for t in range(n_e2e):
+            egtp.plp_step_host_async(ctx, st, lm, head.c, hs_host[t], rs_host[t], None, None, None, 0, slots, 1.0, ys[t], sts[t])
+        p1.record()
+        torch.cuda.synchronize()
+        t1 = time.perf_counter()
+        assert all(int(x.item()) == 0 for x in sts)
+        plp["e2e"]["pipelined_us_per_step"] = p0.elapsed_time(p1) / n_e2e * 1e3
+        plp["e2e"]["pipelined_wall_us_per_step"] = (t1 - t0) / n_e2e * 1e6
+        plp["e2e"]["pipelined_api"] = "plp_step_host_async"
         egtp.egtp_profile_enable(ctx, True)
     except Exception as exc:
         plp["e2e"] = dict(error=str(exc)[:200])

@@ -233,6 +233,19 @@ EGTP_API int plp_step_host(egtp_ctx* ctx, plp_state* st, const egtp_lm_head* lm,
                   const float* src_m, const float* src_s, const float* src_pooled, int32_t n_src,
                   int32_t B_live, float alpha, float* yrem_host, int32_t* status_host, void* stream);
 
+/* plp_step_host without the wait at its end, for a decode loop that hands over step t + 1 while step t is still
+ * running: the call enqueues the copy of hidden_step_host (on a stream the context owns, into one of two halves of
+ * its staging buffer), the step and the copies of yrem_host and status_host (on `stream`), and returns.  The copy
+ * of one call therefore overlaps the kernels of the call before it.  yrem_host and status_host hold the step's
+ * results once `stream` has reached the end of the call's work (synchronise the stream or an event recorded behind
+ * the call); all four host buffers must be pinned and stay untouched until then.  Any number of calls may be in
+ * flight; B_live * d elements must fit half of the staging buffer (EGTP_ERR_CAPACITY otherwise).  Do not mix with
+ * the blocking host entry points while calls are in flight. */
+EGTP_API int plp_step_host_async(egtp_ctx* ctx, plp_state* st, const egtp_lm_head* lm, const egtp_head* head,
+                  const void* hidden_step_host, const int32_t* reset_src_host,
+                  const float* src_m, const float* src_s, const float* src_pooled, int32_t n_src,
+                  int32_t B_live, float alpha, float* yrem_host, int32_t* status_host, void* stream);
+
 /* Prediction head alone, for callers that cannot allocate device memory.  (The paper has no
  * counterpart of this entry point; it exists for deployment reasons only.)
  * Who needs it: code that runs inside a host which owns all GPU memory and rules out cudaMalloc

@@ -39,7 +39,7 @@ EXPORTED_SYMBOLS = [
     "egtp_launch_count", "egtp_lmhead_plan", "egtp_head_forward_static", "egtp_set_lmhead_mode",
     "egtp_entropy_from_logits", "plp_step_from_logits", "egtp_pool_baseline",
     "egtp_entropy_partials", "egtp_entropy_from_partials", "plp_step_from_partials", "egtp_selftest_wait_timeout",
-    "plp_state_bind_head", "egtp_set_lmhead_chunks", "egtp_lmhead_plan_for", "egtp_create_ex", "egtp_set_launch_overlap",
+    "plp_state_bind_head", "egtp_set_lmhead_chunks", "egtp_lmhead_plan_for", "egtp_create_ex", "egtp_set_launch_overlap", "plp_step_host_async",
 ]
 
 
@@ -113,6 +113,7 @@ def load() -> C.CDLL:
                              vp, vp, vp, vp, vp]
     lib.plp_step_host.argtypes = [vp, vp, P(egtp_lm_head), P(egtp_head), vp, vp, vp, vp, vp, i32, i32, f32,
                                   vp, vp, vp]
+    lib.plp_step_host_async.argtypes = lib.plp_step_host.argtypes
     lib.egtp_head_forward_static.argtypes = [P(egtp_head), vp, i64, i32, vp, vp, vp]
     for name in EXPORTED_SYMBOLS:
         fn = getattr(lib, name)
@@ -323,6 +324,18 @@ def plp_step_host(ctx: int, st: int, lm: egtp_lm_head, head: egtp_head, hidden_s
                               _ptr(status_host), _stream(stream))
     if check:
         _check(rc, "plp_step_host")
+    return rc
+
+
+def plp_step_host_async(ctx: int, st: int, lm: egtp_lm_head, head: egtp_head, hidden_step_host, reset_src_host,
+                        src_m, src_s, src_pooled, n_src: int, B_live: int, alpha: float, yrem_host, status_host,
+                        stream=None, check: bool = True) -> int:
+    """plp_step_host without the final wait: results are in yrem_host / status_host once the stream has caught up."""
+    rc = load().plp_step_host_async(ctx, st, C.byref(lm), C.byref(head), _ptr(hidden_step_host), _ptr(reset_src_host),
+                                    _ptr(src_m), _ptr(src_s), _ptr(src_pooled), n_src, B_live, alpha, _ptr(yrem_host),
+                                    _ptr(status_host), _stream(stream))
+    if check:
+        _check(rc, "plp_step_host_async")
     return rc
 
 

@@ -52,7 +52,10 @@ struct egtp_ctx {
   void* hidden_stage = nullptr;   // [max_tokens][max_d] in the widest supported dtype; NULL without host staging
   bool host_staging = true;
   int32_t* offsets_stage = nullptr;  // [max_batch + 1]
-  int32_t* reset_stage = nullptr;    // [max_batch]
+  int32_t* reset_stage = nullptr;    // [2][max_batch]
+  int64_t stage_bytes = 0;           // bytes of hidden_stage
+  cudaEvent_t host_in_ready[2] = {}, host_stage_free[2] = {};   // pipelined host steps: two halves of the staging buffers
+  int host_parity = 0;
   int64_t bytes = 0;
 
   // bookkeeping
@@ -115,6 +118,8 @@ void free_ctx_memory(egtp_ctx* c) {
   if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   for (auto& e : c->piece_ready) if (e) cudaEventDestroy(e);
   if (c->stage_free) cudaEventDestroy(c->stage_free);
+  for (auto& e : c->host_in_ready) if (e) cudaEventDestroy(e);
+  for (auto& e : c->host_stage_free) if (e) cudaEventDestroy(e);
   if (c->fork_ev) cudaEventDestroy(c->fork_ev);
   if (c->join_ev) cudaEventDestroy(c->join_ev);
   for (auto& e : c->pending) { cudaEventDestroy(e.start); cudaEventDestroy(e.stop); }
@@ -676,11 +681,14 @@ int egtp_create_ex(egtp_ctx** out, int device, int64_t max_tokens, int32_t max_b
   if (c->host_staging)
     ok = ok && dev_alloc(c, reinterpret_cast<float**>(&c->hidden_stage), rows_cap * max_d) == cudaSuccess;
   ok = ok && dev_alloc(c, &c->offsets_stage, static_cast<int64_t>(max_batch) + 1) == cudaSuccess;
-  ok = ok && dev_alloc(c, &c->reset_stage, max_batch) == cudaSuccess;
+  ok = ok && dev_alloc(c, &c->reset_stage, 2 * static_cast<int64_t>(max_batch)) == cudaSuccess;
+  c->stage_bytes = c->host_staging ? rows_cap * static_cast<int64_t>(max_d) * 4 : 0;
   ok = ok && cudaMemset(c->status, 0, sizeof(int32_t)) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
   for (auto& e : c->piece_ready) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&c->stage_free, cudaEventDisableTiming) == cudaSuccess;
+  for (auto& e : c->host_in_ready) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+  for (auto& e : c->host_stage_free) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&c->fork_ev, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&c->join_ev, cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
@@ -1172,6 +1180,42 @@ int plp_step_host(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp
   EGTP_CUDA_TRY(cudaMemcpyAsync(yrem_host, c->yhat, sizeof(float) * B_live, cudaMemcpyDeviceToHost, stream));
   EGTP_CUDA_TRY(cudaMemcpyAsync(status_host, c->status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
   EGTP_CUDA_TRY(cudaStreamSynchronize(stream));
+  return EGTP_OK;
+}
+
+int plp_step_host_async(egtp_ctx* c, plp_state* st, const egtp_lm_head* lm, const egtp_head* head,
+                        const void* hidden_step_host, const int32_t* reset_src_host, const float* src_m, const float* src_s,
+                        const float* src_pooled, int32_t n_src, int32_t B_live, float alpha, float* yrem_host,
+                        int32_t* status_host, void* stream_v) {
+  if (!c || !st || !lm || !head || !hidden_step_host || !yrem_host || !status_host) return EGTP_ERR_INVALID_ARG;
+  if (B_live <= 0) return EGTP_ERR_INVALID_ARG;
+  if (!c->host_staging) return EGTP_ERR_UNSUPPORTED;
+  if (lm->dtype != EGTP_F32 && lm->dtype != EGTP_BF16) return EGTP_ERR_UNSUPPORTED;
+  if (B_live > c->max_batch || lm->d > c->max_d) return EGTP_ERR_CAPACITY;
+  const size_t hbytes = static_cast<size_t>(B_live) * lm->d * elem_bytes(lm->dtype);
+  const size_t half = static_cast<size_t>(c->stage_bytes / 2) / 256 * 256;
+  if (hbytes > half) return EGTP_ERR_CAPACITY;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  if (cudaSetDevice(c->device) != cudaSuccess) return EGTP_ERR_CUDA;
+  // Calls alternate between the two halves of the staging buffers.  The copy of this call's rows runs on the
+  // context's copy stream, behind the step that read this half two calls ago and next to the previous call's kernels.
+  const int p = c->host_parity;
+  char* hidden_dev = static_cast<char*>(c->hidden_stage) + p * half;
+  int32_t* reset_dev = c->reset_stage + static_cast<int64_t>(p) * c->max_batch;
+  EGTP_CUDA_TRY(cudaStreamWaitEvent(c->copy_stream, c->host_stage_free[p], 0));
+  EGTP_CUDA_TRY(cudaMemcpyAsync(hidden_dev, hidden_step_host, hbytes, cudaMemcpyHostToDevice, c->copy_stream));
+  if (reset_src_host)
+    EGTP_CUDA_TRY(cudaMemcpyAsync(reset_dev, reset_src_host, sizeof(int32_t) * B_live, cudaMemcpyHostToDevice, c->copy_stream));
+  EGTP_CUDA_TRY(cudaEventRecord(c->host_in_ready[p], c->copy_stream));
+  EGTP_CUDA_TRY(cudaStreamWaitEvent(stream, c->host_in_ready[p], 0));
+  int rc = plp_step(c, st, lm, head, hidden_dev, lm->d, nullptr, reset_src_host ? reset_dev : nullptr, src_m, src_s,
+                    src_pooled, n_src, B_live, alpha, nullptr, nullptr, c->yhat, nullptr, stream);
+  // whatever happened, the half counts as used by `stream` up to here
+  if (cudaEventRecord(c->host_stage_free[p], stream) != cudaSuccess) return EGTP_ERR_CUDA;
+  c->host_parity ^= 1;
+  if (rc != EGTP_OK) return rc;
+  EGTP_CUDA_TRY(cudaMemcpyAsync(yrem_host, c->yhat, sizeof(float) * B_live, cudaMemcpyDeviceToHost, stream));
+  EGTP_CUDA_TRY(cudaMemcpyAsync(status_host, c->status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
   return EGTP_OK;
 }
 

@@ -103,3 +103,19 @@ def test_plp_step_from_logits_matches_oracle_and_plp_step(ctx, bind, slots, m_h)
     yb_n = yb.cpu().numpy().astype(np.float64)
     assert np.abs(ya_n - yb_n).max() <= 2e-3 * max(1.0, np.abs(yb_n).max())
     egtp.plp_state_destroy(st_a); egtp.plp_state_destroy(st_b)
+
+
+def test_entropy_from_logits_many_rows_twice():
+    # more rows than a grid dimension of 65535 would hold, and the same context used twice in a row: the per-row
+    # arrival counters of the in-kernel merge must be back at zero after every call
+    rows, V = 70000, 72
+    rng = np.random.default_rng(5)
+    x = gen.round_to_bf16((rng.standard_normal((rows, V)) * 2.0).astype(np.float32))
+    c = egtp.egtp_create(0, max_tokens=rows, max_batch=64, max_d=64, max_V=1024)
+    try:
+        dev = gu.dev_tensor(x, "bf16")
+        ref = orc.entropy_from_logits(x.astype(np.float64))
+        for _ in range(2):
+            gu.assert_entropy_close(_entropy(c, dev, V), ref)
+    finally:
+        egtp.egtp_destroy(c)

@@ -214,6 +214,20 @@ def test_plp_errors_and_host_entry_point(ctx):
         assert int(sh.item()) == 0
         gu.assert_length_close(y.numpy().astype(np.float64), ref["yrem"][t])
     egtp.plp_state_destroy(st)
+    # the same steps handed over without waiting in between (copy of step t + 1 next to the kernels of step t),
+    # each with its own pinned buffers; one wait at the end
+    st = egtp.plp_state_create(ctx, 8, 128)
+    hs_host = [gu.host_tensor(wl.hidden_steps[t], "bf16") for t in range(3)]
+    rs_host = [torch.from_numpy(wl.reset_src[t].copy()).pin_memory() for t in range(3)]
+    ys = [torch.full((8,), float("nan"), dtype=torch.float32).pin_memory() for _ in range(3)]
+    shs = [torch.full((1,), 99, dtype=torch.int32).pin_memory() for _ in range(3)]
+    for t in range(3):
+        egtp.plp_step_host_async(ctx, st, lm, head.c, hs_host[t], rs_host[t], None, None, None, 0, 8, 1.0, ys[t], shs[t])
+    torch.cuda.synchronize()
+    for t in range(3):
+        assert int(shs[t].item()) == 0
+        gu.assert_length_close(ys[t].numpy().astype(np.float64), ref["yrem"][t])
+    egtp.plp_state_destroy(st)
 
 
 @pytest.mark.parametrize("slots", [40, 150])
