@@ -178,6 +178,11 @@ def test_alpha_and_determinism(ctx):
     _check_all(r1, ref, wl)
     for k in ("H", "weights", "pooled", "yhat", "state_m", "state_s"):
         assert np.array_equal(r1[k], r2[k]), k                          # run-to-run bitwise determinism
+    # a sharp and a flat temperature: H/alpha up to ~170 (the weights span e^-100..1 inside one prompt, rescaled
+    # between 64-token chunks), and weights that are nearly uniform
+    for alpha in (0.05, 20.0):
+        wl.alpha = alpha
+        _check_all(gu.run_egtp(ctx, wl), orc.egtp_predict(wl.hidden, wl.offsets, wl.W, wl.head, alpha, H=ref["H"]), wl)
 
 
 def test_errors_are_reported_not_fatal(ctx):
