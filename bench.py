@@ -119,8 +119,13 @@ class ClockSampler:
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
-        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(smax) if smax else None,
-                    power_w=float(np.median(power)) if power else None, samples=len(sm), reasons=sorted(reasons))
+        out = dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(smax) if smax else None,
+                   power_w=float(np.median(power)) if power else None, samples=len(sm), reasons=sorted(reasons))
+        if t1 - t0 < 0.25:
+            # the driver refreshes the clock and power readings only every 100 ms or so (NVML polled every 2 ms shows
+            # the same values through a 90 ms burst), so a region this short mostly sees the state before it
+            out["note"] = "region shorter than the clock readings' refresh interval: values lag the load"
+        return out
 
 
 def cycles(time_us: float, clk: dict):
