@@ -20,7 +20,11 @@
 // for <= 128 and <= 256 rows, where the step is bound by streaming W from HBM once: every SM
 // gets its own vocabulary range (equal to within 32 columns) and, for 129..256 rows, multiplies
 // both row tiles against each W tile it loads.  The CTA-pair kernel further down (tcgen05.mma.cta_group::2)
-// is the default for 129..256 rows (256 x 512 tiles) and an option for prompts (256 x 256 tiles).
+// is the default for 129..256 rows (256 x 512 tiles) and an option for prompts (256 x 256 or 256 x 512 tiles).
+// fp32 inputs (prompt shape and the <= 128-row decode shape only): every operand is split in shared memory into two
+// tf32 parts and each k step issues three MMAs, which keeps the logits at fp32-level accuracy.
+// Both kernels are launched with programmatic stream serialization: what comes before griddepcontrol.wait touches
+// only the block's own shared and tensor memory.
 //
 // Two more uses of the same machinery (prediction head, Sec. 3.2; PLP, Sec. 3.3): with kFuse the column space
 // continues past the vocabulary with the rows of the head's W1, whose products are written out instead of
